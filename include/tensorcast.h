@@ -1,0 +1,286 @@
+/*
+ * tensorcast.h - C ABI of the descriptor-driven batched tensor mover for NVIDIA B200 (sm_100a).
+ *
+ * One "plan" is a validated, immutable batch of copy descriptors (source tensor/offset,
+ * destination tensor/offset, shape, strides).  Executing a plan is one kernel launch on the
+ * caller's stream.  The plan captures geometry only; data pointers are call arguments, so a
+ * plan can be re-executed on any buffers of the same geometry and re-execution is idempotent
+ * (the paper's call contexts make operations re-entrant, Sec. 3.2 "Plan").
+ *
+ * Operations and the passages of the paper that define them:
+ *   tc_kv_pack             publish(req_id): flush the KV cache of a request's whole context out
+ *                          of the engine's paged pool (Table 2 "Instance Operation"; Sec. 3.2;
+ *                          Sec. 4.5 steps 3-4).  Also the offload leg to pinned host memory and,
+ *                          with a migrate plan, publish fused with hydrate (pool to pool).
+ *   tc_kv_unpack           hydrate(req_id, artifacts): load a request's KV cache into the
+ *                          destination engine's paged pool (Table 2; Sec. 4.5 step 8).
+ *   tc_weights_materialize Artifact.tensor_dict() (materialise), Artifact.view(slice) (one
+ *                          tensor-parallel rank's slice, Sec. 6.2) and transform_into(artifact,
+ *                          spec, target) (fill a caller-owned target buffer) (Table 2; Sec. 5
+ *                          "Tensor Materialization and Transfer").
+ *   tc_plan_create/destroy the lifecycle of the plan object itself.
+ * The paper defines no memory layout; the layouts below are this library's.
+ *
+ * Layouts.  E = bytes per element, D = head dim (contiguous everywhere), H = kv heads,
+ * B = tokens per block, L = layers, c = 0 for K and 1 for V.
+ *   Paged pool, plane (l,c), block b, slot n, head h, element d:
+ *     TC_NHD: plane(l,c) + b*block_stride + ((n*H + h)*D + d)*E
+ *     TC_HND: plane(l,c) + b*block_stride + ((h*B + n)*D + d)*E
+ *     plane(l,c) = bases[l*2 + c]                      when the pool has L*2 table slots
+ *                = bases[0] + (l*2 + c)*plane_stride   when it has one slot
+ *   Token t of request r lives in block bt[bt_off[r] + t / B], slot t % B.
+ *   Packed buffer (always one table slot): requests back to back in request order,
+ *     off_0 = 0, off_{r+1} = off_r + L*2*T_r*H*D*E, and inside request r
+ *     TC_NHD: off_r + ((((l*2 + c)*T_r + t)*H + h)*D + d)*E
+ *     TC_HND: off_r + ((((l*2 + c)*H + h)*T_r + t)*D + d)*E      (request level, no padding)
+ *   Only the T_r valid tokens move; the unused slots of a request's last block are neither
+ *   read nor written, and no other byte of a destination is ever written.
+ *
+ * Ownership.  Every data buffer is caller-leased: the library never allocates, frees or
+ * retains it and touches it only between the call and the completion of the stream work the
+ * call enqueued.  Sources are never written.  The plan object is library-owned: created and
+ * destroyed only through this API.  Spec arrays (T, bt_off, bt, index, rules) are read during
+ * tc_plan_create only and may be freed afterwards.
+ *
+ * Memory spaces.  Pointers inside the *tables* passed to the execute calls are DEVICE-
+ * addressable addresses: device memory, or pinned host memory mapped into the device's
+ * address space (cudaHostAlloc / cudaHostRegister under unified addressing), which the kernel
+ * then reads or writes directly over the host link (zero copy).  The tables themselves, the
+ * spec and every array it points to are HOST memory.
+ *
+ * Synchronisation.  Execute calls are asynchronous on `stream` (a cudaStream_t passed as
+ * void*; NULL = the legacy default stream).  Completion is observed through the stream
+ * (events, cudaStreamSynchronize): operations are lazy handles that block only when awaited
+ * (Sec. 3.2).  The library never synchronises the device.
+ *
+ * Errors.  Every function returns a tc_status.  All detectable errors are raised on the host
+ * before anything is launched; a failed call launches nothing, and a failed tc_plan_create
+ * stores NULL in *out.  There is no rollback after a launch (plans have no transactional
+ * semantics, Sec. 3.2).  No exception crosses the ABI.  Calls on distinct plans are thread
+ * safe; one plan may be executed concurrently on different buffers.
+ */
+#ifndef TENSORCAST_H_
+#define TENSORCAST_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define TC_API __attribute__((visibility("default")))
+#else
+#define TC_API
+#endif
+
+typedef enum {
+    TC_OK = 0,
+    TC_ERR_INVALID_ARG = -1, /* NULL where data is required, bad enum, table length mismatch */
+    TC_ERR_SHAPE = -2,       /* non-positive extent, ndim > 4, split dim not divisible by world */
+    TC_ERR_BOUNDS = -3,      /* block id >= num_blocks, offset past a slot / blob / packed size */
+    TC_ERR_OVERLAP = -4,     /* a destination byte written twice, or read and written in one plan */
+    TC_ERR_KIND = -5,        /* execute call does not match the plan's kind */
+    TC_ERR_OOM = -6,         /* host or device allocation of plan storage failed */
+    TC_ERR_CUDA = -7,        /* a CUDA runtime call failed (no device, launch failure) */
+    TC_ERR_DEADLINE = -8     /* the plan's deadline had already passed at call entry */
+} tc_status;
+
+typedef enum {
+    TC_KV_PACK = 1,    /* paged pool -> packed buffer                    (tc_kv_pack)   */
+    TC_KV_UNPACK = 2,  /* packed buffer -> paged pool                    (tc_kv_unpack) */
+    TC_KV_MIGRATE = 3, /* src pool -> dst pool, one launch               (tc_kv_pack)   */
+    TC_KV_MIXED = 4,   /* offload group src_pool -> dst_pool (tc_kv_pack) plus a reload group
+                          dst_pool -> src_pool (tc_kv_unpack) built and checked together   */
+    TC_WEIGHTS = 5     /* flat blob -> per-parameter tensors             (tc_weights_materialize) */
+} tc_kind;
+
+typedef enum { TC_NHD = 0, TC_HND = 1 } tc_layout;
+
+enum {
+    TC_PLAN_HOST_ONLY = 1u /* validate and lower on the host only: the plan can be inspected
+                              (tc_plan_stats, tc_plan_descriptors) but not executed, and no
+                              CUDA call is made */
+};
+
+#define TC_MAX_TABLE_SLOTS 4000 /* src slots + dst slots of one execute call */
+
+/* Geometry of a paged KV pool (the data pointer(s) come at execute time). */
+typedef struct {
+    int32_t layout;       /* tc_layout inside one block */
+    int32_t reserved;     /* 0 */
+    int64_t num_blocks;   /* NB: valid block ids are [0, NB) */
+    int64_t n_slots;      /* length of the base-pointer table passed at execute: L*2 or 1 */
+    int64_t plane_stride; /* n_slots == 1: bytes from plane (l,c) to the next; else ignored */
+    int64_t block_stride; /* bytes between consecutive blocks of a plane; 0 = tight B*H*D*E */
+    int64_t slot_bytes;   /* byte extent of each table slot, used for bounds checks;
+                             0 = the minimum extent that holds NB blocks */
+} tc_kv_pool_t;
+
+/* A group of R requests.  Host arrays, read at create only. */
+typedef struct {
+    int64_t R;             /* number of requests (0 is legal: the group moves nothing) */
+    const int64_t *T;      /* [R]   valid tokens of each request (0 is legal) */
+    const int64_t *bt_off; /* [R+1] CSR offsets into the block tables; bt_off[r+1]-bt_off[r]
+                                    must equal ceil(T[r] / B) */
+    const int32_t *bt_src; /* block ids in the source pool (NULL when the source is packed) */
+    const int32_t *bt_dst; /* block ids in the destination pool (NULL when the destination
+                              is packed).  No id may appear twice in bt_dst. */
+} tc_kv_group_t;
+
+typedef struct {
+    int64_t L, B, H, D, E;   /* E in {1,2,4,8}; contents are opaque bytes */
+    tc_kv_pool_t src_pool;   /* PACK, MIGRATE, MIXED (the device pool) */
+    tc_kv_pool_t dst_pool;   /* UNPACK, MIGRATE, MIXED (the host pool) */
+    int32_t packed_layout;   /* PACK / UNPACK: tc_layout of the packed buffer */
+    int32_t reserved;        /* 0 */
+    int64_t packed_bytes;    /* PACK / UNPACK: capacity of the packed buffer, for bounds checks;
+                                0 = exactly the required size */
+    tc_kv_group_t group;     /* PACK, UNPACK, MIGRATE; MIXED: the offload group */
+    tc_kv_group_t reload;    /* MIXED only: moves dst_pool[bt_src] -> src_pool[bt_dst] */
+} tc_kv_spec_t;
+
+/* One record of the blob's binary offset index (64 bytes, little endian when stored). */
+typedef struct {
+    uint64_t byte_off;   /* start of the tensor in the blob */
+    uint64_t nbytes;     /* must equal elem_bytes * prod(shape) */
+    uint32_t elem_bytes; /* 1, 2, 4 or 8 */
+    uint32_t ndim;       /* 1..4 */
+    uint64_t shape[4];   /* row-major, tight; unused trailing dims = 1 */
+    uint64_t name_id;    /* opaque: index into the caller's side table of names */
+} tc_index_entry_t;
+
+/* Where tensor i goes.  All-default (rules == NULL): whole tensor, tight, into dst slot i. */
+typedef struct {
+    int32_t split_dim;     /* -1: copy the whole tensor; else rank gets slab
+                              [rank*n/world, (rank+1)*n/world) of this dim (n % world == 0) */
+    int32_t dst_slot;      /* index into dst_ptrs; -1 = i */
+    int64_t dst_off;       /* byte offset inside the slot */
+    int64_t dst_stride[4]; /* byte strides of the destination's dims; all 0 = tight row-major
+                              strides of the (sliced) shape */
+} tc_weight_rule_t;
+
+typedef struct {
+    int64_t n_tensors;
+    const tc_index_entry_t *index; /* [n_tensors] */
+    const tc_weight_rule_t *rules; /* [n_tensors] or NULL */
+    int32_t rank, world;           /* tensor-parallel rank and world size (1 = no sharding) */
+    int64_t blob_bytes;            /* extent of the blob, for bounds checks */
+    int64_t n_dst;                 /* number of destination slots; 0 = n_tensors */
+    const int64_t *dst_bytes;      /* [n_dst] extent of each destination slot, or NULL = each
+                                      slot is exactly as large as its (sliced) tensor */
+} tc_weights_spec_t;
+
+/* Optional knobs; 0 everywhere = the library's defaults. */
+typedef struct {
+    int32_t tile_bytes;   /* target bytes per tile (one CTA iteration) */
+    int32_t ctas_per_sm;  /* resident CTAs per SM for the persistent grid */
+    int32_t max_ctas;     /* cap on the grid (e.g. few CTAs for host-link transfers) */
+    int32_t path;         /* 0 auto; 1 force the register (ld/st) path; 2 force the bulk-copy
+                             (shared-memory staged) path where the geometry allows it */
+} tc_tuning_t;
+
+typedef struct {
+    uint32_t struct_size; /* sizeof(tc_plan_spec_t) */
+    int32_t kind;         /* tc_kind */
+    uint32_t flags;       /* TC_PLAN_* */
+    uint32_t reserved;    /* 0 */
+    uint64_t trace_id;    /* opaque, echoed in tc_plan_stats (the call context's tracing id) */
+    int64_t deadline_ns;  /* absolute CLOCK_MONOTONIC nanoseconds; 0 = none.  A call entered
+                             after the deadline returns TC_ERR_DEADLINE and launches nothing */
+    tc_tuning_t tuning;
+    tc_kv_spec_t kv;           /* kinds 1-4 */
+    tc_weights_spec_t weights; /* kind 5 */
+} tc_plan_spec_t;
+
+typedef struct tc_plan tc_plan_t;
+
+/*
+ * Validate `spec` on the host, lower it to descriptors and tiles, upload them to the current
+ * CUDA device (unless TC_PLAN_HOST_ONLY) and return an immutable plan in *out.
+ * spec, out: host pointers.  On error *out = NULL and nothing stays allocated.
+ */
+TC_API int tc_plan_create(const tc_plan_spec_t *spec, tc_plan_t **out);
+
+/*
+ * Run the gather side of `plan` on `stream`:
+ *   TC_KV_PACK    src_bases = the pool's table (src_pool.n_slots entries), dst_bases = {packed}
+ *   TC_KV_MIGRATE src_bases = source pool table, dst_bases = destination pool table
+ *   TC_KV_MIXED   the offload group: src_bases = src_pool table, dst_bases = dst_pool table
+ * src_bases / dst_bases: HOST arrays of n_src / n_dst device-addressable pointers; they are
+ * read before the call returns.  n_src and n_dst must match the plan (TC_ERR_INVALID_ARG).
+ */
+TC_API int tc_kv_pack(const tc_plan_t *plan, const void *const *src_bases, size_t n_src,
+               void *const *dst_bases, size_t n_dst, void *stream);
+
+/*
+ * Run the scatter side of `plan` on `stream`:
+ *   TC_KV_UNPACK  src_bases = {packed}, dst_bases = the pool's table (dst_pool.n_slots)
+ *   TC_KV_MIXED   the reload group: src_bases = dst_pool table (the host pool it reads),
+ *                 dst_bases = src_pool table (the device pool it fills).  The two groups of a
+ *                 mixed plan touch disjoint blocks and may run concurrently on two streams.
+ * Pool bytes not addressed by the plan keep their contents.
+ */
+TC_API int tc_kv_unpack(const tc_plan_t *plan, const void *const *src_bases, size_t n_src,
+                 void *const *dst_bases, size_t n_dst, void *stream);
+
+/*
+ * Scatter tensors out of the flat blob: dst_ptrs[slot] + dst_off <- blob[byte_off ...], whole
+ * or one rank's slice, per the plan's rules.  blob: device-addressable pointer (device memory
+ * or mapped pinned host memory).  dst_ptrs: HOST array of n_dst device-addressable pointers.
+ */
+TC_API int tc_weights_materialize(const tc_plan_t *plan, const void *blob, void *const *dst_ptrs,
+                           size_t n_dst, void *stream);
+
+/*
+ * Free the plan's host and device storage.  The caller must first have synchronised every
+ * stream that executes it.  NULL is a no-op returning TC_OK.
+ */
+TC_API int tc_plan_destroy(tc_plan_t *plan);
+
+/* ---- off the data path: inspection and diagnostics -------------------------------------- */
+
+typedef struct {
+    uint64_t trace_id;
+    int32_t kind;
+    int32_t executable;            /* 0 for TC_PLAN_HOST_ONLY plans */
+    int64_t n_descriptors[2];      /* [0] pack/migrate/offload/weights group, [1] unpack/reload */
+    int64_t n_tiles[2];
+    int64_t payload_bytes[2];      /* bytes moved by one execution of each group */
+    int64_t packed_bytes_required; /* PACK / UNPACK: sum of L*2*T_r*H*D*E */
+    int64_t device_bytes;          /* plan storage held on the device */
+    int32_t vec_bytes[2];          /* widest access the geometry allows (pointers may narrow it) */
+    int32_t launches_per_execute;  /* kernels one execute call launches (1; 0 if empty) */
+    int32_t path[2];               /* 1 register path, 2 bulk-copy path */
+    int32_t grid[2];               /* CTAs launched per execution */
+} tc_plan_stats_t;
+
+/* Fill *out (host pointer) with the plan's figures. */
+TC_API int tc_plan_stats(const tc_plan_t *plan, tc_plan_stats_t *out);
+
+/* A lowered descriptor as tests and tools may inspect it: a box of n_outer x rows runs of
+ * run_bytes contiguous bytes.  Row k of outer index o starts at
+ *   src: slot src_slot + o*src_slot_step, byte src_off + o*src_outer + (k/n0)*src_s1 + (k%n0)*src_s0
+ *   dst: likewise.  Slots index the src / dst table of the execute call. */
+typedef struct {
+    int64_t src_off, dst_off, src_outer, dst_outer, src_s0, src_s1, dst_s0, dst_s1;
+    uint32_t src_slot, dst_slot, src_slot_step, dst_slot_step;
+    uint32_t run_bytes, n0, rows, n_outer;
+} tc_descriptor_t;
+
+/* Copy up to `cap` descriptors of `group` (0 or 1) into out (host array); *n_out receives the
+ * group's total count. */
+TC_API int tc_plan_descriptors(const tc_plan_t *plan, int group, tc_descriptor_t *out, size_t cap,
+                        size_t *n_out);
+
+/* Static string naming a status code. */
+TC_API const char *tc_strerror(int status);
+
+/* Detail of the calling thread's most recent failure ("" if none); valid until its next call. */
+TC_API const char *tc_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TENSORCAST_H_ */

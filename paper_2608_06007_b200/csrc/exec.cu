@@ -1,0 +1,409 @@
+// Plan lifecycle and the copy-executor kernels (sm_100a).
+//
+// One launch executes one group of a plan.  The grid is persistent: CTAs walk the plan's tile
+// ids with a grid stride; a tile is one outer index (a KV plane) and a row range of one
+// descriptor, about tile_bytes of payload.  Inside a tile every thread moves 16-byte vectors
+// (narrower when the geometry or a base pointer is less aligned): a batch of independent
+// loads first, then the stores, so that many requests per thread are in flight.  Consecutive
+// lanes touch consecutive vectors of a run, so every warp access is one or more whole,
+// aligned segments on both the read and the write side.  Base pointers travel in the kernel
+// parameters; nothing is allocated or copied per execute call.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "plan.h"
+
+namespace tc {
+
+constexpr int kThreads = 256;
+constexpr int kUnrollWide = 8;    // 16-byte vectors in flight per thread
+constexpr int kUnrollNarrow = 4;  // same for the narrower fallback widths
+constexpr int kMinCtasPerSm = 3;
+
+template <int NPTR>
+struct Params {
+    const Desc *descs;
+    const uint32_t *tile_desc;  // null for uniform groups
+    uint32_t n_tiles;
+    uint32_t tiles_per_desc;    // > 0 for uniform groups
+    FastDiv div_tpd;
+    uint32_t log2_ptr_align;    // alignment shared by every base pointer (capped at 4)
+    char *ptr[NPTR];            // src table then dst table
+};
+
+__device__ __forceinline__ uint32_t fastdiv(uint32_t n, FastDiv f) { return (__umulhi(n, f.mul) + n) >> f.shift; }
+
+template <typename V> __device__ __forceinline__ V ld_stream(const char *p);
+template <typename V> __device__ __forceinline__ void st_stream(char *p, V v);
+
+template <> __device__ __forceinline__ uint4 ld_stream<uint4>(const char *p) { return __ldcs(reinterpret_cast<const uint4 *>(p)); }
+template <> __device__ __forceinline__ void st_stream<uint4>(char *p, uint4 v) { __stcs(reinterpret_cast<uint4 *>(p), v); }
+#define TC_NARROW(V)                                                                                  \
+    template <> __device__ __forceinline__ V ld_stream<V>(const char *p) { return *reinterpret_cast<const V *>(p); } \
+    template <> __device__ __forceinline__ void st_stream<V>(char *p, V v) { *reinterpret_cast<V *>(p) = v; }
+TC_NARROW(uint2)
+TC_NARROW(uint32_t)
+TC_NARROW(uint16_t)
+TC_NARROW(uint8_t)
+#undef TC_NARROW
+
+template <int LOGV> struct VecOf;
+template <> struct VecOf<4> { using type = uint4; };
+template <> struct VecOf<3> { using type = uint2; };
+template <> struct VecOf<2> { using type = uint32_t; };
+template <> struct VecOf<1> { using type = uint16_t; };
+template <> struct VecOf<0> { using type = uint8_t; };
+
+// Copy rows [row0, row0 + nrows) of one outer index of descriptor d; src / dst point at row 0.
+// A thread's vectors are kThreads vectors apart, so a warp always covers 32 consecutive
+// vectors of the tile's row space: whole aligned segments on both sides.
+template <int LOGV, int U>
+__device__ __forceinline__ void copy_rows(const Desc &d, const char *src, char *dst, uint32_t row0, uint32_t nrows)
+{
+    using V = typename VecOf<LOGV>::type;
+    const uint32_t nbytes = nrows * d.run;  // <= 1 MiB
+    const uint32_t run = d.run, n0 = d.n0;
+    const FastDiv div_run = d.div_run, div_n0 = d.div_n0;
+    const uint32_t ss0 = d.src_s0, ss1 = d.src_s1, ds0 = d.dst_s0, ds1 = d.dst_s1;
+#pragma unroll 1
+    for (uint32_t base = threadIdx.x << LOGV; base < nbytes; base += (kThreads * U) << LOGV) {
+        V val[U];
+        uint32_t doff[U];
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+            const uint32_t byte = base + ((u * kThreads) << LOGV);
+            if (byte < nbytes) {
+                uint32_t r = fastdiv(byte, div_run);
+                const uint32_t col = byte - r * run;
+                r += row0;
+                const uint32_t i1 = fastdiv(r, div_n0);
+                const uint32_t i0 = r - i1 * n0;
+                doff[u] = i1 * ds1 + i0 * ds0 + col;
+                val[u] = ld_stream<V>(src + (i1 * ss1 + i0 * ss0 + col));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+            const uint32_t byte = base + ((u * kThreads) << LOGV);
+            if (byte < nbytes) st_stream<V>(dst + doff[u], val[u]);
+        }
+    }
+}
+
+// One contiguous run of 16-byte vectors: no row decoding at all.
+template <int U>
+__device__ __forceinline__ void copy_run16(const char *src, char *dst, uint32_t nbytes)
+{
+#pragma unroll 1
+    for (uint32_t base = threadIdx.x << 4; base < nbytes; base += (kThreads * U) << 4) {
+        uint4 val[U];
+#pragma unroll
+        for (int u = 0; u < U; u++)
+            if (base + ((u * kThreads) << 4) < nbytes) val[u] = ld_stream<uint4>(src + base + ((u * kThreads) << 4));
+#pragma unroll
+        for (int u = 0; u < U; u++)
+            if (base + ((u * kThreads) << 4) < nbytes) st_stream<uint4>(dst + base + ((u * kThreads) << 4), val[u]);
+    }
+}
+
+// Three builds of the executor, chosen per group on the host, so that the common cases do not
+// pay registers for the rare ones:
+//   kModeRun   every tile is one 16-byte-aligned contiguous run (same-layout KV blocks, whole
+//              tensors, dim-0 slabs): no row decoding
+//   kModeRows  every access is 16-byte aligned, tiles hold strided rows (layout transforms,
+//              dim-1 slices)
+//   kModeAny   some descriptor or base pointer is less aligned: width picked per tile
+enum { kModeRun = 0, kModeRows = 1, kModeAny = 2 };
+
+template <int NPTR, int MODE>
+__global__ void __launch_bounds__(kThreads, MODE == kModeAny ? 2 : kMinCtasPerSm) tc_copy_kernel(const __grid_constant__ Params<NPTR> prm)
+{
+    __shared__ Desc sdesc[2];
+    int buf = 0;
+    for (uint32_t tile = blockIdx.x; tile < prm.n_tiles; tile += gridDim.x, buf ^= 1) {
+        uint32_t di, t = 0;
+        if (prm.tiles_per_desc) {
+            di = fastdiv(tile, prm.div_tpd);
+            t = tile - di * prm.tiles_per_desc;
+        } else {
+            di = __ldg(prm.tile_desc + tile);
+        }
+        if (threadIdx.x < sizeof(Desc) / 16)
+            reinterpret_cast<uint4 *>(&sdesc[buf])[threadIdx.x] = __ldg(reinterpret_cast<const uint4 *>(prm.descs + di) + threadIdx.x);
+        __syncthreads();
+        const Desc &d = sdesc[buf];
+        if (!prm.tiles_per_desc) t = tile - d.tile0;
+        const uint32_t o = fastdiv(t, d.div_tpo);
+        const uint32_t part = t - o * d.tiles_per_outer;
+        const uint32_t row0 = part * d.rows_per_tile;
+        if (row0 >= d.rows) continue;  // padding tile of a uniform group
+        const uint32_t nrows = min(d.rows_per_tile, d.rows - row0);
+        const char *src = prm.ptr[d.src_slot + o * d.src_slot_step] + d.src_off + o * d.src_outer;
+        char *dst = prm.ptr[d.dst_slot + o * d.dst_slot_step] + d.dst_off + o * d.dst_outer;
+        if (MODE == kModeRun) {
+            const uint32_t i1 = fastdiv(row0, d.div_n0), i0 = row0 - i1 * d.n0;
+            copy_run16<kUnrollWide>(src + (i1 * d.src_s1 + i0 * d.src_s0), dst + (i1 * d.dst_s1 + i0 * d.dst_s0), d.run);
+        } else if (MODE == kModeRows) {
+            copy_rows<4, kUnrollWide>(d, src, dst, row0, nrows);
+        } else {
+            switch (min(d.log2_align, prm.log2_ptr_align)) {
+            case 4: copy_rows<4, kUnrollNarrow>(d, src, dst, row0, nrows); break;
+            case 3: copy_rows<3, kUnrollNarrow>(d, src, dst, row0, nrows); break;
+            case 2: copy_rows<2, kUnrollNarrow>(d, src, dst, row0, nrows); break;
+            case 1: copy_rows<1, kUnrollNarrow>(d, src, dst, row0, nrows); break;
+            default: copy_rows<0, kUnrollNarrow>(d, src, dst, row0, nrows); break;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------ host side
+static int cuda_fail(cudaError_t e, const char *what)
+{
+    return fail(TC_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+static void free_group(Group &g)
+{
+    if (g.d_descs) cudaFree(g.d_descs);
+    if (g.d_tile_desc) cudaFree(g.d_tile_desc);
+    g.d_descs = nullptr;
+    g.d_tile_desc = nullptr;
+}
+
+static int upload_group(tc_plan *plan, Group &g)
+{
+    if (g.descs.empty()) return TC_OK;
+    cudaError_t e;
+    size_t nb = g.descs.size() * sizeof(Desc);
+    if ((e = cudaMalloc(&g.d_descs, nb)) != cudaSuccess)
+        return e == cudaErrorMemoryAllocation ? fail(TC_ERR_OOM, "device allocation of %zu descriptor bytes failed", nb) : cuda_fail(e, "cudaMalloc");
+    if ((e = cudaMemcpy(g.d_descs, g.descs.data(), nb, cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(e, "cudaMemcpy(descriptors)");
+    plan->device_bytes += nb;
+    if (!g.tile_desc.empty()) {
+        nb = g.tile_desc.size() * sizeof(uint32_t);
+        if ((e = cudaMalloc(&g.d_tile_desc, nb)) != cudaSuccess)
+            return e == cudaErrorMemoryAllocation ? fail(TC_ERR_OOM, "device allocation of %zu tile bytes failed", nb) : cuda_fail(e, "cudaMalloc");
+        if ((e = cudaMemcpy(g.d_tile_desc, g.tile_desc.data(), nb, cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(e, "cudaMemcpy(tiles)");
+        plan->device_bytes += nb;
+    }
+    return TC_OK;
+}
+
+// Which executor build a group needs, given the alignment shared by the call's base pointers.
+static int mode_for(const Group &g, uint32_t ptr_align)
+{
+    if (g.log2_align < 4 || ptr_align < 4) return kModeAny;
+    return g.single_run_tiles ? kModeRun : kModeRows;
+}
+
+template <int NPTR, int MODE>
+static int resident_ctas()
+{
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, tc_copy_kernel<NPTR, MODE>, kThreads, 0) != cudaSuccess || n < 1) n = 1;
+    return n;
+}
+
+template <int NPTR>
+static void resident_ctas_all(int out[3])
+{
+    out[kModeRun] = resident_ctas<NPTR, kModeRun>();
+    out[kModeRows] = resident_ctas<NPTR, kModeRows>();
+    out[kModeAny] = resident_ctas<NPTR, kModeAny>();
+}
+
+static void resident_ctas_for(size_t n_ptrs, int out[3])
+{
+    if (n_ptrs <= 8) resident_ctas_all<8>(out);
+    else if (n_ptrs <= 400) resident_ctas_all<400>(out);
+    else resident_ctas_all<TC_MAX_TABLE_SLOTS>(out);
+}
+
+static uint32_t grid_for(const tc_plan *plan, const Group &g, int mode)
+{
+    int per_sm = g.resident_ctas[mode] > 0 ? g.resident_ctas[mode] : 1;
+    if (plan->tuning.ctas_per_sm > 0) per_sm = std::min(per_sm, plan->tuning.ctas_per_sm);
+    uint64_t grid = static_cast<uint64_t>(plan->sm_count > 0 ? plan->sm_count : 148) * per_sm;
+    if (plan->tuning.max_ctas > 0) grid = std::min<uint64_t>(grid, plan->tuning.max_ctas);
+    return static_cast<uint32_t>(std::min<uint64_t>(grid, g.n_tiles));
+}
+
+template <int NPTR>
+static int launch(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t stream)
+{
+    const int mode = mode_for(g, ptr_align);
+    const uint32_t grid = grid_for(plan, g, mode);
+    Params<NPTR> prm;
+    prm.descs = g.d_descs;
+    prm.tile_desc = g.d_tile_desc;
+    prm.n_tiles = static_cast<uint32_t>(g.n_tiles);
+    prm.tiles_per_desc = g.tiles_per_desc;
+    prm.div_tpd = g.div_tpd;
+    prm.log2_ptr_align = ptr_align;
+    for (size_t i = 0; i < g.n_src; i++) prm.ptr[i] = const_cast<char *>(static_cast<const char *>(src[i]));
+    for (size_t i = 0; i < g.n_dst; i++) prm.ptr[g.n_src + i] = static_cast<char *>(dst[i]);
+    for (size_t i = g.n_src + g.n_dst; i < NPTR; i++) prm.ptr[i] = nullptr;
+    switch (mode) {
+    case kModeRun: tc_copy_kernel<NPTR, kModeRun><<<grid, kThreads, 0, stream>>>(prm); break;
+    case kModeRows: tc_copy_kernel<NPTR, kModeRows><<<grid, kThreads, 0, stream>>>(prm); break;
+    default: tc_copy_kernel<NPTR, kModeAny><<<grid, kThreads, 0, stream>>>(prm); break;
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
+    return TC_OK;
+}
+
+static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n_src, void *const *dst, size_t n_dst, void *stream)
+{
+    clear_error();
+    if (!plan) return fail(TC_ERR_INVALID_ARG, "plan is NULL");
+    if (plan->flags & TC_PLAN_HOST_ONLY) return fail(TC_ERR_INVALID_ARG, "a TC_PLAN_HOST_ONLY plan cannot be executed");
+    const Group &g = plan->group[gi];
+    if (n_src != g.n_src || n_dst != g.n_dst)
+        return fail(TC_ERR_INVALID_ARG, "tables of %zu source and %zu destination pointers given, the plan needs %zu and %zu", n_src, n_dst, g.n_src, g.n_dst);
+    if ((n_src && !src) || (n_dst && !dst)) return fail(TC_ERR_INVALID_ARG, "pointer table is NULL");
+    if (plan->deadline_ns && now_ns() > plan->deadline_ns) return fail(TC_ERR_DEADLINE, "deadline passed before the call; nothing launched");
+    if (g.n_tiles == 0) return TC_OK;
+    uint32_t ptr_align = 4;
+    for (size_t i = 0; i < n_src; i++) {
+        if (!src[i]) return fail(TC_ERR_INVALID_ARG, "source table entry %zu is NULL", i);
+        ptr_align = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(src[i]) | 16));
+    }
+    for (size_t i = 0; i < n_dst; i++) {
+        if (!dst[i]) return fail(TC_ERR_INVALID_ARG, "destination table entry %zu is NULL", i);
+        ptr_align = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(dst[i]) | 16));
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t n = n_src + n_dst;
+    if (n <= 8) return launch<8>(plan, g, src, dst, ptr_align, s);
+    if (n <= 400) return launch<400>(plan, g, src, dst, ptr_align, s);
+    return launch<TC_MAX_TABLE_SLOTS>(plan, g, src, dst, ptr_align, s);
+}
+
+}  // namespace tc
+
+using namespace tc;
+
+extern "C" int tc_plan_create(const tc_plan_spec_t *spec, tc_plan_t **out)
+{
+    clear_error();
+    if (out) *out = nullptr;
+    if (!spec || !out) return fail(TC_ERR_INVALID_ARG, "spec and out are required");
+    if (spec->struct_size != sizeof(tc_plan_spec_t))
+        return fail(TC_ERR_INVALID_ARG, "spec.struct_size %u != %zu: header and library disagree", spec->struct_size, sizeof(tc_plan_spec_t));
+    if (spec->deadline_ns && now_ns() > spec->deadline_ns) return fail(TC_ERR_DEADLINE, "deadline passed before the call");
+    tc_plan *plan = new (std::nothrow) tc_plan();
+    if (!plan) return fail(TC_ERR_OOM, "host allocation failed");
+    plan->kind = spec->kind;
+    plan->flags = spec->flags;
+    plan->trace_id = spec->trace_id;
+    plan->deadline_ns = spec->deadline_ns;
+    plan->tuning = spec->tuning;
+    int rc;
+    try {
+        rc = build_plan(spec, plan);
+    } catch (const std::bad_alloc &) {
+        rc = fail(TC_ERR_OOM, "host allocation failed while lowering the plan");
+    }
+    if (rc == TC_OK && !(spec->flags & TC_PLAN_HOST_ONLY)) {
+        cudaError_t e = cudaGetDevice(&plan->device);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&plan->sm_count, cudaDevAttrMultiProcessorCount, plan->device);
+        if (e != cudaSuccess) rc = cuda_fail(e, "querying the current device");
+        for (int k = 0; k < 2 && rc == TC_OK; k++) {
+            rc = upload_group(plan, plan->group[k]);
+            if (plan->group[k].n_tiles) resident_ctas_for(plan->group[k].n_src + plan->group[k].n_dst, plan->group[k].resident_ctas);
+        }
+    }
+    if (rc != TC_OK) {
+        free_group(plan->group[0]);
+        free_group(plan->group[1]);
+        delete plan;
+        return rc;
+    }
+    *out = plan;
+    return TC_OK;
+}
+
+extern "C" int tc_plan_destroy(tc_plan_t *plan)
+{
+    if (!plan) return TC_OK;
+    free_group(plan->group[0]);
+    free_group(plan->group[1]);
+    delete plan;
+    return TC_OK;
+}
+
+extern "C" int tc_kv_pack(const tc_plan_t *plan, const void *const *src_bases, size_t n_src, void *const *dst_bases, size_t n_dst, void *stream)
+{
+    if (plan && plan->kind != TC_KV_PACK && plan->kind != TC_KV_MIGRATE && plan->kind != TC_KV_MIXED) {
+        clear_error();
+        return fail(TC_ERR_KIND, "tc_kv_pack needs a PACK, MIGRATE or MIXED plan (kind %d given)", plan->kind);
+    }
+    return execute(plan, 0, src_bases, n_src, dst_bases, n_dst, stream);
+}
+
+extern "C" int tc_kv_unpack(const tc_plan_t *plan, const void *const *src_bases, size_t n_src, void *const *dst_bases, size_t n_dst, void *stream)
+{
+    if (plan && plan->kind != TC_KV_UNPACK && plan->kind != TC_KV_MIXED) {
+        clear_error();
+        return fail(TC_ERR_KIND, "tc_kv_unpack needs an UNPACK or MIXED plan (kind %d given)", plan->kind);
+    }
+    return execute(plan, 1, src_bases, n_src, dst_bases, n_dst, stream);
+}
+
+extern "C" int tc_weights_materialize(const tc_plan_t *plan, const void *blob, void *const *dst_ptrs, size_t n_dst, void *stream)
+{
+    if (plan && plan->kind != TC_WEIGHTS) {
+        clear_error();
+        return fail(TC_ERR_KIND, "tc_weights_materialize needs a WEIGHTS plan (kind %d given)", plan->kind);
+    }
+    const void *src[1] = {blob};
+    return execute(plan, 0, src, 1, dst_ptrs, n_dst, stream);
+}
+
+extern "C" int tc_plan_stats(const tc_plan_t *plan, tc_plan_stats_t *out)
+{
+    clear_error();
+    if (!plan || !out) return fail(TC_ERR_INVALID_ARG, "plan and out are required");
+    memset(out, 0, sizeof *out);
+    out->trace_id = plan->trace_id;
+    out->kind = plan->kind;
+    out->executable = !(plan->flags & TC_PLAN_HOST_ONLY);
+    for (int k = 0; k < 2; k++) {
+        const Group &g = plan->group[k];
+        out->n_descriptors[k] = static_cast<int64_t>(g.descs.size());
+        out->n_tiles[k] = static_cast<int64_t>(g.n_tiles);
+        out->payload_bytes[k] = g.payload;
+        out->vec_bytes[k] = 1 << g.log2_align;
+        out->path[k] = g.n_tiles ? 1 : 0;
+        out->grid[k] = g.n_tiles ? static_cast<int32_t>(grid_for(plan, g, mode_for(g, 4))) : 0;
+    }
+    out->packed_bytes_required = plan->packed_required;
+    out->device_bytes = plan->device_bytes;
+    out->launches_per_execute = 1;
+    return TC_OK;
+}
+
+extern "C" int tc_plan_descriptors(const tc_plan_t *plan, int group, tc_descriptor_t *out, size_t cap, size_t *n_out)
+{
+    clear_error();
+    if (!plan || group < 0 || group > 1) return fail(TC_ERR_INVALID_ARG, "plan is required and group must be 0 or 1");
+    const Group &g = plan->group[group];
+    if (n_out) *n_out = g.descs.size();
+    if (!out) return TC_OK;
+    for (size_t i = 0; i < g.descs.size() && i < cap; i++) {
+        const Desc &d = g.descs[i];
+        tc_descriptor_t &o = out[i];
+        o.src_off = d.src_off; o.dst_off = d.dst_off; o.src_outer = d.src_outer; o.dst_outer = d.dst_outer;
+        o.src_s0 = d.src_s0; o.src_s1 = d.src_s1; o.dst_s0 = d.dst_s0; o.dst_s1 = d.dst_s1;
+        o.src_slot = d.src_slot; o.dst_slot = d.dst_slot - static_cast<uint32_t>(g.n_src);
+        o.src_slot_step = d.src_slot_step; o.dst_slot_step = d.dst_slot_step;
+        o.run_bytes = d.run; o.n0 = d.n0; o.rows = d.rows; o.n_outer = d.n_outer;
+    }
+    return TC_OK;
+}

@@ -1,0 +1,95 @@
+// Internal plan representation shared by the host-side plan builder and the kernels.
+// Nothing here is part of the public ABI (see include/tensorcast.h).
+#pragma once
+
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "tensorcast.h"
+
+namespace tc {
+
+// Exact unsigned division by a runtime constant for dividends below 2^31:
+//   n / d == (umulhi(n, mul) + n) >> shift
+struct FastDiv {
+    uint32_t mul, shift;
+};
+
+inline FastDiv make_fastdiv(uint32_t d)
+{
+    uint32_t s = 0;
+    while ((1ull << s) < d) s++;
+    uint64_t m = ((1ull << 32) * ((1ull << s) - d)) / d + 1;
+    return FastDiv{static_cast<uint32_t>(m), s};
+}
+
+inline uint32_t fastdiv_host(uint32_t n, FastDiv f)
+{
+    return static_cast<uint32_t>((((static_cast<uint64_t>(n) * f.mul) >> 32) + n) >> f.shift);
+}
+
+// One lowered copy descriptor as the kernels read it (128 bytes, 16-byte aligned).
+// A box of n_outer x rows runs of `run` contiguous bytes; row k of outer index o starts at
+//   table[src_slot + o*src_slot_step] + src_off + o*src_outer + (k / n0)*src_s1 + (k % n0)*src_s0
+// and likewise for dst (dst_slot already includes the offset of the dst table inside the
+// combined pointer table).  The builder guarantees that the row offsets of one descriptor,
+// (k / n0)*s1 + (k % n0)*s0 + run, stay below 2^31 on both sides, so the kernels decode rows in
+// 32-bit arithmetic.  Tiles: outer index o, row range [p*rows_per_tile, ...).
+struct alignas(16) Desc {
+    int64_t src_off, dst_off, src_outer, dst_outer;
+    uint32_t src_s0, src_s1, dst_s0, dst_s1;
+    uint16_t src_slot, dst_slot, src_slot_step, dst_slot_step;
+    FastDiv div_run;  // byte index inside a tile -> row
+    uint32_t run, n0, rows, n_outer;
+    uint32_t rows_per_tile, tiles_per_outer, tile0, log2_align;
+    FastDiv div_n0, div_tpo;
+    uint32_t pad[4];
+};
+static_assert(sizeof(Desc) == 128, "Desc must stay 128 bytes");
+
+struct Group {
+    std::vector<Desc> descs;
+    std::vector<uint32_t> tile_desc;  // tile -> descriptor, only for non-uniform groups
+    uint32_t tiles_per_desc = 0;      // > 0: every descriptor owns exactly this many tile ids
+    FastDiv div_tpd{0, 0};
+    uint64_t n_tiles = 0;
+    int64_t payload = 0;
+    uint32_t log2_align = 4;
+    size_t n_src = 0, n_dst = 0;      // table lengths the execute call must be given
+    bool single_run_tiles = true;     // every tile is one contiguous run
+    int resident_ctas[3] = {0, 0, 0}; // CTAs one SM holds, per executor build
+    // device copies (null for host-only plans and empty groups)
+    Desc *d_descs = nullptr;
+    uint32_t *d_tile_desc = nullptr;
+};
+
+}  // namespace tc
+
+struct tc_plan {
+    int32_t kind = 0;
+    uint32_t flags = 0;
+    uint64_t trace_id = 0;
+    int64_t deadline_ns = 0;
+    tc_tuning_t tuning{};
+    int device = -1;
+    int sm_count = 0;
+    int64_t packed_required = 0;
+    int64_t device_bytes = 0;
+    tc::Group group[2];
+};
+
+namespace tc {
+
+// plan_build.cpp: validate `spec` and lower it into plan->group[*] (host vectors only).
+int build_plan(const tc_plan_spec_t *spec, tc_plan *plan);
+
+// error reporting shared by both translation units
+int fail(int status, const char *fmt, ...);
+void clear_error();
+int64_t now_ns();
+
+constexpr uint32_t kDefaultTileBytes = 32768;
+constexpr uint32_t kMaxTileBytes = 1u << 20;
+
+}  // namespace tc

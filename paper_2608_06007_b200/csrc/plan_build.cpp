@@ -1,0 +1,609 @@
+// Host-side plan builder: validates a tc_plan_spec_t and lowers it to copy descriptors and
+// tiles.  Pure host code (no CUDA call), so it can be exercised on a machine without a GPU.
+//
+// Lowering model.  Every operation of the library (publish, hydrate, migrate, tensor_dict,
+// view, transform_into; Table 2 of the paper) is a set of strided boxes of bytes.  A box is
+// given as a contiguous run plus a list of (extent, src stride, dst stride) dimensions; it is
+// normalised (unit dims dropped, contiguous dims folded into the run, adjacent dims merged,
+// over-long runs cut into tile-sized rows) and emitted as one or more Desc records with at
+// most two strided dimensions, which is what the kernels decode.
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <ctime>
+#include <numeric>
+
+#include "plan.h"
+
+namespace tc {
+
+// ------------------------------------------------------------------------------ errors
+static thread_local std::string g_error;
+
+int fail(int status, const char *fmt, ...)
+{
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_error = buf;
+    return status;
+}
+
+void clear_error() { g_error.clear(); }
+
+int64_t now_ns()
+{
+    timespec ts;
+    clock_gettime(CLOCK_MONOTONIC, &ts);
+    return static_cast<int64_t>(ts.tv_sec) * 1000000000ll + ts.tv_nsec;
+}
+
+const char *last_error() { return g_error.c_str(); }
+
+// ------------------------------------------------------------------------------ boxes
+struct Dim {
+    int64_t ext, s, d;  // extent, source byte stride, destination byte stride
+};
+
+struct Box {
+    int64_t run;              // contiguous bytes of the innermost run
+    std::vector<Dim> dims;    // any order
+    int64_t src_off, dst_off;
+    uint32_t src_slot, dst_slot;
+    // the table-stepping outer dimension (KV planes); n_outer == 1 when unused
+    uint32_t n_outer = 1, src_slot_step = 0, dst_slot_step = 0;
+    int64_t src_outer = 0, dst_outer = 0;
+};
+
+static uint32_t ctz_cap(int64_t v, uint32_t cap = 4)
+{
+    if (v == 0) return cap;
+    uint64_t u = static_cast<uint64_t>(v < 0 ? -v : v);
+    uint32_t n = 0;
+    while (n < cap && !(u & 1)) { u >>= 1; n++; }
+    return n;
+}
+
+static void emit_desc(Group &g, const Box &b, int64_t run, const Dim *inner, const Dim *outer,
+                      int64_t src_off, int64_t dst_off, uint32_t tile_bytes)
+{
+    Desc d{};
+    d.src_off = src_off;
+    d.dst_off = dst_off;
+    d.src_outer = b.src_outer;
+    d.dst_outer = b.dst_outer;
+    d.n0 = inner ? static_cast<uint32_t>(inner->ext) : 1;
+    d.src_s0 = inner ? static_cast<uint32_t>(inner->s) : 0;
+    d.dst_s0 = inner ? static_cast<uint32_t>(inner->d) : 0;
+    uint32_t n1 = outer ? static_cast<uint32_t>(outer->ext) : 1;
+    d.src_s1 = outer ? static_cast<uint32_t>(outer->s) : 0;
+    d.dst_s1 = outer ? static_cast<uint32_t>(outer->d) : 0;
+    d.rows = d.n0 * n1;
+    d.src_slot = static_cast<uint16_t>(b.src_slot);
+    d.dst_slot = static_cast<uint16_t>(b.dst_slot);
+    d.src_slot_step = static_cast<uint16_t>(b.src_slot_step);
+    d.dst_slot_step = static_cast<uint16_t>(b.dst_slot_step);
+    d.run = static_cast<uint32_t>(run);
+    d.n_outer = b.n_outer;
+    d.rows_per_tile = std::max<uint32_t>(1, tile_bytes / d.run);
+    d.rows_per_tile = std::min(d.rows_per_tile, d.rows);
+    d.tiles_per_outer = (d.rows + d.rows_per_tile - 1) / d.rows_per_tile;
+    d.div_run = make_fastdiv(d.run);
+    d.div_n0 = make_fastdiv(d.n0);
+    d.div_tpo = make_fastdiv(d.tiles_per_outer);
+    uint32_t a = std::min({ctz_cap(run), ctz_cap(src_off), ctz_cap(dst_off)});
+    if (d.n0 > 1) a = std::min({a, ctz_cap(d.src_s0), ctz_cap(d.dst_s0)});
+    if (n1 > 1) a = std::min({a, ctz_cap(d.src_s1), ctz_cap(d.dst_s1)});
+    if (d.n_outer > 1) a = std::min({a, ctz_cap(d.src_outer), ctz_cap(d.dst_outer)});
+    d.log2_align = a;
+    g.log2_align = std::min(g.log2_align, a);
+    if (d.rows_per_tile > 1) g.single_run_tiles = false;
+    g.payload += static_cast<int64_t>(d.run) * d.rows * d.n_outer;
+    g.descs.push_back(d);
+}
+
+// Normalise a box and append its descriptors to the group.
+static void lower_box(Group &g, Box b, uint32_t tile_bytes)
+{
+    if (b.run <= 0 || b.n_outer == 0) return;
+    for (const Dim &d : b.dims)
+        if (d.ext <= 0) return;  // empty box
+    // 1. drop unit dims
+    b.dims.erase(std::remove_if(b.dims.begin(), b.dims.end(), [](const Dim &d) { return d.ext == 1; }),
+                 b.dims.end());
+    // 2. fold dims that continue the run on both sides into the run
+    for (bool again = true; again;) {
+        again = false;
+        for (size_t i = 0; i < b.dims.size(); i++)
+            if (b.dims[i].s == b.run && b.dims[i].d == b.run) {
+                b.run *= b.dims[i].ext;
+                b.dims.erase(b.dims.begin() + i);
+                again = true;
+                break;
+            }
+    }
+    // 3. merge pairs of dims that are one dimension in disguise on both sides
+    for (bool again = true; again;) {
+        again = false;
+        for (size_t i = 0; i < b.dims.size() && !again; i++)
+            for (size_t j = 0; j < b.dims.size() && !again; j++)
+                if (i != j && b.dims[j].s == b.dims[i].s * b.dims[i].ext &&
+                    b.dims[j].d == b.dims[i].d * b.dims[i].ext) {
+                    b.dims[i].ext *= b.dims[j].ext;
+                    b.dims.erase(b.dims.begin() + j);
+                    again = true;
+                }
+    }
+    // 4. a run longer than a tile becomes rows of tile_bytes plus a remainder box
+    if (b.run > static_cast<int64_t>(tile_bytes)) {
+        int64_t full = b.run / tile_bytes, rem = b.run % tile_bytes;
+        if (rem) {
+            Box tail = b;
+            tail.run = rem;
+            tail.src_off += full * tile_bytes;
+            tail.dst_off += full * tile_bytes;
+            lower_box(g, tail, tile_bytes);
+        }
+        b.run = tile_bytes;
+        b.dims.push_back(Dim{full, static_cast<int64_t>(tile_bytes), static_cast<int64_t>(tile_bytes)});
+        b.dims.erase(std::remove_if(b.dims.begin(), b.dims.end(), [](const Dim &d) { return d.ext == 1; }),
+                     b.dims.end());
+    }
+    // 5. innermost = smallest destination stride, so that a tile writes as densely as it can
+    std::sort(b.dims.begin(), b.dims.end(), [](const Dim &x, const Dim &y) {
+        return std::llabs(x.d) != std::llabs(y.d) ? std::llabs(x.d) < std::llabs(y.d) : std::llabs(x.s) < std::llabs(y.s);
+    });
+    // 6. one descriptor addresses its rows with 32-bit offsets: cut every dimension so that
+    //    its own span stays below 2^30 bytes (and its extent below 2^20 rows)
+    for (size_t i = 0; i < b.dims.size(); i++) {
+        const int64_t stride = std::max<int64_t>(std::max(b.dims[i].s, b.dims[i].d), 1);
+        const int64_t cap = std::max<int64_t>(1, std::min<int64_t>(1 << 20, ((1ll << 30) - b.run) / stride));
+        if (b.dims[i].ext <= cap || cap <= 1) continue;
+        // ext = q*cap + r: the r-tail becomes its own box, q*cap becomes two dims (cap, q)
+        const int64_t q = b.dims[i].ext / cap, r = b.dims[i].ext % cap;
+        if (r) {
+            Box tail = b;
+            tail.dims[i].ext = r;
+            tail.src_off += q * cap * b.dims[i].s;
+            tail.dst_off += q * cap * b.dims[i].d;
+            lower_box(g, tail, tile_bytes);
+        }
+        Dim hi{q, b.dims[i].s * cap, b.dims[i].d * cap};
+        b.dims[i].ext = cap;
+        b.dims.push_back(hi);  // strides of 2^30 or more: always unrolled on the host below
+    }
+    // 7. at most two strided dims per descriptor, each of span < 2^30; the rest is unrolled here
+    auto span = [](const Dim &d) { return (d.ext - 1) * std::max(d.s, d.d); };
+    const int64_t span_cap = (1ll << 30) - b.run;
+    std::stable_partition(b.dims.begin(), b.dims.end(), [&](const Dim &d) { return span(d) < span_cap && d.ext <= (1 << 20); });
+    size_t keep = 0;
+    while (keep < 2 && keep < b.dims.size() && span(b.dims[keep]) < span_cap && b.dims[keep].ext <= (1 << 20)) keep++;
+    if (keep == 2 && b.dims[0].ext * b.dims[1].ext >= (1ll << 31)) keep = 1;
+    std::vector<int64_t> idx(b.dims.size(), 0);
+    for (;;) {
+        int64_t so = b.src_off, dof = b.dst_off;
+        for (size_t i = keep; i < b.dims.size(); i++) {
+            so += idx[i] * b.dims[i].s;
+            dof += idx[i] * b.dims[i].d;
+        }
+        emit_desc(g, b, b.run, keep >= 1 ? &b.dims[0] : nullptr, keep >= 2 ? &b.dims[1] : nullptr, so, dof,
+                  tile_bytes);
+        size_t i = keep;
+        for (; i < b.dims.size(); i++) {
+            if (++idx[i] < b.dims[i].ext) break;
+            idx[i] = 0;
+        }
+        if (i >= b.dims.size()) break;
+    }
+}
+
+// Assign tile ids.  A group whose descriptors all own (nearly) the same number of tiles is
+// "uniform": tile -> descriptor is a division and short descriptors simply own a few empty
+// tile ids.  Otherwise an explicit tile -> descriptor array is built.
+static int finish_group(Group &g)
+{
+    if (g.descs.empty()) return TC_OK;
+    uint64_t total = 0, max_t = 0;
+    for (const Desc &d : g.descs) {
+        uint64_t t = static_cast<uint64_t>(d.n_outer) * d.tiles_per_outer;
+        total += t;
+        max_t = std::max(max_t, t);
+    }
+    uint64_t padded = max_t * g.descs.size();
+    bool same_shape = true;
+    for (const Desc &d : g.descs)
+        if (d.n_outer != g.descs[0].n_outer) same_shape = false;
+    if (same_shape && padded < (1ull << 31) && total * 10 >= padded * 8) {
+        // uniform: every descriptor is given max tiles_per_outer; extra parts are empty
+        uint32_t tpo = static_cast<uint32_t>(max_t / g.descs[0].n_outer);
+        for (size_t i = 0; i < g.descs.size(); i++) {
+            Desc &d = g.descs[i];
+            d.tiles_per_outer = tpo;
+            d.div_tpo = make_fastdiv(tpo);
+            d.tile0 = static_cast<uint32_t>(i * max_t);
+        }
+        g.tiles_per_desc = static_cast<uint32_t>(max_t);
+        g.div_tpd = make_fastdiv(g.tiles_per_desc);
+        g.n_tiles = padded;
+        return TC_OK;
+    }
+    if (total >= (1ull << 31)) return fail(TC_ERR_INVALID_ARG, "plan has %llu tiles (limit 2^31)", (unsigned long long)total);
+    g.tile_desc.resize(total);
+    uint64_t t0 = 0;
+    for (size_t i = 0; i < g.descs.size(); i++) {
+        Desc &d = g.descs[i];
+        uint64_t t = static_cast<uint64_t>(d.n_outer) * d.tiles_per_outer;
+        d.tile0 = static_cast<uint32_t>(t0);
+        std::fill(g.tile_desc.begin() + t0, g.tile_desc.begin() + t0 + t, static_cast<uint32_t>(i));
+        t0 += t;
+    }
+    g.tiles_per_desc = 0;
+    g.n_tiles = total;
+    return TC_OK;
+}
+
+// ------------------------------------------------------------------------------ KV
+struct PoolView {
+    const tc_kv_pool_t *p;
+    int64_t chunk;         // B*H*D*E
+    int64_t block_stride;  // resolved
+    int64_t plane_stride;  // 0 when the pool has L*2 slots
+    uint32_t slot_step;    // 1 when the pool has L*2 slots
+    int64_t slot_need;     // minimum extent of a slot
+};
+
+static int check_pool(const tc_kv_spec_t &kv, const tc_kv_pool_t &p, const char *name, PoolView *out)
+{
+    const int64_t planes = kv.L * 2, chunk = kv.B * kv.H * kv.D * kv.E;
+    if (p.layout != TC_NHD && p.layout != TC_HND) return fail(TC_ERR_INVALID_ARG, "%s.layout %d is not a tc_layout", name, p.layout);
+    if (p.num_blocks < 0) return fail(TC_ERR_SHAPE, "%s.num_blocks %lld < 0", name, (long long)p.num_blocks);
+    if (p.n_slots != 1 && p.n_slots != planes)
+        return fail(TC_ERR_INVALID_ARG, "%s.n_slots %lld must be 1 or L*2 = %lld", name, (long long)p.n_slots, (long long)planes);
+    int64_t bs = p.block_stride ? p.block_stride : chunk;
+    if (bs < chunk) return fail(TC_ERR_OVERLAP, "%s.block_stride %lld < block bytes %lld: blocks overlap", name, (long long)bs, (long long)chunk);
+    out->p = &p;
+    out->chunk = chunk;
+    out->block_stride = bs;
+    const int64_t nb = std::max<int64_t>(p.num_blocks, 1);
+    if (p.n_slots == 1) {
+        int64_t ps = p.plane_stride;
+        // plane-major (each plane holds all its blocks) or page-first (each block holds all planes)
+        bool plane_major = ps >= (nb - 1) * bs + chunk;
+        bool page_first = ps >= chunk && bs >= (planes - 1) * ps + chunk;
+        if (planes > 1 && !plane_major && !page_first)
+            return fail(TC_ERR_OVERLAP, "%s: plane_stride %lld and block_stride %lld make planes overlap", name, (long long)ps, (long long)bs);
+        out->plane_stride = planes > 1 ? ps : 0;
+        out->slot_step = 0;
+        out->slot_need = (planes - 1) * out->plane_stride + (nb - 1) * bs + chunk;
+    } else {
+        out->plane_stride = 0;
+        out->slot_step = 1;
+        out->slot_need = (nb - 1) * bs + chunk;
+    }
+    if (p.slot_bytes && p.slot_bytes < out->slot_need && p.num_blocks > 0)
+        return fail(TC_ERR_BOUNDS, "%s.slot_bytes %lld < %lld needed for %lld blocks", name, (long long)p.slot_bytes, (long long)out->slot_need, (long long)p.num_blocks);
+    return TC_OK;
+}
+
+static int check_group(const tc_kv_spec_t &kv, const tc_kv_group_t &g, const char *name, bool need_src,
+                       const tc_kv_pool_t *src_pool, bool need_dst, const tc_kv_pool_t *dst_pool)
+{
+    if (g.R < 0) return fail(TC_ERR_SHAPE, "%s.R %lld < 0", name, (long long)g.R);
+    if (g.R == 0) return TC_OK;
+    if (!g.T || !g.bt_off) return fail(TC_ERR_INVALID_ARG, "%s: T and bt_off are required when R > 0", name);
+    if (g.bt_off[0] != 0) return fail(TC_ERR_INVALID_ARG, "%s.bt_off[0] must be 0", name);
+    for (int64_t r = 0; r < g.R; r++) {
+        if (g.T[r] < 0) return fail(TC_ERR_SHAPE, "%s.T[%lld] = %lld < 0", name, (long long)r, (long long)g.T[r]);
+        int64_t n = (g.T[r] + kv.B - 1) / kv.B;
+        if (g.bt_off[r + 1] - g.bt_off[r] != n)
+            return fail(TC_ERR_INVALID_ARG, "%s: request %lld has %lld tokens = %lld blocks but its table holds %lld", name,
+                        (long long)r, (long long)g.T[r], (long long)n, (long long)(g.bt_off[r + 1] - g.bt_off[r]));
+    }
+    const int64_t nblk = g.bt_off[g.R];
+    if (nblk > 0 && need_src && !g.bt_src) return fail(TC_ERR_INVALID_ARG, "%s.bt_src is required", name);
+    if (nblk > 0 && need_dst && !g.bt_dst) return fail(TC_ERR_INVALID_ARG, "%s.bt_dst is required", name);
+    if (need_src)
+        for (int64_t j = 0; j < nblk; j++)
+            if (g.bt_src[j] < 0 || g.bt_src[j] >= src_pool->num_blocks)
+                return fail(TC_ERR_BOUNDS, "%s.bt_src[%lld] = %d outside [0, %lld)", name, (long long)j, g.bt_src[j], (long long)src_pool->num_blocks);
+    if (need_dst) {
+        std::vector<uint8_t> seen(static_cast<size_t>(dst_pool->num_blocks), 0);
+        for (int64_t j = 0; j < nblk; j++) {
+            int32_t b = g.bt_dst[j];
+            if (b < 0 || b >= dst_pool->num_blocks)
+                return fail(TC_ERR_BOUNDS, "%s.bt_dst[%lld] = %d outside [0, %lld)", name, (long long)j, b, (long long)dst_pool->num_blocks);
+            if (seen[b]) return fail(TC_ERR_OVERLAP, "%s.bt_dst names block %d twice: its bytes would be written twice", name, b);
+            seen[b] = 1;
+        }
+    }
+    return TC_OK;
+}
+
+// strides of (slot n, head h) rows of D*E bytes inside one block / one packed request plane
+static void pool_strides(const tc_kv_spec_t &kv, int32_t layout, int64_t *sn, int64_t *sh)
+{
+    const int64_t row = kv.D * kv.E;
+    if (layout == TC_NHD) { *sn = kv.H * row; *sh = row; }
+    else                  { *sn = row;        *sh = kv.B * row; }
+}
+
+static void packed_strides(const tc_kv_spec_t &kv, int32_t layout, int64_t Tr, int64_t *sn, int64_t *sh)
+{
+    const int64_t row = kv.D * kv.E;
+    if (layout == TC_NHD) { *sn = kv.H * row; *sh = row; }
+    else                  { *sn = row;        *sh = Tr * row; }
+}
+
+// Lower one group.  src_pool / dst_pool null = that side is the packed buffer.
+static void lower_kv_group(Group &g, const tc_kv_spec_t &kv, const tc_kv_group_t &grp, const PoolView *src_pool,
+                           const PoolView *dst_pool, int32_t packed_layout, uint32_t tile_bytes)
+{
+    const int64_t row = kv.D * kv.E, planes = kv.L * 2;
+    int64_t off_r = 0;
+    g.descs.reserve(grp.R ? static_cast<size_t>(grp.bt_off[grp.R]) : 0);
+    for (int64_t r = 0; r < grp.R; r++) {
+        const int64_t Tr = grp.T[r];
+        const int64_t plane_bytes = Tr * kv.H * row;  // one (l,c) plane of this request, packed
+        for (int64_t j = 0; j * kv.B < Tr; j++) {
+            const int64_t nvalid = std::min(kv.B, Tr - j * kv.B);
+            const int64_t jj = grp.bt_off[r] + j;
+            Box b;
+            b.run = row;
+            b.n_outer = static_cast<uint32_t>(planes);
+            int64_t ssn, ssh, dsn, dsh;
+            if (src_pool) {
+                pool_strides(kv, src_pool->p->layout, &ssn, &ssh);
+                b.src_off = grp.bt_src[jj] * src_pool->block_stride;
+                b.src_outer = src_pool->plane_stride;
+                b.src_slot_step = src_pool->slot_step;
+            } else {
+                packed_strides(kv, packed_layout, Tr, &ssn, &ssh);
+                b.src_off = off_r + j * kv.B * ssn;
+                b.src_outer = plane_bytes;
+            }
+            if (dst_pool) {
+                pool_strides(kv, dst_pool->p->layout, &dsn, &dsh);
+                b.dst_off = grp.bt_dst[jj] * dst_pool->block_stride;
+                b.dst_outer = dst_pool->plane_stride;
+                b.dst_slot_step = dst_pool->slot_step;
+            } else {
+                packed_strides(kv, packed_layout, Tr, &dsn, &dsh);
+                b.dst_off = off_r + j * kv.B * dsn;
+                b.dst_outer = plane_bytes;
+            }
+            b.src_slot = 0;
+            b.dst_slot = 0;
+            b.dims = {Dim{kv.H, ssh, dsh}, Dim{nvalid, ssn, dsn}};
+            lower_box(g, b, tile_bytes);
+        }
+        off_r += planes * plane_bytes;
+    }
+}
+
+static int build_kv(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t tile_bytes)
+{
+    const tc_kv_spec_t &kv = spec->kv;
+    if (kv.L < 1 || kv.B < 1 || kv.H < 1 || kv.D < 1) return fail(TC_ERR_SHAPE, "L, B, H, D must be >= 1");
+    if (kv.E != 1 && kv.E != 2 && kv.E != 4 && kv.E != 8) return fail(TC_ERR_SHAPE, "E = %lld must be 1, 2, 4 or 8", (long long)kv.E);
+    if (kv.L * 2 > TC_MAX_TABLE_SLOTS / 2) return fail(TC_ERR_INVALID_ARG, "L*2 = %lld exceeds the table limit", (long long)(kv.L * 2));
+    const int kind = spec->kind;
+    const bool src_is_pool = kind != TC_KV_UNPACK, dst_is_pool = kind != TC_KV_PACK;
+    PoolView sp{}, dp{};
+    int rc;
+    if (src_is_pool && (rc = check_pool(kv, kv.src_pool, "src_pool", &sp))) return rc;
+    if (dst_is_pool && (rc = check_pool(kv, kv.dst_pool, "dst_pool", &dp))) return rc;
+    if ((rc = check_group(kv, kv.group, "group", src_is_pool, &kv.src_pool, dst_is_pool, &kv.dst_pool))) return rc;
+    if (kind == TC_KV_PACK || kind == TC_KV_UNPACK) {
+        if (kv.packed_layout != TC_NHD && kv.packed_layout != TC_HND)
+            return fail(TC_ERR_INVALID_ARG, "packed_layout %d is not a tc_layout", kv.packed_layout);
+        int64_t need = 0;
+        for (int64_t r = 0; r < kv.group.R; r++) need += kv.L * 2 * kv.group.T[r] * kv.H * kv.D * kv.E;
+        plan->packed_required = need;
+        if (kv.packed_bytes && kv.packed_bytes < need)
+            return fail(TC_ERR_BOUNDS, "packed_bytes %lld < %lld required", (long long)kv.packed_bytes, (long long)need);
+    }
+    Group &g0 = plan->group[0], &g1 = plan->group[1];
+    if (kind == TC_KV_PACK) {
+        lower_kv_group(g0, kv, kv.group, &sp, nullptr, kv.packed_layout, tile_bytes);
+        g0.n_src = kv.src_pool.n_slots;
+        g0.n_dst = 1;
+    } else if (kind == TC_KV_UNPACK) {
+        lower_kv_group(g1, kv, kv.group, nullptr, &dp, kv.packed_layout, tile_bytes);
+        g1.n_src = 1;
+        g1.n_dst = kv.dst_pool.n_slots;
+    } else if (kind == TC_KV_MIGRATE) {
+        lower_kv_group(g0, kv, kv.group, &sp, &dp, 0, tile_bytes);
+        g0.n_src = kv.src_pool.n_slots;
+        g0.n_dst = kv.dst_pool.n_slots;
+    } else {  // MIXED: offload src_pool -> dst_pool, reload dst_pool -> src_pool
+        if ((rc = check_group(kv, kv.reload, "reload", true, &kv.dst_pool, true, &kv.src_pool))) return rc;
+        const int64_t n_off = kv.group.R ? kv.group.bt_off[kv.group.R] : 0;
+        const int64_t n_rel = kv.reload.R ? kv.reload.bt_off[kv.reload.R] : 0;
+        // the two groups may run concurrently: neither may write what the other reads or writes
+        std::vector<uint8_t> host_used(static_cast<size_t>(kv.dst_pool.num_blocks), 0), dev_used(static_cast<size_t>(kv.src_pool.num_blocks), 0);
+        for (int64_t j = 0; j < n_off; j++) { host_used[kv.group.bt_dst[j]] = 1; dev_used[kv.group.bt_src[j]] = 1; }
+        for (int64_t j = 0; j < n_rel; j++) {
+            if (host_used[kv.reload.bt_src[j]])
+                return fail(TC_ERR_OVERLAP, "block %d of dst_pool is written by the offload group and read by the reload group", kv.reload.bt_src[j]);
+            if (dev_used[kv.reload.bt_dst[j]])
+                return fail(TC_ERR_OVERLAP, "block %d of src_pool is read by the offload group and written by the reload group", kv.reload.bt_dst[j]);
+        }
+        lower_kv_group(g0, kv, kv.group, &sp, &dp, 0, tile_bytes);
+        lower_kv_group(g1, kv, kv.reload, &dp, &sp, 0, tile_bytes);
+        g0.n_src = kv.src_pool.n_slots;
+        g0.n_dst = kv.dst_pool.n_slots;
+        g1.n_src = kv.dst_pool.n_slots;
+        g1.n_dst = kv.src_pool.n_slots;
+    }
+    return TC_OK;
+}
+
+// ------------------------------------------------------------------------------ weights
+struct Span {
+    int64_t lo, hi;
+    int64_t tensor;
+};
+
+static int build_weights(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t tile_bytes)
+{
+    const tc_weights_spec_t &w = spec->weights;
+    if (w.n_tensors < 0) return fail(TC_ERR_SHAPE, "n_tensors %lld < 0", (long long)w.n_tensors);
+    if (w.n_tensors > 0 && !w.index) return fail(TC_ERR_INVALID_ARG, "index is required");
+    if (w.world < 1 || w.rank < 0 || w.rank >= w.world)
+        return fail(TC_ERR_INVALID_ARG, "rank %d / world %d is not a valid tensor-parallel position", w.rank, w.world);
+    const int64_t n_dst = w.n_dst ? w.n_dst : w.n_tensors;
+    if (n_dst + 1 > TC_MAX_TABLE_SLOTS) return fail(TC_ERR_INVALID_ARG, "%lld destination slots exceed the table limit %d", (long long)n_dst, TC_MAX_TABLE_SLOTS - 1);
+    Group &g = plan->group[0];
+    g.n_src = 1;
+    g.n_dst = static_cast<size_t>(n_dst);
+    std::vector<std::vector<Span>> spans(static_cast<size_t>(n_dst));
+    std::vector<Box> boxes;
+    boxes.reserve(static_cast<size_t>(w.n_tensors));
+    for (int64_t i = 0; i < w.n_tensors; i++) {
+        const tc_index_entry_t &t = w.index[i];
+        if (t.ndim < 1 || t.ndim > 4) return fail(TC_ERR_SHAPE, "tensor %lld: ndim %u outside 1..4", (long long)i, t.ndim);
+        if (t.elem_bytes != 1 && t.elem_bytes != 2 && t.elem_bytes != 4 && t.elem_bytes != 8)
+            return fail(TC_ERR_SHAPE, "tensor %lld: elem_bytes %u", (long long)i, t.elem_bytes);
+        int64_t shp[4] = {1, 1, 1, 1}, count = 1;
+        for (uint32_t m = 0; m < 4; m++) {
+            if (m < t.ndim) shp[m] = static_cast<int64_t>(t.shape[m]);
+            else if (t.shape[m] > 1) return fail(TC_ERR_SHAPE, "tensor %lld: shape[%u] = %llu beyond ndim", (long long)i, m, (unsigned long long)t.shape[m]);
+            if (shp[m] < 0 || (shp[m] && count > (1ll << 62) / std::max<int64_t>(shp[m], 1)))
+                return fail(TC_ERR_SHAPE, "tensor %lld: extent overflow", (long long)i);
+            count *= shp[m];
+        }
+        if (static_cast<int64_t>(t.nbytes) != count * t.elem_bytes)
+            return fail(TC_ERR_SHAPE, "tensor %lld: nbytes %llu != elem_bytes * prod(shape) = %lld", (long long)i, (unsigned long long)t.nbytes, (long long)(count * t.elem_bytes));
+        if (static_cast<int64_t>(t.byte_off) < 0 || static_cast<int64_t>(t.byte_off + t.nbytes) > w.blob_bytes)
+            return fail(TC_ERR_BOUNDS, "tensor %lld: bytes [%llu, %llu) lie outside the blob of %lld", (long long)i, (unsigned long long)t.byte_off, (unsigned long long)(t.byte_off + t.nbytes), (long long)w.blob_bytes);
+        tc_weight_rule_t rule{};
+        rule.split_dim = -1;
+        rule.dst_slot = -1;
+        if (w.rules) rule = w.rules[i];
+        int64_t ext[4] = {shp[0], shp[1], shp[2], shp[3]}, shift = 0;
+        int64_t sstr[4];
+        sstr[3] = t.elem_bytes;
+        for (int m = 2; m >= 0; m--) sstr[m] = sstr[m + 1] * shp[m + 1];
+        if (rule.split_dim >= 0) {
+            if (rule.split_dim >= static_cast<int32_t>(t.ndim)) return fail(TC_ERR_SHAPE, "tensor %lld: split_dim %d >= ndim %u", (long long)i, rule.split_dim, t.ndim);
+            if (shp[rule.split_dim] % w.world) return fail(TC_ERR_SHAPE, "tensor %lld: dim %d of extent %lld is not divisible by world %d", (long long)i, rule.split_dim, (long long)shp[rule.split_dim], w.world);
+            ext[rule.split_dim] = shp[rule.split_dim] / w.world;
+            shift = w.rank * ext[rule.split_dim] * sstr[rule.split_dim];
+        } else if (rule.split_dim != -1) {
+            return fail(TC_ERR_INVALID_ARG, "tensor %lld: split_dim %d", (long long)i, rule.split_dim);
+        }
+        int64_t dstr[4];
+        bool tight = !(rule.dst_stride[0] | rule.dst_stride[1] | rule.dst_stride[2] | rule.dst_stride[3]);
+        if (tight) {
+            dstr[3] = t.elem_bytes;
+            for (int m = 2; m >= 0; m--) dstr[m] = dstr[m + 1] * ext[m + 1];
+        } else {
+            for (int m = 0; m < 4; m++) {
+                dstr[m] = rule.dst_stride[m];
+                if (ext[m] > 1 && dstr[m] <= 0) return fail(TC_ERR_INVALID_ARG, "tensor %lld: dst_stride[%d] = %lld must be positive", (long long)i, m, (long long)dstr[m]);
+            }
+        }
+        const int64_t slot = rule.dst_slot < 0 ? i : rule.dst_slot;
+        if (slot >= n_dst) return fail(TC_ERR_INVALID_ARG, "tensor %lld: dst_slot %lld >= n_dst %lld", (long long)i, (long long)slot, (long long)n_dst);
+        if (rule.dst_off < 0) return fail(TC_ERR_BOUNDS, "tensor %lld: dst_off %lld < 0", (long long)i, (long long)rule.dst_off);
+        int64_t n_el = ext[0] * ext[1] * ext[2] * ext[3];
+        if (n_el == 0) continue;
+        int64_t hi = rule.dst_off + t.elem_bytes;
+        for (int m = 0; m < 4; m++) hi += (ext[m] - 1) * dstr[m];
+        const int64_t slot_extent = w.dst_bytes ? w.dst_bytes[slot] : (tight && rule.dst_off == 0 ? n_el * t.elem_bytes : -1);
+        if (slot_extent < 0) return fail(TC_ERR_INVALID_ARG, "tensor %lld: dst_bytes is required when a rule sets dst_off or dst_stride", (long long)i);
+        if (hi > slot_extent) return fail(TC_ERR_BOUNDS, "tensor %lld: writes up to byte %lld of a %lld-byte destination", (long long)i, (long long)hi, (long long)slot_extent);
+        spans[static_cast<size_t>(slot)].push_back(Span{rule.dst_off, hi, i});
+        Box b;
+        b.run = t.elem_bytes;
+        b.src_off = static_cast<int64_t>(t.byte_off) + shift;
+        b.dst_off = rule.dst_off;
+        b.src_slot = 0;
+        b.dst_slot = static_cast<uint32_t>(slot);
+        for (int m = 3; m >= 0; m--) b.dims.push_back(Dim{ext[m], sstr[m], dstr[m]});
+        boxes.push_back(std::move(b));
+    }
+    // exactly-once writes: bounding spans of one slot may not intersect.  (Interleaved strided
+    // destinations whose bounding spans intersect are checked row by row below.)
+    for (size_t s = 0; s < spans.size(); s++) {
+        auto &v = spans[s];
+        std::sort(v.begin(), v.end(), [](const Span &a, const Span &b) { return a.lo < b.lo; });
+        bool clash = false;
+        for (size_t k = 1; k < v.size(); k++)
+            if (v[k].lo < v[k - 1].hi) clash = true;
+        if (!clash) continue;
+        // exact check over the rows of every box that targets this slot
+        Group tmp;
+        for (const Box &b : boxes)
+            if (b.dst_slot == s) lower_box(tmp, b, kMaxTileBytes);
+        std::vector<std::pair<int64_t, int64_t>> rows;
+        uint64_t total_rows = 0;
+        for (const Desc &d : tmp.descs) total_rows += d.rows;
+        if (total_rows > (64ull << 20)) return fail(TC_ERR_OVERLAP, "destination slot %zu: overlapping windows too fine to verify", s);
+        rows.reserve(total_rows);
+        for (const Desc &d : tmp.descs)
+            for (uint32_t k = 0; k < d.rows; k++) {
+                int64_t a = d.dst_off + static_cast<int64_t>(k / d.n0) * d.dst_s1 + static_cast<int64_t>(k % d.n0) * d.dst_s0;
+                rows.emplace_back(a, a + d.run);
+            }
+        std::sort(rows.begin(), rows.end());
+        for (size_t k = 1; k < rows.size(); k++)
+            if (rows[k].first < rows[k - 1].second)
+                return fail(TC_ERR_OVERLAP, "destination slot %zu: byte %lld would be written twice", s, (long long)rows[k].first);
+    }
+    for (const Box &b : boxes) lower_box(g, b, tile_bytes);
+    return TC_OK;
+}
+
+// ------------------------------------------------------------------------------ entry
+int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
+{
+    uint32_t tile_bytes = spec->tuning.tile_bytes > 0 ? static_cast<uint32_t>(spec->tuning.tile_bytes) : kDefaultTileBytes;
+    if (tile_bytes < 512 || tile_bytes > kMaxTileBytes || (tile_bytes & (tile_bytes - 1)))
+        return fail(TC_ERR_INVALID_ARG, "tuning.tile_bytes %u must be a power of two in [512, %u]", tile_bytes, kMaxTileBytes);
+    int rc;
+    switch (spec->kind) {
+    case TC_KV_PACK:
+    case TC_KV_UNPACK:
+    case TC_KV_MIGRATE:
+    case TC_KV_MIXED:
+        rc = build_kv(spec, plan, tile_bytes);
+        break;
+    case TC_WEIGHTS:
+        rc = build_weights(spec, plan, tile_bytes);
+        break;
+    default:
+        return fail(TC_ERR_INVALID_ARG, "kind %d is not a tc_kind", spec->kind);
+    }
+    if (rc) return rc;
+    for (int k = 0; k < 2; k++) {
+        Group &g = plan->group[k];
+        // destination slots follow the source slots in the combined pointer table
+        for (Desc &d : g.descs) d.dst_slot = static_cast<uint16_t>(d.dst_slot + g.n_src);
+        if ((rc = finish_group(g))) return rc;
+    }
+    return TC_OK;
+}
+
+}  // namespace tc
+
+extern "C" const char *tc_last_error(void) { return tc::last_error(); }
+
+extern "C" const char *tc_strerror(int status)
+{
+    switch (status) {
+    case TC_OK: return "TC_OK";
+    case TC_ERR_INVALID_ARG: return "TC_ERR_INVALID_ARG";
+    case TC_ERR_SHAPE: return "TC_ERR_SHAPE";
+    case TC_ERR_BOUNDS: return "TC_ERR_BOUNDS";
+    case TC_ERR_OVERLAP: return "TC_ERR_OVERLAP";
+    case TC_ERR_KIND: return "TC_ERR_KIND";
+    case TC_ERR_OOM: return "TC_ERR_OOM";
+    case TC_ERR_CUDA: return "TC_ERR_CUDA";
+    case TC_ERR_DEADLINE: return "TC_ERR_DEADLINE";
+    default: return "TC_ERR_UNKNOWN";
+    }
+}

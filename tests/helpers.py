@@ -1,0 +1,49 @@
+"""Shared test helpers: a numpy interpreter of lowered descriptors (test-only: it lets the CPU
+suite check the plan builder against the oracle without a GPU) and small case builders."""
+import numpy as np
+
+import oracle
+import paper_2608_06007_b200 as tc
+import workloads as wl
+
+
+def run_descriptors(descs, src_tables, dst_tables, dst_counts=None):
+    """Execute tc_descriptor_t records on flat uint8 numpy buffers, byte-run by byte-run."""
+    for d in descs:
+        for o in range(d.n_outer):
+            s = src_tables[d.src_slot + o * d.src_slot_step]
+            t = dst_tables[d.dst_slot + o * d.dst_slot_step]
+            for k in range(d.rows):
+                i1, i0 = divmod(k, d.n0)
+                a = d.src_off + o * d.src_outer + i1 * d.src_s1 + i0 * d.src_s0
+                b = d.dst_off + o * d.dst_outer + i1 * d.dst_s1 + i0 * d.dst_s0
+                t[b:b + d.run_bytes] = s[a:a + d.run_bytes]
+                if dst_counts is not None:
+                    dst_counts[d.dst_slot + o * d.dst_slot_step][b:b + d.run_bytes] += 1
+
+
+def planes_of(pool, n_planes):
+    per = pool.size // n_planes
+    return [pool[i * per:(i + 1) * per] for i in range(n_planes)]
+
+
+def kv_case(rng, L=2, NB=12, B=4, H=3, D=8, E=2, T=(8, 4, 12), pad_blocks=0):
+    shape = (L, B, H, D, E)
+    chunk = B * H * D * E
+    stride = chunk + pad_blocks
+    pool = rng.integers(0, 256, L * 2 * NB * stride, dtype=np.uint8)
+    T = np.array(T, dtype=np.int64)
+    off = np.concatenate([[0], np.cumsum((T + B - 1) // B)]).astype(np.int64)
+    bt = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    return shape, NB, stride, pool, T, off, bt
+
+
+def small_checkpoint(**kw):
+    return wl.llama_checkpoint(hidden=64, layers=2, q_heads=8, kv_heads=4, head_dim=8, mlp=96,
+                               vocab=160, **kw)
+
+
+def ck_spec(ck, **kw):
+    nbytes = [ck.nbytes(i) for i in range(ck.N)]
+    kw.setdefault("blob_bytes", ck.nbytes_total)
+    return tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, **kw)

@@ -1,0 +1,280 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, byte for byte.
+Everything is copy and indexing, so the bar is exact equality of whole buffers (including
+sentinel-filled destinations and red zones around them)."""
+import itertools
+import time
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2608_06007_b200 as tc
+import workloads as wl
+from helpers import ck_spec, kv_case, planes_of, small_checkpoint
+
+pytestmark = pytest.mark.gpu
+LAYOUTS = [tc.TC_NHD, tc.TC_HND]
+RED = 256  # red-zone bytes on both sides of every destination
+
+
+def dev(a: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(a).cuda()
+
+
+class Guarded:
+    """A device destination of n bytes with sentinel-filled red zones on both sides."""
+
+    def __init__(self, n, fill=0xA5, init=None, shift=0):
+        self.n, self.fill, self.shift = n, fill, shift
+        self.buf = torch.full((n + 2 * RED + shift,), 0x3C, dtype=torch.uint8, device="cuda")
+        self.view = self.buf[RED + shift:RED + shift + n]
+        if init is not None:
+            self.view.copy_(dev(init))
+        else:
+            self.view.fill_(fill)
+
+    def ptr(self, off=0):
+        return self.view.data_ptr() + off
+
+    def result(self):
+        torch.cuda.synchronize()
+        host = self.buf.cpu().numpy()
+        assert (host[:RED + self.shift] == 0x3C).all() and (host[RED + self.shift + self.n:] == 0x3C).all(), "red zone written"
+        return host[RED + self.shift:RED + self.shift + self.n]
+
+
+def pool_tables(g: Guarded, n_planes, slots):
+    per = g.n // n_planes
+    return [g.ptr(p * per) for p in range(n_planes)] if slots == "planes" else [g.ptr()]
+
+
+# --------------------------------------------------------------------------- config 1
+@pytest.mark.parametrize("packed_l", LAYOUTS)
+def test_config1_pack_then_unpack(packed_l):
+    shape, NB, src, dst = wl.config1()
+    s = shape.tuple
+    pool = np.zeros(2 * NB * shape.chunk_bytes, dtype=np.uint8)
+    wl.fill_np(pool, wl.SEED_BASE + 1)
+    planes = planes_of(pool, 2)
+    want = np.zeros(oracle.packed_nbytes(s, src.T), dtype=np.uint8)
+    oracle.kv_pack(s, oracle.NHD, shape.chunk_bytes, planes, src.T, src.bt_off, src.bt, packed_l, want)
+    d_pool = dev(pool)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=pool.size)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=pl, packed_layout=packed_l, T=src.T, bt_off=src.bt_off, bt_src=src.bt))
+    out = Guarded(want.size)
+    tc.tc_kv_pack(plan, [d_pool], [out.ptr()])
+    got = out.result()
+    assert got.size == 1400832 and np.array_equal(got, want)
+    # unpack into a fresh pool filled with the 0xA5A5 sentinel, through an independent table
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(s, oracle.NHD, shape.chunk_bytes, planes_of(want_pool, 2), dst.T, dst.bt_off, dst.bt, packed_l, want)
+    plan2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=pl, packed_layout=packed_l, T=dst.T, bt_off=dst.bt_off, bt_dst=dst.bt))
+    fresh = Guarded(pool.size)
+    tc.tc_kv_unpack(plan2, [out.ptr()], [fresh.ptr()])
+    assert np.array_equal(fresh.result(), want_pool)
+    # idempotent re-execution of both plans gives the same bytes
+    tc.tc_kv_pack(plan, [d_pool], [out.ptr()])
+    tc.tc_kv_unpack(plan2, [out.ptr()], [fresh.ptr()])
+    assert np.array_equal(out.result(), want) and np.array_equal(fresh.result(), want_pool)
+    assert plan.stats().launches_per_execute == 1
+
+
+# --------------------------------------------------------------------------- layouts, tails, tiles
+@pytest.mark.parametrize("pool_l,packed_l", list(itertools.product(LAYOUTS, LAYOUTS)))
+@pytest.mark.parametrize("slots", ["planes", "one"])
+@pytest.mark.parametrize("tile", [0, 2048])
+def test_pack_unpack_all_layouts(pool_l, packed_l, slots, tile):
+    rng = np.random.default_rng(21)
+    # 2 KiB token rows, blocks of 16: several tiles per block with tile=2048, ragged tails
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=3, NB=40, B=16, H=4, D=64, E=2, T=(37, 0, 100, 5, 16, 200), pad_blocks=0)
+    L = shape[0]
+    tune = dict(tile_bytes=tile) if tile else None
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, pool_l, stride, planes_of(pool, L * 2), T, off, bt, packed_l, want)
+    d_pool = Guarded(pool.size, init=pool)
+    if slots == "planes":
+        pl = tc.pool(pool_l, NB, L * 2, block_stride=stride, slot_bytes=pool.size // (L * 2))
+    else:
+        pl = tc.pool(pool_l, NB, 1, plane_stride=pool.size // (L * 2), block_stride=stride, slot_bytes=pool.size)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_src=bt, tuning=tune))
+    out = Guarded(want.size)
+    tc.tc_kv_pack(plan, pool_tables(d_pool, L * 2, slots), [out.ptr()])
+    assert np.array_equal(out.result(), want)
+    assert np.array_equal(d_pool.result(), pool)          # sources are never written
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, pool_l, stride, planes_of(want_pool, L * 2), T, off, bt2, packed_l, want)
+    plan2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_dst=bt2, tuning=tune))
+    fresh = Guarded(pool.size)
+    tc.tc_kv_unpack(plan2, [out.ptr()], pool_tables(fresh, L * 2, slots))
+    assert np.array_equal(fresh.result(), want_pool)
+
+
+@pytest.mark.parametrize("E,D,shift", [(1, 7, 0), (2, 5, 0), (4, 3, 0), (8, 3, 0), (2, 64, 2), (2, 64, 4), (2, 64, 8), (1, 33, 1)])
+def test_odd_shapes_and_misaligned_pointers_fall_back_to_narrow_vectors(E, D, shift):
+    rng = np.random.default_rng(22)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=20, B=4, H=3, D=D, E=E, T=(9, 1, 0, 16, 7), pad_blocks=E * 3)
+    L = shape[0]
+    for pool_l, packed_l in itertools.product(LAYOUTS, LAYOUTS):
+        want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+        oracle.kv_pack(shape, pool_l, stride, planes_of(pool, L * 2), T, off, bt, packed_l, want)
+        d_pool = Guarded(pool.size, init=pool, shift=shift)
+        pl = tc.pool(pool_l, NB, L * 2, block_stride=stride)
+        plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_src=bt))
+        out = Guarded(want.size, shift=shift)
+        tc.tc_kv_pack(plan, pool_tables(d_pool, L * 2, "planes"), [out.ptr()])
+        assert np.array_equal(out.result(), want)
+        want_pool = np.full_like(pool, 0xA5)
+        oracle.kv_unpack(shape, pool_l, stride, planes_of(want_pool, L * 2), T, off, bt, packed_l, want)
+        plan2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_dst=bt))
+        fresh = Guarded(pool.size, shift=shift)
+        tc.tc_kv_unpack(plan2, [out.ptr()], pool_tables(fresh, L * 2, "planes"))
+        assert np.array_equal(fresh.result(), want_pool)
+
+
+# --------------------------------------------------------------------------- migrate, mixed, pinned host
+@pytest.mark.parametrize("src_l,dst_l", list(itertools.product(LAYOUTS, LAYOUTS)))
+def test_migrate_pool_to_pool(src_l, dst_l):
+    rng = np.random.default_rng(23)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=4, NB=48, B=32, H=2, D=128, E=2, T=(512, 33, 1, 300, 64))
+    L, B, H, D, E = shape
+    NB2 = NB + 5
+    bt2 = rng.permutation(NB2)[:off[-1]].astype(np.int32)
+    want = np.full(L * 2 * NB2 * stride, 0xA5, dtype=np.uint8)
+    oracle.kv_migrate(shape, src_l, stride, planes_of(pool, L * 2), dst_l, stride, planes_of(want, L * 2), T, off, bt, bt2, threads=4)
+    sp = tc.pool(src_l, NB, 1, plane_stride=NB * stride)
+    dp = tc.pool(dst_l, NB2, 1, plane_stride=NB2 * stride)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=sp, dst_pool=dp, T=T, bt_off=off, bt_src=bt, bt_dst=bt2))
+    out = Guarded(want.size)
+    tc.tc_kv_pack(plan, [dev(pool)], [out.ptr()])
+    assert np.array_equal(out.result(), want)
+
+
+def test_mixed_plan_offload_and_reload_through_pinned_host_pool():
+    """Device NHD pool <-> pinned page-first HND host pool, both directions of one plan on two
+    streams; the kernels store into / load from host memory directly."""
+    shape = wl.KVShape(L=2, B=16, H=8, D=128, E=2)
+    s = shape.tuple
+    NBd, NBh = 96, 160
+    step = next(wl.config5(NB_dev=NBd, NB_host=NBh, sessions=12, steps=1, shape=shape, p=0.4, max_prefix=6, max_new=3))
+    chunk = shape.chunk_bytes
+    devp = np.zeros(4 * NBd * chunk, dtype=np.uint8)
+    hostp = np.zeros(NBh * 4 * chunk, dtype=np.uint8)
+    wl.fill_np(devp, 1)
+    wl.fill_np(hostp, 2)
+    want_dev, want_host = devp.copy(), hostp.copy()
+    hp = lambda a: [a[p * chunk:] for p in range(4)]
+    oracle.kv_migrate(s, oracle.NHD, chunk, planes_of(devp, 4), oracle.HND, 4 * chunk, hp(want_host), step.offload_T, step.offload_off, step.offload_dev, step.offload_host)
+    oracle.kv_migrate(s, oracle.HND, 4 * chunk, hp(hostp), oracle.NHD, chunk, planes_of(want_dev, 4), step.reload_T, step.reload_off, step.reload_host, step.reload_dev)
+    d_dev = dev(devp)
+    h_host = torch.from_numpy(hostp.copy()).pin_memory()
+    spec = tc.kv_spec(tc.TC_KV_MIXED, s, src_pool=tc.pool(tc.TC_NHD, NBd, 1, plane_stride=NBd * chunk, slot_bytes=devp.size),
+                      dst_pool=tc.pool(tc.TC_HND, NBh, 1, plane_stride=chunk, block_stride=4 * chunk, slot_bytes=hostp.size),
+                      T=step.offload_T, bt_off=step.offload_off, bt_src=step.offload_dev, bt_dst=step.offload_host,
+                      reload=dict(T=step.reload_T, bt_off=step.reload_off, bt_src=step.reload_host, bt_dst=step.reload_dev))
+    plan = tc.tc_plan_create(spec)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    tc.tc_kv_pack(plan, [d_dev], [h_host], stream=s1)
+    tc.tc_kv_unpack(plan, [h_host], [d_dev], stream=s2)
+    torch.cuda.synchronize()
+    assert np.array_equal(d_dev.cpu().numpy(), want_dev)
+    assert np.array_equal(h_host.numpy(), want_host)
+
+
+def test_pack_to_pinned_host_hnd_and_reload():
+    rng = np.random.default_rng(24)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=64, B=16, H=8, D=128, E=2, T=(700, 16, 45, 130))
+    L = shape[0]
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, L * 2), T, off, bt, oracle.HND, want, threads=4)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride)
+    host = torch.zeros(want.size, dtype=torch.uint8).pin_memory()
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_src=bt, tuning=dict(max_ctas=32)))
+    assert plan.stats().grid[0] <= 32
+    tc.tc_kv_pack(plan, [dev(pool)], [host])
+    torch.cuda.synchronize()
+    assert np.array_equal(host.numpy(), want)
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(want_pool, L * 2), T, off, bt2, oracle.HND, want, threads=4)
+    plan2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_dst=bt2))
+    fresh = Guarded(pool.size)
+    tc.tc_kv_unpack(plan2, [host], [fresh.ptr()])
+    assert np.array_equal(fresh.result(), want_pool)
+
+
+# --------------------------------------------------------------------------- weights
+@pytest.mark.parametrize("variant", ["tight", "permuted_misaligned"])
+def test_weights_full_and_every_shard(variant):
+    ck = small_checkpoint() if variant == "tight" else small_checkpoint(order_seed=3, lead_pad=2)
+    blob = np.zeros(ck.nbytes_total + (ck.nbytes_total & 1), dtype=np.uint8)
+    wl.fill_np(blob, 5, "normal")
+    blob = blob[:ck.nbytes_total]
+    d_blob = dev(blob)
+    for world in (1, 4):
+        for rank in range(world):
+            split = ck.split_dim if world > 1 else np.full(ck.N, -1)
+            sizes = [ck.nbytes(i) // (world if split[i] >= 0 else 1) for i in range(ck.N)]
+            want = [np.zeros(n, dtype=np.uint8) for n in sizes]
+            oracle.weights(ck.byte_off, ck.E, ck.shapes, split, rank, world, blob, want)
+            plan = tc.tc_plan_create(ck_spec(ck, split_dim=split, rank=rank, world=world, tuning=dict(tile_bytes=4096)))
+            outs = [Guarded(n, fill=0xEE) for n in sizes]
+            tc.tc_weights_materialize(plan, d_blob, [o.ptr() for o in outs])
+            for i in range(ck.N):
+                assert np.array_equal(outs[i].result(), want[i]), (ck.names[i], world, rank)
+
+
+def test_weights_transform_into_fused_and_strided_targets():
+    ck = small_checkpoint()
+    blob = np.zeros(ck.nbytes_total, dtype=np.uint8)
+    wl.fill_np(blob, 6, "normal")
+    ids = [ck.names.index(f"layers.1.{n}_proj") for n in "qkv"]
+    sizes = [ck.nbytes(i) for i in ids]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    spec = tc.weights_spec(ck.byte_off[ids], sizes, ck.E[ids], ck.ndim[ids], ck.shapes[ids], blob_bytes=blob.size,
+                           dst_slot=[0, 0, 0], dst_off=offs[:3], n_dst=1, dst_bytes=[offs[-1]])
+    fused = Guarded(int(offs[-1]))
+    tc.tc_weights_materialize(tc.tc_plan_create(spec), dev(blob), [fused.ptr()])
+    want = np.zeros(offs[-1], dtype=np.uint8)
+    oracle.weights(ck.byte_off[ids], ck.E[ids], ck.shapes[ids], [-1] * 3, 0, 1, blob, [want] * 3, dst_off=offs[:3])
+    assert np.array_equal(fused.result(), want)
+    # middle-dim split into a strided window of a larger target
+    rng = np.random.default_rng(4)
+    full = rng.integers(0, 2 ** 32, (4, 6, 5), dtype=np.uint32)
+    blob2 = np.concatenate([np.zeros(4, dtype=np.uint8), full.reshape(-1).view(np.uint8)])
+    spec = tc.weights_spec([4], [full.nbytes], [4], [3], [[4, 6, 5, 1]], split_dim=[1], rank=2, world=3, blob_bytes=blob2.size,
+                           dst_slot=[0], dst_off=[12], dst_stride=[[64, 32, 4, 4]], n_dst=1, dst_bytes=[256])
+    target = Guarded(256, fill=0)
+    tc.tc_weights_materialize(tc.tc_plan_create(spec), dev(blob2), [target.ptr()])
+    want2 = np.zeros(256, dtype=np.uint8)
+    oracle.weights([4], [4], [[4, 6, 5, 1]], [1], 2, 3, blob2, [want2], dst_off=[12], dst_stride=[[64, 32, 4, 4]])
+    assert np.array_equal(target.result(), want2)
+
+
+# --------------------------------------------------------------------------- lifecycle on the device
+def test_empty_plan_wrong_tables_and_deadline_launch_nothing():
+    shape, NB, src, dst = wl.config1()
+    s = shape.tuple
+    pl = tc.pool(tc.TC_NHD, NB, 2)
+    empty = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=pl))
+    buf = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    tc.tc_kv_pack(empty, [buf, buf], [buf])                # no-op, returns TC_OK
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=pl, T=src.T, bt_off=src.bt_off, bt_src=src.bt))
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_kv_pack(plan, [buf], [buf])                  # the pool has two table slots
+    assert e.value.status == tc.TC_ERR_INVALID_ARG
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_kv_pack(plan, [buf, 0], [buf])               # NULL table entry
+    assert e.value.status == tc.TC_ERR_INVALID_ARG
+    soon = time.clock_gettime_ns(time.CLOCK_MONOTONIC) + 50_000_000
+    late = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=pl, T=src.T, bt_off=src.bt_off, bt_src=src.bt, deadline_ns=soon))
+    time.sleep(0.1)
+    out = Guarded(1400832)
+    pool = torch.zeros(2 * NB * shape.chunk_bytes, dtype=torch.uint8, device="cuda")
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_kv_pack(late, [pool, pool[NB * shape.chunk_bytes:]], [out.ptr()])
+    assert e.value.status == tc.TC_ERR_DEADLINE
+    assert (out.result() == 0xA5).all()                     # nothing was launched
+    assert plan.stats().device_bytes > 0 and plan.stats().executable

@@ -1,0 +1,325 @@
+"""Host-side tests of the C-ABI library that need no GPU: the exported symbols, the plan
+builder's validation (every error is raised before any launch) and its lowering, checked by
+interpreting the lowered descriptors in numpy and comparing with the oracle byte for byte."""
+import ctypes
+import itertools
+import os
+import re
+import time
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2608_06007_b200 as tc
+import workloads as wl
+from helpers import ck_spec, kv_case, planes_of, run_descriptors, small_checkpoint
+
+HOST = tc.TC_PLAN_HOST_ONLY
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "tensorcast.h")).read()
+    declared = set(re.findall(r"TC_API\s+[\w\s\*]+?\b(tc_\w+)\s*\(", header))
+    assert {"tc_plan_create", "tc_kv_pack", "tc_kv_unpack", "tc_weights_materialize", "tc_plan_destroy"} <= declared
+    lib = tc.load_library()
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert declared == set(tc.EXPORTS)
+    assert ctypes.sizeof(tc.binding.tc_index_entry_t) == 64
+
+
+def test_fast_division_constants_are_exact():
+    # the kernels divide by runtime constants with a multiply-high; replay that arithmetic
+    rng = np.random.default_rng(0)
+    ds = np.unique(np.concatenate([np.arange(1, 300), rng.integers(1, 1 << 20, 300), [1 << 20, (1 << 20) - 1, 3584, 28672]]))
+    ns = np.unique(np.concatenate([np.arange(0, 5000), rng.integers(0, 1 << 31, 5000), [(1 << 31) - 1]])).astype(np.uint64)
+    for d in ds:
+        d = int(d)
+        s = 0
+        while (1 << s) < d:
+            s += 1
+        mul = ((1 << 32) * ((1 << s) - d)) // d + 1
+        assert mul < (1 << 32)
+        q = (((ns * np.uint64(mul)) >> np.uint64(32)) + ns) >> np.uint64(s)
+        assert np.array_equal(q, ns // np.uint64(d)), d
+
+
+# --------------------------------------------------------------------------- KV lowering
+LAYOUTS = [tc.TC_NHD, tc.TC_HND]
+
+
+@pytest.mark.parametrize("pool_l,packed_l", list(itertools.product(LAYOUTS, LAYOUTS)))
+@pytest.mark.parametrize("slots", ["planes", "one"])
+def test_pack_and_unpack_lowering_match_oracle(pool_l, packed_l, slots):
+    rng = np.random.default_rng(1)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, T=(5, 0, 11, 1, 8), pad_blocks=16)
+    L = shape[0]
+    planes = planes_of(pool, L * 2)
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, pool_l, stride, planes, T, off, bt, packed_l, want)
+    if slots == "planes":
+        pl = tc.pool(pool_l, NB, L * 2, block_stride=stride, slot_bytes=planes[0].size)
+        tables = planes
+    else:
+        pl = tc.pool(pool_l, NB, 1, plane_stride=planes[0].size, block_stride=stride, slot_bytes=pool.size)
+        tables = [pool]
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_src=bt, flags=HOST, tuning=dict(tile_bytes=512)))
+    st = plan.stats()
+    assert st.packed_bytes_required == want.size and st.payload_bytes[0] == want.size and not st.executable
+    got = np.full(want.size, 0xCC, dtype=np.uint8)
+    cnt = [np.zeros(want.size, dtype=np.int32)]
+    run_descriptors(plan.descriptors(0), tables, [got], cnt)
+    assert np.array_equal(got, want) and (cnt[0] == 1).all()
+    # unpack through a fresh table into a sentinel pool
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, pool_l, stride, planes_of(want_pool, L * 2), T, off, bt2, packed_l, want)
+    plan2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_dst=bt2, flags=HOST))
+    got_pool = np.full_like(pool, 0xA5)
+    run_descriptors(plan2.descriptors(1), [want], planes_of(got_pool, L * 2) if slots == "planes" else [got_pool])
+    assert np.array_equal(got_pool, want_pool)
+    assert plan2.stats().n_descriptors[0] == 0 and plan2.stats().n_descriptors[1] > 0
+
+
+@pytest.mark.parametrize("src_l,dst_l", list(itertools.product(LAYOUTS, LAYOUTS)))
+def test_migrate_lowering_matches_oracle_including_page_first_pool(src_l, dst_l):
+    rng = np.random.default_rng(2)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, T=(7, 12, 2))
+    L, B, H, D, E = shape
+    chunk = B * H * D * E
+    NB2 = NB + 2
+    bt2 = rng.permutation(NB2)[:off[-1]].astype(np.int32)
+    # destination: page-first pool [block][plane][chunk]
+    dst = np.full(NB2 * L * 2 * chunk, 0x5A, dtype=np.uint8)
+    want = dst.copy()
+    oracle.kv_migrate(shape, src_l, stride, planes_of(pool, L * 2), dst_l, L * 2 * chunk,
+                      [want[p * chunk:] for p in range(L * 2)], T, off, bt, bt2)
+    sp = tc.pool(src_l, NB, L * 2, block_stride=stride)
+    dp = tc.pool(dst_l, NB2, 1, plane_stride=chunk, block_stride=L * 2 * chunk, slot_bytes=dst.size)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=sp, dst_pool=dp, T=T, bt_off=off, bt_src=bt, bt_dst=bt2, flags=HOST))
+    run_descriptors(plan.descriptors(0), planes_of(pool, L * 2), [dst])
+    assert np.array_equal(dst, want)
+
+
+def test_same_layout_full_blocks_lower_to_one_run_per_block():
+    shape, NB, src, dst = wl.config1()
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * shape.chunk_bytes)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape.tuple, src_pool=pl, T=src.T, bt_off=src.bt_off, bt_src=src.bt, flags=HOST))
+    ds = plan.descriptors(0)
+    assert len(ds) == 24                                   # one descriptor per (request, block)
+    assert all(d.rows == 1 and d.n_outer == 2 for d in ds)
+    assert sorted(d.run_bytes for d in ds)[-1] == shape.chunk_bytes
+    st = plan.stats()
+    assert st.payload_bytes[0] == 1400832 and st.vec_bytes[0] == 16 and st.n_tiles[0] == 48
+
+
+def test_mixed_plan_groups_match_oracle():
+    shape = (2, 4, 2, 8, 2)
+    L, B, H, D, E = shape
+    chunk = B * H * D * E
+    step = next(wl.config5(NB_dev=40, NB_host=60, sessions=5, steps=1, shape=wl.KVShape(*shape), p=0.5, max_prefix=4, max_new=2))
+    rng = np.random.default_rng(3)
+    dev = rng.integers(0, 256, L * 2 * 40 * chunk, dtype=np.uint8)        # plane-major, NHD
+    host = rng.integers(0, 256, 60 * L * 2 * chunk, dtype=np.uint8)       # page-first, HND
+    dev_pool = tc.pool(tc.TC_NHD, 40, 1, plane_stride=40 * chunk)
+    host_pool = tc.pool(tc.TC_HND, 60, 1, plane_stride=chunk, block_stride=L * 2 * chunk)
+    spec = tc.kv_spec(tc.TC_KV_MIXED, shape, src_pool=dev_pool, dst_pool=host_pool,
+                      T=step.offload_T, bt_off=step.offload_off, bt_src=step.offload_dev, bt_dst=step.offload_host,
+                      reload=dict(T=step.reload_T, bt_off=step.reload_off, bt_src=step.reload_host, bt_dst=step.reload_dev), flags=HOST)
+    plan = tc.tc_plan_create(spec)
+    want_dev, want_host = dev.copy(), host.copy()
+    hp = lambda a: [a[p * chunk:] for p in range(L * 2)]
+    oracle.kv_migrate(shape, oracle.NHD, chunk, planes_of(dev, L * 2), oracle.HND, L * 2 * chunk, hp(want_host),
+                      step.offload_T, step.offload_off, step.offload_dev, step.offload_host)
+    oracle.kv_migrate(shape, oracle.HND, L * 2 * chunk, hp(host), oracle.NHD, chunk, planes_of(want_dev, L * 2),
+                      step.reload_T, step.reload_off, step.reload_host, step.reload_dev)
+    got_dev, got_host = dev.copy(), host.copy()
+    run_descriptors(plan.descriptors(0), [dev], [got_host])
+    run_descriptors(plan.descriptors(1), [host], [got_dev])
+    assert np.array_equal(got_dev, want_dev) and np.array_equal(got_host, want_host)
+    # an offload target that the reload group reads is refused
+    bad = step.offload_host.copy()
+    bad[0] = step.reload_host[0]
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIXED, shape, src_pool=dev_pool, dst_pool=host_pool,
+                                     T=step.offload_T, bt_off=step.offload_off, bt_src=step.offload_dev, bt_dst=bad,
+                                     reload=dict(T=step.reload_T, bt_off=step.reload_off, bt_src=step.reload_host, bt_dst=step.reload_dev), flags=HOST))
+    assert e.value.status == tc.TC_ERR_OVERLAP
+
+
+# --------------------------------------------------------------------------- weights lowering
+@pytest.mark.parametrize("variant", ["tight", "permuted_misaligned"])
+@pytest.mark.parametrize("world", [1, 4])
+def test_weights_lowering_matches_oracle(variant, world):
+    ck = small_checkpoint() if variant == "tight" else small_checkpoint(order_seed=3, pad_to=1, lead_pad=2)
+    blob = np.random.default_rng(4).integers(0, 256, ck.nbytes_total, dtype=np.uint8)
+    for rank in range(world):
+        split = ck.split_dim if world > 1 else np.full(ck.N, -1)
+        sizes = [ck.nbytes(i) // (world if split[i] >= 0 else 1) for i in range(ck.N)]
+        want = [np.zeros(n, dtype=np.uint8) for n in sizes]
+        oracle.weights(ck.byte_off, ck.E, ck.shapes, split, rank, world, blob, want)
+        plan = tc.tc_plan_create(ck_spec(ck, split_dim=split, rank=rank, world=world, flags=HOST, tuning=dict(tile_bytes=1024)))
+        got = [np.full(n, 0xEE, dtype=np.uint8) for n in sizes]
+        cnt = [np.zeros(n, dtype=np.int32) for n in sizes]
+        run_descriptors(plan.descriptors(0), [blob], got, cnt)
+        for i in range(ck.N):
+            assert np.array_equal(got[i], want[i]), ck.names[i]
+            assert (cnt[i] == 1).all()
+        st = plan.stats()
+        assert st.payload_bytes[0] == sum(sizes)
+        assert st.vec_bytes[0] == (16 if variant == "tight" else 2)
+
+
+def test_weights_transform_into_fused_target():
+    """q, k, v of one layer written side by side into one fused qkv buffer (dst_slot / dst_off),
+    and a middle-dim split written into a strided window."""
+    ck = small_checkpoint()
+    blob = np.random.default_rng(5).integers(0, 256, ck.nbytes_total, dtype=np.uint8)
+    ids = [ck.names.index(f"layers.0.{n}_proj") for n in "qkv"]
+    sizes = [ck.nbytes(i) for i in ids]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    nb = [ck.nbytes(i) for i in ids]
+    spec = tc.weights_spec(ck.byte_off[ids], nb, ck.E[ids], ck.ndim[ids], ck.shapes[ids], blob_bytes=blob.size,
+                           dst_slot=[0, 0, 0], dst_off=offs[:3], n_dst=1, dst_bytes=[offs[-1]], flags=HOST)
+    plan = tc.tc_plan_create(spec)
+    fused = np.zeros(offs[-1], dtype=np.uint8)
+    run_descriptors(plan.descriptors(0), [blob], [fused])
+    want = np.concatenate([blob[ck.byte_off[i]:ck.byte_off[i] + ck.nbytes(i)] for i in ids])
+    assert np.array_equal(fused, want)
+    # overlapping windows are refused
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_plan_create(tc.weights_spec(ck.byte_off[ids], nb, ck.E[ids], ck.ndim[ids], ck.shapes[ids], blob_bytes=blob.size,
+                                          dst_slot=[0, 0, 0], dst_off=[0, sizes[0] - 2, offs[2]], n_dst=1, dst_bytes=[offs[-1]], flags=HOST))
+    assert e.value.status == tc.TC_ERR_OVERLAP
+    # strided window, middle-dim split: same case as the oracle pin
+    rng = np.random.default_rng(4)
+    full = rng.integers(0, 2 ** 32, (4, 6, 5), dtype=np.uint32)
+    blob2 = np.concatenate([np.zeros(3, dtype=np.uint8), full.reshape(-1).view(np.uint8)])
+    spec = tc.weights_spec([3], [full.nbytes], [4], [3], [[4, 6, 5, 1]], split_dim=[1], rank=2, world=3, blob_bytes=blob2.size,
+                           dst_slot=[0], dst_off=[12], dst_stride=[[64, 32, 4, 4]], n_dst=1, dst_bytes=[4 * 2 * 8 * 4], flags=HOST)
+    target = np.zeros((4, 2, 8), dtype=np.uint32)
+    run_descriptors(tc.tc_plan_create(spec).descriptors(0), [blob2], [target.reshape(-1).view(np.uint8)])
+    want = np.zeros_like(target)
+    want[:, :, 3:8] = full[:, 4:6, :]
+    assert np.array_equal(target, want)
+
+
+def test_interleaved_strided_destinations_pass_the_exact_overlap_check():
+    # two [4][3] byte tensors interleaved column-wise into one [4][6] target: bounding spans
+    # intersect but no byte is written twice
+    blob = np.arange(24, dtype=np.uint8)
+    spec = tc.weights_spec([0, 12], [12, 12], [1, 1], [2, 2], [[4, 3, 1, 1]] * 2, blob_bytes=24,
+                           dst_slot=[0, 0], dst_off=[0, 3], dst_stride=[[6, 1, 1, 1]] * 2, n_dst=1, dst_bytes=[24], flags=HOST)
+    out = np.zeros(24, dtype=np.uint8)
+    cnt = [np.zeros(24, dtype=np.int32)]
+    run_descriptors(tc.tc_plan_create(spec).descriptors(0), [blob], [out], cnt)
+    assert (cnt[0] == 1).all()
+    assert np.array_equal(out.reshape(4, 6), np.concatenate([blob[:12].reshape(4, 3), blob[12:].reshape(4, 3)], axis=1))
+
+
+def test_llama3_8b_plans_have_the_expected_size():
+    ck = wl.config3()
+    full = tc.tc_plan_create(ck_spec(ck, flags=HOST)).stats()
+    assert full.payload_bytes[0] == 16060522496 and full.vec_bytes[0] == 16
+    shard = tc.tc_plan_create(ck_spec(ck, split_dim=ck.split_dim, rank=3, world=8, flags=HOST)).stats()
+    assert shard.payload_bytes[0] == 2 * 1004015616
+    # 65 norms of 8 KiB are one tile each; everything else is cut into 32 KiB tiles
+    assert full.n_tiles[0] == (16060522496 - 65 * 8192) // 32768 + 65
+
+
+def test_long_runs_and_wide_spans_are_cut_for_32_bit_row_offsets():
+    # a 6 GiB contiguous tensor and a dim-1 slice whose rows are 3 GiB apart
+    spec = tc.weights_spec([0], [6 << 30], [2], [1], [[3 << 30, 1, 1, 1]], blob_bytes=6 << 30, flags=HOST)
+    ds = tc.tc_plan_create(spec).descriptors(0)
+    assert sum(d.run_bytes * d.rows for d in ds) == 6 << 30
+    for d in ds:
+        assert (d.rows // d.n0) * max(d.src_s1, d.dst_s1) + d.n0 * max(d.src_s0, d.dst_s0) + d.run_bytes < 2 ** 31
+    spec = tc.weights_spec([0], [3 * (3 << 30)], [1], [2], [[3, 3 << 30, 1, 1]], split_dim=[1], rank=1, world=3,
+                           blob_bytes=9 << 30, flags=HOST)
+    ds = tc.tc_plan_create(spec).descriptors(0)
+    assert sum(d.run_bytes * d.rows for d in ds) == 3 << 30
+    starts = sorted(d.src_off for d in ds)
+    assert starts[0] == 1 << 30 and starts[-1] >= (6 << 30) + (1 << 30)
+
+
+# --------------------------------------------------------------------------- validation
+def _pack_spec(**over):
+    shape, NB, src, dst = wl.config1()
+    kw = dict(src_pool=tc.pool(tc.TC_NHD, NB, 2), T=src.T, bt_off=src.bt_off, bt_src=src.bt, flags=HOST)
+    kw.update(over)
+    return tc.kv_spec(kw.pop("kind", tc.TC_KV_PACK), kw.pop("shape", shape.tuple), **kw)
+
+
+def _status(spec):
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_plan_create(spec)
+    return e.value.status
+
+
+def test_validation_rejects_bad_plans_before_any_launch():
+    shape, NB, src, dst = wl.config1()
+    assert _status(_pack_spec(shape=(1, 16, 8, 128, 3))) == tc.TC_ERR_SHAPE
+    bad = src.bt.copy(); bad[5] = NB
+    assert _status(_pack_spec(bt_src=bad)) == tc.TC_ERR_BOUNDS
+    assert _status(_pack_spec(bt_src=None)) == tc.TC_ERR_INVALID_ARG
+    assert _status(_pack_spec(T=[37, 100, 5, 300])) == tc.TC_ERR_INVALID_ARG          # table too short for T
+    assert _status(_pack_spec(packed_bytes=1400831)) == tc.TC_ERR_BOUNDS
+    assert _status(_pack_spec(src_pool=tc.pool(tc.TC_NHD, NB, 3))) == tc.TC_ERR_INVALID_ARG
+    assert _status(_pack_spec(src_pool=tc.pool(tc.TC_NHD, NB, 2, block_stride=100))) == tc.TC_ERR_OVERLAP
+    assert _status(_pack_spec(src_pool=tc.pool(tc.TC_NHD, NB, 2, slot_bytes=1000))) == tc.TC_ERR_BOUNDS
+    assert _status(_pack_spec(src_pool=tc.pool(tc.TC_NHD, NB, 1, plane_stride=4096))) == tc.TC_ERR_OVERLAP
+    assert _status(_pack_spec(kind=9)) == tc.TC_ERR_INVALID_ARG
+    dup = dst.bt.copy(); dup[3] = dup[17]
+    un = dict(kind=tc.TC_KV_UNPACK, src_pool=None, dst_pool=tc.pool(tc.TC_NHD, NB, 2), bt_src=None)
+    assert _status(_pack_spec(bt_dst=dup, **un)) == tc.TC_ERR_OVERLAP                 # a block written twice
+    tc.tc_plan_create(_pack_spec(bt_dst=dst.bt, **un))
+    # prefix sharing on the read side is allowed
+    shared = src.bt.copy(); shared[4] = shared[0]
+    tc.tc_plan_create(_pack_spec(bt_src=shared))
+    spec, keep = _pack_spec()
+    spec.struct_size = 8
+    assert _status(spec) == tc.TC_ERR_INVALID_ARG
+    ck = small_checkpoint()
+    assert _status(ck_spec(ck, split_dim=ck.split_dim, rank=0, world=7, flags=HOST)) == tc.TC_ERR_SHAPE
+    assert _status(ck_spec(ck, split_dim=ck.split_dim, rank=4, world=4, flags=HOST)) == tc.TC_ERR_INVALID_ARG
+    assert _status(ck_spec(ck, blob_bytes=ck.nbytes_total - 1, flags=HOST)) == tc.TC_ERR_BOUNDS
+    nb = [ck.nbytes(i) for i in range(ck.N)]
+    nb[2] += 2
+    assert _status(tc.weights_spec(ck.byte_off, nb, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total + 2, flags=HOST)) == tc.TC_ERR_SHAPE
+    small = [ck.nbytes(i) for i in range(ck.N)]
+    small[1] -= 2
+    assert _status(ck_spec(ck, dst_bytes=small, flags=HOST)) == tc.TC_ERR_BOUNDS
+
+
+def test_empty_plans_deadline_and_kind_checks():
+    shape, NB, src, dst = wl.config1()
+    empty = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape.tuple, src_pool=tc.pool(tc.TC_NHD, NB, 2), flags=HOST))
+    assert empty.stats().n_tiles[0] == 0 and empty.stats().payload_bytes[0] == 0
+    zero_len = tc.tc_plan_create(_pack_spec(T=[0, 0], bt_off=[0, 0, 0], bt_src=[]))
+    assert zero_len.stats().n_descriptors[0] == 0
+    past = time.clock_gettime_ns(time.CLOCK_MONOTONIC) - 1
+    assert _status(_pack_spec(deadline_ns=past)) == tc.TC_ERR_DEADLINE
+    plan = tc.tc_plan_create(_pack_spec(trace_id=77))
+    assert plan.stats().trace_id == 77
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_kv_unpack(plan, [1], [1, 1])
+    assert e.value.status == tc.TC_ERR_KIND
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_kv_pack(plan, [16, 16], [16])            # host-only plans never execute
+    assert e.value.status == tc.TC_ERR_INVALID_ARG
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_weights_materialize(plan, 16, [16])
+    assert e.value.status == tc.TC_ERR_KIND
+    plan.destroy()
+    plan.destroy()                                      # idempotent; NULL destroy is a no-op
+    assert tc.load_library().tc_plan_destroy(None) == 0
+
+
+@pytest.mark.skipif(__import__("torch").cuda.is_available(), reason="only meaningful without a GPU")
+def test_product_path_fails_loudly_without_a_device():
+    """No CPU fallback: without a CUDA device an executable plan cannot even be created."""
+    shape, NB, src, dst = wl.config1()
+    spec = tc.kv_spec(tc.TC_KV_PACK, shape.tuple, src_pool=tc.pool(tc.TC_NHD, NB, 2), T=src.T, bt_off=src.bt_off, bt_src=src.bt)
+    assert _status(spec) == tc.TC_ERR_CUDA
