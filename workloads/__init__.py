@@ -207,16 +207,18 @@ def admit_waves(n_blocks_per_req: np.ndarray, capacity: int):
 
 def config2(NB: int = 20000, R: int = 256, wave_blocks: int | None = None,
             shape: KVShape = LLAMA3_8B_KV, seed: int = SEED_BASE + 2,
-            median: int = 2048, sigma: float = 1.0, max_len: int = 32768):
+            median: int = 2048, sigma: float = 1.0, max_len: int = 32768, NB_dst: int | None = None):
     """Offload/reload waves: log-normal context lengths, fragmented block tables.
 
     Returns (shape, NB, T_all, waves); every wave is (src, dst): the table the wave's
-    requests occupy when packed, and an independent fresh allocation they are reloaded into.
+    requests occupy when packed, and an independent fresh allocation (drawn from a pool of
+    NB_dst blocks, default NB) they are reloaded into.
     """
     ss = np.random.SeedSequence(seed).spawn(3)
     T_all = lognormal_lengths(np.random.default_rng(ss[0]), R, math.log(median), sigma, 1, max_len)
     n_all = (T_all + shape.B - 1) // shape.B
-    cap = NB if wave_blocks is None else min(NB, wave_blocks)
+    NB_dst = NB if NB_dst is None else NB_dst
+    cap = min(NB, NB_dst) if wave_blocks is None else min(NB, NB_dst, wave_blocks)
     # a request larger than the wave capacity is truncated to it (recorded in T_all)
     too_big = n_all > cap
     T_all = np.where(too_big, cap * shape.B, T_all)
@@ -226,7 +228,7 @@ def config2(NB: int = 20000, R: int = 256, wave_blocks: int | None = None,
         T = T_all[ids]
         off = _csr(T, shape.B)
         src = KVRequests(T, off, rng_a.permutation(NB)[:off[-1]].astype(np.int32))
-        dst = KVRequests(T, off, rng_b.permutation(NB)[:off[-1]].astype(np.int32))
+        dst = KVRequests(T, off, rng_b.permutation(NB_dst)[:off[-1]].astype(np.int32))
         waves.append((src, dst))
     return shape, NB, T_all, waves
 
