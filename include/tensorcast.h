@@ -84,7 +84,8 @@ typedef enum {
     TC_ERR_KIND = -5,        /* execute call does not match the plan's kind */
     TC_ERR_OOM = -6,         /* host or device allocation of plan storage failed */
     TC_ERR_CUDA = -7,        /* a CUDA runtime call failed (no device, launch failure) */
-    TC_ERR_DEADLINE = -8     /* the plan's deadline had already passed at call entry */
+    TC_ERR_DEADLINE = -8,    /* the plan's deadline had already passed at call entry */
+    TC_ERR_TOO_LARGE = -9    /* the request exceeds a fixed capacity of the entry point called */
 } tc_status;
 
 typedef enum {
@@ -238,6 +239,38 @@ TC_API int tc_weights_materialize(const tc_plan_t *plan, const void *blob, void 
  * stream that executes it.  NULL is a no-op returning TC_OK.
  */
 TC_API int tc_plan_destroy(tc_plan_t *plan);
+
+/*
+ * tc_kv_pack without any device allocation.  (The paper has no counterpart: this entry point
+ * exists for the library's users, not for one of the paper's operations.)
+ *
+ * tc_plan_create keeps a plan's descriptors in device memory that it obtains with cudaMalloc.
+ * Some callers must not do that: an inference engine that has already handed every free byte
+ * of the GPU to its KV pool (a later cudaMalloc fails or eats into that budget), or a
+ * scheduler loop that cannot afford the device-wide stall an allocation may cause.  For them
+ * this call lowers `spec` (kind TC_KV_PACK, TC_KV_MIGRATE, or the offload group of
+ * TC_KV_MIXED) on the host, copies the descriptors into a fixed scratch area that is part of
+ * the library image, and launches the same kernel as tc_kv_pack on `stream`, all in one call.
+ * It calls no cudaMalloc, cudaFree or other allocating routine; host-side lowering uses
+ * ordinary heap memory.  The data buffers are the caller's, exactly as for tc_kv_pack.
+ *
+ * Capacity: the descriptors and tile list of the call must fit TC_NOALLOC_SCRATCH_BYTES
+ * (1 MiB: about 8,000 KV blocks per call); a larger request returns TC_ERR_TOO_LARGE and
+ * launches nothing.  Every GPU that loads the library holds that 1 MiB until the process exits.
+ *
+ * The first call on a device resolves the scratch area's device address for that device (the
+ * device must be current, as for every call of this library); make that first call before any
+ * stream capture begins.  All calls on a device share the one scratch area, and it keeps the
+ * previous call's contents: each call overwrites the part it uses and nothing in it needs to
+ * start at zero.  Because the area is shared, two calls whose GPU work can overlap - calls on
+ * different streams, or from several threads - race on it; issue them on one stream (where the
+ * copy of the next call's descriptors is ordered after the previous call's kernel) or
+ * synchronise between them.  The descriptor copy comes from pageable host memory, so the call
+ * may block until earlier work on `stream` has drained.
+ */
+#define TC_NOALLOC_SCRATCH_BYTES (1u << 20)
+TC_API int tc_kv_pack_noalloc(const tc_plan_spec_t *spec, const void *const *src_bases, size_t n_src,
+                              void *const *dst_bases, size_t n_dst, void *stream);
 
 /* ---- off the data path: inspection and diagnostics -------------------------------------- */
 

@@ -16,7 +16,8 @@ from . import build as _build
 
 TC_OK = 0
 TC_ERR_INVALID_ARG, TC_ERR_SHAPE, TC_ERR_BOUNDS, TC_ERR_OVERLAP = -1, -2, -3, -4
-TC_ERR_KIND, TC_ERR_OOM, TC_ERR_CUDA, TC_ERR_DEADLINE = -5, -6, -7, -8
+TC_ERR_KIND, TC_ERR_OOM, TC_ERR_CUDA, TC_ERR_DEADLINE, TC_ERR_TOO_LARGE = -5, -6, -7, -8, -9
+TC_NOALLOC_SCRATCH_BYTES = 1 << 20
 TC_KV_PACK, TC_KV_UNPACK, TC_KV_MIGRATE, TC_KV_MIXED, TC_WEIGHTS = 1, 2, 3, 4, 5
 TC_NHD, TC_HND = 0, 1
 TC_PLAN_HOST_ONLY = 1
@@ -84,7 +85,8 @@ class tc_descriptor_t(C.Structure):
 
 
 EXPORTS = ("tc_plan_create", "tc_kv_pack", "tc_kv_unpack", "tc_weights_materialize",
-           "tc_plan_destroy", "tc_plan_stats", "tc_plan_descriptors", "tc_strerror", "tc_last_error")
+           "tc_plan_destroy", "tc_plan_stats", "tc_plan_descriptors", "tc_strerror", "tc_last_error",
+           "tc_kv_pack_noalloc")
 
 _lib = None
 
@@ -106,6 +108,8 @@ def load_library(path: str | None = None):
     lib.tc_plan_destroy.argtypes = [vp]
     lib.tc_plan_stats.argtypes = [vp, C.POINTER(tc_plan_stats_t)]
     lib.tc_plan_descriptors.argtypes = [vp, C.c_int, vp, sz, C.POINTER(sz)]
+    lib.tc_kv_pack_noalloc.argtypes = [C.POINTER(tc_plan_spec_t), vp, sz, vp, sz, vp]
+    lib.tc_kv_pack_noalloc.restype = C.c_int
     lib.tc_strerror.argtypes = [C.c_int]
     lib.tc_strerror.restype = C.c_char_p
     lib.tc_last_error.restype = C.c_char_p
@@ -278,6 +282,18 @@ def tc_kv_pack(plan: Plan, src_bases, dst_bases, stream=None) -> None:
     s, ns = _table(src_bases)
     d, nd = _table(dst_bases)
     _check(load_library().tc_kv_pack(plan.handle, s, ns, d, nd, _stream(stream)))
+
+
+def tc_kv_pack_noalloc(spec, src_bases, dst_bases, stream=None) -> None:
+    """tc_kv_pack for callers that must not allocate device memory: lowers `spec` and runs it
+    in one call, with the descriptors in the library's fixed 1 MiB scratch area instead of a
+    cudaMalloc'ed plan.  Calls whose GPU work may overlap race on that area; keep them on one
+    stream.  Raises TC_ERR_TOO_LARGE when the request does not fit."""
+    if isinstance(spec, tuple):
+        spec = spec[0]
+    s, ns = _table(src_bases)
+    d, nd = _table(dst_bases)
+    _check(load_library().tc_kv_pack_noalloc(C.byref(spec), s, ns, d, nd, _stream(stream)))
 
 
 def tc_kv_unpack(plan: Plan, src_bases, dst_bases, stream=None) -> None:

@@ -604,6 +604,7 @@ extern "C" const char *tc_strerror(int status)
     case TC_ERR_OOM: return "TC_ERR_OOM";
     case TC_ERR_CUDA: return "TC_ERR_CUDA";
     case TC_ERR_DEADLINE: return "TC_ERR_DEADLINE";
+    case TC_ERR_TOO_LARGE: return "TC_ERR_TOO_LARGE";
     default: return "TC_ERR_UNKNOWN";
     }
 }
