@@ -215,7 +215,7 @@ def run_ours(args):
     shape = wl.LLAMA3_8B_KV
     NB = args.kv_blocks
     wave_blocks = args.wave_blocks
-    ck = wl.config3() if not args.small else wl.llama_checkpoint(layers=2, vocab=32064)
+    ck = wl.config3() if not args.small else wl.llama_checkpoint(layers=1, vocab=16032)
     need = NB * shape.block_bytes + 2 * wave_blocks * shape.block_bytes + 2.2 * ck.nbytes_total
     while need > 0.8 * free and NB > 1024:
         NB //= 2
@@ -406,9 +406,12 @@ def run_ours(args):
                 "frac_of_nominal_8TBps": achieved / 8000.0}
 
     threads = os.cpu_count() or 1
-    sample = OracleSample(args.oracle_blocks, threads)
-    cpu_v, _ = sample.run()
-    cpu_desc, threads = sample.desc, sample.threads
+    if args.no_cpu_baseline:
+        cpu_v, cpu_desc = None, "skipped (--no-cpu-baseline)"
+    else:
+        sample = OracleSample(args.oracle_blocks, threads)
+        cpu_v, _ = sample.run()
+        cpu_desc, threads = sample.desc, sample.threads
     line = {
         "metric": "kv_pack_unpack_and_weight_materialise_GBps", "value": value, "unit": "GB/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
@@ -444,6 +447,7 @@ def main():
     ap.add_argument("--shard-rank", type=int, default=0)
     ap.add_argument("--small", action="store_true", help="small case for profiler captures")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiler runs)")
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--e2e-warmup", type=int, default=1)
     ap.add_argument("--oracle-blocks", type=int, default=1536)

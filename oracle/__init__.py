@@ -80,6 +80,13 @@ def _split(n_items: int, threads: int):
     return [(int(edges[k]), int(edges[k + 1])) for k in range(threads) if edges[k] < edges[k + 1]]
 
 
+def _ranges(R, threads, requests):
+    if requests is None:
+        return _split(R, threads)
+    r0, r1 = requests
+    return [(r0 + a, r0 + b) for a, b in _split(r1 - r0, threads)]
+
+
 def _run(fn, ranges, threads):
     if threads <= 1 or len(ranges) <= 1:
         for a, b in ranges:
@@ -96,8 +103,9 @@ def packed_nbytes(shape, T) -> int:
 
 
 def kv_pack(shape, pool_layout, block_stride, planes, T, bt_off, bt, packed_layout,
-            packed, packed_cnt=None, threads=1):
-    """publish / offload: pool planes -> packed buffer (written in place)."""
+            packed, packed_cnt=None, threads=1, requests=None):
+    """publish / offload: pool planes -> packed buffer (written in place).
+    requests=(r0, r1) restricts the loops to requests [r0, r1) (same arithmetic)."""
     lib = _load()
     s, g = _Shape(*shape), _Geom(pool_layout, block_stride)
     T, bt_off, bt = _i64(T), _i64(bt_off), _i32(bt)
@@ -109,7 +117,7 @@ def kv_pack(shape, pool_layout, block_stride, planes, T, bt_off, bt, packed_layo
                            bt.ctypes, C.c_int32(packed_layout), C.c_void_p(_u8(packed).ctypes.data),
                            C.c_void_p(None if packed_cnt is None else _u8(packed_cnt).ctypes.data),
                            C.c_int64(r0), C.c_int64(r1))
-    _run(go, _split(R, threads), threads)
+    _run(go, _ranges(R, threads, requests), threads)
 
 
 def kv_pack_inverse(shape, pool_layout, block_stride, planes, T, bt_off, bt, packed_layout, packed):
@@ -125,7 +133,7 @@ def kv_pack_inverse(shape, pool_layout, block_stride, planes, T, bt_off, bt, pac
 
 
 def kv_unpack(shape, pool_layout, block_stride, planes, T, bt_off, bt, packed_layout,
-              packed, plane_cnt=None, threads=1):
+              packed, plane_cnt=None, threads=1, requests=None):
     """hydrate / reload: packed buffer -> pool planes (written in place)."""
     lib = _load()
     s, g = _Shape(*shape), _Geom(pool_layout, block_stride)
@@ -138,11 +146,11 @@ def kv_unpack(shape, pool_layout, block_stride, planes, T, bt_off, bt, packed_la
         lib.oracle_kv_unpack(C.byref(s), C.byref(g), tbl, cnt, C.c_int64(R), T.ctypes,
                              bt_off.ctypes, bt.ctypes, C.c_int32(packed_layout),
                              C.c_void_p(_u8(packed).ctypes.data), C.c_int64(r0), C.c_int64(r1))
-    _run(go, _split(R, threads), threads)
+    _run(go, _ranges(R, threads, requests), threads)
 
 
 def kv_migrate(shape, src_layout, src_block_stride, src_planes, dst_layout, dst_block_stride,
-               dst_planes, T, bt_off, bt_src, bt_dst, dst_cnt=None, threads=1):
+               dst_planes, T, bt_off, bt_src, bt_dst, dst_cnt=None, threads=1, requests=None):
     """publish then hydrate, fused: src pool -> dst pool through two block tables."""
     lib = _load()
     s = _Shape(*shape)
@@ -156,7 +164,7 @@ def kv_migrate(shape, src_layout, src_block_stride, src_planes, dst_layout, dst_
         lib.oracle_kv_migrate(C.byref(s), C.byref(gs), ts, C.byref(gd), td, cnt, C.c_int64(R),
                               T.ctypes, bt_off.ctypes, bt_src.ctypes, bt_dst.ctypes,
                               C.c_int64(r0), C.c_int64(r1))
-    _run(go, _split(R, threads), threads)
+    _run(go, _ranges(R, threads, requests), threads)
 
 
 def weights(blob_off, E, shapes, split_dim, rank, world, blob, dst, dst_off=None,

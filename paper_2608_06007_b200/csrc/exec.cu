@@ -20,10 +20,21 @@
 
 namespace tc {
 
-constexpr int kThreads = 256;
-constexpr int kUnrollWide = 8;    // 16-byte vectors in flight per thread
-constexpr int kUnrollNarrow = 4;  // same for the narrower fallback widths
-constexpr int kMinCtasPerSm = 3;
+// Three builds of the executor, chosen per group on the host, so that the common cases do not
+// pay registers for the rare ones:
+//   kModeRun   every tile is one 16-byte-aligned contiguous run (same-layout KV blocks, whole
+//              tensors, dim-0 slabs): no row decoding
+//   kModeRows  every access is 16-byte aligned, tiles hold strided rows (layout transforms,
+//              dim-1 slices)
+//   kModeAny   some descriptor or base pointer is less aligned: width picked per tile
+enum { kModeRun = 0, kModeRows = 1, kModeAny = 2 };
+
+// CTA shape per build: threads x vectors in flight per thread (one pass covers a 32 KiB tile)
+// and the residency the register budget is held to.
+template <int MODE> struct Shape;
+template <> struct Shape<kModeRun> { static constexpr int threads = 512, unroll = 4, min_ctas = 3; };
+template <> struct Shape<kModeRows> { static constexpr int threads = 256, unroll = 8, min_ctas = 3; };
+template <> struct Shape<kModeAny> { static constexpr int threads = 256, unroll = 4, min_ctas = 2; };
 
 template <int NPTR>
 struct Params {
@@ -62,7 +73,7 @@ template <> struct VecOf<0> { using type = uint8_t; };
 // Copy rows [row0, row0 + nrows) of one outer index of descriptor d; src / dst point at row 0.
 // A thread's vectors are kThreads vectors apart, so a warp always covers 32 consecutive
 // vectors of the tile's row space: whole aligned segments on both sides.
-template <int LOGV, int U>
+template <int LOGV, int U, int kThreads>
 __device__ __forceinline__ void copy_rows(const Desc &d, const char *src, char *dst, uint32_t row0, uint32_t nrows)
 {
     using V = typename VecOf<LOGV>::type;
@@ -96,7 +107,7 @@ __device__ __forceinline__ void copy_rows(const Desc &d, const char *src, char *
 }
 
 // One contiguous run of 16-byte vectors: no row decoding at all.
-template <int U>
+template <int U, int kThreads>
 __device__ __forceinline__ void copy_run16(const char *src, char *dst, uint32_t nbytes)
 {
 #pragma unroll 1
@@ -111,18 +122,10 @@ __device__ __forceinline__ void copy_run16(const char *src, char *dst, uint32_t 
     }
 }
 
-// Three builds of the executor, chosen per group on the host, so that the common cases do not
-// pay registers for the rare ones:
-//   kModeRun   every tile is one 16-byte-aligned contiguous run (same-layout KV blocks, whole
-//              tensors, dim-0 slabs): no row decoding
-//   kModeRows  every access is 16-byte aligned, tiles hold strided rows (layout transforms,
-//              dim-1 slices)
-//   kModeAny   some descriptor or base pointer is less aligned: width picked per tile
-enum { kModeRun = 0, kModeRows = 1, kModeAny = 2 };
-
 template <int NPTR, int MODE>
-__global__ void __launch_bounds__(kThreads, MODE == kModeAny ? 2 : kMinCtasPerSm) tc_copy_kernel(const __grid_constant__ Params<NPTR> prm)
+__global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) tc_copy_kernel(const __grid_constant__ Params<NPTR> prm)
 {
+    constexpr int kThreads = Shape<MODE>::threads, kUnroll = Shape<MODE>::unroll;
     __shared__ Desc sdesc[2];
     int buf = 0;
     for (uint32_t tile = blockIdx.x; tile < prm.n_tiles; tile += gridDim.x, buf ^= 1) {
@@ -147,16 +150,16 @@ __global__ void __launch_bounds__(kThreads, MODE == kModeAny ? 2 : kMinCtasPerSm
         char *dst = prm.ptr[d.dst_slot + o * d.dst_slot_step] + d.dst_off + o * d.dst_outer;
         if (MODE == kModeRun) {
             const uint32_t i1 = fastdiv(row0, d.div_n0), i0 = row0 - i1 * d.n0;
-            copy_run16<kUnrollWide>(src + (i1 * d.src_s1 + i0 * d.src_s0), dst + (i1 * d.dst_s1 + i0 * d.dst_s0), d.run);
+            copy_run16<kUnroll, kThreads>(src + (i1 * d.src_s1 + i0 * d.src_s0), dst + (i1 * d.dst_s1 + i0 * d.dst_s0), d.run);
         } else if (MODE == kModeRows) {
-            copy_rows<4, kUnrollWide>(d, src, dst, row0, nrows);
+            copy_rows<4, kUnroll, kThreads>(d, src, dst, row0, nrows);
         } else {
             switch (min(d.log2_align, prm.log2_ptr_align)) {
-            case 4: copy_rows<4, kUnrollNarrow>(d, src, dst, row0, nrows); break;
-            case 3: copy_rows<3, kUnrollNarrow>(d, src, dst, row0, nrows); break;
-            case 2: copy_rows<2, kUnrollNarrow>(d, src, dst, row0, nrows); break;
-            case 1: copy_rows<1, kUnrollNarrow>(d, src, dst, row0, nrows); break;
-            default: copy_rows<0, kUnrollNarrow>(d, src, dst, row0, nrows); break;
+            case 4: copy_rows<4, kUnroll, kThreads>(d, src, dst, row0, nrows); break;
+            case 3: copy_rows<3, kUnroll, kThreads>(d, src, dst, row0, nrows); break;
+            case 2: copy_rows<2, kUnroll, kThreads>(d, src, dst, row0, nrows); break;
+            case 1: copy_rows<1, kUnroll, kThreads>(d, src, dst, row0, nrows); break;
+            default: copy_rows<0, kUnroll, kThreads>(d, src, dst, row0, nrows); break;
             }
         }
     }
@@ -206,7 +209,7 @@ template <int NPTR, int MODE>
 static int resident_ctas()
 {
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, tc_copy_kernel<NPTR, MODE>, kThreads, 0) != cudaSuccess || n < 1) n = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, tc_copy_kernel<NPTR, MODE>, Shape<MODE>::threads, 0) != cudaSuccess || n < 1) n = 1;
     return n;
 }
 
@@ -227,11 +230,18 @@ static void resident_ctas_for(size_t n_ptrs, int out[3])
 
 static uint32_t grid_for(const tc_plan *plan, const Group &g, int mode)
 {
-    int per_sm = g.resident_ctas[mode] > 0 ? g.resident_ctas[mode] : 1;
-    if (plan->tuning.ctas_per_sm > 0) per_sm = std::min(per_sm, plan->tuning.ctas_per_sm);
-    uint64_t grid = static_cast<uint64_t>(plan->sm_count > 0 ? plan->sm_count : 148) * per_sm;
+    // Default: one CTA per tile.  The hardware block scheduler then balances the tiles over the
+    // SMs and de-phases the CTAs' load and store bursts, which measured faster than a
+    // persistent grid-stride grid.  tuning.ctas_per_sm / max_ctas select a persistent grid
+    // (few CTAs suit transfers over the host link).
+    uint64_t grid = std::min<uint64_t>(g.n_tiles, 0x7fffffffull);
+    if (plan->tuning.ctas_per_sm > 0) {
+        int per_sm = g.resident_ctas[mode] > 0 ? g.resident_ctas[mode] : 1;
+        per_sm = std::min(per_sm, plan->tuning.ctas_per_sm);
+        grid = std::min<uint64_t>(grid, static_cast<uint64_t>(plan->sm_count > 0 ? plan->sm_count : 148) * per_sm);
+    }
     if (plan->tuning.max_ctas > 0) grid = std::min<uint64_t>(grid, plan->tuning.max_ctas);
-    return static_cast<uint32_t>(std::min<uint64_t>(grid, g.n_tiles));
+    return static_cast<uint32_t>(grid);
 }
 
 template <int NPTR>
@@ -250,9 +260,9 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     for (size_t i = 0; i < g.n_dst; i++) prm.ptr[g.n_src + i] = static_cast<char *>(dst[i]);
     for (size_t i = g.n_src + g.n_dst; i < NPTR; i++) prm.ptr[i] = nullptr;
     switch (mode) {
-    case kModeRun: tc_copy_kernel<NPTR, kModeRun><<<grid, kThreads, 0, stream>>>(prm); break;
-    case kModeRows: tc_copy_kernel<NPTR, kModeRows><<<grid, kThreads, 0, stream>>>(prm); break;
-    default: tc_copy_kernel<NPTR, kModeAny><<<grid, kThreads, 0, stream>>>(prm); break;
+    case kModeRun: tc_copy_kernel<NPTR, kModeRun><<<grid, Shape<kModeRun>::threads, 0, stream>>>(prm); break;
+    case kModeRows: tc_copy_kernel<NPTR, kModeRows><<<grid, Shape<kModeRows>::threads, 0, stream>>>(prm); break;
+    default: tc_copy_kernel<NPTR, kModeAny><<<grid, Shape<kModeAny>::threads, 0, stream>>>(prm); break;
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
