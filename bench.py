@@ -190,6 +190,68 @@ WORKLOAD_NAME = ("configs[1] Llama-3-8B KV offload/reload (20000-block NHD pool,
 # --------------------------------------------------------------------------------------
 # the CUDA arm
 # --------------------------------------------------------------------------------------
+class Ranks:
+    """One process per GPU, replicas only: torch.distributed serves the barrier around the timed
+    region and the max-over-ranks of the device time; no data-path collective exists."""
+
+    def __init__(self, backend: str):
+        import torch.distributed as dist
+        self.dist = dist
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        self.backend = backend
+        if self.world > 1:
+            kw = {}
+            if backend == "nccl":
+                import torch
+                kw["device_id"] = torch.device("cuda", self.local)
+            dist.init_process_group(backend, **kw)
+
+    def barrier(self):
+        if self.backend == "nccl":
+            import torch
+            torch.cuda.synchronize()
+        if self.world > 1:
+            self.dist.barrier()
+            if self.backend == "nccl":
+                import torch
+                torch.cuda.synchronize()
+
+    def max_ms(self, ms: float) -> float:
+        if self.world == 1:
+            return ms
+        import torch
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda" if self.backend == "nccl" else "cpu")
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def throughput(self, bytes_per_rank_per_step: int, steps: int, ms: float) -> float:
+        """Whole-job GB/s: every rank moved the same bytes; the job took the slowest rank's time."""
+        return self.world * bytes_per_rank_per_step * steps / (self.max_ms(ms) * 1e-3) / GB
+
+    def close(self):
+        if self.world > 1:
+            self.dist.destroy_process_group()
+
+
+def run_dry(args):
+    """`--dry-run`: no GPU work; exercises the multi-rank plumbing (rendezvous, barrier,
+    max over ranks, whole-job aggregation) with a made-up per-rank time, for CPU tests."""
+    ranks = Ranks("gloo")
+    ranks.barrier()
+    ms = 100.0 + 50.0 * ranks.rank
+    step_bytes = 10 ** 9
+    value = ranks.throughput(step_bytes, args.steps, ms * args.steps)
+    ranks.barrier()
+    if ranks.rank == 0:
+        print(json.dumps({"metric": "kv_pack_unpack_and_weight_materialise_GBps", "value": value, "unit": "GB/s",
+                          "n_gpus": ranks.world, "steps": args.steps, "warmup": args.warmup, "scaling": "weak",
+                          "ms_per_step": ranks.max_ms(ms) if ranks.world == 1 else 100.0 + 50.0 * (ranks.world - 1),
+                          "dry_run": True}))
+    ranks.close()
+
+
 class Row:
     def __init__(self, name, mode):
         self.name, self.mode = name, mode
@@ -200,16 +262,12 @@ class Row:
 
 def run_ours(args):
     import torch
-    import torch.distributed as dist
 
     import paper_2608_06007_b200 as tc
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    ranks = Ranks("nccl")
+    world, rank, local = ranks.world, ranks.rank, ranks.local
     tc.load_library()
     free, total = torch.cuda.mem_get_info()
     shape = wl.LLAMA3_8B_KV
@@ -252,6 +310,7 @@ def run_ours(args):
     host_tune = dict(tune)
     if args.host_ctas:
         host_tune["max_ctas"] = args.host_ctas
+    host_flags = 0 if args.host_path == "zerocopy" else tc.TC_PLAN_STAGED
     t_plan0 = time.perf_counter()
     plans = []
     for src, dst in waves:
@@ -260,8 +319,8 @@ def run_ours(args):
             pack=tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, packed_bytes=Q.numel(), bt_src=src.bt, tuning=tune or None, **kw)),
             unpack=tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, packed_bytes=Q.numel(), bt_dst=dst.bt, tuning=tune or None, **kw)),
             migrate=tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, s, src_pool=plA, dst_pool=plB, bt_src=src.bt, bt_dst=dst.bt, tuning=tune or None, **kw)),
-            pack_h=tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, packed_bytes=Q.numel(), bt_src=src.bt, tuning=host_tune or None, **kw)),
-            unpack_h=tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, packed_bytes=Q.numel(), bt_dst=dst.bt, tuning=host_tune or None, **kw)),
+            pack_h=tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, packed_bytes=Q.numel(), bt_src=src.bt, tuning=host_tune or None, flags=host_flags, **kw)),
+            unpack_h=tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, packed_bytes=Q.numel(), bt_dst=dst.bt, tuning=host_tune or None, flags=host_flags, **kw)),
             payload=int(src.T.sum()) * shape.token_bytes))
     nbytes = [ck.nbytes(i) for i in range(ck.N)]
     mk_w = lambda tn, **kw: tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total, tuning=tn or None, **kw))
@@ -294,11 +353,7 @@ def run_ours(args):
         timed(rows["a4_weights_full"], lambda: tc.tc_weights_materialize(w_full, blob, full_ptrs, sp), 2 * sum(full_sizes), ev)
         timed(rows["a5_weights_shard"], lambda: tc.tc_weights_materialize(w_shard, blob, shard_ptrs, sp), 2 * sum(shard_sizes), ev)
 
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
+    barrier = ranks.barrier
 
     with torch.cuda.stream(stream):
         for _ in range(args.warmup):
@@ -326,10 +381,8 @@ def run_ours(args):
             rows[k].ms.append(v)
     step_bytes = sum(r.bytes for r in rows.values())
     launches_per_step = sum(r.launches for r in rows.values())
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    e2e_launches = sum(p["pack_h"].stats().launches_per_execute + p["unpack_h"].stats().launches_per_execute for p in plans) + 2
+    total_ms = ranks.max_ms(total_ms)
     value = world * step_bytes * args.steps / (total_ms * 1e-3) / GB
 
     # ---------------- e2e: packed buffer and blob in pinned host memory --------------------
@@ -340,6 +393,22 @@ def run_ours(args):
         blob_h.copy_(blob)
         probe = torch.empty(4096, dtype=torch.uint8).pin_memory()
         torch.cuda.synchronize()
+
+        def ceiling(fn, nbytes):  # cudaMemcpyAsync on the same pinned allocation, best of 3
+            best = 1e9
+            for _ in range(4):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                torch.cuda.synchronize()
+                best = min(best, a.elapsed_time(b))
+            return nbytes / (best * 1e-3) / GB
+
+        with torch.cuda.stream(stream):
+            n_c = min(Qh.numel(), 4 << 30)
+            ceil_h2d = ceiling(lambda: Q[:n_c].copy_(Qh[:n_c], non_blocking=True), n_c)
+            ceil_d2h = ceiling(lambda: Qh[:n_c].copy_(Q[:n_c], non_blocking=True), n_c)
 
         def e2e_step():
             h2d = d2h = 0
@@ -366,21 +435,21 @@ def run_ours(args):
             b.record(stream)
             barrier()
         e_ms = a.elapsed_time(b)
-        if world > 1:
-            t = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+        e_ms = ranks.max_ms(e_ms)
         # same byte convention as `value`: every payload byte is read once and written once
         e2e = {"value": world * 2 * (h2d + d2h - 4096) * args.e2e_steps / (e_ms * 1e-3) / GB, "unit": "GB/s",
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
                "ms_per_step": e_ms / args.e2e_steps,
                "host_link_GBps": world * (h2d + d2h) * args.e2e_steps / (e_ms * 1e-3) / GB,
-               "note": "packed KV buffer and weight blob in pinned host memory; kernels load/store host memory directly"}
+               "host_link_ceiling_GBps": {"h2d_cudaMemcpyAsync": ceil_h2d, "d2h_cudaMemcpyAsync": ceil_d2h},
+               "host_link_frac_of_ceiling": (h2d + d2h) * args.e2e_steps / (e_ms * 1e-3) / GB / ((h2d + d2h) / (h2d / ceil_h2d + d2h / ceil_d2h)),
+               "kv_host_path": args.host_path,
+               "note": "packed KV buffer and weight blob in pinned host memory; KV: copy engines + device staging ring + D2D kernel "
+                       "(staged) or kernel loads/stores on host memory (zerocopy); weights: kernel loads from the pinned blob"}
         del Qh, blob_h
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        ranks.close()
         return
 
     peak, peak_src = measured_peaks()
@@ -401,7 +470,8 @@ def run_ours(args):
     achieved = d["bytes"] / (d["ms"] * 1e-3) / GB
     roofline = {"bound": "hbm", "kernel": f"tc_copy_kernel<{'kModeRows' if dom == 'rows' else 'kModeRun'}>",
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "peak_source": peak_src, "traffic": TRAFFIC_PER_LAUNCH.get(dom),
+                "peak_source": peak_src, "traffic": traffic_per_launch(d["bytes"] / d["launches"]),
+                "traffic_source": "ncu dram bytes of a small case (profiles/), reads scaled by units, writes = payload minus the L2-resident tail",
                 "algorithmic_bytes_per_launch": d["bytes"] / d["launches"], "avg_launch_ms": d["ms"] / d["launches"],
                 "frac_of_nominal_8TBps": achieved / 8000.0}
 
@@ -422,16 +492,20 @@ def run_ours(args):
                    "bytes_per_step": step_bytes, "l2": "every launch moves far more than the 126 MB L2; no flush needed",
                    "parallelism": "replicas only" if world > 1 else "1 GPU", "plans": n_plans, "plan_create_ms_total": plan_ms},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "e2e_gpu_launches_per_step": e2e_launches,
         "roofline": roofline, "rows": per_row,
         "cpu_baseline": {"value": cpu_v, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": cpu_desc},
     }
     print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    ranks.close()
 
 
-# dram bytes per launch of each executor build from the ncu capture summarised under profiles/
-TRAFFIC_PER_LAUNCH = {"rows": None, "run": None}
+def traffic_per_launch(algorithmic_bytes: float) -> float:
+    """DRAM bytes of one full-size launch, scaled from the ncu capture of a small case
+    (profiles/tc_copy_kernel_small_case_full_set.md): reads = 1.0002 x payload (descriptors
+    included); writes = payload less the ~50 MB of dirty lines still in L2 at kernel end."""
+    payload = algorithmic_bytes / 2
+    return 1.0002 * payload + max(payload - 50.7e6, 0.0)
 
 
 def main():
@@ -446,6 +520,7 @@ def main():
     ap.add_argument("--max-waves", type=int, default=0)
     ap.add_argument("--shard-rank", type=int, default=0)
     ap.add_argument("--small", action="store_true", help="small case for profiler captures")
+    ap.add_argument("--dry-run", action="store_true", help="CPU-only check of the multi-rank plumbing (gloo)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiler runs)")
     ap.add_argument("--e2e-steps", type=int, default=1)
@@ -454,8 +529,11 @@ def main():
     ap.add_argument("--tile-bytes", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--host-ctas", type=int, default=0)
+    ap.add_argument("--host-path", default="staged", choices=["staged", "zerocopy"])
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.dry_run:
+        run_dry(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

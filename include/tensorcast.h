@@ -100,9 +100,23 @@ typedef enum {
 typedef enum { TC_NHD = 0, TC_HND = 1 } tc_layout;
 
 enum {
-    TC_PLAN_HOST_ONLY = 1u /* validate and lower on the host only: the plan can be inspected
-                              (tc_plan_stats, tc_plan_descriptors) but not executed, and no
-                              CUDA call is made */
+    TC_PLAN_HOST_ONLY = 1u, /* validate and lower on the host only: the plan can be inspected
+                               (tc_plan_stats, tc_plan_descriptors) but not executed, and no
+                               CUDA call is made */
+    TC_PLAN_STAGED = 2u     /* TC_KV_PACK / TC_KV_UNPACK whose packed buffer is PINNED HOST memory:
+                               instead of letting the kernel load / store host memory directly
+                               (zero copy, the default), move the packed bytes with the copy
+                               engines through a ring of device staging buffers owned by the
+                               library (3 x 64 MiB per device, shared by all staged plans,
+                               allocated when the first such plan is created) and run the kernel
+                               device to device, segment by segment, overlapped on an internal
+                               stream.  This is the streaming pipeline of pinned buffers and
+                               asynchronous streams (Sec. 5) with the scatter / layout
+                               transform fused into its device leg.  The copy engines drive the
+                               host link with larger transactions than SM loads and stores, so
+                               this path is a few percent faster; it costs one launch and one
+                               copy per segment instead of one launch per call.  Staged
+                               executions are serialised with one another by the library. */
 };
 
 #define TC_MAX_TABLE_SLOTS 4000 /* src slots + dst slots of one execute call */
@@ -284,8 +298,10 @@ typedef struct {
     int64_t packed_bytes_required; /* PACK / UNPACK: sum of L*2*T_r*H*D*E */
     int64_t device_bytes;          /* plan storage held on the device */
     int32_t vec_bytes[2];          /* widest access the geometry allows (pointers may narrow it) */
-    int32_t launches_per_execute;  /* kernels one execute call launches (1; 0 if empty) */
-    int32_t path[2];               /* 1 register path, 2 bulk-copy path */
+    int32_t launches_per_execute;  /* kernels one execute call launches (1; one per segment for
+                                      staged plans) */
+    int32_t path[2];               /* 1 direct (zero copy when a buffer is host memory),
+                                      3 staged through the copy engines */
     int32_t grid[2];               /* CTAs launched per execution */
 } tc_plan_stats_t;
 

@@ -21,6 +21,7 @@ TC_NOALLOC_SCRATCH_BYTES = 1 << 20
 TC_KV_PACK, TC_KV_UNPACK, TC_KV_MIGRATE, TC_KV_MIXED, TC_WEIGHTS = 1, 2, 3, 4, 5
 TC_NHD, TC_HND = 0, 1
 TC_PLAN_HOST_ONLY = 1
+TC_PLAN_STAGED = 2
 TC_MAX_TABLE_SLOTS = 4000
 
 

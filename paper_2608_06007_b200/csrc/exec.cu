@@ -44,6 +44,9 @@ struct Params {
     uint32_t tiles_per_desc;    // > 0 for uniform groups
     FastDiv div_tpd;
     uint32_t log2_ptr_align;    // alignment shared by every base pointer (capped at 4)
+    // launch window (win_span == 0: the whole group).  Tile ids then walk plane-major over
+    // descriptors [win_d0, ...) x planes [win_o0, ...): win_span = descriptors x win_tpo.
+    uint32_t win_span, win_d0, win_o0, win_tpo;
     char *ptr[NPTR];            // src table then dst table
 };
 
@@ -130,7 +133,12 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
     int buf = 0;
     for (uint32_t tile = blockIdx.x; tile < prm.n_tiles; tile += gridDim.x, buf ^= 1) {
         uint32_t di, t = 0;
-        if (prm.tiles_per_desc) {
+        if (prm.win_span) {
+            const uint32_t ow = tile / prm.win_span, rem = tile - ow * prm.win_span;
+            const uint32_t dw = rem / prm.win_tpo;
+            di = prm.win_d0 + dw;
+            t = (prm.win_o0 + ow) * prm.win_tpo + (rem - dw * prm.win_tpo);
+        } else if (prm.tiles_per_desc) {
             di = fastdiv(tile, prm.div_tpd);
             t = tile - di * prm.tiles_per_desc;
         } else {
@@ -140,7 +148,7 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
             reinterpret_cast<uint4 *>(&sdesc[buf])[threadIdx.x] = __ldg(reinterpret_cast<const uint4 *>(prm.descs + di) + threadIdx.x);
         __syncthreads();
         const Desc &d = sdesc[buf];
-        if (!prm.tiles_per_desc) t = tile - d.tile0;
+        if (!prm.tiles_per_desc && !prm.win_span) t = tile - d.tile0;
         const uint32_t o = fastdiv(t, d.div_tpo);
         const uint32_t part = t - o * d.tiles_per_outer;
         const uint32_t row0 = part * d.rows_per_tile;
@@ -228,13 +236,14 @@ static void resident_ctas_for(size_t n_ptrs, int out[3])
     else resident_ctas_all<TC_MAX_TABLE_SLOTS>(out);
 }
 
-static uint32_t grid_for(const tc_plan *plan, const Group &g, int mode)
+static uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *win = nullptr)
 {
     // Default: one CTA per tile.  The hardware block scheduler then balances the tiles over the
     // SMs and de-phases the CTAs' load and store bursts, which measured faster than a
     // persistent grid-stride grid.  tuning.ctas_per_sm / max_ctas select a persistent grid
     // (few CTAs suit transfers over the host link).
     uint64_t grid = std::min<uint64_t>(g.n_tiles, 0x7fffffffull);
+    if (win) grid = static_cast<uint64_t>(win->no) * win->nd * (g.tiles_per_desc / g.descs[0].n_outer);
     if (plan->tuning.ctas_per_sm > 0) {
         int per_sm = g.resident_ctas[mode] > 0 ? g.resident_ctas[mode] : 1;
         per_sm = std::min(per_sm, plan->tuning.ctas_per_sm);
@@ -245,14 +254,23 @@ static uint32_t grid_for(const tc_plan *plan, const Group &g, int mode)
 }
 
 template <int NPTR>
-static int launch(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t stream)
+static int launch(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t stream,
+                  const Segment *win = nullptr)
 {
     const int mode = mode_for(g, ptr_align);
-    const uint32_t grid = grid_for(plan, g, mode);
+    const uint32_t grid = grid_for(plan, g, mode, win);
     Params<NPTR> prm;
     prm.descs = g.d_descs;
     prm.tile_desc = g.d_tile_desc;
     prm.n_tiles = static_cast<uint32_t>(g.n_tiles);
+    prm.win_span = prm.win_d0 = prm.win_o0 = prm.win_tpo = 0;
+    if (win) {
+        prm.win_tpo = g.tiles_per_desc / g.descs[0].n_outer;
+        prm.win_span = win->nd * prm.win_tpo;
+        prm.win_d0 = win->d0;
+        prm.win_o0 = win->o0;
+        prm.n_tiles = win->no * prm.win_span;
+    }
     prm.tiles_per_desc = g.tiles_per_desc;
     prm.div_tpd = g.div_tpd;
     prm.log2_ptr_align = ptr_align;
@@ -268,6 +286,129 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
     return TC_OK;
 }
+
+static int launch_any(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s, const Segment *win)
+{
+    const size_t n = g.n_src + g.n_dst;
+    if (n <= 8) return launch<8>(plan, g, src, dst, ptr_align, s, win);
+    if (n <= 400) return launch<400>(plan, g, src, dst, ptr_align, s, win);
+    return launch<TC_MAX_TABLE_SLOTS>(plan, g, src, dst, ptr_align, s, win);
+}
+
+// ---- staged host path: copy engines <-> device staging ring <-> kernel ----------------------
+constexpr int kMaxDevices = 64;
+struct StageArena {
+    char *buf[kStageBuffers] = {};
+    cudaEvent_t ready[kStageBuffers] = {}, freed[kStageBuffers] = {}, entry = nullptr;
+    bool freed_recorded[kStageBuffers] = {};
+    cudaStream_t copy = nullptr;
+    uint64_t next = 0;
+    int refs = 0;
+};
+static StageArena g_stage[kMaxDevices];
+static pthread_mutex_t g_stage_mu = PTHREAD_MUTEX_INITIALIZER;
+
+static void stage_free(StageArena &a)
+{
+    for (int b = 0; b < kStageBuffers; b++) {
+        if (a.buf[b]) cudaFree(a.buf[b]);
+        if (a.ready[b]) cudaEventDestroy(a.ready[b]);
+        if (a.freed[b]) cudaEventDestroy(a.freed[b]);
+    }
+    if (a.entry) cudaEventDestroy(a.entry);
+    if (a.copy) cudaStreamDestroy(a.copy);
+    a = StageArena();
+}
+
+static int stage_acquire(int device, int64_t *bytes)
+{
+    if (device < 0 || device >= kMaxDevices) return fail(TC_ERR_INVALID_ARG, "device ordinal %d is not supported", device);
+    pthread_mutex_lock(&g_stage_mu);
+    StageArena &a = g_stage[device];
+    int rc = TC_OK;
+    if (a.refs == 0) {
+        cudaError_t e = cudaStreamCreateWithFlags(&a.copy, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&a.entry, cudaEventDisableTiming);
+        for (int b = 0; b < kStageBuffers && e == cudaSuccess; b++) {
+            e = cudaMalloc(&a.buf[b], kStageBytes);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&a.ready[b], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&a.freed[b], cudaEventDisableTiming);
+        }
+        if (e != cudaSuccess) {
+            rc = e == cudaErrorMemoryAllocation ? fail(TC_ERR_OOM, "device allocation of the staging ring failed") : cuda_fail(e, "creating the staging ring");
+            stage_free(a);
+        }
+    }
+    if (rc == TC_OK) {
+        a.refs++;
+        *bytes = kStageBytes * kStageBuffers;
+    }
+    pthread_mutex_unlock(&g_stage_mu);
+    return rc;
+}
+
+static void stage_release(int device)
+{
+    if (device < 0 || device >= kMaxDevices) return;
+    pthread_mutex_lock(&g_stage_mu);
+    StageArena &a = g_stage[device];
+    if (a.refs > 0 && --a.refs == 0) {
+        cudaStreamSynchronize(a.copy);
+        stage_free(a);
+    }
+    pthread_mutex_unlock(&g_stage_mu);
+}
+
+#define TC_TRY(call, what)                                   \
+    do {                                                     \
+        cudaError_t e_ = (call);                             \
+        if (e_ != cudaSuccess) { rc = cuda_fail(e_, what); goto out; } \
+    } while (0)
+
+// gi == 0: pack, device pool -> staging (kernel, caller's stream) -> host (copy engine).
+// gi == 1: unpack, host -> staging (copy engine) -> device pool (kernel, caller's stream).
+// Every segment's kernel sees the staging buffer through a base pointer shifted by the
+// segment's packed offset, so the descriptors are used unchanged.
+static int execute_staged(const tc_plan *plan, int gi, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s)
+{
+    StageArena &a = g_stage[plan->device];
+    int rc = TC_OK;
+    pthread_mutex_lock(&g_stage_mu);
+    TC_TRY(cudaEventRecord(a.entry, s), "cudaEventRecord");
+    TC_TRY(cudaStreamWaitEvent(a.copy, a.entry, 0), "cudaStreamWaitEvent");
+    for (const Segment &seg : g.segments) {
+        const int b = static_cast<int>(a.next++ % kStageBuffers);
+        char *shifted = a.buf[b] - seg.lo;
+        const uint32_t pa = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(shifted) | 16));
+        if (gi == 1) {
+            const char *host = static_cast<const char *>(src[0]);
+            if (a.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(a.copy, a.freed[b], 0), "cudaStreamWaitEvent");
+            TC_TRY(cudaMemcpyAsync(a.buf[b], host + seg.lo, static_cast<size_t>(seg.bytes), cudaMemcpyHostToDevice, a.copy), "cudaMemcpyAsync(host to staging)");
+            TC_TRY(cudaEventRecord(a.ready[b], a.copy), "cudaEventRecord");
+            TC_TRY(cudaStreamWaitEvent(s, a.ready[b], 0), "cudaStreamWaitEvent");
+            const void *stage_src[1] = {shifted};
+            if ((rc = launch_any(plan, g, stage_src, dst, pa, s, &seg)) != TC_OK) goto out;
+            TC_TRY(cudaEventRecord(a.freed[b], s), "cudaEventRecord");
+        } else {
+            char *host = static_cast<char *>(dst[0]);
+            if (a.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(s, a.freed[b], 0), "cudaStreamWaitEvent");
+            void *stage_dst[1] = {shifted};
+            if ((rc = launch_any(plan, g, src, stage_dst, pa, s, &seg)) != TC_OK) goto out;
+            TC_TRY(cudaEventRecord(a.ready[b], s), "cudaEventRecord");
+            TC_TRY(cudaStreamWaitEvent(a.copy, a.ready[b], 0), "cudaStreamWaitEvent");
+            TC_TRY(cudaMemcpyAsync(host + seg.lo, a.buf[b], static_cast<size_t>(seg.bytes), cudaMemcpyDeviceToHost, a.copy), "cudaMemcpyAsync(staging to host)");
+            TC_TRY(cudaEventRecord(a.freed[b], a.copy), "cudaEventRecord");
+        }
+        a.freed_recorded[b] = true;
+    }
+    if (gi == 0)  // the caller's stream completes only when the last copies to the host have landed
+        for (int b = 0; b < kStageBuffers; b++)
+            if (a.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(s, a.freed[b], 0), "cudaStreamWaitEvent");
+out:
+    pthread_mutex_unlock(&g_stage_mu);
+    return rc;
+}
+#undef TC_TRY
 
 static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n_src, void *const *dst, size_t n_dst, void *stream)
 {
@@ -290,10 +431,8 @@ static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n
         ptr_align = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(dst[i]) | 16));
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const size_t n = n_src + n_dst;
-    if (n <= 8) return launch<8>(plan, g, src, dst, ptr_align, s);
-    if (n <= 400) return launch<400>(plan, g, src, dst, ptr_align, s);
-    return launch<TC_MAX_TABLE_SLOTS>(plan, g, src, dst, ptr_align, s);
+    if (!g.segments.empty()) return execute_staged(plan, gi, g, src, dst, ptr_align, s);
+    return launch_any(plan, g, src, dst, ptr_align, s, nullptr);
 }
 
 }  // namespace tc
@@ -325,6 +464,13 @@ extern "C" int tc_plan_create(const tc_plan_spec_t *spec, tc_plan_t **out)
         cudaError_t e = cudaGetDevice(&plan->device);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&plan->sm_count, cudaDevAttrMultiProcessorCount, plan->device);
         if (e != cudaSuccess) rc = cuda_fail(e, "querying the current device");
+        if (rc == TC_OK && (!plan->group[0].segments.empty() || !plan->group[1].segments.empty())) {
+            int64_t arena = 0;
+            if ((rc = stage_acquire(plan->device, &arena)) == TC_OK) {
+                plan->staged = true;
+                plan->device_bytes += arena;
+            }
+        }
         for (int k = 0; k < 2 && rc == TC_OK; k++) {
             rc = upload_group(plan, plan->group[k]);
             if (plan->group[k].n_tiles) resident_ctas_for(plan->group[k].n_src + plan->group[k].n_dst, plan->group[k].resident_ctas);
@@ -333,6 +479,7 @@ extern "C" int tc_plan_create(const tc_plan_spec_t *spec, tc_plan_t **out)
     if (rc != TC_OK) {
         free_group(plan->group[0]);
         free_group(plan->group[1]);
+        if (plan->staged) stage_release(plan->device);
         delete plan;
         return rc;
     }
@@ -345,6 +492,7 @@ extern "C" int tc_plan_destroy(tc_plan_t *plan)
     if (!plan) return TC_OK;
     free_group(plan->group[0]);
     free_group(plan->group[1]);
+    if (plan->staged) stage_release(plan->device);
     delete plan;
     return TC_OK;
 }
@@ -391,12 +539,13 @@ extern "C" int tc_plan_stats(const tc_plan_t *plan, tc_plan_stats_t *out)
         out->n_tiles[k] = static_cast<int64_t>(g.n_tiles);
         out->payload_bytes[k] = g.payload;
         out->vec_bytes[k] = 1 << g.log2_align;
-        out->path[k] = g.n_tiles ? 1 : 0;
+        out->path[k] = g.n_tiles ? (g.segments.empty() ? 1 : 3) : 0;
+        if (!g.segments.empty()) out->launches_per_execute = static_cast<int32_t>(g.segments.size());
         out->grid[k] = g.n_tiles ? static_cast<int32_t>(grid_for(plan, g, mode_for(g, 4))) : 0;
     }
     out->packed_bytes_required = plan->packed_required;
     out->device_bytes = plan->device_bytes;
-    out->launches_per_execute = 1;
+    if (out->launches_per_execute == 0) out->launches_per_execute = 1;
     return TC_OK;
 }
 
@@ -427,7 +576,6 @@ extern "C" int tc_plan_descriptors(const tc_plan_t *plan, int group, tc_descript
 static __device__ __align__(256) unsigned char g_noalloc_scratch[TC_NOALLOC_SCRATCH_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 struct NoallocDevice {
     void *scratch = nullptr;  // device address of g_noalloc_scratch on this device
     int sm_count = 0;
@@ -464,6 +612,7 @@ extern "C" int tc_kv_pack_noalloc(const tc_plan_spec_t *spec, const void *const 
     if (spec->kind != TC_KV_PACK && spec->kind != TC_KV_MIGRATE && spec->kind != TC_KV_MIXED)
         return fail(TC_ERR_KIND, "tc_kv_pack_noalloc needs a PACK, MIGRATE or MIXED spec (kind %d given)", spec->kind);
     if (spec->deadline_ns && now_ns() > spec->deadline_ns) return fail(TC_ERR_DEADLINE, "deadline passed before the call");
+    if (spec->flags & TC_PLAN_STAGED) return fail(TC_ERR_INVALID_ARG, "tc_kv_pack_noalloc does not stage: the staging ring is allocated device memory");
     tc_plan plan;  // lives on the host for the duration of this call only
     plan.kind = spec->kind;
     plan.trace_id = spec->trace_id;

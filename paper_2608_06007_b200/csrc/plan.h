@@ -48,9 +48,24 @@ struct alignas(16) Desc {
 };
 static_assert(sizeof(Desc) == 128, "Desc must stay 128 bytes");
 
+// A launch window: descriptors [d0, d0+nd) x planes [o0, o0+no), walked plane-major.
+// A segment of a staged plan is a window whose packed-side bytes are one contiguous range.
+struct Segment {
+    uint32_t d0, nd, o0, no;
+    int64_t lo, bytes;  // the packed-buffer byte range the window touches
+};
+
+// Bookkeeping of one request while a KV group is lowered (staged plans cut segments from it).
+struct RequestSpan {
+    uint32_t d0, d1;      // its descriptors
+    int64_t off, plane_bytes;
+};
+
 struct Group {
     std::vector<Desc> descs;
     std::vector<uint32_t> tile_desc;  // tile -> descriptor, only for non-uniform groups
+    std::vector<RequestSpan> requests; // KV groups with a packed side
+    std::vector<Segment> segments;    // staged plans only
     uint32_t tiles_per_desc = 0;      // > 0: every descriptor owns exactly this many tile ids
     FastDiv div_tpd{0, 0};
     uint64_t n_tiles = 0;
@@ -76,6 +91,7 @@ struct tc_plan {
     int sm_count = 0;
     int64_t packed_required = 0;
     int64_t device_bytes = 0;
+    bool staged = false;  // holds a reference on the device's staging ring
     tc::Group group[2];
 };
 
@@ -90,6 +106,8 @@ void clear_error();
 int64_t now_ns();
 
 constexpr uint32_t kDefaultTileBytes = 32768;
+constexpr int64_t kStageBytes = 64ll << 20;  // one staging buffer
+constexpr int kStageBuffers = 3;
 constexpr uint32_t kMaxTileBytes = 1u << 20;
 
 }  // namespace tc

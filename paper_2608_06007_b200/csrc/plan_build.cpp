@@ -347,6 +347,7 @@ static void lower_kv_group(Group &g, const tc_kv_spec_t &kv, const tc_kv_group_t
     for (int64_t r = 0; r < grp.R; r++) {
         const int64_t Tr = grp.T[r];
         const int64_t plane_bytes = Tr * kv.H * row;  // one (l,c) plane of this request, packed
+        const uint32_t first_desc = static_cast<uint32_t>(g.descs.size());
         for (int64_t j = 0; j * kv.B < Tr; j++) {
             const int64_t nvalid = std::min(kv.B, Tr - j * kv.B);
             const int64_t jj = grp.bt_off[r] + j;
@@ -379,8 +380,43 @@ static void lower_kv_group(Group &g, const tc_kv_spec_t &kv, const tc_kv_group_t
             b.dims = {Dim{kv.H, ssh, dsh}, Dim{nvalid, ssn, dsn}};
             lower_box(g, b, tile_bytes);
         }
+        if (!src_pool || !dst_pool)
+            g.requests.push_back(RequestSpan{first_desc, static_cast<uint32_t>(g.descs.size()), off_r, plane_bytes});
         off_r += planes * plane_bytes;
     }
+}
+
+// Cut a staged group into segments: windows of descriptors x planes whose packed-side bytes
+// are one contiguous range of at most kStageBytes.  Runs of small consecutive requests share
+// a segment; a request larger than a staging buffer is cut at plane boundaries.
+static int build_segments(Group &g, int64_t planes)
+{
+    if (!g.tiles_per_desc) return TC_OK;  // non-uniform group: stays on the zero-copy path
+    for (const Desc &d : g.descs)
+        if (d.n_outer != planes) return TC_OK;
+    size_t i = 0;
+    while (i < g.requests.size()) {
+        const RequestSpan &q = g.requests[i];
+        const int64_t total = planes * q.plane_bytes;
+        if (total == 0) { i++; continue; }
+        if (total <= kStageBytes) {
+            int64_t sum = 0;
+            size_t j = i;
+            while (j < g.requests.size() && sum + planes * g.requests[j].plane_bytes <= kStageBytes) sum += planes * g.requests[j++].plane_bytes;
+            g.segments.push_back(Segment{q.d0, g.requests[j - 1].d1 - q.d0, 0, static_cast<uint32_t>(planes), q.off, sum});
+            i = j;
+        } else {
+            if (q.plane_bytes > kStageBytes)
+                return fail(TC_ERR_TOO_LARGE, "a staged plan needs every (layer, K|V) plane of a request to fit a %lld-byte staging buffer; one has %lld bytes", (long long)kStageBytes, (long long)q.plane_bytes);
+            const int64_t per = kStageBytes / q.plane_bytes;
+            for (int64_t o0 = 0; o0 < planes; o0 += per) {
+                const int64_t no = std::min(per, planes - o0);
+                g.segments.push_back(Segment{q.d0, q.d1 - q.d0, static_cast<uint32_t>(o0), static_cast<uint32_t>(no), q.off + o0 * q.plane_bytes, no * q.plane_bytes});
+            }
+            i++;
+        }
+    }
+    return TC_OK;
 }
 
 static int build_kv(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t tile_bytes)
@@ -584,6 +620,12 @@ int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
         // destination slots follow the source slots in the combined pointer table
         for (Desc &d : g.descs) d.dst_slot = static_cast<uint16_t>(d.dst_slot + g.n_src);
         if ((rc = finish_group(g))) return rc;
+    }
+    if (spec->flags & TC_PLAN_STAGED) {
+        if (spec->kind != TC_KV_PACK && spec->kind != TC_KV_UNPACK)
+            return fail(TC_ERR_KIND, "TC_PLAN_STAGED applies to TC_KV_PACK and TC_KV_UNPACK plans only");
+        Group &g = plan->group[spec->kind == TC_KV_PACK ? 0 : 1];
+        if ((rc = build_segments(g, spec->kv.L * 2))) return rc;
     }
     return TC_OK;
 }

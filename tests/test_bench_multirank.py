@@ -1,0 +1,43 @@
+"""The N>1 path of the benchmark on CPU: two gloo ranks go through the same rendezvous,
+barrier, max-over-ranks and whole-job aggregation code as the NCCL run (replicas only: the
+path has no exchange step, so there is nothing else to distribute)."""
+import json
+import os
+import socket
+import subprocess
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _run(nproc):
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={nproc}",
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port()),
+           os.path.join(ROOT, "bench.py"), "--gpus", str(nproc), "--steps", "4", "--warmup", "3", "--dry-run"]
+    out = subprocess.run(cmd, capture_output=True, text=True, timeout=240, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, out.stdout            # rank 0 alone prints the JSON line
+    return json.loads(lines[0])
+
+
+def test_two_gloo_ranks_aggregate_as_replicas():
+    j = _run(2)
+    assert j["n_gpus"] == 2 and j["scaling"] == "weak"
+    # ranks took 100 and 150 ms per step; the job is as slow as the slowest rank and moved 2x the bytes
+    assert abs(j["ms_per_step"] - 150.0) < 1e-9
+    assert abs(j["value"] - 2 * 1e9 / 0.150 / 1e9) < 1e-9
+
+
+def test_single_process_dry_run():
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--dry-run", "--steps", "2"],
+                         capture_output=True, text=True, timeout=120, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    j = json.loads(out.stdout.strip().splitlines()[-1])
+    assert j["n_gpus"] == 1 and abs(j["value"] - 1e9 / 0.100 / 1e9) < 1e-9

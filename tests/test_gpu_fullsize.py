@@ -97,7 +97,20 @@ def test_config2_full_size_pack_unpack_migrate():
     tc.tc_kv_pack(mig, [poolA], [poolC])
     torch.cuda.synchronize()
     assert torch.equal(poolC, poolB)
-    del poolA, poolB, poolC, Q, A, B
+    # staged host path at full size: offload to pinned host and reload must reproduce the
+    # (oracle-checked) direct results byte for byte
+    Qh = torch.empty(payload, dtype=torch.uint8).pin_memory()
+    pack_s = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, packed_bytes=payload, bt_src=src.bt, flags=tc.TC_PLAN_STAGED, **kw))
+    unpack_s = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, packed_bytes=payload, bt_dst=dst.bt, flags=tc.TC_PLAN_STAGED, **kw))
+    assert pack_s.stats().path[0] == 3 and pack_s.stats().launches_per_execute > 200
+    poolC.fill_(0xA5)
+    tc.tc_kv_pack(pack_s, [poolA], [Qh])
+    tc.tc_kv_unpack(unpack_s, [Qh], [poolC])
+    torch.cuda.synchronize()
+    for lo in range(0, payload, 1 << 30):
+        assert torch.equal(Qh[lo:lo + (1 << 30)].cuda(), Q[lo:lo + (1 << 30)])
+    assert torch.equal(poolC, poolB)
+    del poolA, poolB, poolC, Q, Qh, A, B
     _free()
 
 

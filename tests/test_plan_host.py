@@ -244,6 +244,25 @@ def test_long_runs_and_wide_spans_are_cut_for_32_bit_row_offsets():
     assert starts[0] == 1 << 30 and starts[-1] >= (6 << 30) + (1 << 30)
 
 
+def test_staged_plans_are_cut_into_contiguous_segments():
+    # L=4: 16 KiB per token.  Request 0 (5000 tokens, 80 MB) exceeds a 64 MiB staging buffer and
+    # is cut at plane boundaries (10 MB planes -> 6 + 2 planes); the small requests share one.
+    shape = (4, 16, 8, 128, 2)
+    T = np.array([5000, 37, 0, 100, 700], dtype=np.int64)
+    off = np.concatenate([[0], np.cumsum((T + 15) // 16)])
+    bt = np.arange(off[-1], dtype=np.int32)
+    pl = tc.pool(tc.TC_NHD, int(off[-1]), 1, plane_stride=int(off[-1]) * 16 * 8 * 128 * 2)
+    for kind, kw in ((tc.TC_KV_PACK, dict(src_pool=pl, bt_src=bt)), (tc.TC_KV_UNPACK, dict(dst_pool=pl, bt_dst=bt))):
+        st = tc.tc_plan_create(tc.kv_spec(kind, shape, packed_layout=tc.TC_HND, T=T, bt_off=off, flags=HOST | tc.TC_PLAN_STAGED, **kw)).stats()
+        g = 0 if kind == tc.TC_KV_PACK else 1
+        assert st.path[g] == 3 and st.launches_per_execute == 3
+        st = tc.tc_plan_create(tc.kv_spec(kind, shape, packed_layout=tc.TC_HND, T=T, bt_off=off, flags=HOST, **kw)).stats()
+        assert st.path[g] == 1 and st.launches_per_execute == 1
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl, T=T, bt_off=off, bt_src=bt, bt_dst=bt, flags=HOST | tc.TC_PLAN_STAGED))
+    assert e.value.status == tc.TC_ERR_KIND
+
+
 # --------------------------------------------------------------------------- validation
 def _pack_spec(**over):
     shape, NB, src, dst = wl.config1()
