@@ -448,6 +448,17 @@ def run_ours(args):
                        "(staged) or kernel loads/stores on host memory (zerocopy); weights: kernel loads from the pinned blob"}
         del Qh, blob_h
 
+    extras = None
+    if not args.no_extras and world == 1:
+        for p in plans:
+            for k in ("pack", "unpack", "migrate", "pack_h", "unpack_h"):
+                p[k].destroy()
+        for w in (w_full, w_shard, w_full_h, w_shard_h):
+            w.destroy()
+        del poolA, poolB, Q, blob, dst_full, dst_shard, plans
+        torch.cuda.empty_cache()
+        extras = run_extras(args, tc, torch, stream)
+
     if rank != 0:
         ranks.close()
         return
@@ -493,11 +504,94 @@ def run_ours(args):
                    "parallelism": "replicas only" if world > 1 else "1 GPU", "plans": n_plans, "plan_create_ms_total": plan_ms},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "e2e_gpu_launches_per_step": e2e_launches,
-        "roofline": roofline, "rows": per_row,
+        "roofline": roofline, "rows": per_row, "other_workloads": extras,
         "cpu_baseline": {"value": cpu_v, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": cpu_desc},
     }
     print(json.dumps(line))
     ranks.close()
+
+
+def run_extras(args, tc, torch, stream):
+    """Secondary workloads, reported beside the headline: configs[3] (70B-shaped pool-to-pool
+    migration, one wave) and configs[4] (prefix-reload burst: one mixed plan per scheduler step,
+    created and executed inside the timed region, both directions concurrently over the host
+    link with zero-copy kernels)."""
+    out = {}
+    sp = stream.cuda_stream
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    # ---- configs[3]
+    shape = wl.LLAMA3_70B_KV
+    free, _ = torch.cuda.mem_get_info()
+    NB = 4096
+    while 2 * NB * shape.block_bytes > 0.8 * free:
+        NB //= 2
+    _, _, _, waves = wl.config4(NB=NB, max_waves=1)
+    src, dst = waves[0]
+    A = torch.empty(NB * shape.block_bytes, **u8)
+    A.fill_(7)
+    B = torch.empty(NB * shape.block_bytes, **u8)
+    B.fill_(9)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=A.numel())
+    t0 = time.perf_counter()
+    mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape.tuple, src_pool=pl, dst_pool=pl, T=src.T, bt_off=src.bt_off, bt_src=src.bt, bt_dst=dst.bt))
+    create_ms = 1e3 * (time.perf_counter() - t0)
+    payload = int(src.T.sum()) * shape.token_bytes
+    ms = []
+    with torch.cuda.stream(stream):
+        for i in range(6):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            tc.tc_kv_pack(mig, [A], [B], sp)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                ms.append(a.elapsed_time(b))
+    out["configs[3] 70B KV migrate (one wave)"] = {
+        "pool_blocks": NB, "requests": len(src.T), "blocks": src.n_blocks, "payload_bytes": payload,
+        "GBps": 2 * payload / (statistics.mean(ms) * 1e-3) / GB, "ms": statistics.mean(ms), "plan_create_ms": create_ms}
+    mig.destroy()
+    del A, B
+    torch.cuda.empty_cache()
+    # ---- configs[4]
+    shape = wl.LLAMA3_8B_KV
+    NBd, NBh, n_steps = 20000, args.host_pool_blocks, args.burst_steps
+    dev = torch.empty(NBd * shape.block_bytes, **u8)
+    dev.fill_(3)
+    host = torch.empty(NBh * shape.block_bytes, dtype=torch.uint8).pin_memory()
+    dev_pool = tc.pool(tc.TC_NHD, NBd, 1, plane_stride=NBd * shape.chunk_bytes, slot_bytes=dev.numel())
+    host_pool = tc.pool(tc.TC_HND, NBh, 1, plane_stride=shape.chunk_bytes, block_stride=shape.block_bytes, slot_bytes=host.numel())
+    s2 = torch.cuda.Stream()
+    create, h2d, d2h = [], 0, 0
+    steps = list(wl.config5(NB_dev=NBd, NB_host=NBh, steps=n_steps + 1))
+    torch.cuda.synchronize()
+    t_all = None
+    for i, st in enumerate(steps):
+        if i == 1:  # step 0 is the warm-up
+            torch.cuda.synchronize()
+            t_all = time.perf_counter()
+        t0 = time.perf_counter()
+        plan = tc.tc_plan_create(tc.kv_spec(
+            tc.TC_KV_MIXED, shape.tuple, src_pool=dev_pool, dst_pool=host_pool,
+            T=st.offload_T, bt_off=st.offload_off, bt_src=st.offload_dev, bt_dst=st.offload_host,
+            reload=dict(T=st.reload_T, bt_off=st.reload_off, bt_src=st.reload_host, bt_dst=st.reload_dev)))
+        if i >= 1:
+            create.append(1e3 * (time.perf_counter() - t0))
+            h2d += int(st.reload_T.sum()) * shape.token_bytes
+            d2h += int(st.offload_T.sum()) * shape.token_bytes
+        tc.tc_kv_unpack(plan, [host], [dev], sp)
+        tc.tc_kv_pack(plan, [dev], [host], s2.cuda_stream)
+        torch.cuda.synchronize()   # a scheduler step ends when both directions have landed
+        plan.destroy()
+    wall = time.perf_counter() - t_all
+    out["configs[4] prefix-reload burst (mixed plan per step)"] = {
+        "steps": n_steps, "sessions": 512, "host_pool_blocks": NBh, "device_pool_blocks": NBd,
+        "plans_per_s": n_steps / wall, "ms_per_step_wall": 1e3 * wall / n_steps, "plan_create_ms": statistics.mean(create),
+        "h2d_GBps": h2d / wall / GB, "d2h_GBps": d2h / wall / GB, "link_GBps_both_directions": (h2d + d2h) / wall / GB,
+        "h2d_bytes_per_step": h2d // n_steps, "d2h_bytes_per_step": d2h // n_steps,
+        "note": "wall clock over create + execute + synchronise of every step; reload and offload run concurrently on two streams"}
+    del dev, host
+    torch.cuda.empty_cache()
+    return out
 
 
 def traffic_per_launch(algorithmic_bytes: float) -> float:
@@ -528,6 +622,9 @@ def main():
     ap.add_argument("--oracle-blocks", type=int, default=1536)
     ap.add_argument("--tile-bytes", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--no-extras", action="store_true", help="skip the secondary workloads (configs[3], configs[4])")
+    ap.add_argument("--host-pool-blocks", type=int, default=8192, help="configs[4]: pinned host pool size in 2 MiB blocks")
+    ap.add_argument("--burst-steps", type=int, default=10, help="configs[4]: scheduler steps timed (the workload has 200)")
     ap.add_argument("--host-ctas", type=int, default=0)
     ap.add_argument("--host-path", default="staged", choices=["staged", "zerocopy"])
     args = ap.parse_args()

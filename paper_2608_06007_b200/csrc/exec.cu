@@ -15,6 +15,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "plan.h"
 
@@ -179,29 +180,97 @@ static int cuda_fail(cudaError_t e, const char *what)
     return fail(TC_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
 
-static void free_group(Group &g)
+// Device storage of plans comes from a small per-device cache of power-of-two blocks, so that
+// a caller that creates and destroys one plan per scheduler step pays cudaMalloc / cudaFree
+// (both of which may synchronise the device) only until the cache has warmed up.
+namespace {
+struct CachedBlock {
+    void *ptr;
+    size_t bytes;
+    int device;
+};
+std::vector<CachedBlock> g_block_cache;
+size_t g_block_cache_bytes = 0;
+constexpr size_t kBlockCacheLimit = 256u << 20;
+pthread_mutex_t g_block_mu = PTHREAD_MUTEX_INITIALIZER;
+
+size_t block_size_for(size_t nb)
 {
-    if (g.d_descs) cudaFree(g.d_descs);
-    if (g.d_tile_desc) cudaFree(g.d_tile_desc);
-    g.d_descs = nullptr;
-    g.d_tile_desc = nullptr;
+    size_t s = 64u << 10;
+    while (s < nb) s <<= 1;
+    return s;
 }
 
-static int upload_group(tc_plan *plan, Group &g)
+cudaError_t block_alloc(int device, size_t nb, void **out, size_t *got)
 {
-    if (g.descs.empty()) return TC_OK;
-    cudaError_t e;
-    size_t nb = g.descs.size() * sizeof(Desc);
-    if ((e = cudaMalloc(&g.d_descs, nb)) != cudaSuccess)
-        return e == cudaErrorMemoryAllocation ? fail(TC_ERR_OOM, "device allocation of %zu descriptor bytes failed", nb) : cuda_fail(e, "cudaMalloc");
-    if ((e = cudaMemcpy(g.d_descs, g.descs.data(), nb, cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(e, "cudaMemcpy(descriptors)");
-    plan->device_bytes += nb;
-    if (!g.tile_desc.empty()) {
-        nb = g.tile_desc.size() * sizeof(uint32_t);
-        if ((e = cudaMalloc(&g.d_tile_desc, nb)) != cudaSuccess)
-            return e == cudaErrorMemoryAllocation ? fail(TC_ERR_OOM, "device allocation of %zu tile bytes failed", nb) : cuda_fail(e, "cudaMalloc");
-        if ((e = cudaMemcpy(g.d_tile_desc, g.tile_desc.data(), nb, cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(e, "cudaMemcpy(tiles)");
-        plan->device_bytes += nb;
+    const size_t want = block_size_for(nb);
+    pthread_mutex_lock(&g_block_mu);
+    for (size_t i = 0; i < g_block_cache.size(); i++)
+        if (g_block_cache[i].device == device && g_block_cache[i].bytes == want) {
+            *out = g_block_cache[i].ptr;
+            *got = want;
+            g_block_cache_bytes -= want;
+            g_block_cache.erase(g_block_cache.begin() + i);
+            pthread_mutex_unlock(&g_block_mu);
+            return cudaSuccess;
+        }
+    pthread_mutex_unlock(&g_block_mu);
+    *got = want;
+    return cudaMalloc(out, want);
+}
+
+void block_free(int device, void *ptr, size_t bytes)
+{
+    if (!ptr) return;
+    pthread_mutex_lock(&g_block_mu);
+    if (g_block_cache_bytes + bytes <= kBlockCacheLimit) {
+        g_block_cache.push_back(CachedBlock{ptr, bytes, device});
+        g_block_cache_bytes += bytes;
+        ptr = nullptr;
+    }
+    pthread_mutex_unlock(&g_block_mu);
+    if (ptr) cudaFree(ptr);
+}
+}  // namespace
+
+static void free_plan_storage(tc_plan *plan)
+{
+    block_free(plan->device, plan->d_storage, plan->d_storage_bytes);
+    plan->d_storage = nullptr;
+    for (int k = 0; k < 2; k++) plan->group[k].d_descs = nullptr, plan->group[k].d_tile_desc = nullptr;
+}
+
+// One allocation and one copy per plan: [g0 descriptors | g0 tiles | g1 descriptors | g1 tiles],
+// every part 256-byte aligned.
+static int upload_plan(tc_plan *plan)
+{
+    auto pad = [](size_t n) { return (n + 255) & ~size_t(255); };
+    size_t off[4], total = 0;
+    for (int k = 0; k < 2; k++) {
+        off[2 * k] = total;
+        total += pad(plan->group[k].descs.size() * sizeof(Desc));
+        off[2 * k + 1] = total;
+        total += pad(plan->group[k].tile_desc.size() * sizeof(uint32_t));
+    }
+    if (total == 0) return TC_OK;
+    std::vector<unsigned char> image(total);
+    for (int k = 0; k < 2; k++) {
+        const Group &g = plan->group[k];
+        if (!g.descs.empty()) memcpy(image.data() + off[2 * k], g.descs.data(), g.descs.size() * sizeof(Desc));
+        if (!g.tile_desc.empty()) memcpy(image.data() + off[2 * k + 1], g.tile_desc.data(), g.tile_desc.size() * sizeof(uint32_t));
+    }
+    cudaError_t e = block_alloc(plan->device, total, &plan->d_storage, &plan->d_storage_bytes);
+    if (e != cudaSuccess) {
+        plan->d_storage = nullptr;
+        return e == cudaErrorMemoryAllocation ? fail(TC_ERR_OOM, "device allocation of %zu plan bytes failed", total) : cuda_fail(e, "cudaMalloc");
+    }
+    if ((e = cudaMemcpy(plan->d_storage, image.data(), total, cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(e, "cudaMemcpy(plan)");
+    plan->device_bytes += static_cast<int64_t>(plan->d_storage_bytes);
+    char *base = static_cast<char *>(plan->d_storage);
+    for (int k = 0; k < 2; k++) {
+        Group &g = plan->group[k];
+        if (!g.descs.empty()) g.d_descs = reinterpret_cast<Desc *>(base + off[2 * k]);
+        if (!g.tile_desc.empty()) g.d_tile_desc = reinterpret_cast<uint32_t *>(base + off[2 * k + 1]);
     }
     return TC_OK;
 }
@@ -231,9 +300,19 @@ static void resident_ctas_all(int out[3])
 
 static void resident_ctas_for(size_t n_ptrs, int out[3])
 {
-    if (n_ptrs <= 8) resident_ctas_all<8>(out);
-    else if (n_ptrs <= 400) resident_ctas_all<400>(out);
-    else resident_ctas_all<TC_MAX_TABLE_SLOTS>(out);
+    // queried once per table size class (the answer depends on the kernel, not on the plan)
+    static int cache[3][3];
+    static bool have[3];
+    const int cls = n_ptrs <= 8 ? 0 : n_ptrs <= 400 ? 1 : 2;
+    pthread_mutex_lock(&g_block_mu);
+    if (!have[cls]) {
+        if (cls == 0) resident_ctas_all<8>(cache[cls]);
+        else if (cls == 1) resident_ctas_all<400>(cache[cls]);
+        else resident_ctas_all<TC_MAX_TABLE_SLOTS>(cache[cls]);
+        have[cls] = true;
+    }
+    for (int m = 0; m < 3; m++) out[m] = cache[cls][m];
+    pthread_mutex_unlock(&g_block_mu);
 }
 
 static uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *win = nullptr)
@@ -471,14 +550,12 @@ extern "C" int tc_plan_create(const tc_plan_spec_t *spec, tc_plan_t **out)
                 plan->device_bytes += arena;
             }
         }
-        for (int k = 0; k < 2 && rc == TC_OK; k++) {
-            rc = upload_group(plan, plan->group[k]);
+        if (rc == TC_OK) rc = upload_plan(plan);
+        for (int k = 0; k < 2 && rc == TC_OK; k++)
             if (plan->group[k].n_tiles) resident_ctas_for(plan->group[k].n_src + plan->group[k].n_dst, plan->group[k].resident_ctas);
-        }
     }
     if (rc != TC_OK) {
-        free_group(plan->group[0]);
-        free_group(plan->group[1]);
+        free_plan_storage(plan);
         if (plan->staged) stage_release(plan->device);
         delete plan;
         return rc;
@@ -490,8 +567,7 @@ extern "C" int tc_plan_create(const tc_plan_spec_t *spec, tc_plan_t **out)
 extern "C" int tc_plan_destroy(tc_plan_t *plan)
 {
     if (!plan) return TC_OK;
-    free_group(plan->group[0]);
-    free_group(plan->group[1]);
+    free_plan_storage(plan);
     if (plan->staged) stage_release(plan->device);
     delete plan;
     return TC_OK;

@@ -91,6 +91,8 @@ struct tc_plan {
     int sm_count = 0;
     int64_t packed_required = 0;
     int64_t device_bytes = 0;
+    void *d_storage = nullptr;  // one device block holding both groups' descriptors and tiles
+    size_t d_storage_bytes = 0;
     bool staged = false;  // holds a reference on the device's staging ring
     tc::Group group[2];
 };
