@@ -55,7 +55,7 @@ def _load():
 
 
 def _u8(a: np.ndarray) -> np.ndarray:
-    assert a.dtype == np.uint8 and a.ndim == 1 and a.strides[0] == 1, "oracle buffers are flat uint8"
+    assert a.dtype == np.uint8 and a.ndim == 1 and (a.size == 0 or a.strides[0] == 1), "oracle buffers are flat uint8"
     return a
 
 

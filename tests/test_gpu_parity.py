@@ -286,6 +286,44 @@ def test_weights_transform_into_fused_and_strided_targets():
     assert np.array_equal(target.result(), want2)
 
 
+# --------------------------------------------------------------------------- random geometries
+@pytest.mark.parametrize("seed", range(24))
+def test_random_geometries_on_the_device(seed):
+    rng = np.random.default_rng(1000 + seed)
+    L, B, H = int(rng.integers(1, 4)), int(rng.choice([1, 2, 4, 16, 32])), int(rng.integers(1, 9))
+    D, E = int(rng.choice([3, 8, 16, 64, 128])), int(rng.choice([1, 2, 4, 8]))
+    R = int(rng.integers(1, 7))
+    T = [int(rng.choice([0, 1, B, B + 1, 3 * B - 1, 9 * B, 17 * B + B // 2])) for _ in range(R)]
+    pad = int(rng.choice([0, 0, E, 32]))
+    shift = int(rng.choice([0, 0, 0, E, 16]))
+    tile = int(rng.choice([0, 0, 1024, 8192]))
+    pool_l, other_l = int(rng.integers(0, 2)), int(rng.integers(0, 2))
+    shape = (L, B, H, D, E)
+    T = np.array(T, dtype=np.int64)
+    off = np.concatenate([[0], np.cumsum((T + B - 1) // B)]).astype(np.int64)
+    NB = int(off[-1]) + 2
+    stride = B * H * D * E + pad
+    pool = rng.integers(0, 256, L * 2 * NB * stride, dtype=np.uint8)
+    bt = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    tune = dict(tile_bytes=tile) if tile else None
+    pl = tc.pool(pool_l, NB, L * 2, block_stride=stride, slot_bytes=NB * stride)
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, pool_l, stride, planes_of(pool, L * 2), T, off, bt, other_l, want)
+    d_pool = Guarded(pool.size, init=pool, shift=shift)
+    out = Guarded(max(want.size, 1), shift=shift)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=other_l, T=T, bt_off=off, bt_src=bt, tuning=tune))
+    tc.tc_kv_pack(plan, pool_tables(d_pool, L * 2, "planes"), [out.ptr()])
+    assert np.array_equal(out.result()[:want.size], want)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_migrate(shape, pool_l, stride, planes_of(pool, L * 2), other_l, stride, planes_of(want_pool, L * 2), T, off, bt, bt2)
+    pl2 = tc.pool(other_l, NB, L * 2, block_stride=stride, slot_bytes=NB * stride)
+    mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl2, T=T, bt_off=off, bt_src=bt, bt_dst=bt2, tuning=tune))
+    fresh = Guarded(pool.size, shift=shift)
+    tc.tc_kv_pack(mig, pool_tables(d_pool, L * 2, "planes"), pool_tables(fresh, L * 2, "planes"))
+    assert np.array_equal(fresh.result(), want_pool)
+
+
 # --------------------------------------------------------------------------- lifecycle on the device
 def test_empty_plan_wrong_tables_and_deadline_launch_nothing():
     shape, NB, src, dst = wl.config1()
