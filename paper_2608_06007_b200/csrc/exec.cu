@@ -33,7 +33,7 @@ enum { kModeRun = 0, kModeRows = 1, kModeAny = 2 };
 // CTA shape per build: threads x vectors in flight per thread (one pass covers a 32 KiB tile)
 // and the residency the register budget is held to.
 template <int MODE> struct Shape;
-template <> struct Shape<kModeRun> { static constexpr int threads = 512, unroll = 4, min_ctas = 3; };
+template <> struct Shape<kModeRun> { static constexpr int threads = 256, unroll = 8, min_ctas = 3; };
 template <> struct Shape<kModeRows> { static constexpr int threads = 256, unroll = 8, min_ctas = 3; };
 template <> struct Shape<kModeAny> { static constexpr int threads = 256, unroll = 4, min_ctas = 2; };
 
@@ -44,6 +44,8 @@ struct Params {
     uint32_t n_tiles;
     uint32_t tiles_per_desc;    // > 0 for uniform groups
     FastDiv div_tpd;
+    uint32_t tpo;               // uniform groups: tiles per plane of one descriptor
+    FastDiv div_tpo;
     uint32_t log2_ptr_align;    // alignment shared by every base pointer (capped at 4)
     // launch window (win_span == 0: the whole group).  Tile ids then walk plane-major over
     // descriptors [win_d0, ...) x planes [win_o0, ...): win_span = descriptors x win_tpo.
@@ -133,15 +135,20 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
     __shared__ Desc sdesc[2];
     int buf = 0;
     for (uint32_t tile = blockIdx.x; tile < prm.n_tiles; tile += gridDim.x, buf ^= 1) {
-        uint32_t di, t = 0;
+        // tile id -> descriptor, plane o, part.  For uniform and windowed launches this needs
+        // launch constants only, so it overlaps the descriptor fetch instead of waiting for it.
+        uint32_t di, o = 0, part = 0;
         if (prm.win_span) {
             const uint32_t ow = tile / prm.win_span, rem = tile - ow * prm.win_span;
             const uint32_t dw = rem / prm.win_tpo;
             di = prm.win_d0 + dw;
-            t = (prm.win_o0 + ow) * prm.win_tpo + (rem - dw * prm.win_tpo);
+            o = prm.win_o0 + ow;
+            part = rem - dw * prm.win_tpo;
         } else if (prm.tiles_per_desc) {
             di = fastdiv(tile, prm.div_tpd);
-            t = tile - di * prm.tiles_per_desc;
+            const uint32_t t = tile - di * prm.tiles_per_desc;
+            o = fastdiv(t, prm.div_tpo);
+            part = t - o * prm.tpo;
         } else {
             di = __ldg(prm.tile_desc + tile);
         }
@@ -149,17 +156,24 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
             reinterpret_cast<uint4 *>(&sdesc[buf])[threadIdx.x] = __ldg(reinterpret_cast<const uint4 *>(prm.descs + di) + threadIdx.x);
         __syncthreads();
         const Desc &d = sdesc[buf];
-        if (!prm.tiles_per_desc && !prm.win_span) t = tile - d.tile0;
-        const uint32_t o = fastdiv(t, d.div_tpo);
-        const uint32_t part = t - o * d.tiles_per_outer;
+        if (!prm.tiles_per_desc && !prm.win_span) {
+            const uint32_t t = tile - d.tile0;
+            o = fastdiv(t, d.div_tpo);
+            part = t - o * d.tiles_per_outer;
+        }
         const uint32_t row0 = part * d.rows_per_tile;
         if (row0 >= d.rows) continue;  // padding tile of a uniform group
         const uint32_t nrows = min(d.rows_per_tile, d.rows - row0);
         const char *src = prm.ptr[d.src_slot + o * d.src_slot_step] + d.src_off + o * d.src_outer;
         char *dst = prm.ptr[d.dst_slot + o * d.dst_slot_step] + d.dst_off + o * d.dst_outer;
         if (MODE == kModeRun) {
-            const uint32_t i1 = fastdiv(row0, d.div_n0), i0 = row0 - i1 * d.n0;
-            copy_run16<kUnroll, kThreads>(src + (i1 * d.src_s1 + i0 * d.src_s0), dst + (i1 * d.dst_s1 + i0 * d.dst_s0), d.run);
+            uint32_t so = 0, dof = 0;
+            if (row0) {  // a long run that was cut into rows
+                const uint32_t i1 = fastdiv(row0, d.div_n0), i0 = row0 - i1 * d.n0;
+                so = i1 * d.src_s1 + i0 * d.src_s0;
+                dof = i1 * d.dst_s1 + i0 * d.dst_s0;
+            }
+            copy_run16<kUnroll, kThreads>(src + so, dst + dof, d.run);
         } else if (MODE == kModeRows) {
             copy_rows<4, kUnroll, kThreads>(d, src, dst, row0, nrows);
         } else {
@@ -352,6 +366,8 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     }
     prm.tiles_per_desc = g.tiles_per_desc;
     prm.div_tpd = g.div_tpd;
+    prm.tpo = g.tiles_per_desc ? g.tiles_per_desc / g.descs[0].n_outer : 1;
+    prm.div_tpo = make_fastdiv(prm.tpo);
     prm.log2_ptr_align = ptr_align;
     for (size_t i = 0; i < g.n_src; i++) prm.ptr[i] = const_cast<char *>(static_cast<const char *>(src[i]));
     for (size_t i = 0; i < g.n_dst; i++) prm.ptr[g.n_src + i] = static_cast<char *>(dst[i]);
