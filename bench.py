@@ -538,6 +538,55 @@ def run_extras(args, tc, torch, stream):
     out = {}
     sp = stream.cuda_stream
     u8 = dict(dtype=torch.uint8, device="cuda")
+    # ---- configs[0]: 1.4 MB, launch-latency bound: microseconds and plans per second
+    shape, NB1, src1, dst1 = wl.config1()
+    pool1 = torch.empty(2 * NB1 * shape.chunk_bytes, **u8)
+    wl.fill_torch(pool1, wl.SEED_BASE + 1)
+    fresh1 = torch.empty_like(pool1)
+    packed1 = torch.empty(int(src1.T.sum()) * shape.token_bytes, **u8)
+    pl1 = tc.pool(tc.TC_NHD, NB1, 1, plane_stride=NB1 * shape.chunk_bytes, slot_bytes=pool1.numel())
+    mk_p = lambda: tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape.tuple, src_pool=pl1, packed_layout=tc.TC_HND, T=src1.T, bt_off=src1.bt_off, bt_src=src1.bt))
+    mk_u = lambda: tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape.tuple, dst_pool=pl1, packed_layout=tc.TC_HND, T=dst1.T, bt_off=dst1.bt_off, bt_dst=dst1.bt))
+    p1, u1 = mk_p(), mk_u()
+    with torch.cuda.stream(stream):
+        for _ in range(10):
+            tc.tc_kv_pack(p1, [pool1], [packed1], sp)
+            tc.tc_kv_unpack(u1, [packed1], [fresh1], sp)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(200):
+            tc.tc_kv_pack(p1, [pool1], [packed1], sp)
+            tc.tc_kv_unpack(u1, [packed1], [fresh1], sp)
+        b.record(stream)
+        torch.cuda.synchronize()
+        us_pair = a.elapsed_time(b) * 1e3 / 200
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for _ in range(20):
+                tc.tc_kv_pack(p1, [pool1], [packed1], sp)
+                tc.tc_kv_unpack(u1, [packed1], [fresh1], sp)
+        graph.replay()
+        torch.cuda.synchronize()
+        a.record(stream)
+        for _ in range(10):
+            graph.replay()
+        b.record(stream)
+        torch.cuda.synchronize()
+        us_pair_graph = a.elapsed_time(b) * 1e3 / 200
+    t0 = time.perf_counter()
+    for _ in range(200):
+        pp, uu = mk_p(), mk_u()
+        tc.tc_kv_pack(pp, [pool1], [packed1], sp)
+        tc.tc_kv_unpack(uu, [packed1], [fresh1], sp)
+        torch.cuda.synchronize()
+        pp.destroy()
+        uu.destroy()
+    wall = time.perf_counter() - t0
+    out["configs[0] correctness case (1.4 MB, latency bound)"] = {
+        "us_per_pack_plus_unpack_stream": us_pair, "us_per_pack_plus_unpack_cuda_graph": us_pair_graph,
+        "plans_per_s_create_execute_sync_destroy": 400 / wall, "payload_bytes": packed1.numel()}
+    del pool1, fresh1, packed1
     # ---- configs[3]
     shape = wl.LLAMA3_70B_KV
     free, _ = torch.cuda.mem_get_info()

@@ -324,6 +324,36 @@ def test_random_geometries_on_the_device(seed):
     assert np.array_equal(fresh.result(), want_pool)
 
 
+def test_execute_calls_can_be_captured_in_a_cuda_graph_and_replayed():
+    """Launch-bound use (config 1 moves 1.4 MB): pack + unpack captured once, replayed many
+    times; every replay reproduces the oracle's bytes (re-execution is idempotent)."""
+    shape, NB, src, dst = wl.config1()
+    s = shape.tuple
+    pool = np.zeros(2 * NB * shape.chunk_bytes, dtype=np.uint8)
+    wl.fill_np(pool, wl.SEED_BASE + 1)
+    want = np.zeros(oracle.packed_nbytes(s, src.T), dtype=np.uint8)
+    oracle.kv_pack(s, oracle.NHD, shape.chunk_bytes, planes_of(pool, 2), src.T, src.bt_off, src.bt, oracle.HND, want)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(s, oracle.NHD, shape.chunk_bytes, planes_of(want_pool, 2), dst.T, dst.bt_off, dst.bt, oracle.HND, want)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=pool.size)
+    pack = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=pl, packed_layout=tc.TC_HND, T=src.T, bt_off=src.bt_off, bt_src=src.bt))
+    unpack = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=pl, packed_layout=tc.TC_HND, T=dst.T, bt_off=dst.bt_off, bt_dst=dst.bt))
+    d_pool, packed, fresh = dev(pool), torch.zeros(want.size, dtype=torch.uint8, device="cuda"), Guarded(pool.size)
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph, stream=side):
+        tc.tc_kv_pack(pack, [d_pool], [packed], side.cuda_stream)
+        tc.tc_kv_unpack(unpack, [packed], [fresh.ptr()], side.cuda_stream)
+    for _ in range(3):
+        packed.zero_()
+        fresh.view.fill_(0xA5)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(packed.cpu().numpy(), want)
+        assert np.array_equal(fresh.result(), want_pool)
+
+
 # --------------------------------------------------------------------------- lifecycle on the device
 def test_empty_plan_wrong_tables_and_deadline_launch_nothing():
     shape, NB, src, dst = wl.config1()
