@@ -587,6 +587,33 @@ def run_extras(args, tc, torch, stream):
         "us_per_pack_plus_unpack_stream": us_pair, "us_per_pack_plus_unpack_cuda_graph": us_pair_graph,
         "plans_per_s_create_execute_sync_destroy": 400 / wall, "payload_bytes": packed1.numel()}
     del pool1, fresh1, packed1
+    # ---- configs[2] again, with the integrity checksum folded into the copy
+    ck = wl.config3() if not args.small else wl.llama_checkpoint(layers=1, vocab=16032)
+    blob = torch.empty(ck.nbytes_total, **u8)
+    wl.fill_torch(blob, wl.SEED_BASE + 3, "normal")
+    dstw = torch.empty(ck.nbytes_total, **u8)
+    nbytes = [ck.nbytes(i) for i in range(ck.N)]
+    ptrs = [dstw.data_ptr() + int(o) for o in np.concatenate([[0], np.cumsum(nbytes)])[:-1]]
+    sums = torch.zeros(ck.N, dtype=torch.int64, device="cuda")
+    planc = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total, flags=tc.TC_PLAN_CHECKSUM))
+    res = {}
+    with torch.cuda.stream(stream):
+        for name, fn in (("plain", lambda: tc.tc_weights_materialize(planc, blob, ptrs, sp)),
+                         ("with_checksum", lambda: tc.tc_weights_materialize_checksum(planc, blob, ptrs, sums, sp))):
+            ts = []
+            for i in range(8):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                torch.cuda.synchronize()
+                if i >= 3:
+                    ts.append(a.elapsed_time(b))
+            res[name] = 2 * ck.nbytes_total / (statistics.mean(ts) * 1e-3) / GB
+    out["configs[2] weights full, integrity checksum fused into the copy"] = {"GBps_plain": res["plain"], "GBps_with_checksum": res["with_checksum"]}
+    planc.destroy()
+    del blob, dstw
+    torch.cuda.empty_cache()
     # ---- configs[3]
     shape = wl.LLAMA3_70B_KV
     free, _ = torch.cuda.mem_get_info()

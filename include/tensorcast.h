@@ -103,7 +103,7 @@ enum {
     TC_PLAN_HOST_ONLY = 1u, /* validate and lower on the host only: the plan can be inspected
                                (tc_plan_stats, tc_plan_descriptors) but not executed, and no
                                CUDA call is made */
-    TC_PLAN_STAGED = 2u     /* TC_KV_PACK / TC_KV_UNPACK whose packed buffer is PINNED HOST memory:
+    TC_PLAN_STAGED = 2u,    /* TC_KV_PACK / TC_KV_UNPACK whose packed buffer is PINNED HOST memory:
                                instead of letting the kernel load / store host memory directly
                                (zero copy, the default), move the packed bytes with the copy
                                engines through a ring of device staging buffers owned by the
@@ -117,6 +117,11 @@ enum {
                                this path is a few percent faster; it costs one launch and one
                                copy per segment instead of one launch per call.  Staged
                                executions are serialised with one another by the library. */
+    TC_PLAN_CHECKSUM = 4u   /* TC_WEIGHTS: the plan can also be run by
+                               tc_weights_materialize_checksum, which folds an integrity
+                               checksum of every tensor into the same pass as the copy.  Needs
+                               16-byte aligned geometry and tensors that start on 4-byte
+                               boundaries of the blob (TC_ERR_INVALID_ARG otherwise). */
 };
 
 #define TC_MAX_TABLE_SLOTS 4000 /* src slots + dst slots of one execute call */
@@ -247,6 +252,23 @@ TC_API int tc_kv_unpack(const tc_plan_t *plan, const void *const *src_bases, siz
  */
 TC_API int tc_weights_materialize(const tc_plan_t *plan, const void *blob, void *const *dst_ptrs,
                            size_t n_dst, void *stream);
+
+/*
+ * tc_weights_materialize plus integrity checksums, in one pass over the data (the
+ * materialisation pipeline "verifies integrity" before it hands tensors out, Sec. 5).
+ * `plan` must have been created with TC_PLAN_CHECKSUM.  checksums: DEVICE pointer to
+ * n_tensors uint64 accumulators; the call zeroes them on `stream` and the kernel adds to them.
+ * Definition.  Tensor i is read as little-endian 4-byte words x_u at tensor-relative offsets
+ * 4u.  With  key(u) = ((u * 0x9E3779B1) << 1 | 1) mod 2^32  (an odd 32-bit weight per position),
+ * checksums[i] = sum of x_u * key(u) over the words u of tensor i that this call reads
+ * (all of them, or the rank's slice), modulo 2^64: a position-weighted sum, so any change of
+ * one word and any exchange of two unequal words changes it.  It depends on positions in the SOURCE
+ * tensor, so the checksums of the shards of all ranks add up to the checksum of the whole
+ * tensor, and a publisher can store either.  Comparing with the expected values is the
+ * caller's step (copy the accumulators back after synchronising the stream).
+ */
+TC_API int tc_weights_materialize_checksum(const tc_plan_t *plan, const void *blob, void *const *dst_ptrs,
+                                           size_t n_dst, uint64_t *checksums, void *stream);
 
 /*
  * Free the plan's host and device storage.  The caller must first have synchronised every

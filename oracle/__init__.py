@@ -200,3 +200,23 @@ def weights(blob_off, E, shapes, split_dim, rank, world, blob, dst, dst_off=None
                            td, dst_off.ctypes, dst_stride.ctypes, cnt, C.c_int64(i0), C.c_int64(i1))
     # split per tensor so that skewed sizes still spread over the threads
     _run(go, [(i, i + 1) for i in range(N)] if threads > 1 else [(0, N)], threads)
+
+
+def weights_checksum(blob_off, E, shapes, split_dim, rank, world, blob):
+    """Integrity checksums (uint64 per tensor) of the words the rank's slice covers; raises if a
+    slice covers a 4-byte word only partly."""
+    lib = _load()
+    N = len(blob_off)
+    blob_off, E = _i64(blob_off), _i64(E)
+    shapes = _i64(shapes).reshape(N, 4)
+    split_dim = _i32(split_dim)
+    sums = np.zeros(N, dtype=np.uint64)
+    biggest = int(max((int(np.prod(shapes[i])) * int(E[i]) for i in range(N)), default=0))
+    scratch = np.zeros(max(biggest, 1), dtype=np.uint8)
+    status = C.c_int32(0)
+    lib.oracle_weights_checksum(C.c_int64(N), blob_off.ctypes, E.ctypes, shapes.ctypes, split_dim.ctypes,
+                                C.c_int64(rank), C.c_int64(world), C.c_void_p(_u8(blob).ctypes.data),
+                                sums.ctypes, scratch.ctypes, C.byref(status))
+    if status.value != 0:
+        raise ValueError("a slice covers a 4-byte word only partly: its checksum is undefined")
+    return sums

@@ -236,3 +236,62 @@ void oracle_weights(int64_t N, const int64_t *blob_off, const int64_t *E,
                     }
     }
 }
+
+/*
+ * Integrity checksum folded into weight materialisation (the materialisation pipeline
+ * "verifies integrity", Sec. 5 "Tensor Materialization and Transfer"; the paper does not
+ * define the function, this is the library's, stated in its header).
+ * Tensor i is read as little-endian 4-byte words x_u at tensor-relative byte offsets 4u:
+ *   key(u) = ((u * 0x9E3779B1) << 1 | 1) mod 2^32
+ *   sums[i] = sum of x_u * key(u) over the words the rank's slice covers, modulo 2^64.
+ * Written byte by byte: the slice is first marked in a byte mask of the tensor, then every
+ * fully covered word is added.  A word only partly covered has no defined checksum:
+ * *status is set to -1.  mask_scratch must hold the largest tensor's bytes.
+ */
+void oracle_weights_checksum(int64_t N, const int64_t *blob_off, const int64_t *E,
+                             const int64_t (*shape)[4], const int32_t *split_dim,
+                             int64_t rank, int64_t world, const uint8_t *blob,
+                             uint64_t *sums, uint8_t *mask_scratch, int32_t *status)
+{
+    *status = 0;
+    for (int64_t i = 0; i < N; i++) {
+        int64_t ext[4], shift[4], nbytes = E[i];
+        for (int m = 0; m < 4; m++) {
+            nbytes *= shape[i][m];
+            ext[m] = shape[i][m];
+            shift[m] = 0;
+            if (m == split_dim[i]) {
+                ext[m] = shape[i][m] / world;
+                shift[m] = rank * ext[m];
+            }
+        }
+        for (int64_t p = 0; p < nbytes; p++) mask_scratch[p] = 0;
+        for (int64_t j0 = 0; j0 < ext[0]; j0++)
+            for (int64_t j1 = 0; j1 < ext[1]; j1++)
+                for (int64_t j2 = 0; j2 < ext[2]; j2++)
+                    for (int64_t j3 = 0; j3 < ext[3]; j3++) {
+                        int64_t k = (((j0 + shift[0]) * shape[i][1] + (j1 + shift[1])) * shape[i][2]
+                                     + (j2 + shift[2])) * shape[i][3] + (j3 + shift[3]);
+                        for (int64_t e = 0; e < E[i]; e++) mask_scratch[k * E[i] + e] = 1;
+                    }
+        uint64_t sum = 0;
+        for (int64_t u = 0; u * 4 < nbytes; u++) {
+            int covered = 0;
+            uint32_t x = 0;
+            for (int b = 0; b < 4; b++) {
+                int64_t p = u * 4 + b;
+                if (p < nbytes && mask_scratch[p]) {
+                    covered++;
+                    x |= (uint32_t)blob[blob_off[i] + p] << (8 * b);
+                }
+            }
+            if (covered == 4) {
+                uint32_t key = (((uint32_t)u * 0x9E3779B1u) << 1) | 1u;
+                sum += (uint64_t)x * (uint64_t)key;
+            } else if (covered != 0) {
+                *status = -1;
+            }
+        }
+        sums[i] = sum;
+    }
+}

@@ -22,6 +22,7 @@ TC_KV_PACK, TC_KV_UNPACK, TC_KV_MIGRATE, TC_KV_MIXED, TC_WEIGHTS = 1, 2, 3, 4, 5
 TC_NHD, TC_HND = 0, 1
 TC_PLAN_HOST_ONLY = 1
 TC_PLAN_STAGED = 2
+TC_PLAN_CHECKSUM = 4
 TC_MAX_TABLE_SLOTS = 4000
 
 
@@ -87,7 +88,7 @@ class tc_descriptor_t(C.Structure):
 
 EXPORTS = ("tc_plan_create", "tc_kv_pack", "tc_kv_unpack", "tc_weights_materialize",
            "tc_plan_destroy", "tc_plan_stats", "tc_plan_descriptors", "tc_strerror", "tc_last_error",
-           "tc_kv_pack_noalloc")
+           "tc_kv_pack_noalloc", "tc_weights_materialize_checksum")
 
 _lib = None
 
@@ -111,6 +112,8 @@ def load_library(path: str | None = None):
     lib.tc_plan_descriptors.argtypes = [vp, C.c_int, vp, sz, C.POINTER(sz)]
     lib.tc_kv_pack_noalloc.argtypes = [C.POINTER(tc_plan_spec_t), vp, sz, vp, sz, vp]
     lib.tc_kv_pack_noalloc.restype = C.c_int
+    lib.tc_weights_materialize_checksum.argtypes = [vp, vp, vp, sz, vp, vp]
+    lib.tc_weights_materialize_checksum.restype = C.c_int
     lib.tc_strerror.argtypes = [C.c_int]
     lib.tc_strerror.restype = C.c_char_p
     lib.tc_last_error.restype = C.c_char_p
@@ -306,6 +309,12 @@ def tc_kv_unpack(plan: Plan, src_bases, dst_bases, stream=None) -> None:
 def tc_weights_materialize(plan: Plan, blob, dst_ptrs, stream=None) -> None:
     d, nd = _table(dst_ptrs)
     _check(load_library().tc_weights_materialize(plan.handle, _addr(blob), d, nd, _stream(stream)))
+
+
+def tc_weights_materialize_checksum(plan: Plan, blob, dst_ptrs, checksums, stream=None) -> None:
+    """tc_weights_materialize that also fills `checksums` (device uint64[n_tensors]) in the same pass."""
+    d, nd = _table(dst_ptrs)
+    _check(load_library().tc_weights_materialize_checksum(plan.handle, _addr(blob), d, nd, _addr(checksums), _stream(stream)))
 
 
 def tc_plan_stats(plan: Plan) -> tc_plan_stats_t:

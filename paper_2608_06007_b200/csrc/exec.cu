@@ -50,8 +50,28 @@ struct Params {
     // launch window (win_span == 0: the whole group).  Tile ids then walk plane-major over
     // descriptors [win_d0, ...) x planes [win_o0, ...): win_span = descriptors x win_tpo.
     uint32_t win_span, win_d0, win_o0, win_tpo;
+    unsigned long long *sums;   // checksum accumulators (checked builds only)
     char *ptr[NPTR];            // src table then dst table
 };
+
+// Integrity checksum: position-weighted sum of the source's 4-byte words,
+//   sum of x_u * key(u) mod 2^64,  key(u) = ((u * 0x9E3779B1) << 1 | 1) mod 2^32,
+// u = word index relative to the tensor's first byte.  key(u + 1) = key(u) + 2 * 0x9E3779B1.
+__device__ __forceinline__ unsigned long long csum_vec(uint4 v, unsigned long long byte_pos)
+{
+    constexpr uint32_t kStep = 0x9E3779B1u << 1;
+    uint32_t k = ((static_cast<uint32_t>(byte_pos >> 2) * 0x9E3779B1u) << 1) | 1u;
+    unsigned long long t = static_cast<unsigned long long>(v.x) * k;
+    k += kStep;
+    t += static_cast<unsigned long long>(v.y) * k;
+    k += kStep;
+    t += static_cast<unsigned long long>(v.z) * k;
+    k += kStep;
+    t += static_cast<unsigned long long>(v.w) * k;
+    return t;
+}
+template <typename V> __device__ __forceinline__ unsigned long long csum_of(V, unsigned long long) { return 0; }
+template <> __device__ __forceinline__ unsigned long long csum_of<uint4>(uint4 v, unsigned long long p) { return csum_vec(v, p); }
 
 __device__ __forceinline__ uint32_t fastdiv(uint32_t n, FastDiv f) { return (__umulhi(n, f.mul) + n) >> f.shift; }
 
@@ -76,11 +96,33 @@ template <> struct VecOf<2> { using type = uint32_t; };
 template <> struct VecOf<1> { using type = uint16_t; };
 template <> struct VecOf<0> { using type = uint8_t; };
 
+// Add the CTA's partial checksums to the accumulator: warp shuffles, then one atomic per CTA
+// (many CTAs feed the same tensor's accumulator; same-address atomics are the scarce resource).
+template <int kThreads>
+__device__ __forceinline__ void csum_flush(unsigned long long *sum, unsigned long long acc)
+{
+    __shared__ unsigned long long warp_sums[kThreads / 32];
+#pragma unroll
+    for (int k = 16; k > 0; k >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, k);
+    if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        acc = threadIdx.x < kThreads / 32 ? warp_sums[threadIdx.x] : 0;
+#pragma unroll
+        for (int k = 16; k > 0; k >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, k);
+        if (threadIdx.x == 0) atomicAdd(sum, acc);
+    }
+    __syncthreads();
+}
+
 // Copy rows [row0, row0 + nrows) of one outer index of descriptor d; src / dst point at row 0.
 // A thread's vectors are kThreads vectors apart, so a warp always covers 32 consecutive
 // vectors of the tile's row space: whole aligned segments on both sides.
-template <int LOGV, int U, int kThreads>
-__device__ __forceinline__ void copy_rows(const Desc &d, const char *src, char *dst, uint32_t row0, uint32_t nrows)
+// CHECK: also add the checksum terms of the bytes read to acc; pos0 is the tensor-relative
+// byte position of src.
+template <int LOGV, int U, int kThreads, bool CHECK = false>
+__device__ __forceinline__ void copy_rows(const Desc &d, const char *src, char *dst, uint32_t row0, uint32_t nrows,
+                                          unsigned long long pos0 = 0, unsigned long long *acc = nullptr)
 {
     using V = typename VecOf<LOGV>::type;
     const uint32_t nbytes = nrows * d.run;  // <= 1 MiB
@@ -90,7 +132,7 @@ __device__ __forceinline__ void copy_rows(const Desc &d, const char *src, char *
 #pragma unroll 1
     for (uint32_t base = threadIdx.x << LOGV; base < nbytes; base += (kThreads * U) << LOGV) {
         V val[U];
-        uint32_t doff[U];
+        uint32_t doff[U], soff[CHECK ? U : 1];
 #pragma unroll
         for (int u = 0; u < U; u++) {
             const uint32_t byte = base + ((u * kThreads) << LOGV);
@@ -101,20 +143,25 @@ __device__ __forceinline__ void copy_rows(const Desc &d, const char *src, char *
                 const uint32_t i1 = fastdiv(r, div_n0);
                 const uint32_t i0 = r - i1 * n0;
                 doff[u] = i1 * ds1 + i0 * ds0 + col;
-                val[u] = ld_stream<V>(src + (i1 * ss1 + i0 * ss0 + col));
+                const uint32_t so = i1 * ss1 + i0 * ss0 + col;
+                if (CHECK) soff[u] = so;
+                val[u] = ld_stream<V>(src + so);
             }
         }
 #pragma unroll
         for (int u = 0; u < U; u++) {
             const uint32_t byte = base + ((u * kThreads) << LOGV);
-            if (byte < nbytes) st_stream<V>(dst + doff[u], val[u]);
+            if (byte < nbytes) {
+                st_stream<V>(dst + doff[u], val[u]);
+                if (CHECK) *acc += csum_of<V>(val[u], pos0 + soff[u]);
+            }
         }
     }
 }
 
 // One contiguous run of 16-byte vectors: no row decoding at all.
-template <int U, int kThreads>
-__device__ __forceinline__ void copy_run16(const char *src, char *dst, uint32_t nbytes)
+template <int U, int kThreads, bool CHECK = false>
+__device__ __forceinline__ void copy_run16(const char *src, char *dst, uint32_t nbytes, unsigned long long pos0 = 0, unsigned long long *acc = nullptr)
 {
 #pragma unroll 1
     for (uint32_t base = threadIdx.x << 4; base < nbytes; base += (kThreads * U) << 4) {
@@ -124,11 +171,14 @@ __device__ __forceinline__ void copy_run16(const char *src, char *dst, uint32_t 
             if (base + ((u * kThreads) << 4) < nbytes) val[u] = ld_stream<uint4>(src + base + ((u * kThreads) << 4));
 #pragma unroll
         for (int u = 0; u < U; u++)
-            if (base + ((u * kThreads) << 4) < nbytes) st_stream<uint4>(dst + base + ((u * kThreads) << 4), val[u]);
+            if (base + ((u * kThreads) << 4) < nbytes) {
+                st_stream<uint4>(dst + base + ((u * kThreads) << 4), val[u]);
+                if (CHECK) *acc += csum_vec(val[u], pos0 + base + ((u * kThreads) << 4));
+            }
     }
 }
 
-template <int NPTR, int MODE>
+template <int NPTR, int MODE, bool CHECK = false>
 __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) tc_copy_kernel(const __grid_constant__ Params<NPTR> prm)
 {
     constexpr int kThreads = Shape<MODE>::threads, kUnroll = Shape<MODE>::unroll;
@@ -173,9 +223,21 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
                 so = i1 * d.src_s1 + i0 * d.src_s0;
                 dof = i1 * d.dst_s1 + i0 * d.dst_s0;
             }
-            copy_run16<kUnroll, kThreads>(src + so, dst + dof, d.run);
+            if (CHECK) {
+                unsigned long long acc = 0;
+                copy_run16<kUnroll, kThreads, true>(src + so, dst + dof, d.run, static_cast<unsigned long long>(d.src_off + o * d.src_outer - d.csum_base) + so, &acc);
+                csum_flush<kThreads>(prm.sums + d.tag, acc);
+            } else {
+                copy_run16<kUnroll, kThreads>(src + so, dst + dof, d.run);
+            }
         } else if (MODE == kModeRows) {
-            copy_rows<4, kUnroll, kThreads>(d, src, dst, row0, nrows);
+            if (CHECK) {
+                unsigned long long acc = 0;
+                copy_rows<4, kUnroll, kThreads, true>(d, src, dst, row0, nrows, static_cast<unsigned long long>(d.src_off + o * d.src_outer - d.csum_base), &acc);
+                csum_flush<kThreads>(prm.sums + d.tag, acc);
+            } else {
+                copy_rows<4, kUnroll, kThreads>(d, src, dst, row0, nrows);
+            }
         } else {
             switch (min(d.log2_align, prm.log2_ptr_align)) {
             case 4: copy_rows<4, kUnroll, kThreads>(d, src, dst, row0, nrows); break;
@@ -348,9 +410,10 @@ static uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Se
 
 template <int NPTR>
 static int launch(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t stream,
-                  const Segment *win = nullptr)
+                  const Segment *win = nullptr, unsigned long long *sums = nullptr)
 {
     const int mode = mode_for(g, ptr_align);
+    if (sums && mode == kModeAny) return fail(TC_ERR_INVALID_ARG, "checksums need 16-byte aligned base pointers");
     const uint32_t grid = grid_for(plan, g, mode, win);
     Params<NPTR> prm;
     prm.descs = g.d_descs;
@@ -369,9 +432,14 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     prm.tpo = g.tiles_per_desc ? g.tiles_per_desc / g.descs[0].n_outer : 1;
     prm.div_tpo = make_fastdiv(prm.tpo);
     prm.log2_ptr_align = ptr_align;
+    prm.sums = sums;
     for (size_t i = 0; i < g.n_src; i++) prm.ptr[i] = const_cast<char *>(static_cast<const char *>(src[i]));
     for (size_t i = 0; i < g.n_dst; i++) prm.ptr[g.n_src + i] = static_cast<char *>(dst[i]);
     for (size_t i = g.n_src + g.n_dst; i < NPTR; i++) prm.ptr[i] = nullptr;
+    if (sums) {
+        if (mode == kModeRun) tc_copy_kernel<NPTR, kModeRun, true><<<grid, Shape<kModeRun>::threads, 0, stream>>>(prm);
+        else tc_copy_kernel<NPTR, kModeRows, true><<<grid, Shape<kModeRows>::threads, 0, stream>>>(prm);
+    } else
     switch (mode) {
     case kModeRun: tc_copy_kernel<NPTR, kModeRun><<<grid, Shape<kModeRun>::threads, 0, stream>>>(prm); break;
     case kModeRows: tc_copy_kernel<NPTR, kModeRows><<<grid, Shape<kModeRows>::threads, 0, stream>>>(prm); break;
@@ -382,12 +450,13 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     return TC_OK;
 }
 
-static int launch_any(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s, const Segment *win)
+static int launch_any(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s, const Segment *win,
+                      unsigned long long *sums = nullptr)
 {
     const size_t n = g.n_src + g.n_dst;
-    if (n <= 8) return launch<8>(plan, g, src, dst, ptr_align, s, win);
-    if (n <= 400) return launch<400>(plan, g, src, dst, ptr_align, s, win);
-    return launch<TC_MAX_TABLE_SLOTS>(plan, g, src, dst, ptr_align, s, win);
+    if (n <= 8) return launch<8>(plan, g, src, dst, ptr_align, s, win, sums);
+    if (n <= 400) return launch<400>(plan, g, src, dst, ptr_align, s, win, sums);
+    return launch<TC_MAX_TABLE_SLOTS>(plan, g, src, dst, ptr_align, s, win, sums);
 }
 
 // ---- staged host path: copy engines <-> device staging ring <-> kernel ----------------------
@@ -505,7 +574,8 @@ out:
 }
 #undef TC_TRY
 
-static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n_src, void *const *dst, size_t n_dst, void *stream)
+static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n_src, void *const *dst, size_t n_dst, void *stream,
+                   unsigned long long *sums = nullptr)
 {
     clear_error();
     if (!plan) return fail(TC_ERR_INVALID_ARG, "plan is NULL");
@@ -515,6 +585,10 @@ static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n
         return fail(TC_ERR_INVALID_ARG, "tables of %zu source and %zu destination pointers given, the plan needs %zu and %zu", n_src, n_dst, g.n_src, g.n_dst);
     if ((n_src && !src) || (n_dst && !dst)) return fail(TC_ERR_INVALID_ARG, "pointer table is NULL");
     if (plan->deadline_ns && now_ns() > plan->deadline_ns) return fail(TC_ERR_DEADLINE, "deadline passed before the call; nothing launched");
+    if (sums) {
+        cudaError_t e = cudaMemsetAsync(sums, 0, static_cast<size_t>(plan->n_sums) * sizeof(unsigned long long), static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) return cuda_fail(e, "zeroing the checksum accumulators");
+    }
     if (g.n_tiles == 0) return TC_OK;
     uint32_t ptr_align = 4;
     for (size_t i = 0; i < n_src; i++) {
@@ -527,7 +601,7 @@ static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (!g.segments.empty()) return execute_staged(plan, gi, g, src, dst, ptr_align, s);
-    return launch_any(plan, g, src, dst, ptr_align, s, nullptr);
+    return launch_any(plan, g, src, dst, ptr_align, s, nullptr, sums);
 }
 
 }  // namespace tc
@@ -615,6 +689,16 @@ extern "C" int tc_weights_materialize(const tc_plan_t *plan, const void *blob, v
     }
     const void *src[1] = {blob};
     return execute(plan, 0, src, 1, dst_ptrs, n_dst, stream);
+}
+
+extern "C" int tc_weights_materialize_checksum(const tc_plan_t *plan, const void *blob, void *const *dst_ptrs, size_t n_dst, uint64_t *checksums, void *stream)
+{
+    clear_error();
+    if (plan && (plan->kind != TC_WEIGHTS || !plan->checksummed))
+        return fail(TC_ERR_KIND, "tc_weights_materialize_checksum needs a WEIGHTS plan created with TC_PLAN_CHECKSUM");
+    if (!checksums) return fail(TC_ERR_INVALID_ARG, "checksums is NULL");
+    const void *src[1] = {blob};
+    return execute(plan, 0, src, 1, dst_ptrs, n_dst, stream, reinterpret_cast<unsigned long long *>(checksums));
 }
 
 extern "C" int tc_plan_stats(const tc_plan_t *plan, tc_plan_stats_t *out)

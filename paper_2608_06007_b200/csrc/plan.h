@@ -44,7 +44,9 @@ struct alignas(16) Desc {
     uint32_t run, n0, rows, n_outer;
     uint32_t rows_per_tile, tiles_per_outer, tile0, log2_align;
     FastDiv div_n0, div_tpo;
-    uint32_t pad[4];
+    uint32_t tag;        // checksummed plans: which accumulator (tensor index) this box feeds
+    uint32_t pad;
+    int64_t csum_base;   // checksummed plans: src byte offset of the tensor's first byte
 };
 static_assert(sizeof(Desc) == 128, "Desc must stay 128 bytes");
 
@@ -93,6 +95,8 @@ struct tc_plan {
     int64_t device_bytes = 0;
     void *d_storage = nullptr;  // one device block holding both groups' descriptors and tiles
     size_t d_storage_bytes = 0;
+    bool checksummed = false;  // built with TC_PLAN_CHECKSUM
+    int64_t n_sums = 0;        // accumulators a checksummed execution fills
     bool staged = false;  // holds a reference on the device's staging ring
     tc::Group group[2];
 };

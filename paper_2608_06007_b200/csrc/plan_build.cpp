@@ -56,6 +56,8 @@ struct Box {
     // the table-stepping outer dimension (KV planes); n_outer == 1 when unused
     uint32_t n_outer = 1, src_slot_step = 0, dst_slot_step = 0;
     int64_t src_outer = 0, dst_outer = 0;
+    uint32_t tag = 0;         // checksum accumulator
+    int64_t csum_base = 0;    // source offset that checksum positions are relative to
 };
 
 static uint32_t ctz_cap(int64_t v, uint32_t cap = 4)
@@ -99,6 +101,8 @@ static void emit_desc(Group &g, const Box &b, int64_t run, const Dim *inner, con
     if (n1 > 1) a = std::min({a, ctz_cap(d.src_s1), ctz_cap(d.dst_s1)});
     if (d.n_outer > 1) a = std::min({a, ctz_cap(d.src_outer), ctz_cap(d.dst_outer)});
     d.log2_align = a;
+    d.tag = b.tag;
+    d.csum_base = b.csum_base;
     g.log2_align = std::min(g.log2_align, a);
     if (d.rows_per_tile > 1) g.single_run_tiles = false;
     g.payload += static_cast<int64_t>(d.run) * d.rows * d.n_outer;
@@ -555,6 +559,8 @@ static int build_weights(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t til
         spans[static_cast<size_t>(slot)].push_back(Span{rule.dst_off, hi, i});
         Box b;
         b.run = t.elem_bytes;
+        b.tag = static_cast<uint32_t>(i);
+        b.csum_base = static_cast<int64_t>(t.byte_off);
         b.src_off = static_cast<int64_t>(t.byte_off) + shift;
         b.dst_off = rule.dst_off;
         b.src_slot = 0;
@@ -591,6 +597,15 @@ static int build_weights(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t til
                 return fail(TC_ERR_OVERLAP, "destination slot %zu: byte %lld would be written twice", s, (long long)rows[k].first);
     }
     for (const Box &b : boxes) lower_box(g, b, tile_bytes);
+    if (spec->flags & TC_PLAN_CHECKSUM) {
+        // checksums are sums over aligned 4-byte words of each tensor: every run must be made of
+        // whole words and every access must be 16-byte aligned
+        if (g.log2_align < 4) return fail(TC_ERR_INVALID_ARG, "TC_PLAN_CHECKSUM needs 16-byte aligned offsets, strides and runs");
+        for (int64_t i = 0; i < w.n_tensors; i++)
+            if (w.index[i].byte_off % 4) return fail(TC_ERR_INVALID_ARG, "TC_PLAN_CHECKSUM: tensor %lld starts at byte %llu, not a multiple of 4", (long long)i, (unsigned long long)w.index[i].byte_off);
+        plan->checksummed = true;
+        plan->n_sums = w.n_tensors;
+    }
     return TC_OK;
 }
 
@@ -621,6 +636,8 @@ int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
         for (Desc &d : g.descs) d.dst_slot = static_cast<uint16_t>(d.dst_slot + g.n_src);
         if ((rc = finish_group(g))) return rc;
     }
+    if ((spec->flags & TC_PLAN_CHECKSUM) && spec->kind != TC_WEIGHTS)
+        return fail(TC_ERR_KIND, "TC_PLAN_CHECKSUM applies to TC_WEIGHTS plans only");
     if (spec->flags & TC_PLAN_STAGED) {
         if (spec->kind != TC_KV_PACK && spec->kind != TC_KV_UNPACK)
             return fail(TC_ERR_KIND, "TC_PLAN_STAGED applies to TC_KV_PACK and TC_KV_UNPACK plans only");

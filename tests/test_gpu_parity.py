@@ -286,6 +286,44 @@ def test_weights_transform_into_fused_and_strided_targets():
     assert np.array_equal(target.result(), want2)
 
 
+def test_weights_checksum_fused_with_the_copy():
+    ck = wl.llama_checkpoint(hidden=256, layers=2, q_heads=8, kv_heads=4, head_dim=32, mlp=512, vocab=1024)
+    blob = np.zeros(ck.nbytes_total, dtype=np.uint8)
+    wl.fill_np(blob, 8, "normal")
+    d_blob = dev(blob)
+    nbytes = [ck.nbytes(i) for i in range(ck.N)]
+    for world, ranks in ((1, [0]), (4, [0, 3])):
+        for rank in ranks:
+            split = ck.split_dim if world > 1 else np.full(ck.N, -1)
+            sizes = [n // (world if split[i] >= 0 else 1) for i, n in enumerate(nbytes)]
+            want = [np.zeros(n, dtype=np.uint8) for n in sizes]
+            oracle.weights(ck.byte_off, ck.E, ck.shapes, split, rank, world, blob, want)
+            want_sums = oracle.weights_checksum(ck.byte_off, ck.E, ck.shapes, split, rank, world, blob)
+            plan = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, split_dim=split, rank=rank, world=world,
+                                                     blob_bytes=ck.nbytes_total, flags=tc.TC_PLAN_CHECKSUM, tuning=dict(tile_bytes=4096)))
+            outs = [Guarded(n, fill=0xEE) for n in sizes]
+            sums = torch.full((ck.N,), -1, dtype=torch.int64, device="cuda")
+            for _ in range(2):                                     # accumulators are zeroed by every call
+                tc.tc_weights_materialize_checksum(plan, d_blob, [o.ptr() for o in outs], sums)
+            torch.cuda.synchronize()
+            assert np.array_equal(sums.cpu().numpy().view(np.uint64), want_sums)
+            for i in range(ck.N):
+                assert np.array_equal(outs[i].result(), want[i]), ck.names[i]
+            tc.tc_weights_materialize(plan, d_blob, [o.ptr() for o in outs])   # the plan still runs unchecked
+    # a corrupted blob is detected
+    bad = blob.copy()
+    assert ck.split_dim[1] < 0                                 # a replicated norm: every rank reads all of it
+    bad[ck.byte_off[1] + 100] ^= 0x10
+    tc.tc_weights_materialize_checksum(plan, dev(bad), [o.ptr() for o in outs], sums)
+    torch.cuda.synchronize()
+    got = sums.cpu().numpy().view(np.uint64)
+    assert (got != want_sums).sum() == 1 and got[1] != want_sums[1]
+    plain = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total))
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_weights_materialize_checksum(plain, d_blob, [o.ptr() for o in outs], sums)
+    assert e.value.status == tc.TC_ERR_KIND
+
+
 # --------------------------------------------------------------------------- random geometries
 @pytest.mark.parametrize("seed", range(24))
 def test_random_geometries_on_the_device(seed):

@@ -357,6 +357,46 @@ def test_llama3_8b_index_matches_golden_offsets():
     assert shard_el == g["shard_elements_world8"]
 
 
+# ------------------------------------------------------------------ integrity checksum
+def test_checksum_shards_add_up_to_the_whole_and_replicas_equal_it():
+    ck = small_checkpoint()
+    blob = np.random.default_rng(12).integers(0, 256, ck.nbytes_total, dtype=np.uint8)
+    none = np.full(ck.N, -1)
+    full = oracle.weights_checksum(ck.byte_off, ck.E, ck.shapes, none, 0, 1, blob)
+    W = 4
+    parts = [oracle.weights_checksum(ck.byte_off, ck.E, ck.shapes, ck.split_dim, r, W, blob) for r in range(W)]
+    with np.errstate(over="ignore"):
+        total = np.sum(np.stack(parts), axis=0, dtype=np.uint64)
+    for i in range(ck.N):
+        if ck.split_dim[i] >= 0:
+            assert total[i] == full[i], ck.names[i]          # position-keyed terms: slices partition the sum
+        else:
+            assert all(p[i] == full[i] for p in parts)        # replicated tensors
+
+
+def test_checksum_depends_on_every_bit_and_on_position_but_not_on_the_shape_description():
+    rng = np.random.default_rng(13)
+    blob = rng.integers(0, 256, 4096, dtype=np.uint8)
+    base = oracle.weights_checksum([0], [2], [[32, 64, 1, 1]], [-1], 0, 1, blob)[0]
+    assert base == oracle.weights_checksum([0], [8], [[512, 1, 1, 1]], [-1], 0, 1, blob)[0]     # same bytes, other shape
+    for pos in (0, 7, 8, 1234, 4095):
+        for bit in (0, 7):
+            b2 = blob.copy()
+            b2[pos] ^= 1 << bit
+            assert oracle.weights_checksum([0], [2], [[32, 64, 1, 1]], [-1], 0, 1, b2)[0] != base
+    b2 = blob.copy()
+    b2[0:4], b2[4:8] = blob[4:8], blob[0:4]                                                     # two words swapped
+    assert oracle.weights_checksum([0], [2], [[32, 64, 1, 1]], [-1], 0, 1, b2)[0] != base
+    # one non-zero word (value 3 at word index 2), by hand with Python integers
+    one = np.zeros(16, dtype=np.uint8)
+    one[8] = 3
+    key2 = (((2 * 0x9E3779B1) << 1) | 1) % 2 ** 32
+    assert oracle.weights_checksum([0], [4], [[4, 1, 1, 1]], [-1], 0, 1, one)[0] == 3 * key2
+    # a slice that cuts words in half has no checksum
+    with pytest.raises(ValueError):
+        oracle.weights_checksum([0], [1], [[4, 6, 1, 1]], [1], 0, 3, blob)
+
+
 # ------------------------------------------------------------------ workload generators
 def test_config1_sizes():
     shape, NB, src, dst = wl.config1()
