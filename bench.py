@@ -668,7 +668,8 @@ def run_extras(args, tc, torch, stream):
         plan = tc.tc_plan_create(tc.kv_spec(
             tc.TC_KV_MIXED, shape.tuple, src_pool=dev_pool, dst_pool=host_pool,
             T=st.offload_T, bt_off=st.offload_off, bt_src=st.offload_dev, bt_dst=st.offload_host,
-            reload=dict(T=st.reload_T, bt_off=st.reload_off, bt_src=st.reload_host, bt_dst=st.reload_dev)))
+            reload=dict(T=st.reload_T, bt_off=st.reload_off, bt_src=st.reload_host, bt_dst=st.reload_dev),
+            flags=0 if args.host_path == "zerocopy" else tc.TC_PLAN_STAGED))
         if i >= 1:
             create.append(1e3 * (time.perf_counter() - t0))
             h2d += int(st.reload_T.sum()) * shape.token_bytes
@@ -683,6 +684,7 @@ def run_extras(args, tc, torch, stream):
         "plans_per_s": n_steps / wall, "ms_per_step_wall": 1e3 * wall / n_steps, "plan_create_ms": statistics.mean(create),
         "h2d_GBps": h2d / wall / GB, "d2h_GBps": d2h / wall / GB, "link_GBps_both_directions": (h2d + d2h) / wall / GB,
         "h2d_bytes_per_step": h2d // n_steps, "d2h_bytes_per_step": d2h // n_steps,
+        "host_path": args.host_path,
         "note": "wall clock over create + execute + synchronise of every step; reload and offload run concurrently on two streams"}
     del dev, host
     torch.cuda.empty_cache()

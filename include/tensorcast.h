@@ -103,14 +103,18 @@ enum {
     TC_PLAN_HOST_ONLY = 1u, /* validate and lower on the host only: the plan can be inspected
                                (tc_plan_stats, tc_plan_descriptors) but not executed, and no
                                CUDA call is made */
-    TC_PLAN_STAGED = 2u,    /* TC_KV_PACK / TC_KV_UNPACK whose packed buffer is PINNED HOST memory:
-                               instead of letting the kernel load / store host memory directly
-                               (zero copy, the default), move the packed bytes with the copy
-                               engines through a ring of device staging buffers owned by the
-                               library (3 x 64 MiB per device, shared by all staged plans,
-                               allocated when the first such plan is created) and run the kernel
-                               device to device, segment by segment, overlapped on an internal
-                               stream.  This is the streaming pipeline of pinned buffers and
+    TC_PLAN_STAGED = 2u,    /* TC_KV_PACK / TC_KV_UNPACK whose packed buffer is PINNED HOST memory,
+                               or TC_KV_MIXED whose dst_pool is a page-first pinned host pool in
+                               one allocation (plane_stride = one block of one plane) moved in
+                               full blocks: instead of letting the kernel load / store host
+                               memory directly (zero copy, the default), move the host-side
+                               bytes with the copy engines through rings of device staging
+                               buffers owned by the library (one ring of 3 x 64 MiB per
+                               direction and device, shared by all staged plans, allocated when
+                               the first such plan is created) and run the kernel device to
+                               device, segment by segment, overlapped on internal streams.  A
+                               packed buffer travels in contiguous ranges, a paged host pool
+                               page by page.  Groups that cannot be staged stay zero copy.  This is the streaming pipeline of pinned buffers and
                                asynchronous streams (Sec. 5) with the scatter / layout
                                transform fused into its device leg.  The copy engines drive the
                                host link with larger transactions than SM loads and stores, so

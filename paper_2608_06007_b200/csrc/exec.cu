@@ -461,12 +461,18 @@ static int launch_any(const tc_plan *plan, const Group &g, const void *const *sr
 
 // ---- staged host path: copy engines <-> device staging ring <-> kernel ----------------------
 constexpr int kMaxDevices = 64;
-struct StageArena {
+// One ring per direction (0: device -> host, 1: host -> device), so that an offload and a
+// reload running concurrently on two streams do not wait on each other's buffers.
+struct StageRing {
     char *buf[kStageBuffers] = {};
-    cudaEvent_t ready[kStageBuffers] = {}, freed[kStageBuffers] = {}, entry = nullptr;
+    cudaEvent_t ready[kStageBuffers] = {}, freed[kStageBuffers] = {};
     bool freed_recorded[kStageBuffers] = {};
     cudaStream_t copy = nullptr;
     uint64_t next = 0;
+};
+struct StageArena {
+    StageRing ring[2];
+    cudaEvent_t entry = nullptr;
     int refs = 0;
 };
 static StageArena g_stage[kMaxDevices];
@@ -474,13 +480,15 @@ static pthread_mutex_t g_stage_mu = PTHREAD_MUTEX_INITIALIZER;
 
 static void stage_free(StageArena &a)
 {
-    for (int b = 0; b < kStageBuffers; b++) {
-        if (a.buf[b]) cudaFree(a.buf[b]);
-        if (a.ready[b]) cudaEventDestroy(a.ready[b]);
-        if (a.freed[b]) cudaEventDestroy(a.freed[b]);
+    for (StageRing &r : a.ring) {
+        for (int b = 0; b < kStageBuffers; b++) {
+            if (r.buf[b]) cudaFree(r.buf[b]);
+            if (r.ready[b]) cudaEventDestroy(r.ready[b]);
+            if (r.freed[b]) cudaEventDestroy(r.freed[b]);
+        }
+        if (r.copy) cudaStreamDestroy(r.copy);
     }
     if (a.entry) cudaEventDestroy(a.entry);
-    if (a.copy) cudaStreamDestroy(a.copy);
     a = StageArena();
 }
 
@@ -491,21 +499,23 @@ static int stage_acquire(int device, int64_t *bytes)
     StageArena &a = g_stage[device];
     int rc = TC_OK;
     if (a.refs == 0) {
-        cudaError_t e = cudaStreamCreateWithFlags(&a.copy, cudaStreamNonBlocking);
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&a.entry, cudaEventDisableTiming);
-        for (int b = 0; b < kStageBuffers && e == cudaSuccess; b++) {
-            e = cudaMalloc(&a.buf[b], kStageBytes);
-            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&a.ready[b], cudaEventDisableTiming);
-            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&a.freed[b], cudaEventDisableTiming);
+        cudaError_t e = cudaEventCreateWithFlags(&a.entry, cudaEventDisableTiming);
+        for (StageRing &r : a.ring) {
+            if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&r.copy, cudaStreamNonBlocking);
+            for (int b = 0; b < kStageBuffers && e == cudaSuccess; b++) {
+                e = cudaMalloc(&r.buf[b], kStageBytes);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&r.ready[b], cudaEventDisableTiming);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&r.freed[b], cudaEventDisableTiming);
+            }
         }
         if (e != cudaSuccess) {
-            rc = e == cudaErrorMemoryAllocation ? fail(TC_ERR_OOM, "device allocation of the staging ring failed") : cuda_fail(e, "creating the staging ring");
+            rc = e == cudaErrorMemoryAllocation ? fail(TC_ERR_OOM, "device allocation of the staging rings failed") : cuda_fail(e, "creating the staging rings");
             stage_free(a);
         }
     }
     if (rc == TC_OK) {
         a.refs++;
-        *bytes = kStageBytes * kStageBuffers;
+        *bytes = 2 * kStageBytes * kStageBuffers;
     }
     pthread_mutex_unlock(&g_stage_mu);
     return rc;
@@ -517,7 +527,7 @@ static void stage_release(int device)
     pthread_mutex_lock(&g_stage_mu);
     StageArena &a = g_stage[device];
     if (a.refs > 0 && --a.refs == 0) {
-        cudaStreamSynchronize(a.copy);
+        for (StageRing &r : a.ring) cudaStreamSynchronize(r.copy);
         stage_free(a);
     }
     pthread_mutex_unlock(&g_stage_mu);
@@ -529,45 +539,49 @@ static void stage_release(int device)
         if (e_ != cudaSuccess) { rc = cuda_fail(e_, what); goto out; } \
     } while (0)
 
-// gi == 0: pack, device pool -> staging (kernel, caller's stream) -> host (copy engine).
-// gi == 1: unpack, host -> staging (copy engine) -> device pool (kernel, caller's stream).
+// gi == 0: device pool -> staging (kernel, caller's stream) -> host (copy engine).
+// gi == 1: host -> staging (copy engine) -> device pool (kernel, caller's stream).
+// The host side is table entry 0 of the call (the packed buffer, or the paged host pool).
 // Every segment's kernel sees the staging buffer through a base pointer shifted by the
-// segment's packed offset, so the descriptors are used unchanged.
+// segment's packed offset (0 for paged pools), so the descriptors are used unchanged.
 static int execute_staged(const tc_plan *plan, int gi, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s)
 {
     StageArena &a = g_stage[plan->device];
+    StageRing &r = a.ring[gi];
     int rc = TC_OK;
     pthread_mutex_lock(&g_stage_mu);
     TC_TRY(cudaEventRecord(a.entry, s), "cudaEventRecord");
-    TC_TRY(cudaStreamWaitEvent(a.copy, a.entry, 0), "cudaStreamWaitEvent");
+    TC_TRY(cudaStreamWaitEvent(r.copy, a.entry, 0), "cudaStreamWaitEvent");
     for (const Segment &seg : g.segments) {
-        const int b = static_cast<int>(a.next++ % kStageBuffers);
-        char *shifted = a.buf[b] - seg.lo;
+        const int b = static_cast<int>(r.next++ % kStageBuffers);
+        char *shifted = r.buf[b] - seg.shift;
         const uint32_t pa = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(shifted) | 16));
         if (gi == 1) {
             const char *host = static_cast<const char *>(src[0]);
-            if (a.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(a.copy, a.freed[b], 0), "cudaStreamWaitEvent");
-            TC_TRY(cudaMemcpyAsync(a.buf[b], host + seg.lo, static_cast<size_t>(seg.bytes), cudaMemcpyHostToDevice, a.copy), "cudaMemcpyAsync(host to staging)");
-            TC_TRY(cudaEventRecord(a.ready[b], a.copy), "cudaEventRecord");
-            TC_TRY(cudaStreamWaitEvent(s, a.ready[b], 0), "cudaStreamWaitEvent");
+            if (r.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(r.copy, r.freed[b], 0), "cudaStreamWaitEvent");
+            for (uint32_t c = seg.copy0; c < seg.copy0 + seg.ncopy; c++)
+                TC_TRY(cudaMemcpyAsync(r.buf[b] + g.copies[c].stage_off, host + g.copies[c].host_off, static_cast<size_t>(g.copies[c].bytes), cudaMemcpyHostToDevice, r.copy), "cudaMemcpyAsync(host to staging)");
+            TC_TRY(cudaEventRecord(r.ready[b], r.copy), "cudaEventRecord");
+            TC_TRY(cudaStreamWaitEvent(s, r.ready[b], 0), "cudaStreamWaitEvent");
             const void *stage_src[1] = {shifted};
             if ((rc = launch_any(plan, g, stage_src, dst, pa, s, &seg)) != TC_OK) goto out;
-            TC_TRY(cudaEventRecord(a.freed[b], s), "cudaEventRecord");
+            TC_TRY(cudaEventRecord(r.freed[b], s), "cudaEventRecord");
         } else {
             char *host = static_cast<char *>(dst[0]);
-            if (a.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(s, a.freed[b], 0), "cudaStreamWaitEvent");
+            if (r.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(s, r.freed[b], 0), "cudaStreamWaitEvent");
             void *stage_dst[1] = {shifted};
             if ((rc = launch_any(plan, g, src, stage_dst, pa, s, &seg)) != TC_OK) goto out;
-            TC_TRY(cudaEventRecord(a.ready[b], s), "cudaEventRecord");
-            TC_TRY(cudaStreamWaitEvent(a.copy, a.ready[b], 0), "cudaStreamWaitEvent");
-            TC_TRY(cudaMemcpyAsync(host + seg.lo, a.buf[b], static_cast<size_t>(seg.bytes), cudaMemcpyDeviceToHost, a.copy), "cudaMemcpyAsync(staging to host)");
-            TC_TRY(cudaEventRecord(a.freed[b], a.copy), "cudaEventRecord");
+            TC_TRY(cudaEventRecord(r.ready[b], s), "cudaEventRecord");
+            TC_TRY(cudaStreamWaitEvent(r.copy, r.ready[b], 0), "cudaStreamWaitEvent");
+            for (uint32_t c = seg.copy0; c < seg.copy0 + seg.ncopy; c++)
+                TC_TRY(cudaMemcpyAsync(host + g.copies[c].host_off, r.buf[b] + g.copies[c].stage_off, static_cast<size_t>(g.copies[c].bytes), cudaMemcpyDeviceToHost, r.copy), "cudaMemcpyAsync(staging to host)");
+            TC_TRY(cudaEventRecord(r.freed[b], r.copy), "cudaEventRecord");
         }
-        a.freed_recorded[b] = true;
+        r.freed_recorded[b] = true;
     }
     if (gi == 0)  // the caller's stream completes only when the last copies to the host have landed
         for (int b = 0; b < kStageBuffers; b++)
-            if (a.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(s, a.freed[b], 0), "cudaStreamWaitEvent");
+            if (r.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(s, r.freed[b], 0), "cudaStreamWaitEvent");
 out:
     pthread_mutex_unlock(&g_stage_mu);
     return rc;

@@ -54,7 +54,13 @@ static_assert(sizeof(Desc) == 128, "Desc must stay 128 bytes");
 // A segment of a staged plan is a window whose packed-side bytes are one contiguous range.
 struct Segment {
     uint32_t d0, nd, o0, no;
-    int64_t lo, bytes;  // the packed-buffer byte range the window touches
+    int64_t shift;           // the kernel sees the staging buffer at (buffer - shift)
+    uint32_t copy0, ncopy;   // its copies between host memory and the staging buffer
+};
+
+// One copy-engine transfer of a staged plan.
+struct StageCopy {
+    int64_t stage_off, host_off, bytes;
 };
 
 // Bookkeeping of one request while a KV group is lowered (staged plans cut segments from it).
@@ -68,6 +74,8 @@ struct Group {
     std::vector<uint32_t> tile_desc;  // tile -> descriptor, only for non-uniform groups
     std::vector<RequestSpan> requests; // KV groups with a packed side
     std::vector<Segment> segments;    // staged plans only
+    std::vector<StageCopy> copies;    // staged plans only
+    bool stage_whole_host_pool = false; // staged MIXED group: the host side is a paged pool
     uint32_t tiles_per_desc = 0;      // > 0: every descriptor owns exactly this many tile ids
     FastDiv div_tpd{0, 0};
     uint64_t n_tiles = 0;

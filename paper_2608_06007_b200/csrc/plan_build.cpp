@@ -341,6 +341,24 @@ static void packed_strides(const tc_kv_spec_t &kv, int32_t layout, int64_t Tr, i
     else                  { *sn = row;        *sh = Tr * row; }
 }
 
+static int64_t planes_of(const tc_kv_spec_t &kv) { return kv.L * 2; }
+
+// Staged MIXED group: descriptor k (one per block, in table order) uses ring slot k % slots;
+// a segment is the run of descriptors that fills one staging buffer.
+static void stage_pages(Group &g, const int32_t *host_blocks, int64_t n_blocks, int64_t slots, int64_t page, int64_t host_block_stride)
+{
+    if (static_cast<int64_t>(g.descs.size()) != n_blocks) {  // a block lowered to several descriptors: stay zero copy
+        g.stage_whole_host_pool = false;
+        return;
+    }
+    for (int64_t k0 = 0; k0 < n_blocks; k0 += slots) {
+        const int64_t n = std::min(slots, n_blocks - k0);
+        g.segments.push_back(Segment{static_cast<uint32_t>(k0), static_cast<uint32_t>(n), 0, static_cast<uint32_t>(g.descs[0].n_outer), 0,
+                                     static_cast<uint32_t>(g.copies.size()), static_cast<uint32_t>(n)});
+        for (int64_t k = k0; k < k0 + n; k++) g.copies.push_back(StageCopy{(k - k0) * page, host_blocks[k] * host_block_stride, page});
+    }
+}
+
 // Lower one group.  src_pool / dst_pool null = that side is the packed buffer.
 static void lower_kv_group(Group &g, const tc_kv_spec_t &kv, const tc_kv_group_t &grp, const PoolView *src_pool,
                            const PoolView *dst_pool, int32_t packed_layout, uint32_t tile_bytes)
@@ -407,7 +425,8 @@ static int build_segments(Group &g, int64_t planes)
             int64_t sum = 0;
             size_t j = i;
             while (j < g.requests.size() && sum + planes * g.requests[j].plane_bytes <= kStageBytes) sum += planes * g.requests[j++].plane_bytes;
-            g.segments.push_back(Segment{q.d0, g.requests[j - 1].d1 - q.d0, 0, static_cast<uint32_t>(planes), q.off, sum});
+            g.segments.push_back(Segment{q.d0, g.requests[j - 1].d1 - q.d0, 0, static_cast<uint32_t>(planes), q.off, static_cast<uint32_t>(g.copies.size()), 1});
+            g.copies.push_back(StageCopy{0, q.off, sum});
             i = j;
         } else {
             if (q.plane_bytes > kStageBytes)
@@ -415,7 +434,8 @@ static int build_segments(Group &g, int64_t planes)
             const int64_t per = kStageBytes / q.plane_bytes;
             for (int64_t o0 = 0; o0 < planes; o0 += per) {
                 const int64_t no = std::min(per, planes - o0);
-                g.segments.push_back(Segment{q.d0, q.d1 - q.d0, static_cast<uint32_t>(o0), static_cast<uint32_t>(no), q.off + o0 * q.plane_bytes, no * q.plane_bytes});
+                g.segments.push_back(Segment{q.d0, q.d1 - q.d0, static_cast<uint32_t>(o0), static_cast<uint32_t>(no), q.off + o0 * q.plane_bytes, static_cast<uint32_t>(g.copies.size()), 1});
+                g.copies.push_back(StageCopy{0, q.off + o0 * q.plane_bytes, no * q.plane_bytes});
             }
             i++;
         }
@@ -471,8 +491,36 @@ static int build_kv(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t tile_byt
             if (dev_used[kv.reload.bt_dst[j]])
                 return fail(TC_ERR_OVERLAP, "block %d of src_pool is read by the offload group and written by the reload group", kv.reload.bt_dst[j]);
         }
-        lower_kv_group(g0, kv, kv.group, &sp, &dp, 0, tile_bytes);
-        lower_kv_group(g1, kv, kv.reload, &dp, &sp, 0, tile_bytes);
+        // Staged variant: the host pool's pages travel through the device staging ring with the
+        // copy engines, one transfer per 2 MiB-like page, and the kernels run device to device
+        // against a virtual pool of ring slots.  It needs whole pages on the host side: a
+        // page-first pool in one allocation and groups made of full blocks only.
+        const int64_t page = planes_of(kv) * dp.chunk;
+        auto whole_blocks = [&](const tc_kv_group_t &g) {
+            for (int64_t r = 0; r < g.R; r++)
+                if (g.T[r] % kv.B) return false;
+            return true;
+        };
+        const bool can_stage = (spec->flags & TC_PLAN_STAGED) && kv.dst_pool.n_slots == 1 && dp.plane_stride == dp.chunk &&
+                               page <= kStageBytes && whole_blocks(kv.group) && whole_blocks(kv.reload);
+        if (can_stage) {
+            const int64_t slots = kStageBytes / page;
+            PoolView ring = dp;       // same page layout, block id = slot in the ring buffer
+            ring.block_stride = page;
+            std::vector<int32_t> virt(static_cast<size_t>(std::max(n_off, n_rel)));
+            for (size_t k = 0; k < virt.size(); k++) virt[k] = static_cast<int32_t>(k % slots);
+            tc_kv_group_t off_v = kv.group, rel_v = kv.reload;
+            off_v.bt_dst = virt.data();
+            rel_v.bt_src = virt.data();
+            lower_kv_group(g0, kv, off_v, &sp, &ring, 0, tile_bytes);
+            lower_kv_group(g1, kv, rel_v, &ring, &sp, 0, tile_bytes);
+            g0.stage_whole_host_pool = g1.stage_whole_host_pool = true;
+            stage_pages(g0, kv.group.bt_dst, n_off, slots, page, dp.block_stride);
+            stage_pages(g1, kv.reload.bt_src, n_rel, slots, page, dp.block_stride);
+        } else {
+            lower_kv_group(g0, kv, kv.group, &sp, &dp, 0, tile_bytes);
+            lower_kv_group(g1, kv, kv.reload, &dp, &sp, 0, tile_bytes);
+        }
         g0.n_src = kv.src_pool.n_slots;
         g0.n_dst = kv.dst_pool.n_slots;
         g1.n_src = kv.dst_pool.n_slots;
@@ -639,10 +687,22 @@ int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
     if ((spec->flags & TC_PLAN_CHECKSUM) && spec->kind != TC_WEIGHTS)
         return fail(TC_ERR_KIND, "TC_PLAN_CHECKSUM applies to TC_WEIGHTS plans only");
     if (spec->flags & TC_PLAN_STAGED) {
-        if (spec->kind != TC_KV_PACK && spec->kind != TC_KV_UNPACK)
-            return fail(TC_ERR_KIND, "TC_PLAN_STAGED applies to TC_KV_PACK and TC_KV_UNPACK plans only");
-        Group &g = plan->group[spec->kind == TC_KV_PACK ? 0 : 1];
-        if ((rc = build_segments(g, spec->kv.L * 2))) return rc;
+        if (spec->kind != TC_KV_PACK && spec->kind != TC_KV_UNPACK && spec->kind != TC_KV_MIXED)
+            return fail(TC_ERR_KIND, "TC_PLAN_STAGED applies to TC_KV_PACK, TC_KV_UNPACK and TC_KV_MIXED plans only");
+        if (spec->kind == TC_KV_MIXED) {
+            // segments were cut while lowering; a group that could not be staged must drop them
+            for (int k = 0; k < 2; k++) {
+                Group &g = plan->group[k];
+                if (!g.stage_whole_host_pool || !g.tiles_per_desc) {
+                    if (g.stage_whole_host_pool && !g.descs.empty()) return fail(TC_ERR_INVALID_ARG, "staged MIXED group is not uniform");
+                    g.segments.clear();
+                    g.copies.clear();
+                }
+            }
+        } else {
+            Group &g = plan->group[spec->kind == TC_KV_PACK ? 0 : 1];
+            if ((rc = build_segments(g, spec->kv.L * 2))) return rc;
+        }
     }
     return TC_OK;
 }

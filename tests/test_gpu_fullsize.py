@@ -236,7 +236,8 @@ def test_config4_full_size_migration_70b_shape():
     _free()
 
 
-def test_config5_mixed_steps_device_pool_and_pinned_paged_host_pool():
+@pytest.mark.parametrize("flags", [0, tc.TC_PLAN_STAGED])
+def test_config5_mixed_steps_device_pool_and_pinned_paged_host_pool(flags):
     shape = wl.LLAMA3_8B_KV
     s, chunk, planes = shape.tuple, shape.chunk_bytes, shape.L * 2
     NBd, NBh = 20000, 4096                       # host pool shrunk to 8 GiB of pinned memory
@@ -258,8 +259,9 @@ def test_config5_mixed_steps_device_pool_and_pinned_paged_host_pool():
         before_host_reads = H[step.reload_host].copy()                                       # inputs of the reload
         spec = tc.kv_spec(tc.TC_KV_MIXED, s, src_pool=dev_pool, dst_pool=host_pool,
                           T=step.offload_T, bt_off=step.offload_off, bt_src=step.offload_dev, bt_dst=step.offload_host,
-                          reload=dict(T=step.reload_T, bt_off=step.reload_off, bt_src=step.reload_host, bt_dst=step.reload_dev))
+                          reload=dict(T=step.reload_T, bt_off=step.reload_off, bt_src=step.reload_host, bt_dst=step.reload_dev), flags=flags)
         plan = tc.tc_plan_create(spec)
+        assert plan.stats().path[1] == (3 if flags else 1)
         torch.cuda.synchronize()
         tc.tc_kv_pack(plan, [dev], [host], stream=s1)
         tc.tc_kv_unpack(plan, [host], [dev], stream=s2)

@@ -151,7 +151,8 @@ def test_migrate_pool_to_pool(src_l, dst_l):
     assert np.array_equal(out.result(), want)
 
 
-def test_mixed_plan_offload_and_reload_through_pinned_host_pool():
+@pytest.mark.parametrize("flags", [0, tc.TC_PLAN_STAGED])
+def test_mixed_plan_offload_and_reload_through_pinned_host_pool(flags):
     """Device NHD pool <-> pinned page-first HND host pool, both directions of one plan on two
     streams; the kernels store into / load from host memory directly."""
     shape = wl.KVShape(L=2, B=16, H=8, D=128, E=2)
@@ -172,8 +173,9 @@ def test_mixed_plan_offload_and_reload_through_pinned_host_pool():
     spec = tc.kv_spec(tc.TC_KV_MIXED, s, src_pool=tc.pool(tc.TC_NHD, NBd, 1, plane_stride=NBd * chunk, slot_bytes=devp.size),
                       dst_pool=tc.pool(tc.TC_HND, NBh, 1, plane_stride=chunk, block_stride=4 * chunk, slot_bytes=hostp.size),
                       T=step.offload_T, bt_off=step.offload_off, bt_src=step.offload_dev, bt_dst=step.offload_host,
-                      reload=dict(T=step.reload_T, bt_off=step.reload_off, bt_src=step.reload_host, bt_dst=step.reload_dev))
+                      reload=dict(T=step.reload_T, bt_off=step.reload_off, bt_src=step.reload_host, bt_dst=step.reload_dev), flags=flags)
     plan = tc.tc_plan_create(spec)
+    assert plan.stats().path[0] == (3 if flags else 1) and plan.stats().path[1] == (3 if flags else 1)
     s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
     torch.cuda.synchronize()
     tc.tc_kv_pack(plan, [d_dev], [h_host], stream=s1)
