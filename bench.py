@@ -426,21 +426,63 @@ def run_ours(args):
             ceil_h2d = ceiling(lambda: Q[:n_c].copy_(Qh[:n_c], non_blocking=True), n_c)
             ceil_d2h = ceiling(lambda: Qh[:n_c].copy_(Q[:n_c], non_blocking=True), n_c)
 
+        duplex = args.e2e_schedule == "duplex"
+        Qh2 = torch.empty(max_packed, dtype=torch.uint8).pin_memory() if duplex else Qh
+        Qhs = (Qh, Qh2)
+        stream_u = torch.cuda.Stream() if duplex else stream
+        su = stream_u.cuda_stream
+        ev_packed = [torch.cuda.Event() for _ in range(2)]
+        ev_unpacked = [torch.cuda.Event() for _ in range(2)]
+        ev_fork, ev_join = torch.cuda.Event(), torch.cuda.Event()
+
+        def bidir_ceiling():  # both directions at once with cudaMemcpyAsync, GB/s summed
+            n_c = min(Qh.numel(), 4 << 30)
+            best = 1e9
+            for _ in range(3):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                ev_fork.record(stream)
+                stream_u.wait_event(ev_fork)
+                Qh[:n_c].copy_(Q[:n_c], non_blocking=True)
+                with torch.cuda.stream(stream_u):
+                    poolB[:n_c].copy_(Qh2[:n_c], non_blocking=True)
+                    ev_join.record(stream_u)
+                stream.wait_event(ev_join)
+                b.record(stream)
+                torch.cuda.synchronize()
+                best = min(best, a.elapsed_time(b))
+            return 2 * n_c / (best * 1e-3) / GB
+
         def e2e_step():
+            """Offload every wave to pinned host memory and reload it into the second pool; load the
+            weights from the pinned blob.  duplex: the link is full duplex, so wave k+1 is offloaded
+            (stream) while wave k is reloaded (stream_u), through two host buffers."""
             h2d = d2h = 0
-            for p in plans:
-                tc.tc_kv_pack(p["pack_h"], [poolA], [Qh], sp)      # offload: kernel stores into host memory
-                tc.tc_kv_unpack(p["unpack_h"], [Qh], [poolB], sp)  # reload: kernel loads from host memory
+            ev_fork.record(stream)
+            stream_u.wait_event(ev_fork)
+            tc.tc_weights_materialize(w_full_h, blob_h, full_ptrs, su)
+            tc.tc_weights_materialize(w_shard_h, blob_h, shard_ptrs, su)
+            h2d += sum(full_sizes) + sum(shard_sizes)
+            for k, p in enumerate(plans):
+                i = k % 2 if duplex else 0
+                if k >= (2 if duplex else 1):
+                    stream.wait_event(ev_unpacked[i])                    # the host buffer is free again
+                tc.tc_kv_pack(p["pack_h"], [poolA], [Qhs[i]], sp)        # offload (device -> host)
+                ev_packed[i].record(stream)
+                stream_u.wait_event(ev_packed[i])
+                tc.tc_kv_unpack(p["unpack_h"], [Qhs[i]], [poolB], su)    # reload (host -> device)
+                ev_unpacked[i].record(stream_u)
                 d2h += p["payload"]
                 h2d += p["payload"]
-            tc.tc_weights_materialize(w_full_h, blob_h, full_ptrs, sp)
-            tc.tc_weights_materialize(w_shard_h, blob_h, shard_ptrs, sp)
-            h2d += sum(full_sizes) + sum(shard_sizes)
-            probe.copy_(dst_full[-4096:], non_blocking=True)       # read a result back
+            with torch.cuda.stream(stream_u):
+                probe.copy_(dst_full[-4096:], non_blocking=True)         # read a result back
+                ev_join.record(stream_u)
+            stream.wait_event(ev_join)
             d2h += 4096
             return h2d, d2h
 
         with torch.cuda.stream(stream):
+            ceil_bidir = bidir_ceiling() if duplex else None
             for _ in range(args.e2e_warmup):
                 e2e_step()
             barrier()
@@ -457,12 +499,14 @@ def run_ours(args):
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
                "ms_per_step": e_ms / args.e2e_steps,
                "host_link_GBps": world * (h2d + d2h) * args.e2e_steps / (e_ms * 1e-3) / GB,
-               "host_link_ceiling_GBps": {"h2d_cudaMemcpyAsync": ceil_h2d, "d2h_cudaMemcpyAsync": ceil_d2h},
-               "host_link_frac_of_ceiling": (h2d + d2h) * args.e2e_steps / (e_ms * 1e-3) / GB / ((h2d + d2h) / (h2d / ceil_h2d + d2h / ceil_d2h)),
-               "kv_host_path": args.host_path,
+               "host_link_ceiling_GBps": {"h2d_cudaMemcpyAsync": ceil_h2d, "d2h_cudaMemcpyAsync": ceil_d2h,
+                                          "both_directions_at_once_summed": ceil_bidir},
+               "host_link_frac_of_ceiling": (h2d + d2h) * args.e2e_steps / (e_ms * 1e-3) / GB /
+                                            (ceil_bidir if duplex else (h2d + d2h) / (h2d / ceil_h2d + d2h / ceil_d2h)),
+               "kv_host_path": args.host_path, "schedule": args.e2e_schedule,
                "note": "packed KV buffer and weight blob in pinned host memory; KV: copy engines + device staging ring + D2D kernel "
                        "(staged) or kernel loads/stores on host memory (zerocopy); weights: kernel loads from the pinned blob"}
-        del Qh, blob_h
+        del Qh, Qh2, Qhs, blob_h
 
     extras = None
     if not args.no_extras and world == 1:
@@ -724,6 +768,8 @@ def main():
     ap.add_argument("--burst-steps", type=int, default=10, help="configs[4]: scheduler steps timed (the workload has 200)")
     ap.add_argument("--host-ctas", type=int, default=0)
     ap.add_argument("--host-path", default="staged", choices=["staged", "zerocopy"])
+    ap.add_argument("--e2e-schedule", default="duplex", choices=["duplex", "serial"],
+                    help="duplex: offload wave k+1 while wave k reloads (two streams, two host buffers)")
     args = ap.parse_args()
     if args.dry_run:
         run_dry(args)
