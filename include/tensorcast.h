@@ -111,8 +111,8 @@ enum {
                                bytes with the copy engines through rings of device staging
                                buffers owned by the library (one ring of 3 x 64 MiB per
                                direction and device, shared by all staged plans, allocated when
-                               the first such plan is created) and run the kernel device to
-                               device, segment by segment, overlapped on internal streams.  A
+                               the first such plan is created and kept until the process
+                               exits) and run the kernel device to device, segment by segment, overlapped on internal streams.  A
                                packed buffer travels in contiguous ranges, a paged host pool
                                page by page.  Groups that cannot be staged stay zero copy.  This is the streaming pipeline of pinned buffers and
                                asynchronous streams (Sec. 5) with the scatter / layout

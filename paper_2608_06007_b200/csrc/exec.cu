@@ -499,6 +499,7 @@ static int stage_acquire(int device, int64_t *bytes)
     StageArena &a = g_stage[device];
     int rc = TC_OK;
     if (a.refs == 0) {
+        a.refs = 1;  // the library's own reference: keeps the rings alive between plans
         cudaError_t e = cudaEventCreateWithFlags(&a.entry, cudaEventDisableTiming);
         for (StageRing &r : a.ring) {
             if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&r.copy, cudaStreamNonBlocking);
@@ -510,7 +511,7 @@ static int stage_acquire(int device, int64_t *bytes)
         }
         if (e != cudaSuccess) {
             rc = e == cudaErrorMemoryAllocation ? fail(TC_ERR_OOM, "device allocation of the staging rings failed") : cuda_fail(e, "creating the staging rings");
-            stage_free(a);
+            stage_free(a);  // also resets refs to 0
         }
     }
     if (rc == TC_OK) {
@@ -521,15 +522,14 @@ static int stage_acquire(int device, int64_t *bytes)
     return rc;
 }
 
+// The rings are kept once allocated (like the plan-storage cache): a caller that creates one
+// staged plan per scheduler step must not pay six cudaMalloc / cudaFree pairs per step.
 static void stage_release(int device)
 {
     if (device < 0 || device >= kMaxDevices) return;
     pthread_mutex_lock(&g_stage_mu);
     StageArena &a = g_stage[device];
-    if (a.refs > 0 && --a.refs == 0) {
-        for (StageRing &r : a.ring) cudaStreamSynchronize(r.copy);
-        stage_free(a);
-    }
+    if (a.refs > 1) a.refs--;  // the last reference is never dropped: the rings stay until exit
     pthread_mutex_unlock(&g_stage_mu);
 }
 
