@@ -99,6 +99,12 @@ typedef enum {
 
 typedef enum { TC_NHD = 0, TC_HND = 1 } tc_layout;
 
+/* Order of the packed buffer.  Request-major (default): each request is one self-contained
+ * contiguous region.  Layer-major: plane (l,c) of ALL requests is contiguous,
+ *   plane(l,c) = (l*2 + c) * (sum_q T_q) * Hs*D*E,  request r inside it at (sum_{q<r} T_q) * Hs*D*E,
+ * so that a consumer can start on the first layers while later ones are still in flight. */
+typedef enum { TC_REQUEST_MAJOR = 0, TC_LAYER_MAJOR = 1 } tc_packed_order;
+
 enum {
     TC_PLAN_HOST_ONLY = 1u, /* validate and lower on the host only: the plan can be inspected
                                (tc_plan_stats, tc_plan_descriptors) but not executed, and no
@@ -121,6 +127,11 @@ enum {
                                this path is a few percent faster; it costs one launch and one
                                copy per segment instead of one launch per call.  Staged
                                executions are serialised with one another by the library. */
+    TC_PLAN_SAME_POOL = 8u, /* TC_KV_MIGRATE inside ONE pool (compaction / defragmentation): the
+                               caller will pass the same table as source and destination.
+                               src_pool and dst_pool must describe the same geometry, and no
+                               block may be both read and written (TC_ERR_OVERLAP), so that the
+                               result does not depend on the order in which tiles run. */
     TC_PLAN_CHECKSUM = 4u   /* TC_WEIGHTS: the plan can also be run by
                                tc_weights_materialize_checksum, which folds an integrity
                                checksum of every tensor into the same pass as the copy.  Needs
@@ -158,9 +169,14 @@ typedef struct {
     tc_kv_pool_t src_pool;   /* PACK, MIGRATE, MIXED (the device pool) */
     tc_kv_pool_t dst_pool;   /* UNPACK, MIGRATE, MIXED (the host pool) */
     int32_t packed_layout;   /* PACK / UNPACK: tc_layout of the packed buffer */
-    int32_t reserved;        /* 0 */
+    int32_t packed_order;    /* PACK / UNPACK: tc_packed_order */
     int64_t packed_bytes;    /* PACK / UNPACK: capacity of the packed buffer, for bounds checks;
                                 0 = exactly the required size */
+    int64_t head_begin;      /* PACK / UNPACK: the packed buffer holds heads [head_begin, */
+    int64_t head_count;      /*   head_begin + head_count) only (a tensor-parallel consumer's view
+                                of the request): H becomes Hs = head_count and h becomes
+                                h - head_begin in the packed formulas; the other heads of the
+                                pool are neither read nor written.  head_count 0 = all H heads */
     tc_kv_group_t group;     /* PACK, UNPACK, MIGRATE; MIXED: the offload group */
     tc_kv_group_t reload;    /* MIXED only: moves dst_pool[bt_src] -> src_pool[bt_dst] */
 } tc_kv_spec_t;

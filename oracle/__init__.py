@@ -20,6 +20,7 @@ from concurrent.futures import ThreadPoolExecutor
 import numpy as np
 
 NHD, HND = 0, 1
+REQUEST_MAJOR, LAYER_MAJOR = 0, 1
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "tc_oracle.c")
@@ -42,6 +43,17 @@ class _Shape(C.Structure):
 
 class _Geom(C.Structure):
     _fields_ = [("layout", C.c_int32), ("block_stride", C.c_int64)]
+
+
+class _Packed(C.Structure):
+    _fields_ = [("layout", C.c_int32), ("order", C.c_int32), ("h0", C.c_int64), ("hs", C.c_int64)]
+
+
+def _packed_geom(shape, layout, order, head_begin, head_count):
+    H = shape[2]
+    hs = H - head_begin if head_count is None else head_count
+    assert 0 <= head_begin and hs >= 0 and head_begin + hs <= H
+    return _Packed(layout, order, head_begin, hs)
 
 
 _lib = None
@@ -96,25 +108,29 @@ def _run(fn, ranges, threads):
             list(ex.map(lambda ab: fn(*ab), ranges))
 
 
-def packed_nbytes(shape, T) -> int:
-    """Size of the packed buffer: sum over requests of L*2*T_r*H*D*E."""
+def packed_nbytes(shape, T, head_count=None) -> int:
+    """Size of the packed buffer: sum over requests of L*2*T_r*Hs*D*E (Hs = heads it holds)."""
     L, B, H, D, E = shape
+    H = H if head_count is None else head_count
     return int(sum(L * 2 * int(t) * H * D * E for t in T))
 
 
 def kv_pack(shape, pool_layout, block_stride, planes, T, bt_off, bt, packed_layout,
-            packed, packed_cnt=None, threads=1, requests=None):
+            packed, packed_cnt=None, threads=1, requests=None, order=REQUEST_MAJOR,
+            head_begin=0, head_count=None):
     """publish / offload: pool planes -> packed buffer (written in place).
-    requests=(r0, r1) restricts the loops to requests [r0, r1) (same arithmetic)."""
+    requests=(r0, r1) restricts the loops to requests [r0, r1) (same arithmetic).
+    order / head_begin / head_count: layer-major packed order, head slice of the packed side."""
     lib = _load()
     s, g = _Shape(*shape), _Geom(pool_layout, block_stride)
+    pg = _packed_geom(shape, packed_layout, order, head_begin, head_count)
     T, bt_off, bt = _i64(T), _i64(bt_off), _i32(bt)
     tbl = _ptr_table(planes)
     R = len(T)
 
     def go(r0, r1):
         lib.oracle_kv_pack(C.byref(s), C.byref(g), tbl, C.c_int64(R), T.ctypes, bt_off.ctypes,
-                           bt.ctypes, C.c_int32(packed_layout), C.c_void_p(_u8(packed).ctypes.data),
+                           bt.ctypes, C.byref(pg), C.c_void_p(_u8(packed).ctypes.data),
                            C.c_void_p(None if packed_cnt is None else _u8(packed_cnt).ctypes.data),
                            C.c_int64(r0), C.c_int64(r1))
     _run(go, _ranges(R, threads, requests), threads)
@@ -133,10 +149,12 @@ def kv_pack_inverse(shape, pool_layout, block_stride, planes, T, bt_off, bt, pac
 
 
 def kv_unpack(shape, pool_layout, block_stride, planes, T, bt_off, bt, packed_layout,
-              packed, plane_cnt=None, threads=1, requests=None):
+              packed, plane_cnt=None, threads=1, requests=None, order=REQUEST_MAJOR,
+              head_begin=0, head_count=None):
     """hydrate / reload: packed buffer -> pool planes (written in place)."""
     lib = _load()
     s, g = _Shape(*shape), _Geom(pool_layout, block_stride)
+    pg = _packed_geom(shape, packed_layout, order, head_begin, head_count)
     T, bt_off, bt = _i64(T), _i64(bt_off), _i32(bt)
     tbl = _ptr_table(planes)
     cnt = None if plane_cnt is None else _ptr_table(plane_cnt)
@@ -144,7 +162,7 @@ def kv_unpack(shape, pool_layout, block_stride, planes, T, bt_off, bt, packed_la
 
     def go(r0, r1):
         lib.oracle_kv_unpack(C.byref(s), C.byref(g), tbl, cnt, C.c_int64(R), T.ctypes,
-                             bt_off.ctypes, bt.ctypes, C.c_int32(packed_layout),
+                             bt_off.ctypes, bt.ctypes, C.byref(pg),
                              C.c_void_p(_u8(packed).ctypes.data), C.c_int64(r0), C.c_int64(r1))
     _run(go, _ranges(R, threads, requests), threads)
 

@@ -30,6 +30,14 @@
  *     off_0 = 0, off_{r+1} = off_r + L*2*T_r*H*D*E, and inside request r
  *     NHD: off_r + ((((l*2 + c)*T_r + t)*H + h)*D + d)*E + e
  *     HND: off_r + ((((l*2 + c)*H + h)*T_r + t)*D + d)*E + e
+ *   Two options of the packed side (a consumer's view of the request, Table 2 "view"):
+ *   - head slice [h0, h0+Hs): the packed buffer holds only those heads; H becomes Hs and h
+ *     becomes h - h0 in the formulas above (a tensor-parallel consumer owns a head range);
+ *   - layer-major order: plane (l,c) of ALL requests is contiguous, so that a consumer can
+ *     start on layer 0 while later layers are still in flight:
+ *       plane(l,c) = (l*2 + c) * (sum_q T_q) * Hs*D*E,  req_r = (sum_{q<r} T_q) * Hs*D*E
+ *       NHD: plane + req_r + ((t*Hs + h')*D + d)*E + e
+ *       HND: plane + req_r + ((h'*T_r + t)*D + d)*E + e
  *
  * Every function optionally bumps a per-byte write counter (uint8, saturating)
  * so the tests can prove that each destination byte is written exactly once.
@@ -64,46 +72,53 @@ static int64_t pool_off(const oracle_kv_shape *s, const oracle_pool_geom *g,
     return b * g->block_stride + ((h * s->B + n) * s->D + d) * s->E + e;
 }
 
-/* Byte offset, from the start of request r's packed region, of byte e of (l,c,t,h,d). */
-static int64_t packed_off(const oracle_kv_shape *s, int32_t layout, int64_t Tr,
-                          int64_t l, int64_t c, int64_t t, int64_t h, int64_t d, int64_t e)
-{
-    if (layout == ORACLE_NHD)
-        return ((((l * 2 + c) * Tr + t) * s->H + h) * s->D + d) * s->E + e;
-    return ((((l * 2 + c) * s->H + h) * Tr + t) * s->D + d) * s->E + e;
-}
+enum { ORACLE_REQUEST_MAJOR = 0, ORACLE_LAYER_MAJOR = 1 };
 
-/* Start of request r in the packed buffer: sum of the sizes of the requests before it. */
-static int64_t request_off(const oracle_kv_shape *s, const int64_t *T, int64_t r)
+typedef struct {
+    int32_t layout; /* ORACLE_NHD / ORACLE_HND of the packed buffer */
+    int32_t order;  /* ORACLE_REQUEST_MAJOR / ORACLE_LAYER_MAJOR */
+    int64_t h0, hs; /* head slice [h0, h0 + hs) held by the packed buffer */
+} oracle_packed_geom;
+
+/* Byte offset in the packed buffer of byte e of (request r, l, c, token t, head h, d). */
+static int64_t packed_addr(const oracle_kv_shape *s, const oracle_packed_geom *pg, int64_t R,
+                           const int64_t *T, int64_t r, int64_t l, int64_t c, int64_t t,
+                           int64_t h, int64_t d, int64_t e)
 {
-    int64_t off = 0;
-    for (int64_t q = 0; q < r; q++) off += s->L * 2 * T[q] * s->H * s->D * s->E;
-    return off;
+    int64_t hp = h - pg->h0; /* head index inside the slice */
+    int64_t before = 0, total = 0;
+    for (int64_t q = 0; q < R; q++) {
+        if (q < r) before += T[q];
+        total += T[q];
+    }
+    int64_t inner = (pg->layout == ORACLE_NHD) ? ((t * pg->hs + hp) * s->D + d) * s->E + e
+                                               : ((hp * T[r] + t) * s->D + d) * s->E + e;
+    int64_t tok = pg->hs * s->D * s->E; /* bytes of one token of one plane */
+    if (pg->order == ORACLE_REQUEST_MAJOR)
+        return before * s->L * 2 * tok + (l * 2 + c) * T[r] * tok + inner;
+    return (l * 2 + c) * total * tok + before * tok + inner;
 }
 
 /* publish / offload: gather every valid token of every request into the packed buffer. */
 void oracle_kv_pack(const oracle_kv_shape *s, const oracle_pool_geom *g,
                     const uint8_t *const *pool_base, /* [L*2] plane pointers */
                     int64_t R, const int64_t *T, const int64_t *bt_off, const int32_t *bt,
-                    int32_t packed_layout, uint8_t *packed, uint8_t *packed_cnt,
+                    const oracle_packed_geom *pg, uint8_t *packed, uint8_t *packed_cnt,
                     int64_t r_begin, int64_t r_end)
 {
-    (void)R;
-    for (int64_t r = r_begin; r < r_end; r++) {
-        int64_t off_r = request_off(s, T, r);
+    for (int64_t r = r_begin; r < r_end; r++)
         for (int64_t l = 0; l < s->L; l++)
             for (int64_t c = 0; c < 2; c++)
                 for (int64_t t = 0; t < T[r]; t++) {
                     int64_t b = bt[bt_off[r] + t / s->B], n = t % s->B;
-                    for (int64_t h = 0; h < s->H; h++)
+                    for (int64_t h = pg->h0; h < pg->h0 + pg->hs; h++)
                         for (int64_t d = 0; d < s->D; d++)
                             for (int64_t e = 0; e < s->E; e++) {
-                                int64_t q = off_r + packed_off(s, packed_layout, T[r], l, c, t, h, d, e);
+                                int64_t q = packed_addr(s, pg, R, T, r, l, c, t, h, d, e);
                                 packed[q] = pool_base[l * 2 + c][pool_off(s, g, b, n, h, d, e)];
                                 bump(packed_cnt, q);
                             }
                 }
-    }
 }
 
 /* hydrate / reload: scatter the packed buffer into the blocks named by the table.
@@ -111,26 +126,22 @@ void oracle_kv_pack(const oracle_kv_shape *s, const oracle_pool_geom *g,
 void oracle_kv_unpack(const oracle_kv_shape *s, const oracle_pool_geom *g,
                       uint8_t *const *pool_base, uint8_t *const *pool_cnt,
                       int64_t R, const int64_t *T, const int64_t *bt_off, const int32_t *bt,
-                      int32_t packed_layout, const uint8_t *packed,
+                      const oracle_packed_geom *pg, const uint8_t *packed,
                       int64_t r_begin, int64_t r_end)
 {
-    (void)R;
-    for (int64_t r = r_begin; r < r_end; r++) {
-        int64_t off_r = request_off(s, T, r);
+    for (int64_t r = r_begin; r < r_end; r++)
         for (int64_t l = 0; l < s->L; l++)
             for (int64_t c = 0; c < 2; c++)
                 for (int64_t t = 0; t < T[r]; t++) {
                     int64_t b = bt[bt_off[r] + t / s->B], n = t % s->B;
-                    for (int64_t h = 0; h < s->H; h++)
+                    for (int64_t h = pg->h0; h < pg->h0 + pg->hs; h++)
                         for (int64_t d = 0; d < s->D; d++)
                             for (int64_t e = 0; e < s->E; e++) {
                                 int64_t p = pool_off(s, g, b, n, h, d, e);
-                                pool_base[l * 2 + c][p] =
-                                    packed[off_r + packed_off(s, packed_layout, T[r], l, c, t, h, d, e)];
+                                pool_base[l * 2 + c][p] = packed[packed_addr(s, pg, R, T, r, l, c, t, h, d, e)];
                                 if (pool_cnt) bump(pool_cnt[l * 2 + c], p);
                             }
                 }
-    }
 }
 
 /* publish followed by hydrate, fused: pool to pool through two block tables that

@@ -20,9 +20,11 @@ TC_ERR_KIND, TC_ERR_OOM, TC_ERR_CUDA, TC_ERR_DEADLINE, TC_ERR_TOO_LARGE = -5, -6
 TC_NOALLOC_SCRATCH_BYTES = 1 << 20
 TC_KV_PACK, TC_KV_UNPACK, TC_KV_MIGRATE, TC_KV_MIXED, TC_WEIGHTS = 1, 2, 3, 4, 5
 TC_NHD, TC_HND = 0, 1
+TC_REQUEST_MAJOR, TC_LAYER_MAJOR = 0, 1
 TC_PLAN_HOST_ONLY = 1
 TC_PLAN_STAGED = 2
 TC_PLAN_CHECKSUM = 4
+TC_PLAN_SAME_POOL = 8
 TC_MAX_TABLE_SLOTS = 4000
 
 
@@ -40,7 +42,8 @@ class tc_kv_group_t(C.Structure):
 class tc_kv_spec_t(C.Structure):
     _fields_ = [("L", C.c_int64), ("B", C.c_int64), ("H", C.c_int64), ("D", C.c_int64), ("E", C.c_int64),
                 ("src_pool", tc_kv_pool_t), ("dst_pool", tc_kv_pool_t),
-                ("packed_layout", C.c_int32), ("reserved", C.c_int32), ("packed_bytes", C.c_int64),
+                ("packed_layout", C.c_int32), ("packed_order", C.c_int32), ("packed_bytes", C.c_int64),
+                ("head_begin", C.c_int64), ("head_count", C.c_int64),
                 ("group", tc_kv_group_t), ("reload", tc_kv_group_t)]
 
 
@@ -189,7 +192,7 @@ def group(keep: _Keep, T, bt_off, bt_src=None, bt_dst=None) -> tc_kv_group_t:
 
 def kv_spec(kind, shape, *, src_pool=None, dst_pool=None, packed_layout=TC_NHD, packed_bytes=0,
             T=(), bt_off=(0,), bt_src=None, bt_dst=None, reload=None, flags=0, trace_id=0,
-            deadline_ns=0, tuning=None):
+            deadline_ns=0, tuning=None, packed_order=TC_REQUEST_MAJOR, head_begin=0, head_count=0):
     """Assemble a tc_plan_spec_t for the KV kinds.  shape = (L, B, H, D, E);
     reload = dict(T=, bt_off=, bt_src=, bt_dst=) for TC_KV_MIXED.  Returns (spec, keepalive)."""
     keep = _Keep()
@@ -205,6 +208,7 @@ def kv_spec(kind, shape, *, src_pool=None, dst_pool=None, packed_layout=TC_NHD, 
     if dst_pool is not None:
         kv.dst_pool = dst_pool
     kv.packed_layout, kv.packed_bytes = packed_layout, packed_bytes
+    kv.packed_order, kv.head_begin, kv.head_count = packed_order, head_begin, head_count
     kv.group = group(keep, T, bt_off, bt_src, bt_dst)
     if reload is not None:
         kv.reload = group(keep, reload["T"], reload["bt_off"], reload["bt_src"], reload["bt_dst"])

@@ -334,11 +334,12 @@ static void pool_strides(const tc_kv_spec_t &kv, int32_t layout, int64_t *sn, in
     else                  { *sn = row;        *sh = kv.B * row; }
 }
 
-static void packed_strides(const tc_kv_spec_t &kv, int32_t layout, int64_t Tr, int64_t *sn, int64_t *sh)
+// same for the packed buffer, which holds hs heads of a request of Tr tokens
+static void packed_strides(const tc_kv_spec_t &kv, int32_t layout, int64_t Tr, int64_t hs, int64_t *sn, int64_t *sh)
 {
     const int64_t row = kv.D * kv.E;
-    if (layout == TC_NHD) { *sn = kv.H * row; *sh = row; }
-    else                  { *sn = row;        *sh = Tr * row; }
+    if (layout == TC_NHD) { *sn = hs * row; *sh = row; }
+    else                  { *sn = row;      *sh = Tr * row; }
 }
 
 static int64_t planes_of(const tc_kv_spec_t &kv) { return kv.L * 2; }
@@ -364,11 +365,19 @@ static void lower_kv_group(Group &g, const tc_kv_spec_t &kv, const tc_kv_group_t
                            const PoolView *dst_pool, int32_t packed_layout, uint32_t tile_bytes)
 {
     const int64_t row = kv.D * kv.E, planes = kv.L * 2;
+    const bool has_packed = !src_pool || !dst_pool;
+    // the packed side may hold a head slice and may be ordered layer-major
+    const int64_t h0 = has_packed ? kv.head_begin : 0;
+    const int64_t hs = has_packed && kv.head_count ? kv.head_count : kv.H - h0;
+    const bool layer_major = has_packed && kv.packed_order == TC_LAYER_MAJOR;
+    int64_t total_tokens = 0;
+    for (int64_t r = 0; r < grp.R; r++) total_tokens += grp.T[r];
     int64_t off_r = 0;
     g.descs.reserve(grp.R ? static_cast<size_t>(grp.bt_off[grp.R]) : 0);
     for (int64_t r = 0; r < grp.R; r++) {
         const int64_t Tr = grp.T[r];
-        const int64_t plane_bytes = Tr * kv.H * row;  // one (l,c) plane of this request, packed
+        const int64_t plane_bytes = Tr * hs * row;  // one (l,c) plane of this request, packed
+        const int64_t packed_outer = layer_major ? total_tokens * hs * row : plane_bytes;
         const uint32_t first_desc = static_cast<uint32_t>(g.descs.size());
         for (int64_t j = 0; j * kv.B < Tr; j++) {
             const int64_t nvalid = std::min(kv.B, Tr - j * kv.B);
@@ -379,32 +388,32 @@ static void lower_kv_group(Group &g, const tc_kv_spec_t &kv, const tc_kv_group_t
             int64_t ssn, ssh, dsn, dsh;
             if (src_pool) {
                 pool_strides(kv, src_pool->p->layout, &ssn, &ssh);
-                b.src_off = grp.bt_src[jj] * src_pool->block_stride;
+                b.src_off = grp.bt_src[jj] * src_pool->block_stride + h0 * ssh;
                 b.src_outer = src_pool->plane_stride;
                 b.src_slot_step = src_pool->slot_step;
             } else {
-                packed_strides(kv, packed_layout, Tr, &ssn, &ssh);
+                packed_strides(kv, packed_layout, Tr, hs, &ssn, &ssh);
                 b.src_off = off_r + j * kv.B * ssn;
-                b.src_outer = plane_bytes;
+                b.src_outer = packed_outer;
             }
             if (dst_pool) {
                 pool_strides(kv, dst_pool->p->layout, &dsn, &dsh);
-                b.dst_off = grp.bt_dst[jj] * dst_pool->block_stride;
+                b.dst_off = grp.bt_dst[jj] * dst_pool->block_stride + h0 * dsh;
                 b.dst_outer = dst_pool->plane_stride;
                 b.dst_slot_step = dst_pool->slot_step;
             } else {
-                packed_strides(kv, packed_layout, Tr, &dsn, &dsh);
+                packed_strides(kv, packed_layout, Tr, hs, &dsn, &dsh);
                 b.dst_off = off_r + j * kv.B * dsn;
-                b.dst_outer = plane_bytes;
+                b.dst_outer = packed_outer;
             }
             b.src_slot = 0;
             b.dst_slot = 0;
-            b.dims = {Dim{kv.H, ssh, dsh}, Dim{nvalid, ssn, dsn}};
+            b.dims = {Dim{hs, ssh, dsh}, Dim{nvalid, ssn, dsn}};
             lower_box(g, b, tile_bytes);
         }
-        if (!src_pool || !dst_pool)
+        if (has_packed && !layer_major)  // request-major regions are contiguous: staged plans cut segments from them
             g.requests.push_back(RequestSpan{first_desc, static_cast<uint32_t>(g.descs.size()), off_r, plane_bytes});
-        off_r += planes * plane_bytes;
+        off_r += layer_major ? plane_bytes : planes * plane_bytes;
     }
 }
 
@@ -456,11 +465,18 @@ static int build_kv(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t tile_byt
     if (src_is_pool && (rc = check_pool(kv, kv.src_pool, "src_pool", &sp))) return rc;
     if (dst_is_pool && (rc = check_pool(kv, kv.dst_pool, "dst_pool", &dp))) return rc;
     if ((rc = check_group(kv, kv.group, "group", src_is_pool, &kv.src_pool, dst_is_pool, &kv.dst_pool))) return rc;
+    if (kv.head_begin < 0 || kv.head_count < 0 || kv.head_begin + kv.head_count > kv.H || kv.head_begin >= kv.H)
+        return fail(TC_ERR_BOUNDS, "head slice [%lld, +%lld) lies outside the %lld heads", (long long)kv.head_begin, (long long)kv.head_count, (long long)kv.H);
+    if (kv.packed_order != TC_REQUEST_MAJOR && kv.packed_order != TC_LAYER_MAJOR)
+        return fail(TC_ERR_INVALID_ARG, "packed_order %d is not a tc_packed_order", kv.packed_order);
+    if ((kind == TC_KV_MIGRATE || kind == TC_KV_MIXED) && (kv.head_begin || kv.head_count || kv.packed_order))
+        return fail(TC_ERR_INVALID_ARG, "head slices and packed_order apply to plans with a packed buffer (PACK, UNPACK)");
     if (kind == TC_KV_PACK || kind == TC_KV_UNPACK) {
         if (kv.packed_layout != TC_NHD && kv.packed_layout != TC_HND)
             return fail(TC_ERR_INVALID_ARG, "packed_layout %d is not a tc_layout", kv.packed_layout);
+        const int64_t hs = kv.head_count ? kv.head_count : kv.H - kv.head_begin;
         int64_t need = 0;
-        for (int64_t r = 0; r < kv.group.R; r++) need += kv.L * 2 * kv.group.T[r] * kv.H * kv.D * kv.E;
+        for (int64_t r = 0; r < kv.group.R; r++) need += kv.L * 2 * kv.group.T[r] * hs * kv.D * kv.E;
         plan->packed_required = need;
         if (kv.packed_bytes && kv.packed_bytes < need)
             return fail(TC_ERR_BOUNDS, "packed_bytes %lld < %lld required", (long long)kv.packed_bytes, (long long)need);
@@ -475,6 +491,17 @@ static int build_kv(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t tile_byt
         g1.n_src = 1;
         g1.n_dst = kv.dst_pool.n_slots;
     } else if (kind == TC_KV_MIGRATE) {
+        if (spec->flags & TC_PLAN_SAME_POOL) {
+            const tc_kv_pool_t &a = kv.src_pool, &b = kv.dst_pool;
+            if (a.layout != b.layout || a.num_blocks != b.num_blocks || a.n_slots != b.n_slots || sp.block_stride != dp.block_stride || sp.plane_stride != dp.plane_stride)
+                return fail(TC_ERR_INVALID_ARG, "TC_PLAN_SAME_POOL: src_pool and dst_pool must describe the same pool");
+            const int64_t n = kv.group.R ? kv.group.bt_off[kv.group.R] : 0;
+            std::vector<uint8_t> read(static_cast<size_t>(a.num_blocks), 0);
+            for (int64_t j = 0; j < n; j++) read[kv.group.bt_src[j]] = 1;
+            for (int64_t j = 0; j < n; j++)
+                if (read[kv.group.bt_dst[j]])
+                    return fail(TC_ERR_OVERLAP, "TC_PLAN_SAME_POOL: block %d is both read and written", kv.group.bt_dst[j]);
+        }
         lower_kv_group(g0, kv, kv.group, &sp, &dp, 0, tile_bytes);
         g0.n_src = kv.src_pool.n_slots;
         g0.n_dst = kv.dst_pool.n_slots;
@@ -684,6 +711,8 @@ int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
         for (Desc &d : g.descs) d.dst_slot = static_cast<uint16_t>(d.dst_slot + g.n_src);
         if ((rc = finish_group(g))) return rc;
     }
+    if ((spec->flags & TC_PLAN_SAME_POOL) && spec->kind != TC_KV_MIGRATE)
+        return fail(TC_ERR_KIND, "TC_PLAN_SAME_POOL applies to TC_KV_MIGRATE plans only");
     if ((spec->flags & TC_PLAN_CHECKSUM) && spec->kind != TC_WEIGHTS)
         return fail(TC_ERR_KIND, "TC_PLAN_CHECKSUM applies to TC_WEIGHTS plans only");
     if (spec->flags & TC_PLAN_STAGED) {

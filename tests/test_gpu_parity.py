@@ -151,6 +151,49 @@ def test_migrate_pool_to_pool(src_l, dst_l):
     assert np.array_equal(out.result(), want)
 
 
+@pytest.mark.parametrize("order", [tc.TC_REQUEST_MAJOR, tc.TC_LAYER_MAJOR])
+@pytest.mark.parametrize("packed_l", LAYOUTS)
+def test_head_slice_view_and_layer_major_order(order, packed_l):
+    """A tensor-parallel consumer's view: 2 of 8 KV heads of every request, optionally with the
+    packed buffer ordered layer-major; unpacking writes those heads only."""
+    rng = np.random.default_rng(27)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=3, NB=120, B=16, H=8, D=128, E=2, T=(300, 16, 45, 0, 700))
+    L = shape[0]
+    h0, hs = 4, 2
+    kw = dict(order=order, head_begin=h0, head_count=hs)
+    want = np.zeros(oracle.packed_nbytes(shape, T, hs), dtype=np.uint8)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, L * 2), T, off, bt, packed_l, want, threads=4, **kw)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride)
+    lib_kw = dict(packed_layout=packed_l, packed_order=order, head_begin=h0, head_count=hs, T=T, bt_off=off)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, bt_src=bt, **lib_kw))
+    out = Guarded(want.size)
+    tc.tc_kv_pack(plan, [dev(pool)], [out.ptr()])
+    assert np.array_equal(out.result(), want)
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(want_pool, L * 2), T, off, bt2, packed_l, want, threads=4, **kw)
+    plan2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, bt_dst=bt2, **lib_kw))
+    fresh = Guarded(pool.size)
+    tc.tc_kv_unpack(plan2, [out.ptr()], [fresh.ptr()])
+    assert np.array_equal(fresh.result(), want_pool)
+
+
+def test_same_pool_compaction_in_place():
+    rng = np.random.default_rng(26)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=3, NB=200, B=16, H=8, D=128, E=2, T=(300, 16, 45, 700))
+    L = shape[0]
+    n = int(off[-1])
+    bt = (rng.permutation(NB - n)[:n] + n).astype(np.int32)
+    dst = np.arange(n, dtype=np.int32)
+    want = pool.copy()
+    oracle.kv_migrate(shape, oracle.NHD, stride, planes_of(pool, L * 2), oracle.NHD, stride, planes_of(want, L * 2), T, off, bt, dst, threads=4)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl, T=T, bt_off=off, bt_src=bt, bt_dst=dst, flags=tc.TC_PLAN_SAME_POOL))
+    buf = Guarded(pool.size, init=pool)
+    tc.tc_kv_pack(plan, [buf.ptr()], [buf.ptr()])
+    assert np.array_equal(buf.result(), want)
+
+
 @pytest.mark.parametrize("flags", [0, tc.TC_PLAN_STAGED])
 def test_mixed_plan_offload_and_reload_through_pinned_host_pool(flags):
     """Device NHD pool <-> pinned page-first HND host pool, both directions of one plan on two

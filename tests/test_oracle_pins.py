@@ -357,6 +357,66 @@ def test_llama3_8b_index_matches_golden_offsets():
     assert shard_el == g["shard_elements_world8"]
 
 
+# ------------------------------------------------------------------ packed-side views
+@pytest.mark.parametrize("pool_l,packed_l", list(itertools.product([oracle.NHD, oracle.HND], repeat=2)))
+def test_head_slice_is_a_numpy_slice_of_the_full_pack(pool_l, packed_l):
+    rng = np.random.default_rng(14)
+    shape, NB, stride, pool, T, off, bt = random_case(rng, H=5, T=(7, 0, 12, 1))
+    L, B, H, D, E = shape
+    planes = planes_of(pool, L * 2)
+    full = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, pool_l, stride, planes, T, off, bt, packed_l, full)
+    h0, hs = 1, 3
+    part = np.zeros(oracle.packed_nbytes(shape, T, hs), dtype=np.uint8)
+    cnt = np.zeros_like(part)
+    oracle.kv_pack(shape, pool_l, stride, planes, T, off, bt, packed_l, part, cnt, head_begin=h0, head_count=hs)
+    assert (cnt == 1).all()
+    want, pos = [], 0
+    for t in T:
+        n = L * 2 * int(t) * H * D * E
+        reg = full[pos:pos + n]
+        pos += n
+        if packed_l == oracle.NHD:
+            want.append(reg.reshape(L * 2, int(t), H, D * E)[:, :, h0:h0 + hs].reshape(-1))
+        else:
+            want.append(reg.reshape(L * 2, H, int(t), D * E)[:, h0:h0 + hs].reshape(-1))
+    assert np.array_equal(part, np.concatenate(want))
+    # unpacking the slice writes exactly those heads: the others keep the sentinel
+    pool2 = np.full_like(pool, 0xA5)
+    cnt2 = np.zeros_like(pool)
+    oracle.kv_unpack(shape, pool_l, stride, planes_of(pool2, L * 2), T, off, bt, packed_l, part, planes_of(cnt2, L * 2), head_begin=h0, head_count=hs)
+    assert cnt2.sum() == part.size and cnt2.max() == 1 and (pool2[cnt2 == 0] == 0xA5).all()
+    back = np.zeros_like(part)
+    oracle.kv_pack(shape, pool_l, stride, planes_of(pool2, L * 2), T, off, bt, packed_l, back, head_begin=h0, head_count=hs)
+    assert np.array_equal(back, part)
+
+
+@pytest.mark.parametrize("packed_l", [oracle.NHD, oracle.HND])
+def test_layer_major_order_is_a_regrouping_of_request_major(packed_l):
+    rng = np.random.default_rng(15)
+    shape, NB, stride, pool, T, off, bt = random_case(rng, T=(5, 0, 11, 2))
+    L, B, H, D, E = shape
+    planes = planes_of(pool, L * 2)
+    rm = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    lm = np.zeros_like(rm)
+    cnt = np.zeros_like(rm)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes, T, off, bt, packed_l, rm)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes, T, off, bt, packed_l, lm, cnt, order=oracle.LAYER_MAJOR)
+    assert (cnt == 1).all()
+    per_req, pos = [], 0
+    for t in T:
+        n = L * 2 * int(t) * H * D * E
+        per_req.append(rm[pos:pos + n].reshape(L * 2, -1))     # [plane][bytes of that plane]
+        pos += n
+    want = np.concatenate([np.concatenate([q[p] for q in per_req]) for p in range(L * 2)])
+    assert np.array_equal(lm, want)
+    pool2 = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(pool2, L * 2), T, off, bt, packed_l, lm, order=oracle.LAYER_MAJOR)
+    pool3 = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(pool3, L * 2), T, off, bt, packed_l, rm)
+    assert np.array_equal(pool2, pool3)
+
+
 # ------------------------------------------------------------------ integrity checksum
 def test_checksum_shards_add_up_to_the_whole_and_replicas_equal_it():
     ck = small_checkpoint()

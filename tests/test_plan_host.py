@@ -263,6 +263,64 @@ def test_staged_plans_are_cut_into_contiguous_segments():
     assert e.value.status == tc.TC_ERR_KIND
 
 
+@pytest.mark.parametrize("pool_l,packed_l", list(itertools.product(LAYOUTS, LAYOUTS)))
+@pytest.mark.parametrize("order", [tc.TC_REQUEST_MAJOR, tc.TC_LAYER_MAJOR])
+def test_head_slice_and_layer_major_lowering_match_oracle(pool_l, packed_l, order):
+    rng = np.random.default_rng(7)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=14, B=4, H=5, D=8, E=2, T=(5, 0, 11, 1, 8), pad_blocks=16)
+    L = shape[0]
+    for h0, hs in ((0, 0), (1, 3), (4, 1)):
+        kw = dict(order=order, head_begin=h0, head_count=hs or None)
+        want = np.zeros(oracle.packed_nbytes(shape, T, hs or None), dtype=np.uint8)
+        oracle.kv_pack(shape, pool_l, stride, planes_of(pool, L * 2), T, off, bt, packed_l, want, **kw)
+        pl = tc.pool(pool_l, NB, L * 2, block_stride=stride)
+        lib_kw = dict(packed_layout=packed_l, packed_order=order, head_begin=h0, head_count=hs, T=T, bt_off=off, flags=HOST, tuning=dict(tile_bytes=512))
+        plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, bt_src=bt, **lib_kw))
+        assert plan.stats().packed_bytes_required == want.size
+        got = np.full(want.size, 0xCC, dtype=np.uint8)
+        cnt = [np.zeros(want.size, dtype=np.int32)]
+        run_descriptors(plan.descriptors(0), planes_of(pool, L * 2), [got], cnt)
+        assert np.array_equal(got, want) and (cnt[0] == 1).all()
+        want_pool = np.full_like(pool, 0xA5)
+        oracle.kv_unpack(shape, pool_l, stride, planes_of(want_pool, L * 2), T, off, bt, packed_l, want, **kw)
+        plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, bt_dst=bt, **lib_kw))
+        got_pool = np.full_like(pool, 0xA5)
+        run_descriptors(plan.descriptors(1), [want], planes_of(got_pool, L * 2))
+        assert np.array_equal(got_pool, want_pool)
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, bt_src=bt, packed_layout=packed_l, head_begin=3, head_count=3, T=T, bt_off=off, flags=HOST))
+    assert e.value.status == tc.TC_ERR_BOUNDS
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl, bt_src=bt, bt_dst=bt, head_begin=1, head_count=2, T=T, bt_off=off, flags=HOST))
+    assert e.value.status == tc.TC_ERR_INVALID_ARG
+
+
+def test_same_pool_compaction_lowering_and_its_overlap_check():
+    """Defragmentation: the requests' blocks move to the low block ids of the same pool."""
+    rng = np.random.default_rng(6)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=30, B=4, H=3, D=8, E=2, T=(9, 4, 14))
+    L = shape[0]
+    n = int(off[-1])
+    bt = (rng.permutation(NB - n)[:n] + n).astype(np.int32)       # sources live above the compacted region
+    dst = np.arange(n, dtype=np.int32)
+    want = pool.copy()
+    oracle.kv_migrate(shape, oracle.NHD, stride, planes_of(pool, L * 2), oracle.NHD, stride, planes_of(want, L * 2), T, off, bt, dst)
+    pl = tc.pool(tc.TC_NHD, NB, L * 2, block_stride=stride)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl, T=T, bt_off=off, bt_src=bt, bt_dst=dst, flags=HOST | tc.TC_PLAN_SAME_POOL))
+    got = pool.copy()
+    run_descriptors(plan.descriptors(0), planes_of(pool, L * 2), planes_of(got, L * 2))
+    assert np.array_equal(got, want)
+    clash = dst.copy()
+    clash[0] = bt[3]
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl, T=T, bt_off=off, bt_src=bt, bt_dst=clash, flags=HOST | tc.TC_PLAN_SAME_POOL))
+    assert e.value.status == tc.TC_ERR_OVERLAP
+    other = tc.pool(tc.TC_HND, NB, L * 2, block_stride=stride)
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=other, T=T, bt_off=off, bt_src=bt, bt_dst=dst, flags=HOST | tc.TC_PLAN_SAME_POOL))
+    assert e.value.status == tc.TC_ERR_INVALID_ARG
+
+
 # --------------------------------------------------------------------------- validation
 def _pack_spec(**over):
     shape, NB, src, dst = wl.config1()
