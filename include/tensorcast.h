@@ -48,6 +48,9 @@
  * then reads or writes directly over the host link (zero copy).  The tables themselves, the
  * spec and every array it points to are HOST memory.
  *
+ * Devices.  A plan belongs to the CUDA device that was current when it was created; execute
+ * calls must be made with that device current (TC_ERR_INVALID_ARG otherwise).
+ *
  * Synchronisation.  Execute calls are asynchronous on `stream` (a cudaStream_t passed as
  * void*; NULL = the legacy default stream).  Completion is observed through the stream
  * (events, cudaStreamSynchronize): operations are lazy handles that block only when awaited

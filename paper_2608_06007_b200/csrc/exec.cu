@@ -599,6 +599,9 @@ static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n
         return fail(TC_ERR_INVALID_ARG, "tables of %zu source and %zu destination pointers given, the plan needs %zu and %zu", n_src, n_dst, g.n_src, g.n_dst);
     if ((n_src && !src) || (n_dst && !dst)) return fail(TC_ERR_INVALID_ARG, "pointer table is NULL");
     if (plan->deadline_ns && now_ns() > plan->deadline_ns) return fail(TC_ERR_DEADLINE, "deadline passed before the call; nothing launched");
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess || current != plan->device)
+        return fail(TC_ERR_INVALID_ARG, "the plan lives on device %d but device %d is current", plan->device, current);
     if (sums) {
         cudaError_t e = cudaMemsetAsync(sums, 0, static_cast<size_t>(plan->n_sums) * sizeof(unsigned long long), static_cast<cudaStream_t>(stream));
         if (e != cudaSuccess) return cuda_fail(e, "zeroing the checksum accumulators");

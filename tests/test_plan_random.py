@@ -26,13 +26,16 @@ def kv_cases(draw):
     pad = draw(st.sampled_from([0, E, 16, 48]))
     tile = draw(st.sampled_from([0, 512, 1024, 4096]))
     seed = draw(st.integers(0, 2 ** 31))
-    return (L, B, H, D, E), T, pad, tile, seed, draw(st.sampled_from([0, 1])), draw(st.sampled_from([0, 1])), draw(st.booleans())
+    h0 = draw(st.integers(0, H - 1))
+    hs = draw(st.integers(0, H - h0))   # 0 = all heads from h0... (library: 0 means H - h0)
+    order = draw(st.sampled_from([0, 1]))
+    return (L, B, H, D, E), T, pad, tile, seed, draw(st.sampled_from([0, 1])), draw(st.sampled_from([0, 1])), draw(st.booleans()), h0, hs, order
 
 
 @settings(max_examples=150, **COMMON)
 @given(kv_cases())
 def test_random_kv_pack_unpack_migrate(case):
-    shape, T, pad, tile, seed, pool_l, other_l, one_slot = case
+    shape, T, pad, tile, seed, pool_l, other_l, one_slot, h0, hs, order = case
     L, B, H, D, E = shape
     rng = np.random.default_rng(seed)
     T = np.array(T, dtype=np.int64)
@@ -50,18 +53,20 @@ def test_random_kv_pack_unpack_migrate(case):
     else:
         pl = tc.pool(pool_l, NB, L * 2, block_stride=stride, slot_bytes=NB * stride)
         tabs = lambda a: planes_of(a, L * 2)
-    # pack
-    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
-    oracle.kv_pack(shape, pool_l, stride, planes_of(pool, L * 2), T, off, bt, other_l, want)
-    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=other_l, T=T, bt_off=off, bt_src=bt, flags=HOST, tuning=tune))
+    # pack (the packed side holds heads [h0, h0+hs) in the drawn order)
+    okw = dict(order=order, head_begin=h0, head_count=hs or None)
+    lkw = dict(packed_order=order, head_begin=h0, head_count=hs)
+    want = np.zeros(oracle.packed_nbytes(shape, T, hs or H - h0), dtype=np.uint8)
+    oracle.kv_pack(shape, pool_l, stride, planes_of(pool, L * 2), T, off, bt, other_l, want, **okw)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=other_l, T=T, bt_off=off, bt_src=bt, flags=HOST, tuning=tune, **lkw))
     got = np.full(want.size, 0xCC, dtype=np.uint8)
     cnt = [np.zeros(want.size, dtype=np.int32)]
     run_descriptors(plan.descriptors(0), tabs(pool), [got], cnt)
     assert np.array_equal(got, want) and (cnt[0] == 1).all()
     # unpack
     want_pool = np.full_like(pool, 0xA5)
-    oracle.kv_unpack(shape, pool_l, stride, planes_of(want_pool, L * 2), T, off, bt2, other_l, want)
-    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=other_l, T=T, bt_off=off, bt_dst=bt2, flags=HOST, tuning=tune))
+    oracle.kv_unpack(shape, pool_l, stride, planes_of(want_pool, L * 2), T, off, bt2, other_l, want, **okw)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=other_l, T=T, bt_off=off, bt_dst=bt2, flags=HOST, tuning=tune, **lkw))
     got_pool = np.full_like(pool, 0xA5)
     run_descriptors(plan.descriptors(1), [want], tabs(got_pool))
     assert np.array_equal(got_pool, want_pool)
@@ -74,7 +79,7 @@ def test_random_kv_pack_unpack_migrate(case):
     run_descriptors(plan.descriptors(0), tabs(pool), planes_of(got_pool, L * 2))
     assert np.array_equal(got_pool, want_pool)
     st_ = plan.stats()
-    assert st_.payload_bytes[0] == want.size
+    assert st_.payload_bytes[0] == oracle.packed_nbytes(shape, T)
 
 
 @st.composite
