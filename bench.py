@@ -403,7 +403,21 @@ def run_ours(args):
 
     # ---------------- e2e: packed buffer and blob in pinned host memory --------------------
     e2e = None
+    e2e_skipped = None
     if not args.no_e2e:
+        # pinned host memory is per process: N ranks on one node share the node's RAM
+        try:
+            avail = int(next(l for l in open("/proc/meminfo") if l.startswith("MemAvailable")).split()[1]) * 1024
+        except Exception:
+            avail = 64 << 30
+        budget = 0.6 * avail / world
+        need_duplex, need_serial = 2 * max_packed + ck.nbytes_total, max_packed + ck.nbytes_total
+        if args.e2e_schedule == "duplex" and need_duplex > budget:
+            args.e2e_schedule = "serial"
+        if need_serial > budget:
+            e2e_skipped = (f"skipped: {need_serial / GB:.0f} GB of pinned host memory per rank needed, "
+                           f"{budget / GB:.0f} GB available per rank with {world} ranks on this node")
+    if not args.no_e2e and e2e_skipped is None:
         Qh = torch.empty(max_packed, dtype=torch.uint8).pin_memory()
         blob_h = torch.empty(ck.nbytes_total, dtype=torch.uint8).pin_memory()
         blob_h.copy_(blob)
@@ -565,7 +579,8 @@ def run_ours(args):
                    "weights_bytes": ck.nbytes_total, "shard": f"{args.shard_rank}/8",
                    "bytes_per_step": step_bytes, "l2": "every launch moves far more than the 126 MB L2; no flush needed",
                    "parallelism": "replicas only" if world > 1 else "1 GPU", "plans": n_plans, "plan_create_ms_total": plan_ms},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "clocks": clocks, "e2e": e2e if e2e is not None else ({"value": None, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0, "note": e2e_skipped or "skipped (--no-e2e)"}),
+        "gpu_launches": launches_per_step * args.steps,
         "e2e_gpu_launches_per_step": e2e_launches,
         "roofline": roofline, "rows": per_row, "other_workloads": extras,
         "cpu_baseline": {"value": cpu_v, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": cpu_desc},
