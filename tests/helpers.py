@@ -17,6 +17,9 @@ def run_descriptors(descs, src_tables, dst_tables, dst_counts=None):
                 i1, i0 = divmod(k, d.n0)
                 a = d.src_off + o * d.src_outer + i1 * d.src_s1 + i0 * d.src_s0
                 b = d.dst_off + o * d.dst_outer + i1 * d.dst_s1 + i0 * d.dst_s0
+                # no sanitizer runs on the GPU pool, so every lowered access is bounds-checked here
+                assert 0 <= a and a + d.run_bytes <= s.size, "descriptor reads outside its source slot"
+                assert 0 <= b and b + d.run_bytes <= t.size, "descriptor writes outside its destination slot"
                 t[b:b + d.run_bytes] = s[a:a + d.run_bytes]
                 if dst_counts is not None:
                     dst_counts[d.dst_slot + o * d.dst_slot_step][b:b + d.run_bytes] += 1

@@ -229,6 +229,54 @@ def test_llama3_8b_plans_have_the_expected_size():
     assert full.n_tiles[0] == (16060522496 - 65 * 8192) // 32768 + 65
 
 
+def _extent(descs, side):
+    """Largest byte any descriptor touches, per table slot (src or dst side), computed in closed form."""
+    hi = {}
+    for d in descs:
+        off, outer, s0, s1 = ((d.src_off, d.src_outer, d.src_s0, d.src_s1) if side == "src" else (d.dst_off, d.dst_outer, d.dst_s0, d.dst_s1))
+        slot0, step = (d.src_slot, d.src_slot_step) if side == "src" else (d.dst_slot, d.dst_slot_step)
+        n1 = d.rows // d.n0
+        assert off >= 0 and s0 >= 0 and s1 >= 0 and outer >= 0
+        top = off + (n1 - 1) * s1 + (d.n0 - 1) * s0 + d.run_bytes
+        for o in ((0, d.n_outer - 1) if step else (d.n_outer - 1,)):
+            slot = slot0 + o * step
+            hi[slot] = max(hi.get(slot, 0), top + (0 if step else o * outer))
+    return hi
+
+
+def test_full_size_plans_stay_inside_their_buffers():
+    """Closed-form bounds of every descriptor of the full-size workloads (no sanitizer runs on the
+    GPU pool, so out-of-bounds lowering has to be caught here)."""
+    shape = wl.LLAMA3_8B_KV
+    _, NB, _, waves = wl.config2(wave_blocks=8192, NB_dst=8192)
+    pool_bytes = NB * shape.block_bytes
+    plA = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=pool_bytes)
+    for src, dst in waves[:2]:
+        payload = int(src.T.sum()) * shape.token_bytes
+        for order in (tc.TC_REQUEST_MAJOR, tc.TC_LAYER_MAJOR):
+            plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape.tuple, src_pool=plA, packed_layout=tc.TC_HND, packed_order=order,
+                                                T=src.T, bt_off=src.bt_off, bt_src=src.bt, flags=HOST))
+            ds = plan.descriptors(0)
+            assert max(_extent(ds, "src").values()) <= pool_bytes and _extent(ds, "dst") == {0: payload}
+            assert plan.stats().payload_bytes[0] == payload
+    shape4 = wl.LLAMA3_70B_KV
+    _, NB4, _, w4 = wl.config4(max_waves=1)
+    pl4 = tc.pool(tc.TC_NHD, NB4, shape4.L * 2, slot_bytes=NB4 * shape4.chunk_bytes)
+    ds = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape4.tuple, src_pool=pl4, dst_pool=pl4, T=w4[0][0].T, bt_off=w4[0][0].bt_off,
+                                      bt_src=w4[0][0].bt, bt_dst=w4[0][1].bt, flags=HOST)).descriptors(0)
+    for side in ("src", "dst"):
+        ext = _extent(ds, side)
+        assert set(ext) == {0, shape4.L * 2 - 1} and max(ext.values()) <= NB4 * shape4.chunk_bytes   # first and last plane
+    ck = wl.config3()
+    for kw, total in ((dict(), ck.nbytes_total), (dict(split_dim=ck.split_dim, rank=7, world=8), 2 * 1004015616)):
+        ds = tc.tc_plan_create(ck_spec(ck, flags=HOST, **kw)).descriptors(0)
+        assert max(_extent(ds, "src").values()) <= ck.nbytes_total
+        ext = _extent(ds, "dst")
+        for i in range(ck.N):
+            assert ext[i] == ck.nbytes(i) // (8 if kw and ck.split_dim[i] >= 0 else 1)
+        assert sum(ext.values()) == total
+
+
 def test_long_runs_and_wide_spans_are_cut_for_32_bit_row_offsets():
     # a 6 GiB contiguous tensor and a dim-1 slice whose rows are 3 GiB apart
     spec = tc.weights_spec([0], [6 << 30], [2], [1], [[3 << 30, 1, 1, 1]], blob_bytes=6 << 30, flags=HOST)
