@@ -325,7 +325,8 @@ def run_ours(args):
     nbytes = [ck.nbytes(i) for i in range(ck.N)]
     mk_w = lambda tn, **kw: tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total, tuning=tn or None, **kw))
     w_full, w_shard = mk_w(tune), mk_w(tune, split_dim=ck.split_dim, rank=args.shard_rank, world=W)
-    w_full_h, w_shard_h = mk_w(host_tune), mk_w(host_tune, split_dim=ck.split_dim, rank=args.shard_rank, world=W)
+    w_full_h = mk_w(host_tune, flags=host_flags)
+    w_shard_h = mk_w(host_tune, split_dim=ck.split_dim, rank=args.shard_rank, world=W, flags=host_flags)
     plan_ms = 1e3 * (time.perf_counter() - t_plan0)
     n_plans = 5 * len(waves) + 4
 
@@ -381,7 +382,8 @@ def run_ours(args):
             rows[k].ms.append(v)
     step_bytes = sum(r.bytes for r in rows.values())
     launches_per_step = sum(r.launches for r in rows.values())
-    e2e_launches = sum(p["pack_h"].stats().launches_per_execute + p["unpack_h"].stats().launches_per_execute for p in plans) + 2
+    e2e_launches = (sum(p["pack_h"].stats().launches_per_execute + p["unpack_h"].stats().launches_per_execute for p in plans)
+                    + w_full_h.stats().launches_per_execute + w_shard_h.stats().launches_per_execute)
     total_ms = ranks.max_ms(total_ms)
     value = world * step_bytes * args.steps / (total_ms * 1e-3) / GB
 
@@ -518,8 +520,8 @@ def run_ours(args):
                "host_link_frac_of_ceiling": (h2d + d2h) * args.e2e_steps / (e_ms * 1e-3) / GB /
                                             (ceil_bidir if duplex else (h2d + d2h) / (h2d / ceil_h2d + d2h / ceil_d2h)),
                "kv_host_path": args.host_path, "schedule": args.e2e_schedule,
-               "note": "packed KV buffer and weight blob in pinned host memory; KV: copy engines + device staging ring + D2D kernel "
-                       "(staged) or kernel loads/stores on host memory (zerocopy); weights: kernel loads from the pinned blob"}
+               "note": "packed KV buffer and weight blob in pinned host memory. staged: copy engines + device staging rings + "
+                       "D2D kernel (the TP shard's strided slices stay zero copy); zerocopy: kernel loads/stores on host memory"}
         del Qh, Qh2, Qhs, blob_h
 
     extras = None

@@ -113,9 +113,12 @@ enum {
                                (tc_plan_stats, tc_plan_descriptors) but not executed, and no
                                CUDA call is made */
     TC_PLAN_STAGED = 2u,    /* TC_KV_PACK / TC_KV_UNPACK whose packed buffer is PINNED HOST memory,
-                               or TC_KV_MIXED whose dst_pool is a page-first pinned host pool in
+                               TC_KV_MIXED whose dst_pool is a page-first pinned host pool in
                                one allocation (plane_stride = one block of one plane) moved in
-                               full blocks: instead of letting the kernel load / store host
+                               full blocks, or TC_WEIGHTS whose blob is pinned host memory and
+                               whose tensors are read in contiguous pieces (whole tensors and
+                               dim-0 slabs; strided slices stay zero copy, which fetches only
+                               the bytes it needs): instead of letting the kernel load / store host
                                memory directly (zero copy, the default), move the host-side
                                bytes with the copy engines through rings of device staging
                                buffers owned by the library (one ring of 3 x 64 MiB per

@@ -50,6 +50,7 @@ struct Params {
     // launch window (win_span == 0: the whole group).  Tile ids then walk plane-major over
     // descriptors [win_d0, ...) x planes [win_o0, ...): win_span = descriptors x win_tpo.
     uint32_t win_span, win_d0, win_o0, win_tpo;
+    uint32_t tile_base;         // first global tile id of this launch (tile-range segments)
     unsigned long long *sums;   // checksum accumulators (checked builds only)
     char *ptr[NPTR];            // src table then dst table
 };
@@ -184,7 +185,7 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
     constexpr int kThreads = Shape<MODE>::threads, kUnroll = Shape<MODE>::unroll;
     __shared__ Desc sdesc[2];
     int buf = 0;
-    for (uint32_t tile = blockIdx.x; tile < prm.n_tiles; tile += gridDim.x, buf ^= 1) {
+    for (uint32_t tile = blockIdx.x + prm.tile_base; tile < prm.n_tiles; tile += gridDim.x, buf ^= 1) {
         // tile id -> descriptor, plane o, part.  For uniform and windowed launches this needs
         // launch constants only, so it overlaps the descriptor fetch instead of waiting for it.
         uint32_t di, o = 0, part = 0;
@@ -398,7 +399,7 @@ static uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Se
     // persistent grid-stride grid.  tuning.ctas_per_sm / max_ctas select a persistent grid
     // (few CTAs suit transfers over the host link).
     uint64_t grid = std::min<uint64_t>(g.n_tiles, 0x7fffffffull);
-    if (win) grid = static_cast<uint64_t>(win->no) * win->nd * (g.tiles_per_desc / g.descs[0].n_outer);
+    if (win) grid = win->nd ? static_cast<uint64_t>(win->no) * win->nd * (g.tiles_per_desc / g.descs[0].n_outer) : win->no;
     if (plan->tuning.ctas_per_sm > 0) {
         int per_sm = g.resident_ctas[mode] > 0 ? g.resident_ctas[mode] : 1;
         per_sm = std::min(per_sm, plan->tuning.ctas_per_sm);
@@ -419,8 +420,11 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     prm.descs = g.d_descs;
     prm.tile_desc = g.d_tile_desc;
     prm.n_tiles = static_cast<uint32_t>(g.n_tiles);
-    prm.win_span = prm.win_d0 = prm.win_o0 = prm.win_tpo = 0;
-    if (win) {
+    prm.win_span = prm.win_d0 = prm.win_o0 = prm.win_tpo = prm.tile_base = 0;
+    if (win && win->nd == 0) {  // a range of global tile ids
+        prm.tile_base = win->d0;
+        prm.n_tiles = win->d0 + win->no;
+    } else if (win) {
         prm.win_tpo = g.tiles_per_desc / g.descs[0].n_outer;
         prm.win_span = win->nd * prm.win_tpo;
         prm.win_d0 = win->d0;
@@ -539,16 +543,19 @@ static void stage_release(int device)
         if (e_ != cudaSuccess) { rc = cuda_fail(e_, what); goto out; } \
     } while (0)
 
-// gi == 0: device pool -> staging (kernel, caller's stream) -> host (copy engine).
-// gi == 1: host -> staging (copy engine) -> device pool (kernel, caller's stream).
+// to the host:   device -> staging (kernel, caller's stream) -> host (copy engine).
+// to the device: host -> staging (copy engine) -> device (kernel, caller's stream).
 // The host side is table entry 0 of the call (the packed buffer, or the paged host pool).
 // Every segment's kernel sees the staging buffer through a base pointer shifted by the
 // segment's packed offset (0 for paged pools), so the descriptors are used unchanged.
-static int execute_staged(const tc_plan *plan, int gi, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s)
+static int execute_staged(const tc_plan *plan, int gi, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s,
+                          unsigned long long *sums = nullptr)
 {
     StageArena &a = g_stage[plan->device];
-    StageRing &r = a.ring[gi];
+    const bool to_device = g.host_is_src;
+    StageRing &r = a.ring[to_device ? 1 : 0];
     int rc = TC_OK;
+    (void)gi;
     pthread_mutex_lock(&g_stage_mu);
     TC_TRY(cudaEventRecord(a.entry, s), "cudaEventRecord");
     TC_TRY(cudaStreamWaitEvent(r.copy, a.entry, 0), "cudaStreamWaitEvent");
@@ -556,7 +563,7 @@ static int execute_staged(const tc_plan *plan, int gi, const Group &g, const voi
         const int b = static_cast<int>(r.next++ % kStageBuffers);
         char *shifted = r.buf[b] - seg.shift;
         const uint32_t pa = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(shifted) | 16));
-        if (gi == 1) {
+        if (to_device) {
             const char *host = static_cast<const char *>(src[0]);
             if (r.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(r.copy, r.freed[b], 0), "cudaStreamWaitEvent");
             for (uint32_t c = seg.copy0; c < seg.copy0 + seg.ncopy; c++)
@@ -564,7 +571,7 @@ static int execute_staged(const tc_plan *plan, int gi, const Group &g, const voi
             TC_TRY(cudaEventRecord(r.ready[b], r.copy), "cudaEventRecord");
             TC_TRY(cudaStreamWaitEvent(s, r.ready[b], 0), "cudaStreamWaitEvent");
             const void *stage_src[1] = {shifted};
-            if ((rc = launch_any(plan, g, stage_src, dst, pa, s, &seg)) != TC_OK) goto out;
+            if ((rc = launch_any(plan, g, stage_src, dst, pa, s, &seg, sums)) != TC_OK) goto out;
             TC_TRY(cudaEventRecord(r.freed[b], s), "cudaEventRecord");
         } else {
             char *host = static_cast<char *>(dst[0]);
@@ -579,7 +586,7 @@ static int execute_staged(const tc_plan *plan, int gi, const Group &g, const voi
         }
         r.freed_recorded[b] = true;
     }
-    if (gi == 0)  // the caller's stream completes only when the last copies to the host have landed
+    if (!to_device)  // the caller's stream completes only when the last copies to the host have landed
         for (int b = 0; b < kStageBuffers; b++)
             if (r.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(s, r.freed[b], 0), "cudaStreamWaitEvent");
 out:
@@ -617,7 +624,7 @@ static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n
         ptr_align = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(dst[i]) | 16));
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (!g.segments.empty()) return execute_staged(plan, gi, g, src, dst, ptr_align, s);
+    if (!g.segments.empty()) return execute_staged(plan, gi, g, src, dst, ptr_align, s, sums);
     return launch_any(plan, g, src, dst, ptr_align, s, nullptr, sums);
 }
 

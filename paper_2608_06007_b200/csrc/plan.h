@@ -53,7 +53,8 @@ static_assert(sizeof(Desc) == 128, "Desc must stay 128 bytes");
 // A launch window: descriptors [d0, d0+nd) x planes [o0, o0+no), walked plane-major.
 // A segment of a staged plan is a window whose packed-side bytes are one contiguous range.
 struct Segment {
-    uint32_t d0, nd, o0, no;
+    uint32_t d0, nd, o0, no; // window of descriptors x planes; nd == 0: a range of global tile
+                             // ids instead, [d0, d0 + no) (non-uniform groups, e.g. weights)
     int64_t shift;           // the kernel sees the staging buffer at (buffer - shift)
     uint32_t copy0, ncopy;   // its copies between host memory and the staging buffer
 };
@@ -76,6 +77,7 @@ struct Group {
     std::vector<Segment> segments;    // staged plans only
     std::vector<StageCopy> copies;    // staged plans only
     bool stage_whole_host_pool = false; // staged MIXED group: the host side is a paged pool
+    bool host_is_src = false;          // staged groups: direction (host -> device when true)
     uint32_t tiles_per_desc = 0;      // > 0: every descriptor owns exactly this many tile ids
     FastDiv div_tpd{0, 0};
     uint64_t n_tiles = 0;

@@ -672,6 +672,7 @@ static int build_weights(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t til
                 return fail(TC_ERR_OVERLAP, "destination slot %zu: byte %lld would be written twice", s, (long long)rows[k].first);
     }
     for (const Box &b : boxes) lower_box(g, b, tile_bytes);
+    g.host_is_src = true;
     if (spec->flags & TC_PLAN_CHECKSUM) {
         // checksums are sums over aligned 4-byte words of each tensor: every run must be made of
         // whole words and every access must be 16-byte aligned
@@ -682,6 +683,38 @@ static int build_weights(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t til
         plan->n_sums = w.n_tensors;
     }
     return TC_OK;
+}
+
+// Staged weights (blob in pinned host memory): a segment is a range of global tile ids whose
+// source bytes are one contiguous range of the blob of at most kStageBytes.  That needs a
+// non-uniform group (tile ids follow the descriptors) in which every tile reads one contiguous
+// piece - whole tensors and dim-0 slabs; strided slices stay on the zero-copy path, which reads
+// only the bytes it needs.
+static void build_segments_blob(Group &g)
+{
+    if (g.descs.empty() || g.tiles_per_desc) return;
+    for (const Desc &d : g.descs) {
+        const bool rows_contiguous = d.rows == 1 || (d.src_s0 == d.run && (d.rows == d.n0 || d.src_s1 == d.n0 * d.run));
+        if (d.n_outer != 1 || !rows_contiguous || d.src_slot != 0) return;
+    }
+    int64_t seg_lo = -1, seg_hi = -1;
+    uint32_t seg_t0 = 0, t = 0;
+    auto flush = [&](uint32_t t_end) {
+        if (seg_lo < 0) return;
+        g.segments.push_back(Segment{seg_t0, 0, 0, t_end - seg_t0, seg_lo, static_cast<uint32_t>(g.copies.size()), 1});
+        g.copies.push_back(StageCopy{0, seg_lo, seg_hi - seg_lo});
+        seg_lo = -1;
+    };
+    for (const Desc &d : g.descs)
+        for (uint32_t p = 0; p < d.tiles_per_outer; p++, t++) {
+            const uint32_t row0 = p * d.rows_per_tile, nrows = std::min(d.rows_per_tile, d.rows - row0);
+            const int64_t lo = d.src_off + static_cast<int64_t>(row0 / d.n0) * d.src_s1 + static_cast<int64_t>(row0 % d.n0) * d.src_s0;
+            const int64_t hi = lo + static_cast<int64_t>(nrows) * d.run;
+            if (seg_lo >= 0 && (lo != seg_hi || hi - seg_lo > kStageBytes)) flush(t);
+            if (seg_lo < 0) { seg_lo = lo; seg_t0 = t; }
+            seg_hi = hi;
+        }
+    flush(t);
 }
 
 // ------------------------------------------------------------------------------ entry
@@ -715,10 +748,13 @@ int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
         return fail(TC_ERR_KIND, "TC_PLAN_SAME_POOL applies to TC_KV_MIGRATE plans only");
     if ((spec->flags & TC_PLAN_CHECKSUM) && spec->kind != TC_WEIGHTS)
         return fail(TC_ERR_KIND, "TC_PLAN_CHECKSUM applies to TC_WEIGHTS plans only");
+    plan->group[1].host_is_src = true;  // UNPACK / reload read the host side
     if (spec->flags & TC_PLAN_STAGED) {
-        if (spec->kind != TC_KV_PACK && spec->kind != TC_KV_UNPACK && spec->kind != TC_KV_MIXED)
-            return fail(TC_ERR_KIND, "TC_PLAN_STAGED applies to TC_KV_PACK, TC_KV_UNPACK and TC_KV_MIXED plans only");
-        if (spec->kind == TC_KV_MIXED) {
+        if (spec->kind == TC_KV_MIGRATE)
+            return fail(TC_ERR_KIND, "TC_PLAN_STAGED does not apply to TC_KV_MIGRATE plans (no host side)");
+        if (spec->kind == TC_WEIGHTS) {
+            build_segments_blob(plan->group[0]);
+        } else if (spec->kind == TC_KV_MIXED) {
             // segments were cut while lowering; a group that could not be staged must drop them
             for (int k = 0; k < 2; k++) {
                 Group &g = plan->group[k];

@@ -304,6 +304,44 @@ def test_weights_full_and_every_shard(variant):
                 assert np.array_equal(outs[i].result(), want[i]), (ck.names[i], world, rank)
 
 
+def test_weights_from_a_pinned_blob_zero_copy_and_staged():
+    ck = wl.llama_checkpoint(hidden=512, layers=3, q_heads=8, kv_heads=4, head_dim=64, mlp=2048, vocab=70000)   # 190 MB: several staging buffers
+    blob = np.zeros(ck.nbytes_total, dtype=np.uint8)
+    wl.fill_np(blob, 9, "normal")
+    h_blob = torch.from_numpy(blob).pin_memory()
+    nbytes = [ck.nbytes(i) for i in range(ck.N)]
+    want = [np.zeros(n, dtype=np.uint8) for n in nbytes]
+    oracle.weights(ck.byte_off, ck.E, ck.shapes, np.full(ck.N, -1), 0, 1, blob, want, threads=8)
+    want_sums = oracle.weights_checksum(ck.byte_off, ck.E, ck.shapes, np.full(ck.N, -1), 0, 1, blob)
+    for flags in (0, tc.TC_PLAN_STAGED, tc.TC_PLAN_STAGED | tc.TC_PLAN_CHECKSUM):
+        plan = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total, flags=flags))
+        st = plan.stats()
+        assert st.path[0] == (3 if flags & tc.TC_PLAN_STAGED else 1)
+        if flags & tc.TC_PLAN_STAGED:
+            assert st.launches_per_execute >= 3
+        outs = [Guarded(n, fill=0xEE) for n in nbytes]
+        if flags & tc.TC_PLAN_CHECKSUM:
+            sums = torch.zeros(ck.N, dtype=torch.int64, device="cuda")
+            tc.tc_weights_materialize_checksum(plan, h_blob, [o.ptr() for o in outs], sums)
+            torch.cuda.synchronize()
+            assert np.array_equal(sums.cpu().numpy().view(np.uint64), want_sums)
+        else:
+            tc.tc_weights_materialize(plan, h_blob, [o.ptr() for o in outs])
+        for i in range(ck.N):
+            assert np.array_equal(outs[i].result(), want[i]), (ck.names[i], flags)
+    # a shard reads strided slices: it stays on the zero-copy path even when staging is asked for
+    plan = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, split_dim=ck.split_dim, rank=1, world=4,
+                                             blob_bytes=ck.nbytes_total, flags=tc.TC_PLAN_STAGED))
+    assert plan.stats().path[0] == 1
+    sizes = [n // (4 if ck.split_dim[i] >= 0 else 1) for i, n in enumerate(nbytes)]
+    want = [np.zeros(n, dtype=np.uint8) for n in sizes]
+    oracle.weights(ck.byte_off, ck.E, ck.shapes, ck.split_dim, 1, 4, blob, want, threads=8)
+    outs = [Guarded(n, fill=0xEE) for n in sizes]
+    tc.tc_weights_materialize(plan, h_blob, [o.ptr() for o in outs])
+    for i in range(ck.N):
+        assert np.array_equal(outs[i].result(), want[i]), ck.names[i]
+
+
 def test_weights_transform_into_fused_and_strided_targets():
     ck = small_checkpoint()
     blob = np.zeros(ck.nbytes_total, dtype=np.uint8)
