@@ -342,6 +342,57 @@ def test_weights_from_a_pinned_blob_zero_copy_and_staged():
         assert np.array_equal(outs[i].result(), want[i]), ck.names[i]
 
 
+def test_moe_checkpoint_many_tensors_and_expert_stacking():
+    """A MoE-shaped checkpoint: (a) 1 500+ tensors, one destination each - the pointer table of
+    the launch grows to thousands of slots; (b) transform_into with expert stacking: the gate and
+    up matrices of all experts of a layer land in one fused [experts, 2*moe_mlp/W, hidden] buffer
+    as rank r's shard, the down matrices in one [experts, hidden, moe_mlp/W] buffer (strided)."""
+    ck = wl.moe_checkpoint(hidden=64, layers=4, experts=128, moe_mlp=32)
+    assert ck.N > 1500
+    blob = np.zeros(ck.nbytes_total, dtype=np.uint8)
+    wl.fill_np(blob, 11, "normal")
+    d_blob = dev(blob)
+    nbytes = [ck.nbytes(i) for i in range(ck.N)]
+    W, rank = 2, 1
+    sizes = [n // (W if ck.split_dim[i] >= 0 else 1) for i, n in enumerate(nbytes)]
+    want = [np.zeros(n, dtype=np.uint8) for n in sizes]
+    oracle.weights(ck.byte_off, ck.E, ck.shapes, ck.split_dim, rank, W, blob, want)
+    plan = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, split_dim=ck.split_dim, rank=rank, world=W, blob_bytes=ck.nbytes_total))
+    arena = Guarded(sum(sizes), fill=0xEE)
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    tc.tc_weights_materialize(plan, d_blob, [arena.ptr(int(o)) for o in offs[:-1]])
+    got = arena.result()
+    for i in range(ck.N):
+        assert np.array_equal(got[offs[i]:offs[i + 1]], want[i]), ck.names[i]
+    # (b) expert stacking for layer 2
+    experts, mlp, hidden, E = 128, 32, 64, 2
+    ids, slot, doff, dstride = [], [], [], []
+    gu_row = hidden * E                     # one row of a gate/up shard
+    gu_exp = 2 * (mlp // W) * gu_row        # one expert of the fused gate_up buffer
+    dn_exp = hidden * (mlp // W) * E        # one expert of the stacked down buffer
+    for e in range(experts):
+        for k, nm in enumerate(("gate_proj", "up_proj")):
+            ids.append(ck.names.index(f"layers.2.experts.{e}.{nm}"))
+            slot.append(0)
+            doff.append(e * gu_exp + k * (mlp // W) * gu_row)
+            dstride.append([gu_row, E, E, E])
+        ids.append(ck.names.index(f"layers.2.experts.{e}.down_proj"))
+        slot.append(1)
+        doff.append(e * dn_exp)
+        dstride.append([(mlp // W) * E, E, E, E])
+    ids = np.array(ids)
+    nb = [nbytes[i] for i in ids]
+    spec = tc.weights_spec(ck.byte_off[ids], nb, ck.E[ids], ck.ndim[ids], ck.shapes[ids], split_dim=ck.split_dim[ids], rank=rank, world=W,
+                           blob_bytes=ck.nbytes_total, dst_slot=slot, dst_off=doff, dst_stride=dstride, n_dst=2, dst_bytes=[experts * gu_exp, experts * dn_exp])
+    gate_up, down = Guarded(experts * gu_exp), Guarded(experts * dn_exp)
+    tc.tc_weights_materialize(tc.tc_plan_create(spec), d_blob, [gate_up.ptr(), down.ptr()])
+    want_gu, want_dn = np.full(experts * gu_exp, 0xA5, dtype=np.uint8), np.full(experts * dn_exp, 0xA5, dtype=np.uint8)
+    oracle.weights(ck.byte_off[ids], ck.E[ids], ck.shapes[ids], ck.split_dim[ids], rank, W, blob,
+                   [want_gu if s_ == 0 else want_dn for s_ in slot], dst_off=doff, dst_stride=dstride)
+    assert np.array_equal(gate_up.result(), want_gu) and np.array_equal(down.result(), want_dn)
+    assert not (want_gu == 0xA5).all()
+
+
 def test_weights_transform_into_fused_and_strided_targets():
     ck = small_checkpoint()
     blob = np.zeros(ck.nbytes_total, dtype=np.uint8)

@@ -359,3 +359,31 @@ def shard_shape(ck: Checkpoint, i: int, world: int):
     if ck.split_dim[i] >= 0:
         s[ck.split_dim[i]] //= world
     return s
+
+
+def moe_checkpoint(hidden=64, layers=2, experts=16, moe_mlp=32, q_heads=4, kv_heads=2, head_dim=16, vocab=128, E=2) -> Checkpoint:
+    """Mixture-of-experts-shaped state dict (the paper's loader experiments use Qwen3 MoE
+    checkpoints): per layer attention projections plus `experts` x [gate, up, down] matrices
+    stored one tensor per expert, which an engine wants stacked into [experts, ...] buffers."""
+    items = [("embed_tokens", (vocab, hidden), 0)]
+    for l in range(layers):
+        p = f"layers.{l}."
+        items += [(p + "input_layernorm", (hidden,), -1), (p + "q_proj", (q_heads * head_dim, hidden), 0),
+                  (p + "k_proj", (kv_heads * head_dim, hidden), 0), (p + "v_proj", (kv_heads * head_dim, hidden), 0),
+                  (p + "o_proj", (hidden, q_heads * head_dim), 1), (p + "router", (experts, hidden), -1)]
+        for e in range(experts):
+            q = p + f"experts.{e}."
+            items += [(q + "gate_proj", (moe_mlp, hidden), 0), (q + "up_proj", (moe_mlp, hidden), 0), (q + "down_proj", (hidden, moe_mlp), 1)]
+    items += [("norm", (hidden,), -1), ("lm_head", (vocab, hidden), 0)]
+    N = len(items)
+    shapes = np.ones((N, 4), dtype=np.int64)
+    ndim = np.zeros(N, dtype=np.int32)
+    byte_off = np.zeros(N, dtype=np.int64)
+    off = 0
+    for i, (_, shp, _) in enumerate(items):
+        shapes[i, :len(shp)] = shp
+        ndim[i] = len(shp)
+        byte_off[i] = off
+        off += int(np.prod(shp)) * E
+    return Checkpoint(names=[it[0] for it in items], shapes=shapes, ndim=ndim, E=np.full(N, E, dtype=np.int64),
+                      byte_off=byte_off, split_dim=np.array([it[2] for it in items], dtype=np.int32), nbytes_total=off)
