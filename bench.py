@@ -143,6 +143,8 @@ class OracleSample:
         self.planes = [pool[p * per:(p + 1) * per] for p in range(shape.L * 2)]
         self.packed = np.zeros(oracle.packed_nbytes(shape.tuple, self.src.T), dtype=np.uint8)
         pool2 = np.zeros_like(pool)
+        pool2.fill(0)            # touch the pages now: page faults are not part of the oracle's time
+        self.packed.fill(0)
         self.planes2 = [pool2[p * per:(p + 1) * per] for p in range(shape.L * 2)]
         self.desc = (f"oracle kv_pack NHD->HND + kv_unpack of {len(self.src.T)} requests / {self.src.n_blocks} blocks "
                      f"({self.packed.size / GB:.2f} GB payload) of the Llama-3-8B KV workload, {threads} threads")
