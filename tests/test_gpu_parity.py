@@ -526,6 +526,54 @@ def test_execute_calls_can_be_captured_in_a_cuda_graph_and_replayed():
         assert np.array_equal(fresh.result(), want_pool)
 
 
+def test_concurrent_threads_create_execute_destroy():
+    """Calls on distinct plans are thread safe (plan-storage cache, staging rings, per-thread error
+    text): four threads each create, run on their own stream and destroy plans in a loop."""
+    import threading
+    rng = np.random.default_rng(28)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=64, B=16, H=8, D=128, E=2, T=(100, 37, 16, 5, 200))
+    L = shape[0]
+    d_pool = dev(pool)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride)
+    wants = {}
+    for lay in LAYOUTS:
+        w = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+        oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, L * 2), T, off, bt, lay, w, threads=4)
+        wants[lay] = w
+    errors = []
+
+    def worker(k):
+        try:
+            stream = torch.cuda.Stream()
+            lay = LAYOUTS[k % 2]
+            out = torch.zeros(wants[lay].size, dtype=torch.uint8, device="cuda")
+            host = torch.zeros(wants[lay].size, dtype=torch.uint8).pin_memory()
+            for it in range(25):
+                flags = tc.TC_PLAN_STAGED if (it + k) % 3 == 0 else 0
+                plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=lay, T=T, bt_off=off, bt_src=bt, flags=flags))
+                target = host if flags else out
+                tc.tc_kv_pack(plan, [d_pool], [target], stream.cuda_stream)
+                stream.synchronize()
+                got = target.cpu().numpy() if not flags else host.numpy().copy()
+                if not np.array_equal(got, wants[lay]):
+                    errors.append((k, it, "mismatch"))
+                try:
+                    tc.tc_kv_unpack(plan, [target], [d_pool])      # wrong kind: error text is per thread
+                except tc.TensorCastError as e:
+                    if e.status != tc.TC_ERR_KIND or "tc_kv_unpack" not in str(e):
+                        errors.append((k, it, str(e)))
+                plan.destroy()
+        except Exception as e:  # noqa: BLE001
+            errors.append((k, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(k,)) for k in range(4)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors[:3]
+
+
 # --------------------------------------------------------------------------- lifecycle on the device
 def test_empty_plan_wrong_tables_and_deadline_launch_nothing():
     shape, NB, src, dst = wl.config1()
