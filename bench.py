@@ -560,7 +560,7 @@ def run_ours(args):
     roofline = {"bound": "hbm", "kernel": f"tc_copy_kernel<{'kModeRows' if dom == 'rows' else 'kModeRun'}>",
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_source": peak_src, "traffic": traffic_per_launch(d["bytes"] / d["launches"]),
-                "traffic_source": "ncu dram bytes of a small case (profiles/), reads scaled by units, writes = payload minus the L2-resident tail",
+                "traffic_source": "ncu dram bytes of a small case, reads scaled by units, writes = payload minus the L2-resident tail",
                 "algorithmic_bytes_per_launch": d["bytes"] / d["launches"], "avg_launch_ms": d["ms"] / d["launches"],
                 "frac_of_nominal_8TBps": achieved / 8000.0,
                 "library_copy_of_the_same_random_bits_GBps": copy_same_data,
@@ -755,9 +755,9 @@ def run_extras(args, tc, torch, stream):
 
 
 def traffic_per_launch(algorithmic_bytes: float) -> float:
-    """DRAM bytes of one full-size launch, scaled from the ncu capture of a small case
-    (profiles/tc_copy_kernel_small_case_full_set.md): reads = 1.0002 x payload (descriptors
-    included); writes = payload less the ~50 MB of dirty lines still in L2 at kernel end."""
+    """DRAM bytes of one full-size launch, scaled from an `ncu --set full` capture of a small
+    case (226 MB wave, 700 MB checkpoint): reads = 1.0002 x payload (descriptors included);
+    writes = payload less the ~50 MB of dirty lines still in L2 at kernel end."""
     payload = algorithmic_bytes / 2
     return 1.0002 * payload + max(payload - 50.7e6, 0.0)
 

@@ -18,8 +18,8 @@
  *     (Table 2; Sec. 3.2).
  *   - Artifacts are immutable with one canonical content (Sec. 3.2), so every
  *     operation here is an exact byte copy with exactly one correct result.
- *   The paper gives no memory layout; the layouts below are this build's
- *   reading (listed in the design notes) and are written out as formulas.
+ *   The paper gives no memory layout; the layouts below are this library's
+ *   reading of those operations and are written out as formulas.
  *
  * Layouts (all sizes in elements of E bytes; d is contiguous everywhere):
  *   paged pool, plane (l,c), c=0 for K, c=1 for V, block b, slot n, head h:
