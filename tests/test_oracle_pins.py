@@ -154,6 +154,28 @@ def test_pack_nhd_equals_numpy_gather_when_blocks_are_full():
     assert np.array_equal(got_h, want_h)
 
 
+def test_unpack_equals_numpy_scatter_when_blocks_are_full():
+    rng = np.random.default_rng(31)
+    shape, NB, stride, pool, T, off, bt = random_case(rng)
+    L, B, H, D, E = shape
+    packed = rng.integers(0, 256, oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    for packed_l in (oracle.NHD, oracle.HND):
+        got = np.full_like(pool, 0xA5)
+        oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(got, L * 2), T, off, bt, packed_l, packed)
+        want = np.full_like(pool, 0xA5).reshape(L * 2, NB, B, H, D * E)
+        pos = 0
+        for r, t in enumerate(T):
+            n = L * 2 * int(t) * H * D * E
+            reg = packed[pos:pos + n]
+            pos += n
+            if packed_l == oracle.NHD:
+                tok = reg.reshape(L * 2, int(t), H, D * E)
+            else:
+                tok = reg.reshape(L * 2, H, int(t), D * E).transpose(0, 2, 1, 3)
+            want[:, bt[off[r]:off[r + 1]]] = tok.reshape(L * 2, -1, B, H, D * E)
+        assert np.array_equal(got, want.reshape(-1))
+
+
 def test_hnd_pool_is_per_block_transpose_of_nhd_pool():
     rng = np.random.default_rng(4)
     shape, NB, stride, pool, T, off, bt = random_case(rng, T=(7, 4, 9))
