@@ -223,8 +223,9 @@ typedef struct {
     int32_t tile_bytes;   /* target bytes per tile (one CTA iteration) */
     int32_t ctas_per_sm;  /* resident CTAs per SM for the persistent grid */
     int32_t max_ctas;     /* cap on the grid (e.g. few CTAs for host-link transfers) */
-    int32_t path;         /* 0 auto; 1 force the register (ld/st) path; 2 force the bulk-copy
-                             (shared-memory staged) path where the geometry allows it */
+    int32_t tile_order;   /* 0 auto: KV groups run plane-major over descriptors sorted by
+                             destination offset (ascending writes); 1: request / descriptor order
+                             as given, planes of one block consecutively */
 } tc_tuning_t;
 
 typedef struct {

@@ -413,6 +413,12 @@ template <int NPTR>
 static int launch(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t stream,
                   const Segment *win = nullptr, unsigned long long *sums = nullptr)
 {
+    // Uniform groups with planes (KV) are walked plane-major by default: all blocks of plane 0,
+    // then plane 1, ...  Together with descriptors sorted by destination offset, every plane
+    // pass writes ascending addresses (and pack / unpack stream through the packed buffer),
+    // which measured 3-5 % faster than walking the planes of one block after another.
+    Segment whole{0, static_cast<uint32_t>(g.descs.size()), 0, g.descs.empty() ? 0 : g.descs[0].n_outer, 0, 0, 0};
+    if (!win && g.tiles_per_desc && !g.descs.empty() && g.descs[0].n_outer > 1 && plan->tuning.tile_order != 1) win = &whole;
     const int mode = mode_for(g, ptr_align);
     if (sums && mode == kModeAny) return fail(TC_ERR_INVALID_ARG, "checksums need 16-byte aligned base pointers");
     const uint32_t grid = grid_for(plan, g, mode, win);

@@ -742,6 +742,12 @@ int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
         Group &g = plan->group[k];
         // destination slots follow the source slots in the combined pointer table
         for (Desc &d : g.descs) d.dst_slot = static_cast<uint16_t>(d.dst_slot + g.n_src);
+        // KV groups that are not staged: ascending destination offsets (descriptors are
+        // independent, so their order is free; staged groups keep request order, which their
+        // segments are cut from)
+        const bool kv_kind = spec->kind != TC_WEIGHTS;
+        if (kv_kind && !(spec->flags & TC_PLAN_STAGED) && spec->tuning.tile_order != 1)
+            std::stable_sort(g.descs.begin(), g.descs.end(), [](const Desc &a, const Desc &b) { return a.dst_off < b.dst_off; });
         if ((rc = finish_group(g))) return rc;
     }
     if ((spec->flags & TC_PLAN_SAME_POOL) && spec->kind != TC_KV_MIGRATE)
