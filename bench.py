@@ -271,6 +271,15 @@ def run_ours(args):
     ranks = Ranks("nccl")
     world, rank, local = ranks.world, ranks.rank, ranks.local
     tc.load_library()
+    # the CPU baseline goes first, while the host's memory is still unfragmented (the 50+ GB of
+    # pinned buffers allocated and freed below slow the oracle down 3-4x if it runs after them)
+    threads = os.cpu_count() or 1
+    cpu_v, cpu_desc = None, "skipped"
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sample = OracleSample(args.oracle_blocks, threads)
+        cpu_v, _ = sample.run()
+        cpu_desc, threads = sample.desc, sample.threads
+        del sample
     free, total = torch.cuda.mem_get_info()
     shape = wl.LLAMA3_8B_KV
     NB = args.kv_blocks
@@ -567,13 +576,6 @@ def run_ours(args):
                 "note": "peak is the driver-measured copy ceiling; cudaMemcpyAsync of this workload's own random bits, "
                         "sustained, is given beside it (random contents put the GPU at its power cap)"}
 
-    threads = os.cpu_count() or 1
-    if args.no_cpu_baseline:
-        cpu_v, cpu_desc = None, "skipped (--no-cpu-baseline)"
-    else:
-        sample = OracleSample(args.oracle_blocks, threads)
-        cpu_v, _ = sample.run()
-        cpu_desc, threads = sample.desc, sample.threads
     line = {
         "metric": "kv_pack_unpack_and_weight_materialise_GBps", "value": value, "unit": "GB/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
