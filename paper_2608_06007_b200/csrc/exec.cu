@@ -1,13 +1,20 @@
 // Plan lifecycle and the copy-executor kernels (sm_100a).
 //
-// One launch executes one group of a plan.  The grid is persistent: CTAs walk the plan's tile
-// ids with a grid stride; a tile is one outer index (a KV plane) and a row range of one
-// descriptor, about tile_bytes of payload.  Inside a tile every thread moves 16-byte vectors
+// One launch executes one group of a plan (a staged plan: one launch per segment).  By default
+// the grid has one CTA per tile - a tile is one plane of one descriptor and a row range of it,
+// about tile_bytes (32 KiB) of payload - and the hardware block scheduler spreads the tiles over
+// the SMs; KV groups walk their tiles plane-major over descriptors sorted by destination offset,
+// so every plane pass writes ascending addresses.  tuning.ctas_per_sm / max_ctas turn the same
+// kernel into a persistent grid-stride loop.  Inside a tile every thread moves 16-byte vectors
 // (narrower when the geometry or a base pointer is less aligned): a batch of independent
-// loads first, then the stores, so that many requests per thread are in flight.  Consecutive
-// lanes touch consecutive vectors of a run, so every warp access is one or more whole,
-// aligned segments on both the read and the write side.  Base pointers travel in the kernel
-// parameters; nothing is allocated or copied per execute call.
+// streaming loads first, then the stores, so that many requests per thread are in flight.
+// Consecutive lanes touch consecutive vectors of a run, so every warp access is one or more
+// whole, aligned lines on both the read and the write side.  Base pointers travel in the
+// kernel parameters; nothing is allocated or copied per execute call.
+//
+// Host memory: pointers to mapped pinned memory work in every call (the kernel loads / stores
+// over the host link).  Staged plans instead move the host-side bytes with the copy engines
+// through device staging rings and run the kernel device to device (see execute_staged).
 #include <cuda_runtime.h>
 #include <pthread.h>
 
