@@ -43,9 +43,11 @@
  * tc_plan_create only and may be freed afterwards.
  *
  * Memory spaces.  Pointers inside the *tables* passed to the execute calls are DEVICE-
- * addressable addresses: device memory, or pinned host memory mapped into the device's
+ * addressable addresses: device memory, pinned host memory mapped into the device's
  * address space (cudaHostAlloc / cudaHostRegister under unified addressing), which the kernel
- * then reads or writes directly over the host link (zero copy).  The tables themselves, the
+ * then reads or writes directly over the host link (zero copy), or another GPU's memory once
+ * peer access is enabled (every CTA then moves its own tile with plain loads and stores over
+ * NVLink; the library issues no multicast or bulk-tensor copy).  The tables themselves, the
  * spec and every array it points to are HOST memory.
  *
  * Devices.  A plan belongs to the CUDA device that was current when it was created; execute
