@@ -739,8 +739,10 @@ def run_extras(args, tc, torch, stream):
             create.append(1e3 * (time.perf_counter() - t0))
             h2d += int(st.reload_T.sum()) * shape.token_bytes
             d2h += int(st.offload_T.sum()) * shape.token_bytes
-        tc.tc_kv_unpack(plan, [host], [dev], sp)
+        # the short offload is enqueued first: the reload's ~6 000 page copies fill the driver's
+        # stream queue, so whatever is enqueued after it only starts when it is nearly done
         tc.tc_kv_pack(plan, [dev], [host], s2.cuda_stream)
+        tc.tc_kv_unpack(plan, [host], [dev], sp)
         torch.cuda.synchronize()   # a scheduler step ends when both directions have landed
         plan.destroy()
     wall = time.perf_counter() - t_all
