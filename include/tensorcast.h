@@ -114,27 +114,33 @@ enum {
     TC_PLAN_HOST_ONLY = 1u, /* validate and lower on the host only: the plan can be inspected
                                (tc_plan_stats, tc_plan_descriptors) but not executed, and no
                                CUDA call is made */
-    TC_PLAN_STAGED = 2u,    /* TC_KV_PACK / TC_KV_UNPACK whose packed buffer is PINNED HOST memory,
-                               TC_KV_MIXED whose dst_pool is a page-first pinned host pool in
-                               one allocation (plane_stride = one block of one plane) moved in
-                               full blocks, or TC_WEIGHTS whose blob is pinned host memory and
-                               whose tensors are read in contiguous pieces (whole tensors and
-                               dim-0 slabs; strided slices stay zero copy, which fetches only
-                               the bytes it needs): instead of letting the kernel load / store host
-                               memory directly (zero copy, the default), move the host-side
-                               bytes with the copy engines through rings of device staging
-                               buffers owned by the library (one ring of 3 x 64 MiB per
-                               direction and device, shared by all staged plans, allocated when
-                               the first such plan is created and kept until the process
-                               exits) and run the kernel device to device, segment by segment, overlapped on internal streams.  A
-                               packed buffer travels in contiguous ranges, a paged host pool
-                               page by page.  Groups that cannot be staged stay zero copy.  This is the streaming pipeline of pinned buffers and
-                               asynchronous streams (Sec. 5) with the scatter / layout
-                               transform fused into its device leg.  The copy engines drive the
-                               host link with larger transactions than SM loads and stores, so
-                               this path is a few percent faster; it costs one launch and one
-                               copy per segment instead of one launch per call.  Staged
-                               executions are serialised with one another by the library. */
+    TC_PLAN_STAGED = 2u,    /* The host side of the plan is PINNED HOST memory and should travel
+                               through the copy engines instead of being loaded / stored by the
+                               kernel itself (zero copy, the default):
+                                 - TC_KV_PACK / TC_KV_UNPACK: the packed buffer (request-major);
+                                 - TC_KV_MIXED: dst_pool, a page-first host pool in one
+                                   allocation (plane_stride = one block of one plane), moved in
+                                   full blocks;
+                                 - TC_WEIGHTS: the blob, for tensors read in contiguous pieces
+                                   (whole tensors, dim-0 slabs).
+                               The library cuts the plan into segments whose host bytes are
+                               contiguous ranges of at most 64 MiB (a paged pool: runs of 2 MiB
+                               pages), copies each segment between host memory and a ring of
+                               device staging buffers on an internal stream, and runs the same
+                               kernel device to device on the caller's stream, segment by
+                               segment, chained by events: the streaming pipeline of pinned
+                               buffers and asynchronous streams (Sec. 5) with the scatter /
+                               layout transform fused into its device leg.  The copy engines
+                               drive the host link with larger transactions than SM loads and
+                               stores, so this path is faster (and stays fast when both
+                               directions of the link are busy); it costs one launch and one or
+                               more copies per segment instead of one launch per call.  The
+                               rings (3 x 64 MiB per direction and device) are allocated when
+                               the first staged plan is created and kept until the process
+                               exits.  Groups that cannot be staged (strided slices of a blob,
+                               partial blocks of a paged pool, layer-major packed buffers) stay
+                               zero copy.  Staged executions are serialised with one another
+                               by the library while they are enqueued. */
     TC_PLAN_SAME_POOL = 8u, /* TC_KV_MIGRATE inside ONE pool (compaction / defragmentation): the
                                caller will pass the same table as source and destination.
                                src_pool and dst_pool must describe the same geometry, and no
@@ -223,8 +229,9 @@ typedef struct {
 /* Optional knobs; 0 everywhere = the library's defaults. */
 typedef struct {
     int32_t tile_bytes;   /* target bytes per tile (one CTA iteration) */
-    int32_t ctas_per_sm;  /* resident CTAs per SM for the persistent grid */
-    int32_t max_ctas;     /* cap on the grid (e.g. few CTAs for host-link transfers) */
+    int32_t ctas_per_sm;  /* > 0: a persistent grid-stride grid of this many CTAs per SM instead
+                             of one CTA per tile */
+    int32_t max_ctas;     /* > 0: cap on the grid (persistent grid-stride loop) */
     int32_t tile_order;   /* 0 auto: KV groups run plane-major over descriptors sorted by
                              destination offset (ascending writes); 1: request / descriptor order
                              as given, planes of one block consecutively */
