@@ -30,6 +30,18 @@ def test_library_exports_every_declared_symbol():
     assert ctypes.sizeof(tc.binding.tc_index_entry_t) == 64
 
 
+def test_header_is_plain_c_and_the_library_runs_from_a_c_client(tmp_path):
+    """tests/c_abi_check.c is compiled as C11 against include/tensorcast.h and linked with the
+    library; it lowers the worked micro-example and executes the descriptors by hand."""
+    import subprocess
+    lib = tc.build_library()
+    exe = tmp_path / "c_abi_check"
+    subprocess.check_call(["gcc", "-std=c11", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+                           os.path.join(ROOT, "tests", "c_abi_check.c"), "-o", str(exe), lib, "-Wl,-rpath," + os.path.dirname(lib)])
+    out = subprocess.run([str(exe)], capture_output=True, text=True, timeout=60)
+    assert out.returncode == 0 and out.stdout.strip() == "ok", out.stdout + out.stderr
+
+
 def test_fast_division_constants_are_exact():
     # the kernels divide by runtime constants with a multiply-high; replay that arithmetic
     rng = np.random.default_rng(0)
