@@ -47,7 +47,9 @@
  * address space (cudaHostAlloc / cudaHostRegister under unified addressing), which the kernel
  * then reads or writes directly over the host link (zero copy), or another GPU's memory once
  * peer access is enabled (every CTA then moves its own tile with plain loads and stores over
- * NVLink; the library issues no multicast or bulk-tensor copy).  The tables themselves, the
+ * NVLink; the library issues no multicast or bulk-tensor copy).  Pageable host memory is not
+ * addressable by the device: the execute calls refuse it (TC_ERR_INVALID_ARG) instead of
+ * letting a kernel fault.  The tables themselves, the
  * spec and every array it points to are HOST memory.
  *
  * Devices.  A plan belongs to the CUDA device that was current when it was created; execute

@@ -608,6 +608,26 @@ out:
 }
 #undef TC_TRY
 
+// A table entry must be memory the device can address: device memory, managed memory, or host
+// memory that is pinned and mapped.  Plain pageable host memory would make the kernel fault, so
+// it is refused here, on the host.  Large tables are spot-checked (first, last and evenly spaced
+// entries) to keep the call cheap.
+static int check_addressable(const void *const *table, size_t n, const char *what)
+{
+    const size_t step = n <= 32 ? 1 : n / 32;
+    for (size_t i = 0; i < n; i = (i + step < n || i == n - 1) ? i + step : n - 1) {
+        cudaPointerAttributes attr;
+        cudaError_t e = cudaPointerGetAttributes(&attr, table[i]);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return fail(TC_ERR_INVALID_ARG, "%s table entry %zu (%p) is not a valid address for this device", what, i, table[i]);
+        }
+        if (attr.type == cudaMemoryTypeUnregistered)
+            return fail(TC_ERR_INVALID_ARG, "%s table entry %zu (%p) is pageable host memory: pin it (cudaHostAlloc / cudaHostRegister) or use device memory", what, i, table[i]);
+    }
+    return TC_OK;
+}
+
 static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n_src, void *const *dst, size_t n_dst, void *stream,
                    unsigned long long *sums = nullptr)
 {
@@ -636,6 +656,9 @@ static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n
         if (!dst[i]) return fail(TC_ERR_INVALID_ARG, "destination table entry %zu is NULL", i);
         ptr_align = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(dst[i]) | 16));
     }
+    int rc;
+    if ((rc = check_addressable(src, n_src, "source")) != TC_OK) return rc;
+    if ((rc = check_addressable(const_cast<const void *const *>(dst), n_dst, "destination")) != TC_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (!g.segments.empty()) return execute_staged(plan, gi, g, src, dst, ptr_align, s, sums);
     return launch_any(plan, g, src, dst, ptr_align, s, nullptr, sums);

@@ -589,6 +589,11 @@ def test_empty_plan_wrong_tables_and_deadline_launch_nothing():
     with pytest.raises(tc.TensorCastError) as e:
         tc.tc_kv_pack(plan, [buf, 0], [buf])               # NULL table entry
     assert e.value.status == tc.TC_ERR_INVALID_ARG
+    pageable = np.zeros(1400832, dtype=np.uint8)           # ordinary host memory: the kernel could not address it
+    pool_ok = torch.zeros(2 * NB * shape.chunk_bytes, dtype=torch.uint8, device="cuda")
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_kv_pack(plan, [pool_ok, pool_ok[NB * shape.chunk_bytes:]], [pageable])
+    assert e.value.status == tc.TC_ERR_INVALID_ARG and "pageable" in str(e.value)
     soon = time.clock_gettime_ns(time.CLOCK_MONOTONIC) + 50_000_000
     late = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=pl, T=src.T, bt_off=src.bt_off, bt_src=src.bt, deadline_ns=soon))
     time.sleep(0.1)
