@@ -383,6 +383,12 @@ typedef struct {
 TC_API int tc_plan_descriptors(const tc_plan_t *plan, int group, tc_descriptor_t *out, size_t cap,
                         size_t *n_out);
 
+/* Give back what the library caches between plans: the pool of device blocks that plan storage
+ * is carved from and, if no staged plan exists on the device any more, its staging rings.
+ * Synchronises the internal copy streams first.  Safe to call at any time; later calls simply
+ * allocate again. */
+TC_API int tc_trim(void);
+
 /* Static string naming a status code. */
 TC_API const char *tc_strerror(int status);
 

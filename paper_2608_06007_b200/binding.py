@@ -91,7 +91,7 @@ class tc_descriptor_t(C.Structure):
 
 EXPORTS = ("tc_plan_create", "tc_kv_pack", "tc_kv_unpack", "tc_weights_materialize",
            "tc_plan_destroy", "tc_plan_stats", "tc_plan_descriptors", "tc_strerror", "tc_last_error",
-           "tc_kv_pack_noalloc", "tc_weights_materialize_checksum")
+           "tc_kv_pack_noalloc", "tc_weights_materialize_checksum", "tc_trim")
 
 _lib = None
 
@@ -117,6 +117,8 @@ def load_library(path: str | None = None):
     lib.tc_kv_pack_noalloc.restype = C.c_int
     lib.tc_weights_materialize_checksum.argtypes = [vp, vp, vp, sz, vp, vp]
     lib.tc_weights_materialize_checksum.restype = C.c_int
+    lib.tc_trim.argtypes = []
+    lib.tc_trim.restype = C.c_int
     lib.tc_strerror.argtypes = [C.c_int]
     lib.tc_strerror.restype = C.c_char_p
     lib.tc_last_error.restype = C.c_char_p
@@ -319,6 +321,11 @@ def tc_weights_materialize_checksum(plan: Plan, blob, dst_ptrs, checksums, strea
     """tc_weights_materialize that also fills `checksums` (device uint64[n_tensors]) in the same pass."""
     d, nd = _table(dst_ptrs)
     _check(load_library().tc_weights_materialize_checksum(plan.handle, _addr(blob), d, nd, _addr(checksums), _stream(stream)))
+
+
+def tc_trim() -> None:
+    """Release the device memory the library caches between plans (plan-storage blocks, idle staging rings)."""
+    _check(load_library().tc_trim())
 
 
 def tc_plan_stats(plan: Plan) -> tc_plan_stats_t:

@@ -761,6 +761,25 @@ extern "C" int tc_weights_materialize_checksum(const tc_plan_t *plan, const void
     return execute(plan, 0, src, 1, dst_ptrs, n_dst, stream, reinterpret_cast<unsigned long long *>(checksums));
 }
 
+extern "C" int tc_trim(void)
+{
+    clear_error();
+    pthread_mutex_lock(&g_block_mu);
+    for (const CachedBlock &b : g_block_cache) cudaFree(b.ptr);
+    g_block_cache.clear();
+    g_block_cache_bytes = 0;
+    pthread_mutex_unlock(&g_block_mu);
+    pthread_mutex_lock(&g_stage_mu);
+    for (StageArena &a : g_stage)
+        if (a.refs == 1) {  // only the library's own reference is left
+            for (StageRing &r : a.ring)
+                if (r.copy) cudaStreamSynchronize(r.copy);
+            stage_free(a);
+        }
+    pthread_mutex_unlock(&g_stage_mu);
+    return TC_OK;
+}
+
 extern "C" int tc_plan_stats(const tc_plan_t *plan, tc_plan_stats_t *out)
 {
     clear_error();

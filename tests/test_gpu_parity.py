@@ -604,3 +604,17 @@ def test_empty_plan_wrong_tables_and_deadline_launch_nothing():
     assert e.value.status == tc.TC_ERR_DEADLINE
     assert (out.result() == 0xA5).all()                     # nothing was launched
     assert plan.stats().device_bytes > 0 and plan.stats().executable
+    # the caches can be dropped at any time; the library allocates again on demand
+    free0 = torch.cuda.mem_get_info()[0]
+    staged = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=pl, T=src.T, bt_off=src.bt_off, bt_src=src.bt, flags=tc.TC_PLAN_STAGED))
+    staged.destroy()
+    plan.destroy()
+    late.destroy()
+    empty.destroy()
+    tc.tc_trim()
+    assert torch.cuda.mem_get_info()[0] >= free0
+    again = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=pl, T=src.T, bt_off=src.bt_off, bt_src=src.bt, flags=tc.TC_PLAN_STAGED))
+    host = torch.zeros(1400832, dtype=torch.uint8).pin_memory()
+    tc.tc_kv_pack(again, [pool_ok, pool_ok[NB * shape.chunk_bytes:]], [host])
+    torch.cuda.synchronize()
+    assert not host.numpy().any()                         # an all-zero pool packs to zeros

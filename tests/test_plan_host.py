@@ -449,6 +449,7 @@ def test_empty_plans_deadline_and_kind_checks():
     with pytest.raises(tc.TensorCastError) as e:
         tc.tc_weights_materialize(plan, 16, [16])
     assert e.value.status == tc.TC_ERR_KIND
+    tc.tc_trim()                                        # nothing cached here: still fine
     plan.destroy()
     plan.destroy()                                      # idempotent; NULL destroy is a no-op
     assert tc.load_library().tc_plan_destroy(None) == 0
