@@ -430,6 +430,33 @@ def test_validation_rejects_bad_plans_before_any_launch():
     assert _status(ck_spec(ck, dst_bytes=small, flags=HOST)) == tc.TC_ERR_BOUNDS
 
 
+def test_documented_limits_are_enforced():
+    shape, NB, src, dst = wl.config1()
+    # pointer-table capacity: L*2 planes per pool, src + dst slots of one call
+    big_l = (1001, 16, 8, 128, 2)
+    assert _status(tc.kv_spec(tc.TC_KV_PACK, big_l, src_pool=tc.pool(tc.TC_NHD, 4, 2002), flags=HOST)) == tc.TC_ERR_INVALID_ARG
+    n = tc.TC_MAX_TABLE_SLOTS
+    spec = tc.weights_spec(np.arange(n) * 16, [16] * n, [2] * n, [1] * n, [[8, 1, 1, 1]] * n, blob_bytes=16 * n, flags=HOST)
+    assert _status(spec) == tc.TC_ERR_INVALID_ARG
+    ok = n - 1
+    plan = tc.tc_plan_create(tc.weights_spec(np.arange(ok) * 16, [16] * ok, [2] * ok, [1] * ok, [[8, 1, 1, 1]] * ok, blob_bytes=16 * ok, flags=HOST))
+    assert plan.stats().n_descriptors[0] == ok
+    # more than 2^31 tiles in one plan
+    huge = 1 << 47
+    assert _status(tc.weights_spec([0], [huge], [1], [1], [[huge, 1, 1, 1]], blob_bytes=huge, flags=HOST)) == tc.TC_ERR_INVALID_ARG
+    # tile size knob must be a power of two in range
+    assert _status(_pack_spec(tuning=dict(tile_bytes=3000))) == tc.TC_ERR_INVALID_ARG
+    assert _status(_pack_spec(tuning=dict(tile_bytes=1 << 21))) == tc.TC_ERR_INVALID_ARG
+    # the longest request the configs allow (32 768 tokens) and a single-token one, in one plan
+    T = np.array([32768, 1], dtype=np.int64)
+    off = np.array([0, 2048, 2049], dtype=np.int64)
+    bt = np.arange(2049, dtype=np.int32)
+    s8 = wl.LLAMA3_8B_KV
+    st = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s8.tuple, src_pool=tc.pool(tc.TC_NHD, 2049, 1, plane_stride=2049 * s8.chunk_bytes),
+                                      packed_layout=tc.TC_HND, T=T, bt_off=off, bt_src=bt, flags=HOST)).stats()
+    assert st.payload_bytes[0] == 32769 * s8.token_bytes and st.n_descriptors[0] == 2049 and st.n_tiles[0] == 2049 * 64
+
+
 def test_empty_plans_deadline_and_kind_checks():
     shape, NB, src, dst = wl.config1()
     empty = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape.tuple, src_pool=tc.pool(tc.TC_NHD, NB, 2), flags=HOST))
