@@ -218,6 +218,46 @@ def test_weights_transform_into_fused_target():
     assert np.array_equal(target, want)
 
 
+def test_tp_resharding_8_to_2_and_2_to_8_by_composition_of_rules():
+    """A checkpoint saved as W shard blobs, loaded at another TP degree W'.  8 -> 2: rank r' of 2
+    concatenates four source shards along the split dim (dst_off / dst_stride windows, one plan
+    per source blob).  2 -> 8: rank r' of 8 takes a quarter of one source shard (split of the
+    shard).  Both must equal the oracle's direct W' shard of the full tensor."""
+    rng = np.random.default_rng(8)
+    shp, E = (16, 24), 2                                   # one [out, in] matrix, bf16-sized elements
+    full = rng.integers(0, 256, shp[0] * shp[1] * E, dtype=np.uint8)
+    for dim in (0, 1):
+        def shard(rank, world):
+            out = np.zeros(full.size // world, dtype=np.uint8)
+            oracle.weights([0], [E], [[shp[0], shp[1], 1, 1]], [dim], rank, world, full, [out])
+            return out
+        sshape = lambda world: [shp[0] // world if dim == 0 else shp[0], shp[1] // world if dim == 1 else shp[1], 1, 1]
+        # 8 -> 2
+        for r2 in range(2):
+            want = shard(r2, 2)
+            got = np.full(want.size, 0xEE, dtype=np.uint8)
+            cnt = [np.zeros(want.size, dtype=np.int32)]
+            d2 = sshape(2)
+            for k in range(4):                              # source shards 4*r2 .. 4*r2+3
+                src_blob = shard(4 * r2 + k, 8)
+                s8 = sshape(8)
+                if dim == 0:
+                    off, stride = k * src_blob.size, [d2[1] * E, E, E, E]
+                else:
+                    off, stride = k * s8[1] * E, [d2[1] * E, E, E, E]
+                spec = tc.weights_spec([0], [src_blob.size], [E], [2], [s8], blob_bytes=src_blob.size, dst_slot=[0], dst_off=[off],
+                                       dst_stride=[stride], n_dst=1, dst_bytes=[want.size], flags=HOST)
+                run_descriptors(tc.tc_plan_create(spec).descriptors(0), [src_blob], [got], cnt)
+            assert np.array_equal(got, want) and (cnt[0] == 1).all(), (dim, r2)
+        # 2 -> 8
+        for r8 in range(8):
+            src_blob = shard(r8 // 4, 2)
+            spec = tc.weights_spec([0], [src_blob.size], [E], [2], [sshape(2)], split_dim=[dim], rank=r8 % 4, world=4, blob_bytes=src_blob.size, flags=HOST)
+            got = np.full(full.size // 8, 0xEE, dtype=np.uint8)
+            run_descriptors(tc.tc_plan_create(spec).descriptors(0), [src_blob], [got])
+            assert np.array_equal(got, shard(r8, 8)), (dim, r8)
+
+
 def test_interleaved_strided_destinations_pass_the_exact_overlap_check():
     # two [4][3] byte tensors interleaved column-wise into one [4][6] target: bounding spans
     # intersect but no byte is written twice
