@@ -56,12 +56,12 @@ def test_config2_full_size_pack_unpack_migrate():
     wl.fill_torch(poolA, wl.SEED_BASE + 2)
     poolB = torch.full((WB * shape.block_bytes,), 0xA5, **u8)
     payload = int(src.T.sum()) * shape.token_bytes
-    Q = torch.full((payload,), 0x5A, **u8)
+    Q = torch.full((max(int(w[0].T.sum()) for w in waves) * shape.token_bytes,), 0x5A, **u8)
     plA = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * chunk, slot_bytes=poolA.numel())
     plB = tc.pool(tc.TC_NHD, WB, 1, plane_stride=WB * chunk, slot_bytes=poolB.numel())
     kw = dict(T=src.T, bt_off=src.bt_off)
-    pack = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, packed_bytes=payload, bt_src=src.bt, **kw))
-    unpack = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, packed_bytes=payload, bt_dst=dst.bt, **kw))
+    pack = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, packed_bytes=Q.numel(), bt_src=src.bt, **kw))
+    unpack = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, packed_bytes=Q.numel(), bt_dst=dst.bt, **kw))
     assert pack.stats().payload_bytes[0] == payload and pack.stats().grid[0] == pack.stats().n_tiles[0]
     tc.tc_kv_pack(pack, [poolA], [Q])
     tc.tc_kv_unpack(unpack, [Q], [poolB])
@@ -97,6 +97,37 @@ def test_config2_full_size_pack_unpack_migrate():
     tc.tc_kv_pack(mig, [poolA], [poolC])
     torch.cuda.synchronize()
     assert torch.equal(poolC, poolB)
+    # every other wave of the workload: the any-size properties over all bytes (full blocks land
+    # in their destination blocks, unused destination blocks keep the sentinel), both through
+    # pack + unpack and through the fused migrate
+    for w_src, w_dst in waves[1:]:
+        wkw = dict(T=w_src.T, bt_off=w_src.bt_off)
+        wp = int(w_src.T.sum()) * shape.token_bytes
+        assert wp <= Q.numel()
+        pk = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, bt_src=w_src.bt, **wkw))
+        up = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, bt_dst=w_dst.bt, **wkw))
+        mg = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, s, src_pool=plA, dst_pool=plB, bt_src=w_src.bt, bt_dst=w_dst.bt, **wkw))
+        poolB.fill_(0xA5)
+        poolC.fill_(0xA5)
+        tc.tc_kv_pack(pk, [poolA], [Q])
+        tc.tc_kv_unpack(up, [Q], [poolB])
+        tc.tc_kv_pack(mg, [poolA], [poolC])
+        torch.cuda.synchronize()
+        assert torch.equal(poolB, poolC)
+        fullw = np.concatenate([np.arange(w_src.bt_off[r], w_src.bt_off[r] + w_src.T[r] // shape.B) for r in range(len(w_src.T))])
+        sbw = torch.as_tensor(w_src.bt[fullw], dtype=torch.long, device="cuda")
+        dbw = torch.as_tensor(w_dst.bt[fullw], dtype=torch.long, device="cuda")
+        for p in range(0, planes, 5):
+            assert torch.equal(A[p][sbw], B[p][dbw])
+        ubw = torch.as_tensor(np.setdiff1d(np.arange(WB), w_dst.bt), dtype=torch.long, device="cuda")
+        assert bool((B[::7, ubw] == 0xA5).all())
+        for pl_ in (pk, up, mg):
+            pl_.destroy()
+    # restore wave 0's results for the staged comparison below
+    poolB.fill_(0xA5)
+    tc.tc_kv_pack(pack, [poolA], [Q])
+    tc.tc_kv_unpack(unpack, [Q], [poolB])
+    torch.cuda.synchronize()
     # staged host path at full size: offload to pinned host and reload must reproduce the
     # (oracle-checked) direct results byte for byte
     Qh = torch.empty(payload, dtype=torch.uint8).pin_memory()
@@ -108,7 +139,8 @@ def test_config2_full_size_pack_unpack_migrate():
     tc.tc_kv_unpack(unpack_s, [Qh], [poolC])
     torch.cuda.synchronize()
     for lo in range(0, payload, 1 << 30):
-        assert torch.equal(Qh[lo:lo + (1 << 30)].cuda(), Q[lo:lo + (1 << 30)])
+        hi = min(lo + (1 << 30), payload)
+        assert torch.equal(Qh[lo:hi].cuda(), Q[lo:hi])
     assert torch.equal(poolC, poolB)
     del poolA, poolB, poolC, Q, Qh, A, B
     _free()
