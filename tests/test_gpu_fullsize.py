@@ -81,7 +81,16 @@ def test_config2_full_size_pack_unpack_migrate():
         oracle.kv_unpack(s, oracle.NHD, chunk, [want_blocks[p].reshape(-1) for p in range(planes)], [src.T[r]], [0, n], np.arange(n), oracle.HND, want)
         got_blocks = _blocks_to_host(poolB, planes, WB, chunk, dst.bt[dst.bt_off[r]:dst.bt_off[r + 1]])
         assert np.array_equal(got_blocks, want_blocks), f"request {r} unpacked"
-    # (b) every full block arrives; every block outside the table keeps the sentinel
+    # (b) every byte of the packed buffer, as the library routine it reduces to: gather the
+    # request's blocks, keep the valid tokens, swap the (token, head) axes (request-level HND)
+    A5 = poolA.view(planes, NB, shape.B, shape.H, shape.D * shape.E)
+    for r in range(len(src.T)):
+        ids = torch.as_tensor(src.bt[src.bt_off[r]:src.bt_off[r + 1]], dtype=torch.long, device="cuda")
+        Tr = int(src.T[r])
+        tok = A5[:, ids].reshape(planes, -1, shape.H, shape.D * shape.E)[:, :Tr]
+        assert torch.equal(tok.permute(0, 2, 1, 3).reshape(-1), Q[int(offs[r]):int(offs[r + 1])]), f"request {r}"
+        del tok
+    # every full block arrives; every block outside the table keeps the sentinel
     full = np.concatenate([np.arange(src.bt_off[r], src.bt_off[r] + src.T[r] // shape.B) for r in range(len(src.T))])
     sb = torch.as_tensor(src.bt[full], dtype=torch.long, device="cuda")
     db = torch.as_tensor(dst.bt[full], dtype=torch.long, device="cuda")
