@@ -111,6 +111,30 @@ def test_pack_unpack_all_layouts(pool_l, packed_l, slots, tile):
     assert np.array_equal(fresh.result(), want_pool)
 
 
+@pytest.mark.parametrize("tune", [dict(tile_order=1), dict(ctas_per_sm=2), dict(max_ctas=7), dict(tile_bytes=65536), dict(tile_bytes=1024, ctas_per_sm=1, tile_order=1)])
+def test_tuning_knobs_change_the_schedule_not_the_bytes(tune):
+    rng = np.random.default_rng(29)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=3, NB=90, B=32, H=8, D=128, E=2, T=(700, 33, 0, 64, 1200))
+    L = shape[0]
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride)
+    d_pool = dev(pool)
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, L * 2), T, off, bt, oracle.HND, want, threads=8)
+    out = Guarded(want.size)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_src=bt, tuning=tune))
+    tc.tc_kv_pack(plan, [d_pool], [out.ptr()])
+    assert np.array_equal(out.result(), want)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_migrate(shape, oracle.NHD, stride, planes_of(pool, L * 2), oracle.NHD, stride, planes_of(want_pool, L * 2), T, off, bt, bt2, threads=8)
+    mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl, T=T, bt_off=off, bt_src=bt, bt_dst=bt2, tuning=tune))
+    fresh = Guarded(pool.size)
+    tc.tc_kv_pack(mig, [d_pool], [fresh.ptr()])
+    assert np.array_equal(fresh.result(), want_pool)
+    if "max_ctas" in tune:
+        assert plan.stats().grid[0] == 7
+
+
 @pytest.mark.parametrize("E,D,shift", [(1, 7, 0), (2, 5, 0), (4, 3, 0), (8, 3, 0), (2, 64, 2), (2, 64, 4), (2, 64, 8), (1, 33, 1)])
 def test_odd_shapes_and_misaligned_pointers_fall_back_to_narrow_vectors(E, D, shift):
     rng = np.random.default_rng(22)
