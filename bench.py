@@ -595,6 +595,95 @@ def run_ours(args):
     ranks.close()
 
 
+def cold_path(args, tc, torch, stream):
+    """Weight loading from a FILE (storage -> pinned ring -> device, scatter and slicing fused
+    into the device leg): wall-clock GB/s of blob bytes, next to the plain rate at which the
+    same file can be read into pinned memory and to the unpipelined sequence (read everything,
+    then materialise from pinned memory)."""
+    import shutil
+    import tempfile
+    sp = stream.cuda_stream
+    ck = wl.llama_checkpoint(layers=1, vocab=16032) if args.small else wl.llama_checkpoint(layers=args.cold_layers, vocab=32064)
+    root = "/dev/shm" if os.path.isdir("/dev/shm") and shutil.disk_usage("/dev/shm").free > 2 * ck.nbytes_total else tempfile.gettempdir()
+    if shutil.disk_usage(root).free < 2 * ck.nbytes_total:
+        return {"skipped": f"no room for a {ck.nbytes_total} byte file under {root}"}
+    blob = torch.empty(ck.nbytes_total, dtype=torch.uint8, device="cuda")
+    wl.fill_torch(blob, wl.SEED_BASE + 3, "normal")
+    host = torch.empty(ck.nbytes_total, dtype=torch.uint8).pin_memory()
+    host.copy_(blob)
+    header = 4096 + 8 * ck.N
+    fdw, path = tempfile.mkstemp(prefix="tc_cold_", suffix=".bin", dir=root)
+    out = {"file": f"{ck.nbytes_total} B blob behind a {header} B header, in {root} (page cache)"}
+    try:
+        with os.fdopen(fdw, "wb") as f:
+            f.write(bytes(header))
+            host.numpy().tofile(f)
+        nbytes = [ck.nbytes(i) for i in range(ck.N)]
+        dstw = torch.empty(ck.nbytes_total, dtype=torch.uint8, device="cuda")
+        ptrs = [dstw.data_ptr() + int(o) for o in np.concatenate([[0], np.cumsum(nbytes)])[:-1]]
+        sums = torch.zeros(ck.N, dtype=torch.int64, device="cuda")
+        fd = os.open(path, os.O_RDONLY)
+        n_readers = max(1, min(8, (os.cpu_count() or 2) - 1))
+
+        def read_all():  # the storage leg alone: the whole blob into pinned memory, same thread count
+            view = memoryview(host.numpy())
+            part = -(-ck.nbytes_total // n_readers)
+
+            def rd(i):
+                lo, hi = i * part, min(ck.nbytes_total, (i + 1) * part)
+                while lo < hi:
+                    k = os.preadv(fd, [view[lo:min(hi, lo + (64 << 20))]], header + lo)
+                    lo += k
+            th = [threading.Thread(target=rd, args=(i,)) for i in range(n_readers)]
+            [t.start() for t in th]
+            [t.join() for t in th]
+
+        def wall(fn, reps=3):
+            best = []
+            for i in range(reps + 1):
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                fn()
+                torch.cuda.synchronize()
+                if i:
+                    best.append(time.perf_counter() - t0)
+            return statistics.mean(best)
+
+        plan = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total,
+                                                 flags=tc.TC_PLAN_STREAM | tc.TC_PLAN_CHECKSUM))
+        staged = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total, flags=tc.TC_PLAN_STAGED))
+        t_read = wall(read_all)
+        with torch.cuda.stream(stream):
+            t_stream = wall(lambda: tc.tc_weights_materialize_file(plan, fd, header, ptrs, stream=sp))
+            same = bool(torch.equal(dstw, blob))
+            t_check = wall(lambda: tc.tc_weights_materialize_file(plan, fd, header, ptrs, checksums=sums, stream=sp))
+            t_seq = wall(lambda: (read_all(), tc.tc_weights_materialize(staged, host, ptrs, sp)))
+        W = 8
+        sizes = [n // (W if ck.split_dim[i] >= 0 else 1) for i, n in enumerate(nbytes)]
+        sptrs = [dstw.data_ptr() + int(o) for o in np.concatenate([[0], np.cumsum(sizes)])[:-1]]
+        shard = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, split_dim=ck.split_dim, rank=args.shard_rank, world=W,
+                                                  blob_bytes=ck.nbytes_total, flags=tc.TC_PLAN_STREAM))
+        read_bytes = sum(sg.bytes for sg in shard.segments(0))
+        with torch.cuda.stream(stream):
+            t_shard = wall(lambda: tc.tc_weights_materialize_file(shard, fd, header, sptrs, stream=sp))
+        os.close(fd)
+        out.update({
+            "readers": n_readers, "chunks": plan.stats().launches_per_execute, "bytes_match_after_streaming": same,
+            "GBps_file_read_into_pinned_only": ck.nbytes_total / t_read / GB,
+            "GBps_streamed_full": ck.nbytes_total / t_stream / GB,
+            "GBps_streamed_full_with_checksum": ck.nbytes_total / t_check / GB,
+            "GBps_read_everything_then_materialize": ck.nbytes_total / t_seq / GB,
+            "shard_1_of_8": {"payload_bytes": sum(sizes), "file_bytes_read": read_bytes, "chunks": shard.stats().launches_per_execute,
+                             "ms": 1e3 * t_shard, "GBps_of_file_bytes": read_bytes / t_shard / GB}})
+        for p_ in (plan, staged, shard):
+            p_.destroy()
+    finally:
+        os.unlink(path)
+    del blob, host
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_extras(args, tc, torch, stream):
     """Secondary workloads, reported beside the headline: configs[3] (70B-shaped pool-to-pool
     migration, one wave) and configs[4] (prefix-reload burst: one mixed plan per scheduler step,
@@ -679,6 +768,7 @@ def run_extras(args, tc, torch, stream):
     planc.destroy()
     del blob, dstw
     torch.cuda.empty_cache()
+    out["weights cold path: blob streamed from a file"] = cold_path(args, tc, torch, stream)
     # ---- configs[3]
     shape = wl.LLAMA3_70B_KV
     free, _ = torch.cuda.mem_get_info()
@@ -789,6 +879,7 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary workloads (configs[3], configs[4])")
     ap.add_argument("--host-pool-blocks", type=int, default=8192, help="configs[4]: pinned host pool size in 2 MiB blocks")
     ap.add_argument("--burst-steps", type=int, default=10, help="configs[4]: scheduler steps timed (the workload has 200)")
+    ap.add_argument("--cold-layers", type=int, default=8, help="cold-path extra: layers of the checkpoint written to a file (8: 4.0 GB)")
     ap.add_argument("--host-ctas", type=int, default=0)
     ap.add_argument("--host-path", default="staged", choices=["staged", "zerocopy"])
     ap.add_argument("--e2e-schedule", default="duplex", choices=["duplex", "serial"],

@@ -92,7 +92,8 @@ typedef enum {
     TC_ERR_OOM = -6,         /* host or device allocation of plan storage failed */
     TC_ERR_CUDA = -7,        /* a CUDA runtime call failed (no device, launch failure) */
     TC_ERR_DEADLINE = -8,    /* the plan's deadline had already passed at call entry */
-    TC_ERR_TOO_LARGE = -9    /* the request exceeds a fixed capacity of the entry point called */
+    TC_ERR_TOO_LARGE = -9,   /* the request exceeds a fixed capacity of the entry point called */
+    TC_ERR_IO = -10          /* reading the blob file failed or hit end of file early */
 } tc_status;
 
 typedef enum {
@@ -148,11 +149,20 @@ enum {
                                src_pool and dst_pool must describe the same geometry, and no
                                block may be both read and written (TC_ERR_OVERLAP), so that the
                                result does not depend on the order in which tiles run. */
-    TC_PLAN_CHECKSUM = 4u   /* TC_WEIGHTS: the plan can also be run by
+    TC_PLAN_CHECKSUM = 4u,  /* TC_WEIGHTS: the plan can also be run by
                                tc_weights_materialize_checksum, which folds an integrity
                                checksum of every tensor into the same pass as the copy.  Needs
                                16-byte aligned geometry and tensors that start on 4-byte
                                boundaries of the blob (TC_ERR_INVALID_ARG otherwise). */
+    TC_PLAN_STREAM = 16u    /* TC_WEIGHTS: the blob is streamed chunk by chunk, from a file
+                               (tc_weights_materialize_file) or from pinned host memory
+                               (tc_weights_materialize), through the staging ring.  Unlike
+                               TC_PLAN_STAGED every tensor is staged: a strided slice travels
+                               as the byte range that covers it (whole rows, as a loader
+                               reading from storage fetches them) and is cut out on the
+                               device.  Chunks start on 4 KiB boundaries of the blob and are at
+                               most 64 MiB; a tile whose covering range is larger cannot be
+                               streamed (TC_ERR_TOO_LARGE at create). */
 };
 
 #define TC_MAX_TABLE_SLOTS 4000 /* src slots + dst slots of one execute call */
@@ -309,6 +319,31 @@ TC_API int tc_weights_materialize_checksum(const tc_plan_t *plan, const void *bl
                                            size_t n_dst, uint64_t *checksums, void *stream);
 
 /*
+ * Cold path of weight loading: tc_weights_materialize with the blob in a FILE (the
+ * storage -> pinned staging buffer -> device memory pipeline of Sec. 5, with the scatter, the
+ * rank's slicing and optionally the integrity checksum fused into the device leg).
+ * `plan`: a TC_WEIGHTS plan created with TC_PLAN_STREAM.  fd: a file descriptor open for
+ * reading (ordinary buffered I/O; the library only calls pread / posix_fadvise on it and never
+ * closes it); the blob starts at byte `file_offset` of the file, so a container format's header
+ * may precede it.  checksums: NULL, or as for tc_weights_materialize_checksum (the plan then
+ * also needs TC_PLAN_CHECKSUM).
+ * Per chunk of the plan the call reads the chunk's byte range with a few reader threads into
+ * one of three 64 MiB pinned host buffers that the library owns (allocated by the first call
+ * on a device, kept until tc_trim or exit), hands it to the copy engine and launches the kernel
+ * for the chunk's tiles on `stream`; reading chunk k+1 overlaps transfer and scatter of chunk k.
+ * The call RETURNS when the last chunk has been read and enqueued, so unlike the other entry
+ * points it blocks for about the time the storage reads take; device work completes on
+ * `stream` as usual.  Calls on one device are serialised with one another.
+ * Errors: everything tc_weights_materialize checks, before the first read; TC_ERR_KIND for a
+ * plan without TC_PLAN_STREAM; TC_ERR_IO when a read fails or the file ends early - chunks
+ * before the failing one have been enqueued and will still complete, the destination tensors
+ * are then partly written (there is no rollback, as for any failure after launch).
+ */
+TC_API int tc_weights_materialize_file(const tc_plan_t *plan, int fd, int64_t file_offset,
+                                       void *const *dst_ptrs, size_t n_dst, uint64_t *checksums,
+                                       void *stream);
+
+/*
  * Free the plan's host and device storage.  The caller must first have synchronised every
  * stream that executes it.  NULL is a no-op returning TC_OK.
  */
@@ -376,12 +411,31 @@ typedef struct {
     int64_t src_off, dst_off, src_outer, dst_outer, src_s0, src_s1, dst_s0, dst_s1;
     uint32_t src_slot, dst_slot, src_slot_step, dst_slot_step;
     uint32_t run_bytes, n0, rows, n_outer;
+    uint32_t rows_per_tile;   /* rows one tile (one CTA pass) moves */
+    uint32_t tiles_per_outer; /* tile ids per outer index; parts past the last row are empty */
+    uint32_t tile0;           /* global id of tile (outer 0, part 0); tile (o, p) has id
+                                 tile0 + o*tiles_per_outer + p */
+    uint32_t reserved;
 } tc_descriptor_t;
 
 /* Copy up to `cap` descriptors of `group` (0 or 1) into out (host array); *n_out receives the
  * group's total count. */
 TC_API int tc_plan_descriptors(const tc_plan_t *plan, int group, tc_descriptor_t *out, size_t cap,
                         size_t *n_out);
+
+/* One chunk of a staged or streamed TC_WEIGHTS plan, or one segment of a staged request-major
+ * packed buffer: the tiles [tile0, tile0 + n_tiles) run against host bytes [host_off,
+ * host_off + bytes) of the blob / packed buffer, which the kernel sees at the start of a
+ * staging buffer.  (n_tiles = 0: the segment is a window of descriptors x planes, not a tile
+ * range, as staged KV plans use; only host_off and bytes are meaningful then.) */
+typedef struct {
+    int64_t host_off, bytes;
+    uint32_t tile0, n_tiles;
+} tc_segment_t;
+
+/* Copy up to `cap` segments of `group` into out (host array); *n_out receives the count
+ * (0 for plans that are not staged). */
+TC_API int tc_plan_segments(const tc_plan_t *plan, int group, tc_segment_t *out, size_t cap, size_t *n_out);
 
 /* Give back what the library caches between plans: the pool of device blocks that plan storage
  * is carved from and, if no staged plan exists on the device any more, its staging rings.

@@ -16,7 +16,7 @@ from . import build as _build
 
 TC_OK = 0
 TC_ERR_INVALID_ARG, TC_ERR_SHAPE, TC_ERR_BOUNDS, TC_ERR_OVERLAP = -1, -2, -3, -4
-TC_ERR_KIND, TC_ERR_OOM, TC_ERR_CUDA, TC_ERR_DEADLINE, TC_ERR_TOO_LARGE = -5, -6, -7, -8, -9
+TC_ERR_KIND, TC_ERR_OOM, TC_ERR_CUDA, TC_ERR_DEADLINE, TC_ERR_TOO_LARGE, TC_ERR_IO = -5, -6, -7, -8, -9, -10
 TC_NOALLOC_SCRATCH_BYTES = 1 << 20
 TC_KV_PACK, TC_KV_UNPACK, TC_KV_MIGRATE, TC_KV_MIXED, TC_WEIGHTS = 1, 2, 3, 4, 5
 TC_NHD, TC_HND = 0, 1
@@ -25,6 +25,7 @@ TC_PLAN_HOST_ONLY = 1
 TC_PLAN_STAGED = 2
 TC_PLAN_CHECKSUM = 4
 TC_PLAN_SAME_POOL = 8
+TC_PLAN_STREAM = 16
 TC_MAX_TABLE_SLOTS = 4000
 
 
@@ -86,12 +87,18 @@ class tc_descriptor_t(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("src_off", "dst_off", "src_outer", "dst_outer",
                                           "src_s0", "src_s1", "dst_s0", "dst_s1")] + \
                [(n, C.c_uint32) for n in ("src_slot", "dst_slot", "src_slot_step", "dst_slot_step",
-                                          "run_bytes", "n0", "rows", "n_outer")]
+                                          "run_bytes", "n0", "rows", "n_outer",
+                                          "rows_per_tile", "tiles_per_outer", "tile0", "reserved")]
+
+
+class tc_segment_t(C.Structure):
+    _fields_ = [("host_off", C.c_int64), ("bytes", C.c_int64), ("tile0", C.c_uint32), ("n_tiles", C.c_uint32)]
 
 
 EXPORTS = ("tc_plan_create", "tc_kv_pack", "tc_kv_unpack", "tc_weights_materialize",
            "tc_plan_destroy", "tc_plan_stats", "tc_plan_descriptors", "tc_strerror", "tc_last_error",
-           "tc_kv_pack_noalloc", "tc_weights_materialize_checksum", "tc_trim")
+           "tc_kv_pack_noalloc", "tc_weights_materialize_checksum", "tc_trim",
+           "tc_weights_materialize_file", "tc_plan_segments")
 
 _lib = None
 
@@ -117,6 +124,10 @@ def load_library(path: str | None = None):
     lib.tc_kv_pack_noalloc.restype = C.c_int
     lib.tc_weights_materialize_checksum.argtypes = [vp, vp, vp, sz, vp, vp]
     lib.tc_weights_materialize_checksum.restype = C.c_int
+    lib.tc_weights_materialize_file.argtypes = [vp, C.c_int, C.c_int64, vp, sz, vp, vp]
+    lib.tc_weights_materialize_file.restype = C.c_int
+    lib.tc_plan_segments.argtypes = [vp, C.c_int, vp, sz, C.POINTER(sz)]
+    lib.tc_plan_segments.restype = C.c_int
     lib.tc_trim.argtypes = []
     lib.tc_trim.restype = C.c_int
     lib.tc_strerror.argtypes = [C.c_int]
@@ -275,6 +286,9 @@ class Plan:
     def descriptors(self, group: int = 0):
         return tc_plan_descriptors(self, group)
 
+    def segments(self, group: int = 0):
+        return tc_plan_segments(self, group)
+
 
 def tc_plan_create(spec, keep=None) -> Plan:
     if isinstance(spec, tuple):
@@ -321,6 +335,25 @@ def tc_weights_materialize_checksum(plan: Plan, blob, dst_ptrs, checksums, strea
     """tc_weights_materialize that also fills `checksums` (device uint64[n_tensors]) in the same pass."""
     d, nd = _table(dst_ptrs)
     _check(load_library().tc_weights_materialize_checksum(plan.handle, _addr(blob), d, nd, _addr(checksums), _stream(stream)))
+
+
+def tc_weights_materialize_file(plan: Plan, fd: int, file_offset: int, dst_ptrs, checksums=None, stream=None) -> None:
+    """tc_weights_materialize with the blob read from file descriptor `fd`, starting at byte
+    `file_offset` (plan created with TC_PLAN_STREAM).  Blocks while the file is read; the device
+    work completes on `stream`."""
+    d, nd = _table(dst_ptrs)
+    cs = _addr(checksums) if checksums is not None else None
+    _check(load_library().tc_weights_materialize_file(plan.handle, int(fd), int(file_offset), d, nd, cs, _stream(stream)))
+
+
+def tc_plan_segments(plan: Plan, group: int = 0):
+    """Chunks of a staged / streamed plan as a list of tc_segment_t."""
+    lib = load_library()
+    n = C.c_size_t()
+    _check(lib.tc_plan_segments(plan.handle, group, None, 0, C.byref(n)))
+    arr = (tc_segment_t * max(1, n.value))()
+    _check(lib.tc_plan_segments(plan.handle, group, C.cast(arr, C.c_void_p), n.value, C.byref(n)))
+    return list(arr[:n.value])
 
 
 def tc_trim() -> None:

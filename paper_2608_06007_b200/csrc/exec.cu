@@ -16,12 +16,17 @@
 // over the host link).  Staged plans instead move the host-side bytes with the copy engines
 // through device staging rings and run the kernel device to device (see execute_staged).
 #include <cuda_runtime.h>
+#include <fcntl.h>
 #include <pthread.h>
+#include <unistd.h>
 
 #include <algorithm>
+#include <atomic>
+#include <cerrno>
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <thread>
 #include <vector>
 
 #include "plan.h"
@@ -487,8 +492,17 @@ struct StageRing {
     cudaStream_t copy = nullptr;
     uint64_t next = 0;
 };
+// Pinned host buffers that file chunks are read into (tc_weights_materialize_file).
+constexpr int kHostBuffers = 3;
+struct HostRing {
+    char *buf[kHostBuffers] = {};
+    cudaEvent_t freed[kHostBuffers] = {};  // the copy engine has finished reading the buffer
+    bool used[kHostBuffers] = {};
+    uint64_t next = 0;
+};
 struct StageArena {
     StageRing ring[2];
+    HostRing host;
     cudaEvent_t entry = nullptr;
     int refs = 0;
 };
@@ -504,6 +518,10 @@ static void stage_free(StageArena &a)
             if (r.freed[b]) cudaEventDestroy(r.freed[b]);
         }
         if (r.copy) cudaStreamDestroy(r.copy);
+    }
+    for (int b = 0; b < kHostBuffers; b++) {
+        if (a.host.buf[b]) cudaFreeHost(a.host.buf[b]);
+        if (a.host.freed[b]) cudaEventDestroy(a.host.freed[b]);
     }
     if (a.entry) cudaEventDestroy(a.entry);
     a = StageArena();
@@ -606,6 +624,128 @@ out:
     pthread_mutex_unlock(&g_stage_mu);
     return rc;
 }
+
+// ---- cold path: file -> pinned host ring -> staging ring -> kernel ---------------------------
+static pthread_mutex_t g_file_mu = PTHREAD_MUTEX_INITIALIZER;  // one file stream per process at a time
+
+// Read [off, off + len) of fd into dst with a few threads (buffered reads of a cached or
+// striped file scale with the number of readers).  The range is handed out in 2 MiB pieces
+// from a shared counter, so the readers finish within one piece of each other.  Returns 0, an
+// errno, or -1 at end of file.
+static int read_range(int fd, int64_t off, int64_t len, char *dst)
+{
+    constexpr int64_t kPiece = 2ll << 20;
+    const int64_t n_pieces = (len + kPiece - 1) / kPiece;
+    const unsigned hw = std::thread::hardware_concurrency();
+    const int64_t max_readers = std::min<int64_t>(8, hw > 1 ? hw - 1 : 1);
+    const int n = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(max_readers, n_pieces / 2)));
+    std::atomic<int> err{0};
+    std::atomic<int64_t> next{0};
+    auto work = [&]() {
+        for (;;) {
+            const int64_t k = next.fetch_add(1, std::memory_order_relaxed);
+            if (k >= n_pieces || err.load(std::memory_order_relaxed)) return;
+            int64_t lo = off + k * kPiece;
+            const int64_t hi = std::min(off + len, lo + kPiece);
+            while (lo < hi) {
+                const ssize_t got = pread(fd, dst + (lo - off), static_cast<size_t>(hi - lo), static_cast<off_t>(lo));
+                if (got < 0) {
+                    if (errno == EINTR) continue;
+                    err = errno ? errno : EIO;
+                    return;
+                }
+                if (got == 0) {
+                    err = -1;
+                    return;
+                }
+                lo += got;
+            }
+        }
+    };
+    std::vector<std::thread> pool;
+    try {
+        for (int i = 1; i < n; i++) pool.emplace_back(work);
+    } catch (...) {
+        // thread creation failed: the readers that exist, and this thread, share the pieces
+    }
+    work();
+    for (std::thread &t : pool) t.join();
+    return err;
+}
+
+static int host_ring_acquire(HostRing &h)
+{
+    if (h.buf[0]) return TC_OK;
+    for (int b = 0; b < kHostBuffers; b++) {
+        cudaError_t e = cudaHostAlloc(reinterpret_cast<void **>(&h.buf[b]), kStageBytes, cudaHostAllocDefault);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h.freed[b], cudaEventDisableTiming);
+        if (e != cudaSuccess) {
+            for (int k = 0; k <= b; k++) {
+                if (h.buf[k]) cudaFreeHost(h.buf[k]);
+                if (h.freed[k]) cudaEventDestroy(h.freed[k]);
+            }
+            h = HostRing();
+            return e == cudaErrorMemoryAllocation ? fail(TC_ERR_OOM, "pinned allocation of the file staging buffers failed") : cuda_fail(e, "creating the file staging buffers");
+        }
+    }
+    return TC_OK;
+}
+
+// Per chunk: wait until the pinned buffer's previous transfer is done, read the chunk's bytes
+// from the file (this is where the call spends its time), then enqueue copy, kernel and events
+// exactly as execute_staged does.  The ring lock is taken per chunk, not per call, so staged
+// KV traffic of other threads keeps flowing while a checkpoint streams in.
+static int execute_streamed(const tc_plan *plan, const Group &g, int fd, int64_t file_off, void *const *dst, uint32_t ptr_align, cudaStream_t s,
+                            unsigned long long *sums)
+{
+    StageArena &a = g_stage[plan->device];
+    StageRing &r = a.ring[1];
+    HostRing &h = a.host;
+    int rc = TC_OK;
+    pthread_mutex_lock(&g_file_mu);
+    pthread_mutex_lock(&g_stage_mu);
+    rc = host_ring_acquire(h);
+    pthread_mutex_unlock(&g_stage_mu);
+    for (size_t i = 0; i < g.segments.size() && rc == TC_OK; i++) {
+        const Segment &seg = g.segments[i];
+        const StageCopy &c = g.copies[seg.copy0];
+        const int hb = static_cast<int>(h.next++ % kHostBuffers);
+        if (h.used[hb]) {
+            cudaError_t e = cudaEventSynchronize(h.freed[hb]);
+            if (e != cudaSuccess) { rc = cuda_fail(e, "cudaEventSynchronize"); break; }
+        }
+        if (i + 1 < g.segments.size()) {  // start read-ahead of the next chunk
+            const StageCopy &nx = g.copies[g.segments[i + 1].copy0];
+            posix_fadvise(fd, static_cast<off_t>(file_off + nx.host_off), static_cast<off_t>(nx.bytes), POSIX_FADV_WILLNEED);
+        }
+        const int err = read_range(fd, file_off + c.host_off, c.bytes, h.buf[hb]);
+        if (err) {
+            rc = err < 0 ? fail(TC_ERR_IO, "the file ends inside blob bytes [%lld, %lld)", (long long)c.host_off, (long long)(c.host_off + c.bytes))
+                         : fail(TC_ERR_IO, "reading blob bytes [%lld, %lld): %s", (long long)c.host_off, (long long)(c.host_off + c.bytes), strerror(err));
+            break;
+        }
+        pthread_mutex_lock(&g_stage_mu);
+        {
+            const int b = static_cast<int>(r.next++ % kStageBuffers);
+            char *shifted = r.buf[b] - seg.shift;
+            const uint32_t pa = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(shifted) | 16));
+            const void *stage_src[1] = {shifted};
+            if (r.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(r.copy, r.freed[b], 0), "cudaStreamWaitEvent");
+            TC_TRY(cudaMemcpyAsync(r.buf[b] + c.stage_off, h.buf[hb], static_cast<size_t>(c.bytes), cudaMemcpyHostToDevice, r.copy), "cudaMemcpyAsync(host to staging)");
+            TC_TRY(cudaEventRecord(h.freed[hb], r.copy), "cudaEventRecord");
+            h.used[hb] = true;
+            TC_TRY(cudaEventRecord(r.ready[b], r.copy), "cudaEventRecord");
+            TC_TRY(cudaStreamWaitEvent(s, r.ready[b], 0), "cudaStreamWaitEvent");
+            if ((rc = launch_any(plan, g, stage_src, dst, pa, s, &seg, sums)) != TC_OK) goto out;
+            TC_TRY(cudaEventRecord(r.freed[b], s), "cudaEventRecord");
+            r.freed_recorded[b] = true;
+        }
+    out:
+        pthread_mutex_unlock(&g_stage_mu);
+    }
+    pthread_mutex_unlock(&g_file_mu);
+    return rc;
+}
 #undef TC_TRY
 
 // A table entry must be memory the device can address: device memory, managed memory, or host
@@ -628,8 +768,13 @@ static int check_addressable(const void *const *table, size_t n, const char *wha
     return TC_OK;
 }
 
+struct FileSource {
+    int fd;
+    int64_t offset;
+};
+
 static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n_src, void *const *dst, size_t n_dst, void *stream,
-                   unsigned long long *sums = nullptr)
+                   unsigned long long *sums = nullptr, const FileSource *file = nullptr)
 {
     clear_error();
     if (!plan) return fail(TC_ERR_INVALID_ARG, "plan is NULL");
@@ -637,7 +782,8 @@ static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n
     const Group &g = plan->group[gi];
     if (n_src != g.n_src || n_dst != g.n_dst)
         return fail(TC_ERR_INVALID_ARG, "tables of %zu source and %zu destination pointers given, the plan needs %zu and %zu", n_src, n_dst, g.n_src, g.n_dst);
-    if ((n_src && !src) || (n_dst && !dst)) return fail(TC_ERR_INVALID_ARG, "pointer table is NULL");
+    if ((n_src && !src && !file) || (n_dst && !dst)) return fail(TC_ERR_INVALID_ARG, "pointer table is NULL");
+    if (file && g.n_tiles && g.segments.empty()) return fail(TC_ERR_KIND, "the plan was not cut into chunks: create it with TC_PLAN_STREAM");
     if (plan->deadline_ns && now_ns() > plan->deadline_ns) return fail(TC_ERR_DEADLINE, "deadline passed before the call; nothing launched");
     int current = -1;
     if (cudaGetDevice(&current) != cudaSuccess || current != plan->device)
@@ -648,7 +794,7 @@ static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n
     }
     if (g.n_tiles == 0) return TC_OK;
     uint32_t ptr_align = 4;
-    for (size_t i = 0; i < n_src; i++) {
+    for (size_t i = 0; i < n_src && !file; i++) {
         if (!src[i]) return fail(TC_ERR_INVALID_ARG, "source table entry %zu is NULL", i);
         ptr_align = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(src[i]) | 16));
     }
@@ -657,9 +803,10 @@ static int execute(const tc_plan *plan, int gi, const void *const *src, size_t n
         ptr_align = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(dst[i]) | 16));
     }
     int rc;
-    if ((rc = check_addressable(src, n_src, "source")) != TC_OK) return rc;
+    if (!file && (rc = check_addressable(src, n_src, "source")) != TC_OK) return rc;
     if ((rc = check_addressable(const_cast<const void *const *>(dst), n_dst, "destination")) != TC_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (file) return execute_streamed(plan, g, file->fd, file->offset, dst, ptr_align, s, sums);
     if (!g.segments.empty()) return execute_staged(plan, gi, g, src, dst, ptr_align, s, sums);
     return launch_any(plan, g, src, dst, ptr_align, s, nullptr, sums);
 }
@@ -761,6 +908,18 @@ extern "C" int tc_weights_materialize_checksum(const tc_plan_t *plan, const void
     return execute(plan, 0, src, 1, dst_ptrs, n_dst, stream, reinterpret_cast<unsigned long long *>(checksums));
 }
 
+extern "C" int tc_weights_materialize_file(const tc_plan_t *plan, int fd, int64_t file_offset, void *const *dst_ptrs, size_t n_dst, uint64_t *checksums,
+                                           void *stream)
+{
+    clear_error();
+    if (plan && (plan->kind != TC_WEIGHTS || !(plan->flags & TC_PLAN_STREAM)))
+        return fail(TC_ERR_KIND, "tc_weights_materialize_file needs a WEIGHTS plan created with TC_PLAN_STREAM");
+    if (plan && checksums && !plan->checksummed) return fail(TC_ERR_KIND, "checksums need a plan created with TC_PLAN_CHECKSUM");
+    if (fd < 0 || file_offset < 0) return fail(TC_ERR_INVALID_ARG, "fd %d / file_offset %lld: both must be >= 0", fd, (long long)file_offset);
+    const FileSource file{fd, file_offset};
+    return execute(plan, 0, nullptr, 1, dst_ptrs, n_dst, stream, reinterpret_cast<unsigned long long *>(checksums), &file);
+}
+
 extern "C" int tc_trim(void)
 {
     clear_error();
@@ -819,6 +978,26 @@ extern "C" int tc_plan_descriptors(const tc_plan_t *plan, int group, tc_descript
         o.src_slot = d.src_slot; o.dst_slot = d.dst_slot - static_cast<uint32_t>(g.n_src);
         o.src_slot_step = d.src_slot_step; o.dst_slot_step = d.dst_slot_step;
         o.run_bytes = d.run; o.n0 = d.n0; o.rows = d.rows; o.n_outer = d.n_outer;
+        o.rows_per_tile = d.rows_per_tile; o.tiles_per_outer = d.tiles_per_outer; o.tile0 = d.tile0; o.reserved = 0;
+    }
+    return TC_OK;
+}
+
+extern "C" int tc_plan_segments(const tc_plan_t *plan, int group, tc_segment_t *out, size_t cap, size_t *n_out)
+{
+    clear_error();
+    if (!plan || group < 0 || group > 1) return fail(TC_ERR_INVALID_ARG, "plan is required and group must be 0 or 1");
+    const Group &g = plan->group[group];
+    if (n_out) *n_out = g.segments.size();
+    if (!out) return TC_OK;
+    for (size_t i = 0; i < g.segments.size() && i < cap; i++) {
+        const Segment &seg = g.segments[i];
+        tc_segment_t &o = out[i];
+        o.host_off = seg.ncopy ? g.copies[seg.copy0].host_off : 0;
+        o.bytes = 0;
+        for (uint32_t c = seg.copy0; c < seg.copy0 + seg.ncopy; c++) o.bytes += g.copies[c].bytes;
+        o.tile0 = seg.nd ? 0 : seg.d0;
+        o.n_tiles = seg.nd ? 0 : seg.no;
     }
     return TC_OK;
 }

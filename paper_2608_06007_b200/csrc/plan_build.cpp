@@ -687,36 +687,71 @@ static int build_weights(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t til
     return TC_OK;
 }
 
-// Staged weights (blob in pinned host memory): a segment is a range of global tile ids whose
-// source bytes are one contiguous range of the blob of at most kStageBytes.  That needs a
-// non-uniform group (tile ids follow the descriptors) in which every tile reads one contiguous
-// piece - whole tensors and dim-0 slabs; strided slices stay on the zero-copy path, which reads
-// only the bytes it needs.
-static void build_segments_blob(Group &g)
+// Byte range of the blob that tile (outer o, part p) of descriptor d reads: [*lo, *hi).
+static void tile_cover(const Desc &d, uint32_t o, uint32_t p, int64_t *lo, int64_t *hi)
 {
-    if (g.descs.empty() || g.tiles_per_desc) return;
-    for (const Desc &d : g.descs) {
-        const bool rows_contiguous = d.rows == 1 || (d.src_s0 == d.run && (d.rows == d.n0 || d.src_s1 == d.n0 * d.run));
-        if (d.n_outer != 1 || !rows_contiguous || d.src_slot != 0) return;
+    const uint32_t row0 = p * d.rows_per_tile, last = std::min(d.rows, row0 + d.rows_per_tile) - 1;
+    const uint32_t i1a = row0 / d.n0, i0a = row0 % d.n0, i1b = last / d.n0, i0b = last % d.n0;
+    auto at = [&](uint32_t i1, uint32_t i0) { return static_cast<int64_t>(i1) * d.src_s1 + static_cast<int64_t>(i0) * d.src_s0; };
+    int64_t first = at(i1a, i0a), end = at(i1b, i0b);
+    if (i1a != i1b) {  // the tile wraps over the inner index: its extremes may sit at the wrap
+        first = std::min(first, at(i1a + 1, 0));
+        end = std::max(end, at(i1b - 1, d.n0 - 1));
     }
+    const int64_t base = d.src_off + static_cast<int64_t>(o) * d.src_outer;
+    *lo = base + first;
+    *hi = base + end + d.run;
+}
+
+// Weights: cut the tile sequence into segments whose blob bytes form one range of at most one
+// staging buffer.  Plain staging (blob in pinned memory) takes only tensors read in contiguous
+// pieces, back to back; anything else leaves the whole group zero copy (the kernel then fetches
+// exactly the bytes it needs over the link).  Streaming (`covering`) takes every descriptor: a
+// strided slice travels as the byte range that covers it, as a loader reading whole rows from
+// storage would, and tiles whose ranges are close (gap no longer than the tile's own range)
+// share a segment.  Segment starts are rounded down to 4 KiB: file reads start on page
+// boundaries and every byte keeps its alignment modulo 16 inside the staging buffer.
+static int build_segments_blob(Group &g, bool covering)
+{
+    if (g.descs.empty()) return TC_OK;
+    if (!covering)
+        for (const Desc &d : g.descs) {
+            const bool rows_contiguous = d.rows == 1 || (d.src_s0 == d.run && (d.rows == d.n0 || d.src_s1 == d.n0 * d.run));
+            if (d.n_outer != 1 || !rows_contiguous || d.src_slot != 0) return TC_OK;
+        }
     int64_t seg_lo = -1, seg_hi = -1;
-    uint32_t seg_t0 = 0, t = 0;
-    auto flush = [&](uint32_t t_end) {
+    uint32_t seg_t0 = 0, seg_t1 = 0;
+    auto flush = [&]() {
         if (seg_lo < 0) return;
-        g.segments.push_back(Segment{seg_t0, 0, 0, t_end - seg_t0, seg_lo, static_cast<uint32_t>(g.copies.size()), 1});
+        g.segments.push_back(Segment{seg_t0, 0, 0, seg_t1 - seg_t0, seg_lo, static_cast<uint32_t>(g.copies.size()), 1});
         g.copies.push_back(StageCopy{0, seg_lo, seg_hi - seg_lo});
         seg_lo = -1;
     };
     for (const Desc &d : g.descs)
-        for (uint32_t p = 0; p < d.tiles_per_outer; p++, t++) {
-            const uint32_t row0 = p * d.rows_per_tile, nrows = std::min(d.rows_per_tile, d.rows - row0);
-            const int64_t lo = d.src_off + static_cast<int64_t>(row0 / d.n0) * d.src_s1 + static_cast<int64_t>(row0 % d.n0) * d.src_s0;
-            const int64_t hi = lo + static_cast<int64_t>(nrows) * d.run;
-            if (seg_lo >= 0 && (lo != seg_hi || hi - seg_lo > kStageBytes)) flush(t);
-            if (seg_lo < 0) { seg_lo = lo; seg_t0 = t; }
-            seg_hi = hi;
-        }
-    flush(t);
+        for (uint32_t o = 0; o < d.n_outer; o++)
+            for (uint32_t p = 0; p < d.tiles_per_outer; p++) {
+                if (p * d.rows_per_tile >= d.rows) continue;  // padding part of a uniform group: empty
+                const uint32_t t = d.tile0 + o * d.tiles_per_outer + p;
+                int64_t lo, hi;
+                tile_cover(d, o, p, &lo, &hi);
+                const int64_t gap_ok = covering ? hi - lo : 0;
+                const bool joins = seg_lo >= 0 && lo >= seg_lo && lo - seg_hi <= gap_ok && (covering || lo == seg_hi);
+                if (!joins || std::max(hi, seg_hi) - seg_lo > kStageBytes) flush();
+                if (seg_lo < 0) {
+                    seg_lo = covering ? lo & ~int64_t(4095) : lo;
+                    seg_hi = hi;
+                    seg_t0 = t;
+                    if (hi - seg_lo > kStageBytes) {
+                        g.segments.clear();
+                        g.copies.clear();
+                        return fail(TC_ERR_TOO_LARGE, "a tile of the plan reads a blob range of %lld bytes, more than one %lld-byte staging buffer: the slice is too sparse to stream", (long long)(hi - seg_lo), (long long)kStageBytes);
+                    }
+                }
+                seg_hi = std::max(seg_hi, hi);
+                seg_t1 = t + 1;
+            }
+    flush();
+    return TC_OK;
 }
 
 // ------------------------------------------------------------------------------ entry
@@ -757,11 +792,13 @@ int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
     if ((spec->flags & TC_PLAN_CHECKSUM) && spec->kind != TC_WEIGHTS)
         return fail(TC_ERR_KIND, "TC_PLAN_CHECKSUM applies to TC_WEIGHTS plans only");
     plan->group[1].host_is_src = true;  // UNPACK / reload read the host side
-    if (spec->flags & TC_PLAN_STAGED) {
+    if ((spec->flags & TC_PLAN_STREAM) && spec->kind != TC_WEIGHTS)
+        return fail(TC_ERR_KIND, "TC_PLAN_STREAM applies to TC_WEIGHTS plans only");
+    if (spec->flags & (TC_PLAN_STAGED | TC_PLAN_STREAM)) {
         if (spec->kind == TC_KV_MIGRATE)
             return fail(TC_ERR_KIND, "TC_PLAN_STAGED does not apply to TC_KV_MIGRATE plans (no host side)");
         if (spec->kind == TC_WEIGHTS) {
-            build_segments_blob(plan->group[0]);
+            if ((rc = build_segments_blob(plan->group[0], (spec->flags & TC_PLAN_STREAM) != 0))) return rc;
         } else if (spec->kind == TC_KV_MIXED) {
             // segments were cut while lowering; a group that could not be staged must drop them
             for (int k = 0; k < 2; k++) {
@@ -797,6 +834,7 @@ extern "C" const char *tc_strerror(int status)
     case TC_ERR_CUDA: return "TC_ERR_CUDA";
     case TC_ERR_DEADLINE: return "TC_ERR_DEADLINE";
     case TC_ERR_TOO_LARGE: return "TC_ERR_TOO_LARGE";
+    case TC_ERR_IO: return "TC_ERR_IO";
     default: return "TC_ERR_UNKNOWN";
     }
 }

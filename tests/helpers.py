@@ -25,6 +25,28 @@ def run_descriptors(descs, src_tables, dst_tables, dst_counts=None):
                     dst_counts[d.dst_slot + o * d.dst_slot_step][b:b + d.run_bytes] += 1
 
 
+def run_tile_range(descs, tile0, n_tiles, src_tables, dst_tables, dst_counts=None, src_shift=0):
+    """Execute only the tiles [tile0, tile0 + n_tiles) of the descriptors, as one launch of a
+    staged / streamed segment does; source addresses are taken relative to `src_shift` (the
+    segment's first host byte sits at the start of the staging buffer)."""
+    for d in descs:
+        for o in range(d.n_outer):
+            s = src_tables[d.src_slot + o * d.src_slot_step]
+            t = dst_tables[d.dst_slot + o * d.dst_slot_step]
+            for p in range(d.tiles_per_outer):
+                if not tile0 <= d.tile0 + o * d.tiles_per_outer + p < tile0 + n_tiles:
+                    continue
+                for k in range(p * d.rows_per_tile, min(d.rows, (p + 1) * d.rows_per_tile)):
+                    i1, i0 = divmod(k, d.n0)
+                    a = d.src_off + o * d.src_outer + i1 * d.src_s1 + i0 * d.src_s0 - src_shift
+                    b = d.dst_off + o * d.dst_outer + i1 * d.dst_s1 + i0 * d.dst_s0
+                    assert 0 <= a and a + d.run_bytes <= s.size, "tile reads outside its segment's staged bytes"
+                    assert 0 <= b and b + d.run_bytes <= t.size, "tile writes outside its destination slot"
+                    t[b:b + d.run_bytes] = s[a:a + d.run_bytes]
+                    if dst_counts is not None:
+                        dst_counts[d.dst_slot + o * d.dst_slot_step][b:b + d.run_bytes] += 1
+
+
 def planes_of(pool, n_planes):
     per = pool.size // n_planes
     return [pool[i * per:(i + 1) * per] for i in range(n_planes)]

@@ -2,6 +2,7 @@
 Everything is copy and indexing, so the bar is exact equality of whole buffers (including
 sentinel-filled destinations and red zones around them)."""
 import itertools
+import os
 import time
 
 import numpy as np
@@ -415,6 +416,61 @@ def test_moe_checkpoint_many_tensors_and_expert_stacking():
                    [want_gu if s_ == 0 else want_dn for s_ in slot], dst_off=doff, dst_stride=dstride)
     assert np.array_equal(gate_up.result(), want_gu) and np.array_equal(down.result(), want_dn)
     assert not (want_gu == 0xA5).all()
+
+
+def test_weights_streamed_from_a_file(tmp_path):
+    """Cold path: the blob sits in a file behind a header; chunks travel file -> pinned ring ->
+    staging ring -> kernel.  Full checkpoint (with fused checksums) and a shard whose strided
+    slices stream as covering ranges."""
+    ck = wl.llama_checkpoint(hidden=512, layers=3, q_heads=8, kv_heads=4, head_dim=64, mlp=2048, vocab=70000)   # 190 MB: several chunks
+    blob = np.zeros(ck.nbytes_total, dtype=np.uint8)
+    wl.fill_np(blob, 9, "normal")
+    header = 4099                                             # the blob need not start on any boundary of the file
+    path = tmp_path / "checkpoint.bin"
+    with open(path, "wb") as f:
+        f.write(bytes(header))
+        f.write(blob.tobytes())
+    nbytes = [ck.nbytes(i) for i in range(ck.N)]
+    fd = os.open(path, os.O_RDONLY)
+    try:
+        for world, rank in ((1, 0), (4, 1), (4, 3)):
+            split = ck.split_dim if world > 1 else np.full(ck.N, -1)
+            sizes = [n // (world if split[i] >= 0 else 1) for i, n in enumerate(nbytes)]
+            want = [np.zeros(n, dtype=np.uint8) for n in sizes]
+            oracle.weights(ck.byte_off, ck.E, ck.shapes, split, rank, world, blob, want, threads=8)
+            want_sums = oracle.weights_checksum(ck.byte_off, ck.E, ck.shapes, split, rank, world, blob)
+            plan = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, split_dim=split, rank=rank, world=world,
+                                                     blob_bytes=ck.nbytes_total, flags=tc.TC_PLAN_STREAM | tc.TC_PLAN_CHECKSUM))
+            st = plan.stats()
+            assert st.path[0] == 3 and st.launches_per_execute >= 3
+            sums = torch.full((ck.N,), -1, dtype=torch.int64, device="cuda")
+            for rep in range(2):                               # the second pass reuses every ring buffer
+                outs = [Guarded(n, fill=0xEE) for n in sizes]
+                tc.tc_weights_materialize_file(plan, fd, header, [o.ptr() for o in outs], checksums=sums if rep else None)
+                for i in range(ck.N):
+                    assert np.array_equal(outs[i].result(), want[i]), (ck.names[i], world, rank, rep)
+            assert np.array_equal(sums.cpu().numpy().view(np.uint64), want_sums)
+            # the same chunked plan also takes the blob from pinned memory
+            h_blob = torch.from_numpy(blob).pin_memory()
+            outs = [Guarded(n, fill=0xEE) for n in sizes]
+            tc.tc_weights_materialize(plan, h_blob, [o.ptr() for o in outs])
+            for i in range(ck.N):
+                assert np.array_equal(outs[i].result(), want[i]), (ck.names[i], world, rank, "pinned")
+        # the file ends early: reported, nothing hangs, the context stays usable
+        with pytest.raises(tc.TensorCastError) as e:
+            tc.tc_weights_materialize_file(plan, fd, header + (100 << 20), [o.ptr() for o in outs])
+        assert e.value.status == tc.TC_ERR_IO and "ends" in str(e.value)
+        torch.cuda.synchronize()
+        plain = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total, flags=tc.TC_PLAN_STAGED))
+        full = [Guarded(n, fill=0xEE) for n in nbytes]
+        with pytest.raises(tc.TensorCastError) as e:
+            tc.tc_weights_materialize_file(plain, fd, header, [o.ptr() for o in full])
+        assert e.value.status == tc.TC_ERR_KIND
+        with pytest.raises(tc.TensorCastError) as e:
+            tc.tc_weights_materialize_file(plan, -1, 0, [o.ptr() for o in outs])
+        assert e.value.status == tc.TC_ERR_INVALID_ARG
+    finally:
+        os.close(fd)
 
 
 def test_weights_transform_into_fused_and_strided_targets():

@@ -13,7 +13,7 @@ import pytest
 import oracle
 import paper_2608_06007_b200 as tc
 import workloads as wl
-from helpers import ck_spec, kv_case, planes_of, run_descriptors, small_checkpoint
+from helpers import run_tile_range, ck_spec, kv_case, planes_of, run_descriptors, small_checkpoint
 
 HOST = tc.TC_PLAN_HOST_ONLY
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -360,6 +360,65 @@ def test_staged_plans_are_cut_into_contiguous_segments():
         assert st.path[g] == 1 and st.launches_per_execute == 1
     with pytest.raises(tc.TensorCastError) as e:
         tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl, T=T, bt_off=off, bt_src=bt, bt_dst=bt, flags=HOST | tc.TC_PLAN_STAGED))
+    assert e.value.status == tc.TC_ERR_KIND
+
+
+@pytest.mark.parametrize("variant", ["tight", "permuted_misaligned"])
+@pytest.mark.parametrize("world", [1, 4])
+@pytest.mark.parametrize("mode", ["stream", "staged"])
+def test_weight_chunks_hold_every_byte_their_tiles_read(variant, world, mode):
+    """Streamed (and staged) weight plans run chunk by chunk against a staging buffer that holds
+    only the chunk's blob range: emulate exactly that, tile range by tile range."""
+    ck = small_checkpoint() if variant == "tight" else small_checkpoint(order_seed=3, pad_to=1, lead_pad=2)
+    blob = np.random.default_rng(4).integers(0, 256, ck.nbytes_total, dtype=np.uint8)
+    flag = tc.TC_PLAN_STREAM if mode == "stream" else tc.TC_PLAN_STAGED
+    for rank in range(world):
+        split = ck.split_dim if world > 1 else np.full(ck.N, -1)
+        sizes = [ck.nbytes(i) // (world if split[i] >= 0 else 1) for i in range(ck.N)]
+        want = [np.zeros(n, dtype=np.uint8) for n in sizes]
+        oracle.weights(ck.byte_off, ck.E, ck.shapes, split, rank, world, blob, want)
+        plan = tc.tc_plan_create(ck_spec(ck, split_dim=split, rank=rank, world=world, flags=HOST | flag, tuning=dict(tile_bytes=512)))
+        segs, descs, st = plan.segments(0), plan.descriptors(0), plan.stats()
+        if mode == "staged" and world > 1:
+            assert not segs and st.path[0] == 1          # strided slices: plain staging declines, zero copy
+            continue
+        assert segs and st.path[0] == 3 and st.launches_per_execute == len(segs)
+        got = [np.full(n, 0xEE, dtype=np.uint8) for n in sizes]
+        cnt = [np.zeros(n, dtype=np.int32) for n in sizes]
+        end = 0
+        for sg in segs:
+            assert sg.n_tiles > 0 and sg.tile0 >= end          # ascending, disjoint tile ranges
+            end = sg.tile0 + sg.n_tiles
+            assert 0 <= sg.host_off and sg.host_off + sg.bytes <= blob.size and sg.bytes <= 64 << 20
+            if mode == "stream":
+                assert sg.host_off % 4096 == 0
+            stage = blob[sg.host_off:sg.host_off + sg.bytes].copy()
+            run_tile_range(descs, sg.tile0, sg.n_tiles, [stage], got, cnt, src_shift=sg.host_off)
+        assert end <= st.n_tiles[0]
+        for i in range(ck.N):
+            assert np.array_equal(got[i], want[i]), ck.names[i]
+            assert (cnt[i] == 1).all()                         # every tile ran in exactly one chunk
+        if world > 1:                                          # slabs of different tensors are far apart: several chunks
+            assert len(segs) > 1
+            assert sum(sg.bytes for sg in segs) < blob.size    # ... that do not read the whole blob
+
+
+def test_stream_flag_limits():
+    # 2 KiB pieces of 8 MiB rows, 16 rows per 32 KiB tile: one tile's covering range is 120 MiB
+    spec = tc.weights_spec([0], [64 * (8 << 20)], [2], [2], [[64, 4 << 20, 1, 1]], split_dim=[1], rank=5, world=4096,
+                           blob_bytes=64 * (8 << 20), flags=HOST | tc.TC_PLAN_STREAM)
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_plan_create(spec)
+    assert e.value.status == tc.TC_ERR_TOO_LARGE and "sparse" in str(e.value)
+    spec = tc.weights_spec([0], [64 * (8 << 20)], [2], [2], [[64, 4 << 20, 1, 1]], split_dim=[1], rank=5, world=4096,
+                           blob_bytes=64 * (8 << 20), flags=HOST | tc.TC_PLAN_STREAM, tuning=dict(tile_bytes=8192))
+    segs = tc.tc_plan_create(spec).segments(0)                 # 4 rows per tile: 24 MiB per tile, two tiles per chunk
+    assert len(segs) == 8 and all(sg.bytes <= 64 << 20 for sg in segs)
+    shape = (1, 4, 2, 8, 2)
+    pl = tc.pool(tc.TC_NHD, 4, 1, plane_stride=4 * 4 * 2 * 8 * 2)
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, bt_src=np.arange(2, dtype=np.int32), T=np.array([8]),
+                                     bt_off=np.array([0, 2]), flags=HOST | tc.TC_PLAN_STREAM))
     assert e.value.status == tc.TC_ERR_KIND
 
 
