@@ -327,13 +327,14 @@ TC_API int tc_weights_materialize_checksum(const tc_plan_t *plan, const void *bl
  * closes it); the blob starts at byte `file_offset` of the file, so a container format's header
  * may precede it.  checksums: NULL, or as for tc_weights_materialize_checksum (the plan then
  * also needs TC_PLAN_CHECKSUM).
- * Per chunk of the plan the call reads the chunk's byte range with a few reader threads into
- * one of three 64 MiB pinned host buffers that the library owns (allocated by the first call
- * on a device, kept until tc_trim or exit), hands it to the copy engine and launches the kernel
- * for the chunk's tiles on `stream`; reading chunk k+1 overlaps transfer and scatter of chunk k.
+ * Reader threads that live for the duration of the call (up to 8) read the plan's chunks, in
+ * order, into three 64 MiB pinned host buffers that the library owns (allocated by the first
+ * call on a device, kept until tc_trim or exit); as each chunk completes the calling thread
+ * hands it to the copy engine and launches the kernel for the chunk's tiles on `stream`.
+ * Reading runs up to two chunks ahead of transfer and scatter.
  * The call RETURNS when the last chunk has been read and enqueued, so unlike the other entry
  * points it blocks for about the time the storage reads take; device work completes on
- * `stream` as usual.  Calls on one device are serialised with one another.
+ * `stream` as usual.  Calls are serialised with one another.
  * Errors: everything tc_weights_materialize checks, before the first read; TC_ERR_KIND for a
  * plan without TC_PLAN_STREAM; TC_ERR_IO when a read fails or the file ends early - chunks
  * before the failing one have been enqueued and will still complete, the destination tensors

@@ -23,6 +23,8 @@
 #include <algorithm>
 #include <atomic>
 #include <cerrno>
+#include <condition_variable>
+#include <mutex>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -628,50 +630,107 @@ out:
 // ---- cold path: file -> pinned host ring -> staging ring -> kernel ---------------------------
 static pthread_mutex_t g_file_mu = PTHREAD_MUTEX_INITIALIZER;  // one file stream per process at a time
 
-// Read [off, off + len) of fd into dst with a few threads (buffered reads of a cached or
-// striped file scale with the number of readers).  The range is handed out in 2 MiB pieces
-// from a shared counter, so the readers finish within one piece of each other.  Returns 0, an
-// errno, or -1 at end of file.
-static int read_range(int fd, int64_t off, int64_t len, char *dst)
-{
-    constexpr int64_t kPiece = 2ll << 20;
-    const int64_t n_pieces = (len + kPiece - 1) / kPiece;
-    const unsigned hw = std::thread::hardware_concurrency();
-    const int64_t max_readers = std::min<int64_t>(8, hw > 1 ? hw - 1 : 1);
-    const int n = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(max_readers, n_pieces / 2)));
-    std::atomic<int> err{0};
-    std::atomic<int64_t> next{0};
-    auto work = [&]() {
-        for (;;) {
-            const int64_t k = next.fetch_add(1, std::memory_order_relaxed);
-            if (k >= n_pieces || err.load(std::memory_order_relaxed)) return;
-            int64_t lo = off + k * kPiece;
-            const int64_t hi = std::min(off + len, lo + kPiece);
-            while (lo < hi) {
-                const ssize_t got = pread(fd, dst + (lo - off), static_cast<size_t>(hi - lo), static_cast<off_t>(lo));
-                if (got < 0) {
-                    if (errno == EINTR) continue;
-                    err = errno ? errno : EIO;
-                    return;
-                }
-                if (got == 0) {
-                    err = -1;
-                    return;
-                }
+// Reader threads of one tc_weights_materialize_file call.  Every chunk of the plan is a job of
+// 1 MiB pieces; the caller opens jobs in order as pinned buffers become free, the readers take
+// pieces of the oldest open job from a shared counter and move on to the next open job without
+// waiting for one another, so the file is read continuously across chunk boundaries (buffered
+// reads of a cached or striped file scale with the number of readers).
+struct ReadJob {
+    int64_t off = 0, len = 0, n_pieces = 0;
+    char *dst = nullptr;
+    std::atomic<int64_t> next{0}, done{0};
+};
+struct ReaderPool {
+    static constexpr int64_t kPiece = 1ll << 20;
+    int fd;
+    std::vector<ReadJob> jobs;
+    size_t opened = 0;  // jobs [0, opened) may be read (guarded by mu)
+    bool quit = false;
+    std::atomic<int> err{0};  // 0, an errno, or -1 at end of file
+    std::mutex mu;
+    std::condition_variable cv;
+    std::vector<std::thread> threads;
+
+    ReaderPool(int fd_, size_t n_jobs) : fd(fd_), jobs(n_jobs) {}
+
+    void start()
+    {
+        const unsigned hw = std::thread::hardware_concurrency();
+        const int n = static_cast<int>(std::min<unsigned>(8, hw > 2 ? hw - 2 : 1));
+        try {
+            for (int i = 0; i < n; i++) threads.emplace_back([this] { run(); });
+        } catch (...) {
+            // fewer readers than wished for; with none at all the caller reads (see wait)
+        }
+    }
+    void open(size_t j, int64_t off, int64_t len, char *dst)
+    {
+        ReadJob &job = jobs[j];
+        job.off = off;
+        job.len = len;
+        job.dst = dst;
+        job.n_pieces = (len + kPiece - 1) / kPiece;
+        std::lock_guard<std::mutex> lk(mu);
+        opened = j + 1;
+        cv.notify_all();
+    }
+    bool read_piece(ReadJob &job)
+    {
+        const int64_t k = job.next.fetch_add(1, std::memory_order_relaxed);
+        if (k >= job.n_pieces) return false;
+        int64_t lo = job.off + k * kPiece;
+        const int64_t hi = std::min(job.off + job.len, lo + kPiece);
+        while (lo < hi && !err.load(std::memory_order_relaxed)) {
+            const ssize_t got = pread(fd, job.dst + (lo - job.off), static_cast<size_t>(hi - lo), static_cast<off_t>(lo));
+            if (got < 0) {
+                if (errno == EINTR) continue;
+                err = errno ? errno : EIO;
+            } else if (got == 0) {
+                err = -1;
+            } else {
                 lo += got;
             }
         }
-    };
-    std::vector<std::thread> pool;
-    try {
-        for (int i = 1; i < n; i++) pool.emplace_back(work);
-    } catch (...) {
-        // thread creation failed: the readers that exist, and this thread, share the pieces
+        if (job.done.fetch_add(1, std::memory_order_acq_rel) + 1 == job.n_pieces) {
+            std::lock_guard<std::mutex> lk(mu);
+            cv.notify_all();
+        }
+        return true;
     }
-    work();
-    for (std::thread &t : pool) t.join();
-    return err;
-}
+    void run()
+    {
+        size_t j = 0;
+        while (j < jobs.size()) {
+            {
+                std::unique_lock<std::mutex> lk(mu);
+                cv.wait(lk, [&] { return quit || opened > j; });
+                if (quit) return;
+            }
+            while (read_piece(jobs[j])) {}
+            j++;
+        }
+    }
+    // Block until job j has been read completely (or a read failed).  Returns err.
+    int wait(size_t j)
+    {
+        ReadJob &job = jobs[j];
+        if (threads.empty())
+            while (read_piece(job)) {}
+        std::unique_lock<std::mutex> lk(mu);
+        cv.wait(lk, [&] { return job.done.load(std::memory_order_acquire) >= job.n_pieces; });
+        return err.load();
+    }
+    ~ReaderPool()
+    {
+        {
+            std::lock_guard<std::mutex> lk(mu);
+            quit = true;
+            err = err.load() ? err.load() : ECANCELED;  // readers in the middle of a job stop at the next piece
+            cv.notify_all();
+        }
+        for (std::thread &t : threads) t.join();
+    }
+};
 
 static int host_ring_acquire(HostRing &h)
 {
@@ -691,58 +750,77 @@ static int host_ring_acquire(HostRing &h)
     return TC_OK;
 }
 
-// Per chunk: wait until the pinned buffer's previous transfer is done, read the chunk's bytes
-// from the file (this is where the call spends its time), then enqueue copy, kernel and events
-// exactly as execute_staged does.  The ring lock is taken per chunk, not per call, so staged
-// KV traffic of other threads keeps flowing while a checkpoint streams in.
+// The caller's thread is the conductor: it opens chunk i + 2 for the readers as soon as the copy
+// engine has drained that chunk's pinned buffer, waits until chunk i has been read, and enqueues
+// copy, kernel and events for it exactly as execute_staged does.  Reading (where the call
+// spends its time) thus runs two chunks ahead of the transfers.  The ring lock is taken per
+// chunk, not per call, so staged KV traffic of other threads keeps flowing while a checkpoint
+// streams in.
 static int execute_streamed(const tc_plan *plan, const Group &g, int fd, int64_t file_off, void *const *dst, uint32_t ptr_align, cudaStream_t s,
                             unsigned long long *sums)
 {
     StageArena &a = g_stage[plan->device];
     StageRing &r = a.ring[1];
     HostRing &h = a.host;
+    const size_t n = g.segments.size();
     int rc = TC_OK;
     pthread_mutex_lock(&g_file_mu);
     pthread_mutex_lock(&g_stage_mu);
     rc = host_ring_acquire(h);
     pthread_mutex_unlock(&g_stage_mu);
-    for (size_t i = 0; i < g.segments.size() && rc == TC_OK; i++) {
-        const Segment &seg = g.segments[i];
-        const StageCopy &c = g.copies[seg.copy0];
-        const int hb = static_cast<int>(h.next++ % kHostBuffers);
-        if (h.used[hb]) {
-            cudaError_t e = cudaEventSynchronize(h.freed[hb]);
-            if (e != cudaSuccess) { rc = cuda_fail(e, "cudaEventSynchronize"); break; }
-        }
-        if (i + 1 < g.segments.size()) {  // start read-ahead of the next chunk
-            const StageCopy &nx = g.copies[g.segments[i + 1].copy0];
-            posix_fadvise(fd, static_cast<off_t>(file_off + nx.host_off), static_cast<off_t>(nx.bytes), POSIX_FADV_WILLNEED);
-        }
-        const int err = read_range(fd, file_off + c.host_off, c.bytes, h.buf[hb]);
-        if (err) {
-            rc = err < 0 ? fail(TC_ERR_IO, "the file ends inside blob bytes [%lld, %lld)", (long long)c.host_off, (long long)(c.host_off + c.bytes))
-                         : fail(TC_ERR_IO, "reading blob bytes [%lld, %lld): %s", (long long)c.host_off, (long long)(c.host_off + c.bytes), strerror(err));
-            break;
-        }
-        pthread_mutex_lock(&g_stage_mu);
-        {
-            const int b = static_cast<int>(r.next++ % kStageBuffers);
-            char *shifted = r.buf[b] - seg.shift;
-            const uint32_t pa = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(shifted) | 16));
-            const void *stage_src[1] = {shifted};
-            if (r.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(r.copy, r.freed[b], 0), "cudaStreamWaitEvent");
-            TC_TRY(cudaMemcpyAsync(r.buf[b] + c.stage_off, h.buf[hb], static_cast<size_t>(c.bytes), cudaMemcpyHostToDevice, r.copy), "cudaMemcpyAsync(host to staging)");
-            TC_TRY(cudaEventRecord(h.freed[hb], r.copy), "cudaEventRecord");
-            h.used[hb] = true;
-            TC_TRY(cudaEventRecord(r.ready[b], r.copy), "cudaEventRecord");
-            TC_TRY(cudaStreamWaitEvent(s, r.ready[b], 0), "cudaStreamWaitEvent");
-            if ((rc = launch_any(plan, g, stage_src, dst, pa, s, &seg, sums)) != TC_OK) goto out;
-            TC_TRY(cudaEventRecord(r.freed[b], s), "cudaEventRecord");
-            r.freed_recorded[b] = true;
-        }
-    out:
-        pthread_mutex_unlock(&g_stage_mu);
+    if (rc != TC_OK) {
+        pthread_mutex_unlock(&g_file_mu);
+        return rc;
     }
+    {
+        ReaderPool pool(fd, n);
+        const uint64_t first = h.next;
+        h.next += n;
+        auto host_buf = [&](size_t i) { return static_cast<int>((first + i) % kHostBuffers); };
+        auto open = [&](size_t i) -> int {
+            const int hb = host_buf(i);
+            if (h.used[hb]) {
+                cudaError_t e = cudaEventSynchronize(h.freed[hb]);
+                if (e != cudaSuccess) return cuda_fail(e, "cudaEventSynchronize");
+            }
+            const StageCopy &c = g.copies[g.segments[i].copy0];
+            posix_fadvise(fd, static_cast<off_t>(file_off + c.host_off), static_cast<off_t>(c.bytes), POSIX_FADV_WILLNEED);
+            pool.open(i, file_off + c.host_off, c.bytes, h.buf[hb]);
+            return TC_OK;
+        };
+        pool.start();
+        for (size_t i = 0; i < n && i < kHostBuffers - 1 && rc == TC_OK; i++) rc = open(i);
+        for (size_t i = 0; i < n && rc == TC_OK; i++) {
+            if (i + kHostBuffers - 1 < n && (rc = open(i + kHostBuffers - 1)) != TC_OK) break;
+            const Segment &seg = g.segments[i];
+            const StageCopy &c = g.copies[seg.copy0];
+            const int err = pool.wait(i);
+            if (err) {
+                rc = err < 0 ? fail(TC_ERR_IO, "the file ends inside blob bytes [%lld, %lld)", (long long)c.host_off, (long long)(c.host_off + c.bytes))
+                             : fail(TC_ERR_IO, "reading blob bytes [%lld, %lld): %s", (long long)c.host_off, (long long)(c.host_off + c.bytes), strerror(err));
+                break;
+            }
+            const int hb = host_buf(i);
+            pthread_mutex_lock(&g_stage_mu);
+            {
+                const int b = static_cast<int>(r.next++ % kStageBuffers);
+                char *shifted = r.buf[b] - seg.shift;
+                const uint32_t pa = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(shifted) | 16));
+                const void *stage_src[1] = {shifted};
+                if (r.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(r.copy, r.freed[b], 0), "cudaStreamWaitEvent");
+                TC_TRY(cudaMemcpyAsync(r.buf[b] + c.stage_off, h.buf[hb], static_cast<size_t>(c.bytes), cudaMemcpyHostToDevice, r.copy), "cudaMemcpyAsync(host to staging)");
+                TC_TRY(cudaEventRecord(h.freed[hb], r.copy), "cudaEventRecord");
+                h.used[hb] = true;
+                TC_TRY(cudaEventRecord(r.ready[b], r.copy), "cudaEventRecord");
+                TC_TRY(cudaStreamWaitEvent(s, r.ready[b], 0), "cudaStreamWaitEvent");
+                if ((rc = launch_any(plan, g, stage_src, dst, pa, s, &seg, sums)) != TC_OK) goto out;
+                TC_TRY(cudaEventRecord(r.freed[b], s), "cudaEventRecord");
+                r.freed_recorded[b] = true;
+            }
+        out:
+            pthread_mutex_unlock(&g_stage_mu);
+        }
+    }  // the pool's destructor stops and joins the readers
     pthread_mutex_unlock(&g_file_mu);
     return rc;
 }
