@@ -120,7 +120,7 @@ enum {
     TC_PLAN_STAGED = 2u,    /* The host side of the plan is PINNED HOST memory and should travel
                                through the copy engines instead of being loaded / stored by the
                                kernel itself (zero copy, the default):
-                                 - TC_KV_PACK / TC_KV_UNPACK: the packed buffer (request-major);
+                                 - TC_KV_PACK / TC_KV_UNPACK: the packed buffer;
                                  - TC_KV_MIXED: dst_pool, a page-first host pool in one
                                    allocation (plane_stride = one block of one plane), moved in
                                    full blocks;
@@ -141,8 +141,9 @@ enum {
                                rings (3 x 64 MiB per direction and device) are allocated when
                                the first staged plan is created and kept until the process
                                exits.  Groups that cannot be staged (strided slices of a blob,
-                               partial blocks of a paged pool, layer-major packed buffers) stay
-                               zero copy.  Staged executions are serialised with one another
+                               partial blocks of a paged pool) stay zero copy.  Layer-major
+                               packed buffers are cut into runs of whole planes, in layer
+                               order.  Staged executions are serialised with one another
                                by the library while they are enqueued. */
     TC_PLAN_SAME_POOL = 8u, /* TC_KV_MIGRATE inside ONE pool (compaction / defragmentation): the
                                caller will pass the same table as source and destination.
@@ -424,14 +425,17 @@ typedef struct {
 TC_API int tc_plan_descriptors(const tc_plan_t *plan, int group, tc_descriptor_t *out, size_t cap,
                         size_t *n_out);
 
-/* One chunk of a staged or streamed TC_WEIGHTS plan, or one segment of a staged request-major
- * packed buffer: the tiles [tile0, tile0 + n_tiles) run against host bytes [host_off,
- * host_off + bytes) of the blob / packed buffer, which the kernel sees at the start of a
- * staging buffer.  (n_tiles = 0: the segment is a window of descriptors x planes, not a tile
- * range, as staged KV plans use; only host_off and bytes are meaningful then.) */
+/* One segment (chunk) of a staged or streamed plan: the host bytes [host_off, host_off + bytes)
+ * of the blob / packed buffer (a paged host pool: the total of its page runs, host_off = the
+ * first run) travel through one staging buffer, and one launch runs
+ *   - the tiles [tile0, tile0 + n_tiles) (TC_WEIGHTS plans; n_descs = 0), or
+ *   - the window of descriptors [desc0, desc0 + n_descs) x outer indices (planes)
+ *     [outer0, outer0 + n_outer) (KV plans; n_tiles = 0)
+ * against it, seeing byte host_off of the host side at the start of the staging buffer. */
 typedef struct {
     int64_t host_off, bytes;
     uint32_t tile0, n_tiles;
+    uint32_t desc0, n_descs, outer0, n_outer;
 } tc_segment_t;
 
 /* Copy up to `cap` segments of `group` into out (host array); *n_out receives the count

@@ -92,7 +92,8 @@ class tc_descriptor_t(C.Structure):
 
 
 class tc_segment_t(C.Structure):
-    _fields_ = [("host_off", C.c_int64), ("bytes", C.c_int64), ("tile0", C.c_uint32), ("n_tiles", C.c_uint32)]
+    _fields_ = [("host_off", C.c_int64), ("bytes", C.c_int64), ("tile0", C.c_uint32), ("n_tiles", C.c_uint32),
+                ("desc0", C.c_uint32), ("n_descs", C.c_uint32), ("outer0", C.c_uint32), ("n_outer", C.c_uint32)]
 
 
 EXPORTS = ("tc_plan_create", "tc_kv_pack", "tc_kv_unpack", "tc_weights_materialize",

@@ -1076,6 +1076,10 @@ extern "C" int tc_plan_segments(const tc_plan_t *plan, int group, tc_segment_t *
         for (uint32_t c = seg.copy0; c < seg.copy0 + seg.ncopy; c++) o.bytes += g.copies[c].bytes;
         o.tile0 = seg.nd ? 0 : seg.d0;
         o.n_tiles = seg.nd ? 0 : seg.no;
+        o.desc0 = seg.nd ? seg.d0 : 0;
+        o.n_descs = seg.nd;
+        o.outer0 = seg.nd ? seg.o0 : 0;
+        o.n_outer = seg.nd ? seg.no : 0;
     }
     return TC_OK;
 }

@@ -413,7 +413,7 @@ static void lower_kv_group(Group &g, const tc_kv_spec_t &kv, const tc_kv_group_t
             b.dims = {Dim{hs, ssh, dsh}, Dim{nvalid, ssn, dsn}};
             lower_box(g, b, tile_bytes);
         }
-        if (has_packed && !layer_major)  // request-major regions are contiguous: staged plans cut segments from them
+        if (has_packed)  // staged plans cut segments from the requests' contiguous regions
             g.requests.push_back(RequestSpan{first_desc, static_cast<uint32_t>(g.descs.size()), off_r, plane_bytes});
         off_r += layer_major ? plane_bytes : planes * plane_bytes;
     }
@@ -422,11 +422,51 @@ static void lower_kv_group(Group &g, const tc_kv_spec_t &kv, const tc_kv_group_t
 // Cut a staged group into segments: windows of descriptors x planes whose packed-side bytes
 // are one contiguous range of at most kStageBytes.  Runs of small consecutive requests share
 // a segment; a request larger than a staging buffer is cut at plane boundaries.
-static int build_segments(Group &g, int64_t planes)
+//
+// Layer-major packed buffers: plane (l,c) of ALL requests is contiguous (stride P = one plane of
+// every request), and q.off is the request's offset inside a plane.  A segment is a run of whole
+// planes when P fits a staging buffer several times, else a run of requests inside one plane;
+// segments come out in buffer order, plane 0 first, so a consumer of the host buffer (or of the
+// pool, on reload) sees the layers complete one after the other.
+static int build_segments(Group &g, int64_t planes, bool layer_major)
 {
     if (!g.tiles_per_desc) return TC_OK;  // non-uniform group: stays on the zero-copy path
     for (const Desc &d : g.descs)
         if (d.n_outer != planes) return TC_OK;
+    if (layer_major) {
+        int64_t P = 0;
+        for (const RequestSpan &q : g.requests) {
+            if (q.plane_bytes > kStageBytes)
+                return fail(TC_ERR_TOO_LARGE, "a staged plan needs every (layer, K|V) plane of a request to fit a %lld-byte staging buffer; one has %lld bytes", (long long)kStageBytes, (long long)q.plane_bytes);
+            P += q.plane_bytes;
+        }
+        if (P == 0) return TC_OK;
+        const uint32_t nd_all = static_cast<uint32_t>(g.descs.size());
+        if (P <= kStageBytes) {
+            const int64_t per = kStageBytes / P;
+            for (int64_t o0 = 0; o0 < planes; o0 += per) {
+                const int64_t no = std::min(per, planes - o0);
+                g.segments.push_back(Segment{0, nd_all, static_cast<uint32_t>(o0), static_cast<uint32_t>(no), o0 * P, static_cast<uint32_t>(g.copies.size()), 1});
+                g.copies.push_back(StageCopy{0, o0 * P, no * P});
+            }
+            return TC_OK;
+        }
+        for (int64_t o = 0; o < planes; o++) {
+            size_t i = 0;
+            while (i < g.requests.size()) {
+                int64_t sum = 0;
+                size_t j = i;
+                while (j < g.requests.size() && sum + g.requests[j].plane_bytes <= kStageBytes) sum += g.requests[j++].plane_bytes;
+                const RequestSpan &q = g.requests[i];
+                if (sum > 0) {
+                    g.segments.push_back(Segment{q.d0, g.requests[j - 1].d1 - q.d0, static_cast<uint32_t>(o), 1, o * P + q.off, static_cast<uint32_t>(g.copies.size()), 1});
+                    g.copies.push_back(StageCopy{0, o * P + q.off, sum});
+                }
+                i = j;
+            }
+        }
+        return TC_OK;
+    }
     size_t i = 0;
     while (i < g.requests.size()) {
         const RequestSpan &q = g.requests[i];
@@ -811,7 +851,7 @@ int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
             }
         } else {
             Group &g = plan->group[spec->kind == TC_KV_PACK ? 0 : 1];
-            if ((rc = build_segments(g, spec->kv.L * 2))) return rc;
+            if ((rc = build_segments(g, spec->kv.L * 2, spec->kv.packed_order == TC_LAYER_MAJOR))) return rc;
         }
     }
     return TC_OK;

@@ -25,6 +25,25 @@ def run_descriptors(descs, src_tables, dst_tables, dst_counts=None):
                     dst_counts[d.dst_slot + o * d.dst_slot_step][b:b + d.run_bytes] += 1
 
 
+def run_window(descs, seg, src_tables, dst_tables, dst_counts=None, src_shift=0, dst_shift=0):
+    """Execute the window of descriptors x planes of one staged KV segment; the staged side's
+    addresses are taken relative to the segment's first host byte (src_shift or dst_shift)."""
+    for d in descs[seg.desc0:seg.desc0 + seg.n_descs]:
+        for o in range(seg.outer0, seg.outer0 + seg.n_outer):
+            assert o < d.n_outer
+            s = src_tables[d.src_slot + o * d.src_slot_step]
+            t = dst_tables[d.dst_slot + o * d.dst_slot_step]
+            for k in range(d.rows):
+                i1, i0 = divmod(k, d.n0)
+                a = d.src_off + o * d.src_outer + i1 * d.src_s1 + i0 * d.src_s0 - src_shift
+                b = d.dst_off + o * d.dst_outer + i1 * d.dst_s1 + i0 * d.dst_s0 - dst_shift
+                assert 0 <= a and a + d.run_bytes <= s.size, "window reads outside its source"
+                assert 0 <= b and b + d.run_bytes <= t.size, "window writes outside its destination"
+                t[b:b + d.run_bytes] = s[a:a + d.run_bytes]
+                if dst_counts is not None:
+                    dst_counts[d.dst_slot + o * d.dst_slot_step][b:b + d.run_bytes] += 1
+
+
 def run_tile_range(descs, tile0, n_tiles, src_tables, dst_tables, dst_counts=None, src_shift=0):
     """Execute only the tiles [tile0, tile0 + n_tiles) of the descriptors, as one launch of a
     staged / streamed segment does; source addresses are taken relative to `src_shift` (the

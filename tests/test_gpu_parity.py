@@ -276,7 +276,8 @@ def test_pack_to_pinned_host_hnd_and_reload():
 
 
 @pytest.mark.parametrize("packed_l", LAYOUTS)
-def test_staged_offload_and_reload_through_the_copy_engines(packed_l):
+@pytest.mark.parametrize("order", [tc.TC_REQUEST_MAJOR, tc.TC_LAYER_MAJOR])
+def test_staged_offload_and_reload_through_the_copy_engines(packed_l, order):
     """TC_PLAN_STAGED: packed buffer in pinned host memory, moved by the copy engines through
     the device staging ring; one request is larger than a staging buffer (cut at planes), the
     small ones share a segment.  Run twice to reuse ring buffers across calls."""
@@ -284,15 +285,15 @@ def test_staged_offload_and_reload_through_the_copy_engines(packed_l):
     shape, NB, stride, pool, T, off, bt = kv_case(rng, L=4, NB=400, B=16, H=8, D=128, E=2, T=(5000, 37, 0, 100, 700))
     L = shape[0]
     want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
-    oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, L * 2), T, off, bt, packed_l, want, threads=8)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, L * 2), T, off, bt, packed_l, want, order=order, threads=8)
     pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride)
     d_pool = dev(pool)
-    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_src=bt, flags=tc.TC_PLAN_STAGED))
-    assert plan.stats().path[0] == 3 and plan.stats().launches_per_execute == 3
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=packed_l, packed_order=order, T=T, bt_off=off, bt_src=bt, flags=tc.TC_PLAN_STAGED))
+    assert plan.stats().path[0] == 3 and plan.stats().launches_per_execute == (3 if order == tc.TC_REQUEST_MAJOR else 2)
     bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
     want_pool = np.full_like(pool, 0xA5)
-    oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(want_pool, L * 2), T, off, bt2, packed_l, want, threads=8)
-    plan2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_dst=bt2, flags=tc.TC_PLAN_STAGED))
+    oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(want_pool, L * 2), T, off, bt2, packed_l, want, order=order, threads=8)
+    plan2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=packed_l, packed_order=order, T=T, bt_off=off, bt_dst=bt2, flags=tc.TC_PLAN_STAGED))
     stream = torch.cuda.Stream()
     for _ in range(2):
         host = torch.full((want.size + 4096,), 0x77, dtype=torch.uint8).pin_memory()

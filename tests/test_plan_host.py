@@ -13,7 +13,7 @@ import pytest
 import oracle
 import paper_2608_06007_b200 as tc
 import workloads as wl
-from helpers import run_tile_range, ck_spec, kv_case, planes_of, run_descriptors, small_checkpoint
+from helpers import run_tile_range, run_window, ck_spec, kv_case, planes_of, run_descriptors, small_checkpoint
 
 HOST = tc.TC_PLAN_HOST_ONLY
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -361,6 +361,56 @@ def test_staged_plans_are_cut_into_contiguous_segments():
     with pytest.raises(tc.TensorCastError) as e:
         tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl, T=T, bt_off=off, bt_src=bt, bt_dst=bt, flags=HOST | tc.TC_PLAN_STAGED))
     assert e.value.status == tc.TC_ERR_KIND
+
+
+@pytest.mark.parametrize("order,L,T,n_seg", [
+    (tc.TC_REQUEST_MAJOR, 4, (5000, 37, 0, 100, 700), 3),      # 80 MB request cut at planes (6 + 2), small ones share one
+    (tc.TC_LAYER_MAJOR, 4, (5000, 37, 0, 100, 700), 2),        # 12 MB per plane of all requests: 5 + 3 planes
+    (tc.TC_LAYER_MAJOR, 1, (0, 20000, 15000, 0, 3000, 0), 4),  # 78 MB per plane: cut inside planes at requests
+])
+def test_staged_kv_segments_hold_every_byte_their_windows_touch(order, L, T, n_seg):
+    """Emulate the staged path segment by segment against a staging array that holds only the
+    segment's host bytes, for offload (pack) and reload (unpack)."""
+    rng = np.random.default_rng(31)
+    B, H, D, E = 16, 8, 128, 2
+    shape = (L, B, H, D, E)
+    T = np.array(T, dtype=np.int64)
+    off = np.concatenate([[0], np.cumsum((T + B - 1) // B)]).astype(np.int64)
+    NB = int(off[-1]) + 3
+    chunk = B * H * D * E
+    pool = rng.integers(0, 256, L * 2 * NB * chunk, dtype=np.uint8)
+    bt = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, oracle.NHD, chunk, planes_of(pool, L * 2), T, off, bt, oracle.NHD, want, order=order, threads=8)
+    pl = tc.pool(tc.TC_NHD, NB, L * 2, block_stride=chunk)
+    kw = dict(packed_layout=tc.TC_NHD, packed_order=order, T=T, bt_off=off, flags=HOST | tc.TC_PLAN_STAGED)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, bt_src=bt, **kw))
+    segs = plan.segments(0)
+    assert len(segs) == n_seg == plan.stats().launches_per_execute and plan.stats().path[0] == 3
+    host = np.full(want.size, 0x77, dtype=np.uint8)
+    cnt = np.zeros(want.size, dtype=np.int32)
+    end = 0
+    for sg in segs:
+        assert sg.n_descs > 0 and sg.n_outer > 0 and sg.n_tiles == 0 and 0 < sg.bytes <= 64 << 20
+        assert sg.host_off == end                             # segments follow the buffer order without gaps
+        end = sg.host_off + sg.bytes
+        stage, c = np.full(sg.bytes, 0x55, dtype=np.uint8), np.zeros(sg.bytes, dtype=np.int32)
+        run_window(plan.descriptors(0), sg, planes_of(pool, L * 2), [stage], [c], dst_shift=sg.host_off)
+        assert (c == 1).all()                                 # the copy back to the host carries no stale byte
+        host[sg.host_off:end] = stage
+        cnt[sg.host_off:end] += 1
+    assert end == want.size and (cnt == 1).all() and np.array_equal(host, want)
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, oracle.NHD, chunk, planes_of(want_pool, L * 2), T, off, bt2, oracle.NHD, want, order=order, threads=8)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, bt_dst=bt2, **kw))
+    segs = plan.segments(1)
+    assert len(segs) == n_seg
+    got_pool = np.full_like(pool, 0xA5)
+    for sg in segs:
+        stage = want[sg.host_off:sg.host_off + sg.bytes].copy()
+        run_window(plan.descriptors(1), sg, [stage], planes_of(got_pool, L * 2), src_shift=sg.host_off)
+    assert np.array_equal(got_pool, want_pool)
 
 
 @pytest.mark.parametrize("variant", ["tight", "permuted_misaligned"])
