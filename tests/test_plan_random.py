@@ -8,7 +8,7 @@ from hypothesis import HealthCheck, given, settings, strategies as st
 
 import oracle
 import paper_2608_06007_b200 as tc
-from helpers import planes_of, run_descriptors
+from helpers import planes_of, run_descriptors, run_tile_range
 
 HOST = tc.TC_PLAN_HOST_ONLY
 COMMON = dict(deadline=None, suppress_health_check=[HealthCheck.too_slow, HealthCheck.data_too_large])
@@ -128,5 +128,16 @@ def test_random_weight_specs(case):
     got = [np.full(n, 0xEE, dtype=np.uint8) for n in sizes]
     cnt = [np.zeros(n, dtype=np.int32) for n in sizes]
     run_descriptors(plan.descriptors(0), [blob], got, cnt)
+    for g, w, c in zip(got, want, cnt):
+        assert np.array_equal(g, w) and (c == 1).all()
+    # the same spec cut into chunks for streaming: every chunk's staging bytes cover what its tiles read
+    plan = tc.tc_plan_create(tc.weights_spec(offs, nbytes, E, ndim, shapes, split_dim=split, rank=rank, world=world, blob_bytes=blob.size,
+                                             flags=HOST | tc.TC_PLAN_STREAM, tuning=dict(tile_bytes=tile) if tile else None))
+    got = [np.full(n, 0xEE, dtype=np.uint8) for n in sizes]
+    cnt = [np.zeros(n, dtype=np.int32) for n in sizes]
+    descs = plan.descriptors(0)
+    for sg in plan.segments(0):
+        assert sg.host_off % 4096 == 0 and sg.host_off + sg.bytes <= blob.size
+        run_tile_range(descs, sg.tile0, sg.n_tiles, [blob[sg.host_off:sg.host_off + sg.bytes].copy()], got, cnt, src_shift=sg.host_off)
     for g, w, c in zip(got, want, cnt):
         assert np.array_equal(g, w) and (c == 1).all()
