@@ -655,6 +655,67 @@ def test_concurrent_threads_create_execute_destroy():
     assert not errors, errors[:3]
 
 
+def test_file_stream_and_staged_reload_share_the_staging_ring(tmp_path):
+    """A checkpoint streams in from a file while another thread reloads KV through the same
+    host-to-device staging ring: the ring is locked per chunk, so the two interleave."""
+    import threading
+    ck = wl.llama_checkpoint(hidden=512, layers=3, q_heads=8, kv_heads=4, head_dim=64, mlp=2048, vocab=70000)
+    blob = np.zeros(ck.nbytes_total, dtype=np.uint8)
+    wl.fill_np(blob, 11, "normal")
+    path = tmp_path / "blob.bin"
+    blob.tofile(path)
+    nbytes = [ck.nbytes(i) for i in range(ck.N)]
+    wplan = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total, flags=tc.TC_PLAN_STREAM))
+    rng = np.random.default_rng(29)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=4, NB=400, B=16, H=8, D=128, E=2, T=(5000, 37, 0, 100, 700))
+    L = shape[0]
+    packed = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    wl.fill_np(packed[:packed.size & ~1], 12)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(want_pool, L * 2), T, off, bt, oracle.HND, packed, threads=8)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride)
+    uplan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_dst=bt, flags=tc.TC_PLAN_STAGED))
+    h_packed = torch.from_numpy(packed).pin_memory()
+    errors = []
+
+    def loader():
+        try:
+            fd = os.open(path, os.O_RDONLY)
+            stream = torch.cuda.Stream()
+            out = torch.empty(ck.nbytes_total, dtype=torch.uint8, device="cuda")
+            ptrs = [out.data_ptr() + int(o) for o in np.concatenate([[0], np.cumsum(nbytes)])[:-1]]
+            for it in range(4):
+                out.fill_(0xEE)
+                torch.cuda.current_stream().synchronize()
+                tc.tc_weights_materialize_file(wplan, fd, 0, ptrs, stream=stream.cuda_stream)
+                stream.synchronize()
+                if not np.array_equal(out.cpu().numpy(), blob):   # tight canonical order: the outputs concatenate to the blob
+                    errors.append(("loader", it))
+            os.close(fd)
+        except Exception as e:  # noqa: BLE001
+            errors.append(("loader", repr(e)))
+
+    def reloader():
+        try:
+            stream = torch.cuda.Stream()
+            for it in range(12):
+                fresh = Guarded(pool.size)
+                torch.cuda.current_stream().synchronize()
+                tc.tc_kv_unpack(uplan, [h_packed], [fresh.ptr()], stream.cuda_stream)
+                stream.synchronize()
+                if not np.array_equal(fresh.result(), want_pool):
+                    errors.append(("reloader", it))
+        except Exception as e:  # noqa: BLE001
+            errors.append(("reloader", repr(e)))
+
+    threads = [threading.Thread(target=loader), threading.Thread(target=reloader)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors[:3]
+
+
 # --------------------------------------------------------------------------- lifecycle on the device
 def test_empty_plan_wrong_tables_and_deadline_launch_nothing():
     shape, NB, src, dst = wl.config1()
