@@ -766,6 +766,27 @@ def run_extras(args, tc, torch, stream):
             res[name] = 2 * ck.nbytes_total / (statistics.mean(ts) * 1e-3) / GB
     out["configs[2] weights full, integrity checksum fused into the copy"] = {"GBps_plain": res["plain"], "GBps_with_checksum": res["with_checksum"]}
     planc.destroy()
+    # ---- configs[2]: every rank's shard of W = 8, each timed alone
+    W = 8
+    sizes = [n // (W if ck.split_dim[i] >= 0 else 1) for i, n in enumerate(nbytes)]
+    sptrs = [dstw.data_ptr() + int(o) for o in np.concatenate([[0], np.cumsum(sizes)])[:-1]]
+    per_rank = []
+    with torch.cuda.stream(stream):
+        for rank in range(W):
+            sh = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, split_dim=ck.split_dim, rank=rank, world=W, blob_bytes=ck.nbytes_total))
+            ts = []
+            for i in range(8):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                tc.tc_weights_materialize(sh, blob, sptrs, sp)
+                b.record(stream)
+                torch.cuda.synchronize()
+                if i >= 3:
+                    ts.append(a.elapsed_time(b))
+            per_rank.append(2 * sum(sizes) / (statistics.mean(ts) * 1e-3) / GB)
+            sh.destroy()
+    out["configs[2] weights TP shard, every rank of 8 (timed alone, back to back: the 4 GB of traffic partly stays in L2)"] = {
+        "payload_bytes": sum(sizes), "GBps_per_rank": per_rank}
     del blob, dstw
     torch.cuda.empty_cache()
     out["weights cold path: blob streamed from a file"] = cold_path(args, tc, torch, stream)
@@ -800,6 +821,45 @@ def run_extras(args, tc, torch, stream):
         "pool_blocks": NB, "requests": len(src.T), "blocks": src.n_blocks, "payload_bytes": payload,
         "GBps": 2 * payload / (statistics.mean(ms) * 1e-3) / GB, "ms": statistics.mean(ms), "plan_create_ms": create_ms}
     mig.destroy()
+    # the same wave into an HND pool (layout transform fused into the migration) ...
+    pl_hnd = tc.pool(tc.TC_HND, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=A.numel())
+    mig_t = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape.tuple, src_pool=pl, dst_pool=pl_hnd, T=src.T, bt_off=src.bt_off, bt_src=src.bt, bt_dst=dst.bt))
+
+    def timed(fn):
+        ts = []
+        with torch.cuda.stream(stream):
+            for i in range(6):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                torch.cuda.synchronize()
+                if i >= 3:
+                    ts.append(a.elapsed_time(b))
+        return statistics.mean(ts)
+    ms_t = timed(lambda: tc.tc_kv_pack(mig_t, [A], [B], sp))
+    mig_t.destroy()
+    out["configs[3] 70B KV migrate (one wave)"]["GBps_into_an_HND_pool"] = 2 * payload / (ms_t * 1e-3) / GB
+    # ... and, for comparison, unfused: pack into a device buffer, then unpack (twice the traffic).
+    # The buffer takes what memory is left, so only the first requests that fit take part.
+    free, _ = torch.cuda.mem_get_info()
+    budget = int(0.8 * free)
+    k = int(np.searchsorted(np.cumsum(src.T) * shape.token_bytes, budget, side="right"))
+    if k > 0:
+        Tk, offk = src.T[:k], src.bt_off[:k + 1]
+        nblk = int(offk[-1])
+        part = int(Tk.sum()) * shape.token_bytes
+        Q = torch.empty(part, **u8)
+        pk = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape.tuple, src_pool=pl, packed_layout=tc.TC_NHD, T=Tk, bt_off=offk, bt_src=src.bt[:nblk]))
+        up = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape.tuple, dst_pool=pl, packed_layout=tc.TC_NHD, T=Tk, bt_off=offk, bt_dst=dst.bt[:nblk]))
+        fused = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape.tuple, src_pool=pl, dst_pool=pl, T=Tk, bt_off=offk, bt_src=src.bt[:nblk], bt_dst=dst.bt[:nblk]))
+        ms_two = timed(lambda: (tc.tc_kv_pack(pk, [A], [Q], sp), tc.tc_kv_unpack(up, [Q], [B], sp)))
+        ms_one = timed(lambda: tc.tc_kv_pack(fused, [A], [B], sp))
+        out["configs[3] 70B KV migrate (one wave)"]["fused_vs_pack_then_unpack"] = {
+            "requests": k, "payload_bytes": part, "ms_fused_migrate": ms_one, "ms_pack_then_unpack_through_a_device_buffer": ms_two}
+        for p_ in (pk, up, fused):
+            p_.destroy()
+        del Q
     del A, B
     torch.cuda.empty_cache()
     # ---- configs[4]
