@@ -750,9 +750,10 @@ def run_extras(args, tc, torch, stream):
     ptrs = [dstw.data_ptr() + int(o) for o in np.concatenate([[0], np.cumsum(nbytes)])[:-1]]
     sums = torch.zeros(ck.N, dtype=torch.int64, device="cuda")
     planc = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total, flags=tc.TC_PLAN_CHECKSUM))
+    planp = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total))
     res = {}
     with torch.cuda.stream(stream):
-        for name, fn in (("plain", lambda: tc.tc_weights_materialize(planc, blob, ptrs, sp)),
+        for name, fn in (("plain", lambda: tc.tc_weights_materialize(planp, blob, ptrs, sp)),
                          ("with_checksum", lambda: tc.tc_weights_materialize_checksum(planc, blob, ptrs, sums, sp))):
             ts = []
             for i in range(8):
@@ -766,6 +767,7 @@ def run_extras(args, tc, torch, stream):
             res[name] = 2 * ck.nbytes_total / (statistics.mean(ts) * 1e-3) / GB
     out["configs[2] weights full, integrity checksum fused into the copy"] = {"GBps_plain": res["plain"], "GBps_with_checksum": res["with_checksum"]}
     planc.destroy()
+    planp.destroy()
     # ---- configs[2]: every rank's shard of W = 8, each timed alone
     W = 8
     sizes = [n // (W if ck.split_dim[i] >= 0 else 1) for i, n in enumerate(nbytes)]

@@ -154,7 +154,8 @@ enum {
                                tc_weights_materialize_checksum, which folds an integrity
                                checksum of every tensor into the same pass as the copy.  Needs
                                16-byte aligned geometry and tensors that start on 4-byte
-                               boundaries of the blob (TC_ERR_INVALID_ARG otherwise). */
+                               boundaries of the blob (TC_ERR_INVALID_ARG otherwise).  Such
+                               plans default to 64 KiB tiles (tuning.tile_bytes overrides). */
     TC_PLAN_STREAM = 16u    /* TC_WEIGHTS: the blob is streamed chunk by chunk, from a file
                                (tc_weights_materialize_file) or from pinned host memory
                                (tc_weights_materialize), through the staging ring.  Unlike
