@@ -91,3 +91,21 @@ def ck_spec(ck, **kw):
     nbytes = [ck.nbytes(i) for i in range(ck.N)]
     kw.setdefault("blob_bytes", ck.nbytes_total)
     return tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, **kw)
+
+
+def ipc_pack_child(q_in, q_out):
+    """Runs in a spawned process: receives a pool another process allocated (torch maps it through
+    CUDA IPC), packs from it with this process's own plan and returns the packed bytes."""
+    try:
+        import torch
+        pool_t, shape, pool_args, T, off, bt, packed_l, n = q_in.get()
+        pl = tc.pool(*pool_args[0], **pool_args[1])
+        plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_src=bt))
+        out = torch.zeros(n, dtype=torch.uint8, device="cuda")
+        tc.tc_kv_pack(plan, [pool_t], [out])
+        torch.cuda.synchronize()
+        q_out.put(("ok", out.cpu().numpy()))
+        plan.destroy()
+        del pool_t
+    except Exception as e:  # noqa: BLE001
+        q_out.put(("error", repr(e)))

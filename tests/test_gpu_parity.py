@@ -716,6 +716,34 @@ def test_file_stream_and_staged_reload_share_the_staging_ring(tmp_path):
     assert not errors, errors[:3]
 
 
+def test_pool_of_another_process_through_cuda_ipc():
+    """Same-host sharing: a KV pool allocated by this process is opened by a second process
+    through CUDA IPC and used there as the source table of its own plan (data buffers are
+    caller-leased plain pointers, so nothing in the library is special-cased for this)."""
+    import torch.multiprocessing as mp
+    from helpers import ipc_pack_child
+    rng = np.random.default_rng(33)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=40, B=16, H=8, D=128, E=2, T=(100, 37, 16, 5, 200))
+    L = shape[0]
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, L * 2), T, off, bt, oracle.HND, want, threads=4)
+    d_pool = dev(pool)
+    torch.cuda.synchronize()
+    ctx = mp.get_context("spawn")
+    q_in, q_out = ctx.Queue(), ctx.Queue()
+    child = ctx.Process(target=ipc_pack_child, args=(q_in, q_out))
+    child.start()
+    try:
+        q_in.put((d_pool, shape, ((tc.TC_NHD, NB, 1), dict(plane_stride=NB * stride)), T, off, bt, tc.TC_HND, want.size))
+        status, got = q_out.get(timeout=300)
+    finally:
+        child.join(timeout=60)
+        if child.is_alive():
+            child.kill()
+    assert status == "ok", got
+    assert np.array_equal(got, want)
+
+
 # --------------------------------------------------------------------------- lifecycle on the device
 def test_empty_plan_wrong_tables_and_deadline_launch_nothing():
     shape, NB, src, dst = wl.config1()
