@@ -684,6 +684,67 @@ def cold_path(args, tc, torch, stream):
     return out
 
 
+def moe_stacking(args, tc, torch, stream):
+    """transform_into with expert stacking on a mixture-of-experts checkpoint of the shape the
+    paper's loader experiments use (Qwen3-30B-A3B: hidden 2048, 128 experts of 768, some of its
+    48 layers): per layer the gate and up matrices of all experts land in one fused
+    [experts, 2*mlp, hidden] buffer and the down matrices in one [experts, hidden, mlp] buffer;
+    every other tensor gets its own destination."""
+    import re
+    sp = stream.cuda_stream
+    layers, experts, mlp, hidden = (1 if args.small else args.moe_layers), 128, 768, 2048
+    ck = wl.moe_checkpoint(hidden=hidden, layers=layers, experts=experts, moe_mlp=mlp, q_heads=32, kv_heads=4, head_dim=128, vocab=151936)
+    E = 2
+    nbytes = [ck.nbytes(i) for i in range(ck.N)]
+    gu_exp, dn_exp = 2 * mlp * hidden * E, hidden * mlp * E
+    slot, doff, dst_bytes = [], [], []
+    fused = {}
+    pat = re.compile(r"layers\.(\d+)\.experts\.(\d+)\.(gate|up|down)_proj")
+    for i, name in enumerate(ck.names):
+        m = pat.fullmatch(name)
+        if not m:
+            slot.append(len(dst_bytes))
+            doff.append(0)
+            dst_bytes.append(nbytes[i])
+            continue
+        l, e, kind = int(m.group(1)), int(m.group(2)), m.group(3)
+        key = (l, "down" if kind == "down" else "gate_up")
+        if key not in fused:
+            fused[key] = len(dst_bytes)
+            dst_bytes.append(experts * (dn_exp if kind == "down" else gu_exp))
+        slot.append(fused[key])
+        doff.append(e * dn_exp if kind == "down" else e * gu_exp + (mlp * hidden * E if kind == "up" else 0))
+    blob = torch.empty(ck.nbytes_total, dtype=torch.uint8, device="cuda")
+    wl.fill_torch(blob, wl.SEED_BASE + 6, "normal")
+    arena = torch.empty(sum(dst_bytes), dtype=torch.uint8, device="cuda")
+    starts = np.concatenate([[0], np.cumsum(dst_bytes)])[:-1]
+    ptrs = [arena.data_ptr() + int(o) for o in starts]
+    t0 = time.perf_counter()
+    plan = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total,
+                                             dst_slot=slot, dst_off=doff, n_dst=len(dst_bytes), dst_bytes=dst_bytes))
+    create_ms = 1e3 * (time.perf_counter() - t0)
+    ts = []
+    with torch.cuda.stream(stream):
+        for i in range(8):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            tc.tc_weights_materialize(plan, blob, ptrs, sp)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b))
+    # spot check: expert 5 of the last layer, up_proj, sits behind its gate_proj in the fused buffer
+    i = ck.names.index(f"layers.{layers - 1}.experts.5.up_proj")
+    lo = int(starts[slot[i]]) + doff[i]
+    ok = bool(torch.equal(arena[lo:lo + nbytes[i]], blob[int(ck.byte_off[i]):int(ck.byte_off[i]) + nbytes[i]]))
+    st = plan.stats()
+    plan.destroy()
+    del blob, arena
+    torch.cuda.empty_cache()
+    return {"layers": layers, "tensors": ck.N, "destination_buffers": len(dst_bytes), "bytes": ck.nbytes_total, "tiles": int(st.n_tiles[0]),
+            "plan_create_ms": create_ms, "ms": statistics.mean(ts), "GBps": 2 * ck.nbytes_total / (statistics.mean(ts) * 1e-3) / GB, "spot_check": ok}
+
+
 def run_extras(args, tc, torch, stream):
     """Secondary workloads, reported beside the headline: configs[3] (70B-shaped pool-to-pool
     migration, one wave) and configs[4] (prefix-reload burst: one mixed plan per scheduler step,
@@ -792,6 +853,7 @@ def run_extras(args, tc, torch, stream):
     del blob, dstw
     torch.cuda.empty_cache()
     out["weights cold path: blob streamed from a file"] = cold_path(args, tc, torch, stream)
+    out["transform_into: MoE expert stacking (Qwen3-30B-A3B-shaped layers)"] = moe_stacking(args, tc, torch, stream)
     # ---- configs[3]
     shape = wl.LLAMA3_70B_KV
     free, _ = torch.cuda.mem_get_info()
@@ -942,6 +1004,7 @@ def main():
     ap.add_argument("--host-pool-blocks", type=int, default=8192, help="configs[4]: pinned host pool size in 2 MiB blocks")
     ap.add_argument("--burst-steps", type=int, default=10, help="configs[4]: scheduler steps timed (the workload has 200)")
     ap.add_argument("--cold-layers", type=int, default=8, help="cold-path extra: layers of the checkpoint written to a file (8: 4.0 GB)")
+    ap.add_argument("--moe-layers", type=int, default=8, help="expert-stacking extra: layers of the MoE checkpoint (8: 11 GB)")
     ap.add_argument("--host-ctas", type=int, default=0)
     ap.add_argument("--host-path", default="staged", choices=["staged", "zerocopy"])
     ap.add_argument("--e2e-schedule", default="duplex", choices=["duplex", "serial"],
