@@ -719,9 +719,11 @@ def moe_stacking(args, tc, torch, stream):
     arena = torch.empty(sum(dst_bytes), dtype=torch.uint8, device="cuda")
     starts = np.concatenate([[0], np.cumsum(dst_bytes)])[:-1]
     ptrs = [arena.data_ptr() + int(o) for o in starts]
+    spec = tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total,
+                           dst_slot=slot, dst_off=doff, n_dst=len(dst_bytes), dst_bytes=dst_bytes)
+    torch.cuda.synchronize()  # the fill above is still running; plan upload would wait for it
     t0 = time.perf_counter()
-    plan = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total,
-                                             dst_slot=slot, dst_off=doff, n_dst=len(dst_bytes), dst_bytes=dst_bytes))
+    plan = tc.tc_plan_create(spec)
     create_ms = 1e3 * (time.perf_counter() - t0)
     ts = []
     with torch.cuda.stream(stream):
@@ -867,6 +869,7 @@ def run_extras(args, tc, torch, stream):
     B = torch.empty(NB * shape.block_bytes, **u8)
     B.fill_(9)
     pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=A.numel())
+    torch.cuda.synchronize()  # the fills above are still running; plan upload would wait for them
     t0 = time.perf_counter()
     mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape.tuple, src_pool=pl, dst_pool=pl, T=src.T, bt_off=src.bt_off, bt_src=src.bt, bt_dst=dst.bt))
     create_ms = 1e3 * (time.perf_counter() - t0)
