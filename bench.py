@@ -595,6 +595,24 @@ def run_ours(args):
     ranks.close()
 
 
+def b2b_ms(torch, stream, fn, reps=5, warm=2):
+    """Device milliseconds per call of fn: `reps` calls enqueued back to back inside one event pair,
+    behind `warm` untimed ones that are still running when the first event is enqueued.  The host
+    side of a call (marshalling the pointer table, checks, the launch itself) then overlaps the GPU
+    work of the call before it; with a synchronise before every timed launch a short kernel would be
+    charged for the time the idle GPU waits for the host."""
+    with torch.cuda.stream(stream):
+        for _ in range(warm):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
 def cold_path(args, tc, torch, stream):
     """Weight loading from a FILE (storage -> pinned ring -> device, scatter and slicing fused
     into the device leg): wall-clock GB/s of blob bytes, next to the plain rate at which the
@@ -725,16 +743,7 @@ def moe_stacking(args, tc, torch, stream):
     t0 = time.perf_counter()
     plan = tc.tc_plan_create(spec)
     create_ms = 1e3 * (time.perf_counter() - t0)
-    ts = []
-    with torch.cuda.stream(stream):
-        for i in range(8):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            tc.tc_weights_materialize(plan, blob, ptrs, sp)
-            b.record(stream)
-            torch.cuda.synchronize()
-            if i >= 3:
-                ts.append(a.elapsed_time(b))
+    ms = b2b_ms(torch, stream, lambda: tc.tc_weights_materialize(plan, blob, ptrs, sp))
     # spot check: expert 5 of the last layer, up_proj, sits behind its gate_proj in the fused buffer
     i = ck.names.index(f"layers.{layers - 1}.experts.5.up_proj")
     lo = int(starts[slot[i]]) + doff[i]
@@ -744,7 +753,7 @@ def moe_stacking(args, tc, torch, stream):
     del blob, arena
     torch.cuda.empty_cache()
     return {"layers": layers, "tensors": ck.N, "destination_buffers": len(dst_bytes), "bytes": ck.nbytes_total, "tiles": int(st.n_tiles[0]),
-            "plan_create_ms": create_ms, "ms": statistics.mean(ts), "GBps": 2 * ck.nbytes_total / (statistics.mean(ts) * 1e-3) / GB, "spot_check": ok}
+            "plan_create_ms": create_ms, "ms": ms, "GBps": 2 * ck.nbytes_total / (ms * 1e-3) / GB, "spot_check": ok}
 
 
 def run_extras(args, tc, torch, stream):
@@ -815,19 +824,9 @@ def run_extras(args, tc, torch, stream):
     planc = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total, flags=tc.TC_PLAN_CHECKSUM))
     planp = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total))
     res = {}
-    with torch.cuda.stream(stream):
-        for name, fn in (("plain", lambda: tc.tc_weights_materialize(planp, blob, ptrs, sp)),
-                         ("with_checksum", lambda: tc.tc_weights_materialize_checksum(planc, blob, ptrs, sums, sp))):
-            ts = []
-            for i in range(8):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream)
-                fn()
-                b.record(stream)
-                torch.cuda.synchronize()
-                if i >= 3:
-                    ts.append(a.elapsed_time(b))
-            res[name] = 2 * ck.nbytes_total / (statistics.mean(ts) * 1e-3) / GB
+    for name, fn in (("plain", lambda: tc.tc_weights_materialize(planp, blob, ptrs, sp)),
+                     ("with_checksum", lambda: tc.tc_weights_materialize_checksum(planc, blob, ptrs, sums, sp))):
+        res[name] = 2 * ck.nbytes_total / (b2b_ms(torch, stream, fn) * 1e-3) / GB
     out["configs[2] weights full, integrity checksum fused into the copy"] = {"GBps_plain": res["plain"], "GBps_with_checksum": res["with_checksum"]}
     planc.destroy()
     planp.destroy()
@@ -836,21 +835,12 @@ def run_extras(args, tc, torch, stream):
     sizes = [n // (W if ck.split_dim[i] >= 0 else 1) for i, n in enumerate(nbytes)]
     sptrs = [dstw.data_ptr() + int(o) for o in np.concatenate([[0], np.cumsum(sizes)])[:-1]]
     per_rank = []
-    with torch.cuda.stream(stream):
-        for rank in range(W):
-            sh = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, split_dim=ck.split_dim, rank=rank, world=W, blob_bytes=ck.nbytes_total))
-            ts = []
-            for i in range(8):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream)
-                tc.tc_weights_materialize(sh, blob, sptrs, sp)
-                b.record(stream)
-                torch.cuda.synchronize()
-                if i >= 3:
-                    ts.append(a.elapsed_time(b))
-            per_rank.append(2 * sum(sizes) / (statistics.mean(ts) * 1e-3) / GB)
-            sh.destroy()
-    out["configs[2] weights TP shard, every rank of 8 (timed alone, back to back: the 4 GB of traffic partly stays in L2)"] = {
+    for rank in range(W):
+        sh = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, split_dim=ck.split_dim, rank=rank, world=W, blob_bytes=ck.nbytes_total))
+        ms = b2b_ms(torch, stream, lambda: tc.tc_weights_materialize(sh, blob, sptrs, sp), reps=10)
+        per_rank.append(2 * sum(sizes) / (ms * 1e-3) / GB)
+        sh.destroy()
+    out["configs[2] weights TP shard, every rank of 8 (10 launches back to back per rank; 4 GB of traffic per launch)"] = {
         "payload_bytes": sum(sizes), "GBps_per_rank": per_rank}
     del blob, dstw
     torch.cuda.empty_cache()
@@ -874,36 +864,17 @@ def run_extras(args, tc, torch, stream):
     mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape.tuple, src_pool=pl, dst_pool=pl, T=src.T, bt_off=src.bt_off, bt_src=src.bt, bt_dst=dst.bt))
     create_ms = 1e3 * (time.perf_counter() - t0)
     payload = int(src.T.sum()) * shape.token_bytes
-    ms = []
-    with torch.cuda.stream(stream):
-        for i in range(6):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            tc.tc_kv_pack(mig, [A], [B], sp)
-            b.record(stream)
-            torch.cuda.synchronize()
-            if i >= 3:
-                ms.append(a.elapsed_time(b))
+    ms_mig = b2b_ms(torch, stream, lambda: tc.tc_kv_pack(mig, [A], [B], sp), reps=3)
     out["configs[3] 70B KV migrate (one wave)"] = {
         "pool_blocks": NB, "requests": len(src.T), "blocks": src.n_blocks, "payload_bytes": payload,
-        "GBps": 2 * payload / (statistics.mean(ms) * 1e-3) / GB, "ms": statistics.mean(ms), "plan_create_ms": create_ms}
+        "GBps": 2 * payload / (ms_mig * 1e-3) / GB, "ms": ms_mig, "plan_create_ms": create_ms}
     mig.destroy()
     # the same wave into an HND pool (layout transform fused into the migration) ...
     pl_hnd = tc.pool(tc.TC_HND, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=A.numel())
     mig_t = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape.tuple, src_pool=pl, dst_pool=pl_hnd, T=src.T, bt_off=src.bt_off, bt_src=src.bt, bt_dst=dst.bt))
 
     def timed(fn):
-        ts = []
-        with torch.cuda.stream(stream):
-            for i in range(6):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream)
-                fn()
-                b.record(stream)
-                torch.cuda.synchronize()
-                if i >= 3:
-                    ts.append(a.elapsed_time(b))
-        return statistics.mean(ts)
+        return b2b_ms(torch, stream, fn, reps=3)
     ms_t = timed(lambda: tc.tc_kv_pack(mig_t, [A], [B], sp))
     mig_t.destroy()
     out["configs[3] 70B KV migrate (one wave)"]["GBps_into_an_HND_pool"] = 2 * payload / (ms_t * 1e-3) / GB

@@ -168,11 +168,9 @@ enum {
 };
 
 #define TC_MAX_TABLE_SLOTS 4000 /* src slots + dst slots of one execute call.  The table travels in the
-                                   kernel parameters; looking a pointer up in a table of thousands of
-                                   entries costs bandwidth (measured: none up to ~60 slots, 2 % at
-                                   400, 15 % at 3000), so a checkpoint of thousands of small tensors
-                                   moves fastest into a few large buffers addressed by
-                                   tc_weight_rule_t.dst_slot / dst_off. */
+                                   kernel parameters; its size does not change the kernel's speed
+                                   (measured: 6.97 TB/s with 1 to 3072 destination slots), only the
+                                   host time of the call (one check and one copy per entry). */
 
 /* Geometry of a paged KV pool (the data pointer(s) come at execute time). */
 typedef struct {
