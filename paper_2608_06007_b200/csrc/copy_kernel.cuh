@@ -32,6 +32,7 @@ struct Params {
     const Desc *descs;
     const uint32_t *tile_desc;  // null for uniform groups
     uint32_t n_tiles;
+    uint32_t n_descs;           // descriptors of the group (bounds the look-ahead prefetch)
     uint32_t tiles_per_desc;    // > 0 for uniform groups
     FastDiv div_tpd;
     uint32_t tpo;               // uniform groups: tiles per plane of one descriptor
@@ -65,6 +66,12 @@ template <typename V> __device__ __forceinline__ unsigned long long csum_of(V, u
 template <> __device__ __forceinline__ unsigned long long csum_of<uint4>(uint4 v, unsigned long long p) { return csum_vec(v, p); }
 
 __device__ __forceinline__ uint32_t fastdiv(uint32_t n, FastDiv f) { return (__umulhi(n, f.mul) + n) >> f.shift; }
+
+// Metadata look-ahead distances: about two waves of resident CTAs (148 SMs x 3), and for
+// listed groups, where the descriptor of a later tile is not known without a load, a fixed
+// number of descriptors.
+constexpr uint32_t kLookAheadTiles = 1024, kLookAheadDescs = 16;
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 template <typename V> __device__ __forceinline__ V ld_stream(const char *p);
 template <typename V> __device__ __forceinline__ void st_stream(char *p, V v);
@@ -195,6 +202,23 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
         }
         if (threadIdx.x < sizeof(Desc) / 16)
             reinterpret_cast<uint4 *>(&sdesc[buf])[threadIdx.x] = __ldg(reinterpret_cast<const uint4 *>(prm.descs + di) + threadIdx.x);
+        // Look-ahead: pull the metadata of tiles a few waves ahead into L2.  Consecutive tiles
+        // start almost together, so without this every tile of a short descriptor waits on the
+        // same DRAM miss (and, in listed groups, on the tile-list line before it).
+        if (threadIdx.x == kThreads - 1) {
+            const uint32_t ahead = tile + kLookAheadTiles;
+            uint32_t da;
+            if (prm.win_span) {
+                const uint32_t rem = ahead % prm.win_span;
+                da = prm.win_d0 + rem / prm.win_tpo;
+            } else if (prm.tiles_per_desc) {
+                da = fastdiv(ahead, prm.div_tpd);
+            } else {
+                if (ahead < prm.n_tiles) prefetch_l2(prm.tile_desc + ahead);
+                da = di + kLookAheadDescs;
+            }
+            if (da < prm.n_descs) prefetch_l2(prm.descs + da);
+        }
         __syncthreads();
         const Desc &d = sdesc[buf];
         if (!prm.tiles_per_desc && !prm.win_span) {

@@ -86,6 +86,7 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     prm.descs = g.d_descs;
     prm.tile_desc = g.d_tile_desc;
     prm.n_tiles = static_cast<uint32_t>(g.n_tiles);
+    prm.n_descs = static_cast<uint32_t>(g.descs.size());
     prm.win_span = prm.win_d0 = prm.win_o0 = prm.win_tpo = prm.tile_base = 0;
     if (win && win->nd == 0) {  // a range of global tile ids
         prm.tile_base = win->d0;
