@@ -256,10 +256,11 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
         } else {
             switch (min(d.log2_align, prm.log2_ptr_align)) {
             case 4: copy_rows<4, kUnroll, kThreads>(d, src, dst, row0, nrows); break;
-            case 3: copy_rows<3, kUnroll, kThreads>(d, src, dst, row0, nrows); break;
-            case 2: copy_rows<2, kUnroll, kThreads>(d, src, dst, row0, nrows); break;
-            case 1: copy_rows<1, kUnroll, kThreads>(d, src, dst, row0, nrows); break;
-            default: copy_rows<0, kUnroll, kThreads>(d, src, dst, row0, nrows); break;
+            // narrower vectors cost fewer registers each, so more of them can be in flight
+            case 3: copy_rows<3, 2 * kUnroll, kThreads>(d, src, dst, row0, nrows); break;
+            case 2: copy_rows<2, 2 * kUnroll, kThreads>(d, src, dst, row0, nrows); break;
+            case 1: copy_rows<1, 2 * kUnroll, kThreads>(d, src, dst, row0, nrows); break;
+            default: copy_rows<0, 2 * kUnroll, kThreads>(d, src, dst, row0, nrows); break;
             }
         }
     }
