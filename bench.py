@@ -756,6 +756,44 @@ def moe_stacking(args, tc, torch, stream):
             "plan_create_ms": create_ms, "ms": ms, "GBps": 2 * ck.nbytes_total / (ms * 1e-3) / GB, "spot_check": ok}
 
 
+def kv_shapes(args, tc, torch, stream):
+    """Rows a1-a3 on other KV geometries than the headline one: few KV heads (what a tensor-parallel
+    rank or a GQA / MQA model holds: planes of 4-16 KiB per block), larger blocks, small head_dim."""
+    sp = stream.cuda_stream
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    out = {}
+    K = wl.KVShape
+    cases = [("8 KV heads (headline shape)", K(32, 16, 8, 128)), ("4 KV heads", K(28, 16, 4, 128)), ("2 KV heads", K(28, 16, 2, 128)),
+             ("1 KV head", K(32, 16, 1, 128)), ("32 heads of 64", K(32, 16, 32, 64)), ("block 128", K(32, 128, 8, 128))]
+    for label, shape in cases[:2 if args.small else None]:
+        s = shape.tuple
+        NB = int(((1 if args.small else 8) << 30) // shape.block_bytes)
+        WB = NB // 2
+        _, _, _, waves = wl.config2(NB=NB, R=256, wave_blocks=WB, NB_dst=WB, shape=shape)
+        src, dst = waves[0]
+        poolA = torch.empty(NB * shape.block_bytes, **u8)
+        wl.fill_torch(poolA, wl.SEED_BASE + 7)
+        poolB = torch.empty(WB * shape.block_bytes, **u8)
+        payload = int(src.T.sum()) * shape.token_bytes
+        Q = torch.empty(payload, **u8)
+        plA = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=poolA.numel())
+        plB = tc.pool(tc.TC_NHD, WB, 1, plane_stride=WB * shape.chunk_bytes, slot_bytes=poolB.numel())
+        kw = dict(T=src.T, bt_off=src.bt_off)
+        pk = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, bt_src=src.bt, **kw))
+        up = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, bt_dst=dst.bt, **kw))
+        mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, s, src_pool=plA, dst_pool=plB, bt_src=src.bt, bt_dst=dst.bt, **kw))
+        res = {"plane_KiB": shape.chunk_bytes // 1024, "planes_per_tile": int(mig.descriptors(0)[0].planes_per_tile), "payload_bytes": payload}
+        for name, fn in (("pack", lambda: tc.tc_kv_pack(pk, [poolA], [Q], sp)), ("unpack", lambda: tc.tc_kv_unpack(up, [Q], [poolB], sp)),
+                         ("migrate", lambda: tc.tc_kv_pack(mig, [poolA], [poolB], sp))):
+            res["GBps_" + name] = 2 * payload / (b2b_ms(torch, stream, fn, reps=8, warm=3) * 1e-3) / GB
+        out[label + f" L{shape.L} B{shape.B} H{shape.H} D{shape.D}"] = res
+        for p_ in (pk, up, mig):
+            p_.destroy()
+        del poolA, poolB, Q
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_extras(args, tc, torch, stream):
     """Secondary workloads, reported beside the headline: configs[3] (70B-shaped pool-to-pool
     migration, one wave) and configs[4] (prefix-reload burst: one mixed plan per scheduler step,
@@ -846,6 +884,7 @@ def run_extras(args, tc, torch, stream):
     torch.cuda.empty_cache()
     out["weights cold path: blob streamed from a file"] = cold_path(args, tc, torch, stream)
     out["transform_into: MoE expert stacking (Qwen3-30B-A3B-shaped layers)"] = moe_stacking(args, tc, torch, stream)
+    out["rows a1-a3 on other KV geometries (8 GiB pools, first wave)"] = kv_shapes(args, tc, torch, stream)
     # ---- configs[3]
     shape = wl.LLAMA3_70B_KV
     free, _ = torch.cuda.mem_get_info()

@@ -420,8 +420,9 @@ typedef struct {
     uint32_t rows_per_tile;   /* rows one tile (one CTA pass) moves */
     uint32_t tiles_per_outer; /* tile ids per outer index; parts past the last row are empty */
     uint32_t tile0;           /* global id of tile (outer 0, part 0); tile (o, p) has id
-                                 tile0 + o*tiles_per_outer + p */
-    uint32_t reserved;
+                                 tile0 + (o / planes_per_tile)*tiles_per_outer + p */
+    uint32_t planes_per_tile; /* 1, or - small planes, a few KiB each - how many consecutive
+                                 outer indices of the descriptor one tile moves */
 } tc_descriptor_t;
 
 /* Copy up to `cap` descriptors of `group` (0 or 1) into out (host array); *n_out receives the

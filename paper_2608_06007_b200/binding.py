@@ -88,7 +88,7 @@ class tc_descriptor_t(C.Structure):
                                           "src_s0", "src_s1", "dst_s0", "dst_s1")] + \
                [(n, C.c_uint32) for n in ("src_slot", "dst_slot", "src_slot_step", "dst_slot_step",
                                           "run_bytes", "n0", "rows", "n_outer",
-                                          "rows_per_tile", "tiles_per_outer", "tile0", "reserved")]
+                                          "rows_per_tile", "tiles_per_outer", "tile0", "planes_per_tile")]
 
 
 class tc_segment_t(C.Structure):

@@ -41,6 +41,8 @@ struct Params {
     // launch window (win_span == 0: the whole group).  Tile ids then walk plane-major over
     // descriptors [win_d0, ...) x planes [win_o0, ...): win_span = descriptors x win_tpo.
     uint32_t win_span, win_d0, win_o0, win_tpo;
+    uint32_t win_o_end;         // first plane past the window
+    uint32_t ppt, log2_unit;    // multi-plane tiles (MULTI builds): planes per tile, log2 of the padded plane
     uint32_t tile_base;         // first global tile id of this launch (tile-range segments)
     unsigned long long *sums;   // checksum accumulators (checked builds only)
     char *ptr[NPTR];            // src table then dst table
@@ -157,6 +159,51 @@ __device__ __forceinline__ void copy_rows(const Desc &d, const char *src, char *
     }
 }
 
+// A tile of n_units consecutive planes of one descriptor (small planes, see Group::ppt).  The
+// tile's byte space gives every plane 2^log2_unit bytes, of which the first rows * run are real;
+// plane k sits k * outer bytes behind plane 0 on each side.  ROWS: decode rows inside a plane,
+// else every plane is one run.  src / dst point at row 0 of the tile's first plane.
+template <int LOGV, int U, int kThreads, bool ROWS>
+__device__ __forceinline__ void copy_multi(const Desc &d, const char *src, char *dst, uint32_t n_units, uint32_t log2_unit)
+{
+    using V = typename VecOf<LOGV>::type;
+    const uint32_t unit_bytes = d.rows * d.run, mask = (1u << log2_unit) - 1;
+    const uint32_t nbytes = n_units << log2_unit;
+    const uint32_t run = d.run, n0 = d.n0;
+    const FastDiv div_run = d.div_run, div_n0 = d.div_n0;
+    const uint32_t ss0 = d.src_s0, ss1 = d.src_s1, ds0 = d.dst_s0, ds1 = d.dst_s1;
+    const long long src_outer = d.src_outer, dst_outer = d.dst_outer;
+#pragma unroll 1
+    for (uint32_t base = threadIdx.x << LOGV; base < nbytes; base += (kThreads * U) << LOGV) {
+        V val[U];
+        uint32_t doff[U];
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+            const uint32_t byte = base + ((u * kThreads) << LOGV);
+            const uint32_t k = byte >> log2_unit, w = byte & mask;
+            if (byte < nbytes && w < unit_bytes) {
+                uint32_t so = w;
+                doff[u] = w;
+                if (ROWS) {
+                    const uint32_t r = fastdiv(w, div_run);
+                    const uint32_t col = w - r * run;
+                    const uint32_t i1 = fastdiv(r, div_n0);
+                    const uint32_t i0 = r - i1 * n0;
+                    doff[u] = i1 * ds1 + i0 * ds0 + col;
+                    so = i1 * ss1 + i0 * ss0 + col;
+                }
+                val[u] = ld_stream<V>(src + k * src_outer + so);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+            const uint32_t byte = base + ((u * kThreads) << LOGV);
+            const uint32_t k = byte >> log2_unit, w = byte & mask;
+            if (byte < nbytes && w < unit_bytes) st_stream<V>(dst + k * dst_outer + doff[u], val[u]);
+        }
+    }
+}
+
 // One contiguous run of 16-byte vectors: no row decoding at all.
 template <int U, int kThreads, bool CHECK = false>
 __device__ __forceinline__ void copy_run16(const char *src, char *dst, uint32_t nbytes, unsigned long long pos0 = 0, unsigned long long *acc = nullptr)
@@ -176,7 +223,7 @@ __device__ __forceinline__ void copy_run16(const char *src, char *dst, uint32_t 
     }
 }
 
-template <int NPTR, int MODE, bool CHECK = false>
+template <int NPTR, int MODE, bool CHECK = false, bool MULTI = false>
 __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) tc_copy_kernel(const __grid_constant__ Params<NPTR> prm)
 {
     constexpr int kThreads = Shape<MODE>::threads, kUnroll = Shape<MODE>::unroll;
@@ -190,13 +237,14 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
             const uint32_t ow = tile / prm.win_span, rem = tile - ow * prm.win_span;
             const uint32_t dw = rem / prm.win_tpo;
             di = prm.win_d0 + dw;
-            o = prm.win_o0 + ow;
+            o = prm.win_o0 + (MULTI ? ow * prm.ppt : ow);
             part = rem - dw * prm.win_tpo;
         } else if (prm.tiles_per_desc) {
             di = fastdiv(tile, prm.div_tpd);
             const uint32_t t = tile - di * prm.tiles_per_desc;
             o = fastdiv(t, prm.div_tpo);
             part = t - o * prm.tpo;
+            if (MULTI) o *= prm.ppt;
         } else {
             di = __ldg(prm.tile_desc + tile);
         }
@@ -225,6 +273,27 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
             const uint32_t t = tile - d.tile0;
             o = fastdiv(t, d.div_tpo);
             part = t - o * d.tiles_per_outer;
+        }
+        if (MULTI) {  // several whole planes of one descriptor (uniform groups, one part per plane)
+            const uint32_t o_end = prm.win_span ? prm.win_o_end : d.n_outer;
+            if (o >= o_end) continue;
+            const uint32_t n_units = min(prm.ppt, o_end - o);
+            const char *msrc = prm.ptr[d.src_slot] + d.src_off + o * d.src_outer;
+            char *mdst = prm.ptr[d.dst_slot] + d.dst_off + o * d.dst_outer;
+            if (MODE == kModeRun) {
+                copy_multi<4, kUnroll, kThreads, false>(d, msrc, mdst, n_units, prm.log2_unit);
+            } else if (MODE == kModeRows) {
+                copy_multi<4, kUnroll, kThreads, true>(d, msrc, mdst, n_units, prm.log2_unit);
+            } else {
+                switch (min(d.log2_align, prm.log2_ptr_align)) {
+                case 4: copy_multi<4, kUnroll, kThreads, true>(d, msrc, mdst, n_units, prm.log2_unit); break;
+                case 3: copy_multi<3, 2 * kUnroll, kThreads, true>(d, msrc, mdst, n_units, prm.log2_unit); break;
+                case 2: copy_multi<2, 2 * kUnroll, kThreads, true>(d, msrc, mdst, n_units, prm.log2_unit); break;
+                case 1: copy_multi<1, 2 * kUnroll, kThreads, true>(d, msrc, mdst, n_units, prm.log2_unit); break;
+                default: copy_multi<0, 2 * kUnroll, kThreads, true>(d, msrc, mdst, n_units, prm.log2_unit); break;
+                }
+            }
+            continue;
         }
         const uint32_t row0 = part * d.rows_per_tile;
         if (row0 >= d.rows) continue;  // padding tile of a uniform group

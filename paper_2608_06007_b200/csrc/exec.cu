@@ -336,7 +336,7 @@ extern "C" int tc_plan_descriptors(const tc_plan_t *plan, int group, tc_descript
         o.src_slot = d.src_slot; o.dst_slot = d.dst_slot - static_cast<uint32_t>(g.n_src);
         o.src_slot_step = d.src_slot_step; o.dst_slot_step = d.dst_slot_step;
         o.run_bytes = d.run; o.n0 = d.n0; o.rows = d.rows; o.n_outer = d.n_outer;
-        o.rows_per_tile = d.rows_per_tile; o.tiles_per_outer = d.tiles_per_outer; o.tile0 = d.tile0; o.reserved = 0;
+        o.rows_per_tile = d.rows_per_tile; o.tiles_per_outer = d.tiles_per_outer; o.tile0 = d.tile0; o.planes_per_tile = g.ppt;
     }
     return TC_OK;
 }

@@ -52,6 +52,9 @@ void resident_ctas_for(size_t n_ptrs, int out[3])
     pthread_mutex_unlock(&g_occupancy_mu);
 }
 
+// Tile rows per descriptor: planes, or groups of ppt planes.
+static uint32_t outer_groups(const Group &g) { return (g.descs[0].n_outer + g.ppt - 1) / g.ppt; }
+
 uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *win)
 {
     // Default: one CTA per tile.  The hardware block scheduler then balances the tiles over the
@@ -59,7 +62,7 @@ uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *
     // persistent grid-stride grid.  tuning.ctas_per_sm / max_ctas select a persistent grid
     // (few CTAs suit transfers over the host link).
     uint64_t grid = std::min<uint64_t>(g.n_tiles, 0x7fffffffull);
-    if (win) grid = win->nd ? static_cast<uint64_t>(win->no) * win->nd * (g.tiles_per_desc / g.descs[0].n_outer) : win->no;
+    if (win) grid = win->nd ? static_cast<uint64_t>((win->no + g.ppt - 1) / g.ppt) * win->nd * (g.tiles_per_desc / outer_groups(g)) : win->no;
     if (plan->tuning.ctas_per_sm > 0) {
         int per_sm = g.resident_ctas[mode] > 0 ? g.resident_ctas[mode] : 1;
         per_sm = std::min(per_sm, plan->tuning.ctas_per_sm);
@@ -87,27 +90,40 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     prm.tile_desc = g.d_tile_desc;
     prm.n_tiles = static_cast<uint32_t>(g.n_tiles);
     prm.n_descs = static_cast<uint32_t>(g.descs.size());
-    prm.win_span = prm.win_d0 = prm.win_o0 = prm.win_tpo = prm.tile_base = 0;
+    prm.win_span = prm.win_d0 = prm.win_o0 = prm.win_tpo = prm.win_o_end = prm.tile_base = 0;
+    prm.ppt = g.ppt;
+    prm.log2_unit = g.log2_unit;
     if (win && win->nd == 0) {  // a range of global tile ids
         prm.tile_base = win->d0;
         prm.n_tiles = win->d0 + win->no;
     } else if (win) {
-        prm.win_tpo = g.tiles_per_desc / g.descs[0].n_outer;
+        prm.win_tpo = g.tiles_per_desc / outer_groups(g);
         prm.win_span = win->nd * prm.win_tpo;
         prm.win_d0 = win->d0;
         prm.win_o0 = win->o0;
-        prm.n_tiles = win->no * prm.win_span;
+        prm.win_o_end = win->o0 + win->no;
+        prm.n_tiles = (win->no + g.ppt - 1) / g.ppt * prm.win_span;
     }
     prm.tiles_per_desc = g.tiles_per_desc;
     prm.div_tpd = g.div_tpd;
-    prm.tpo = g.tiles_per_desc ? g.tiles_per_desc / g.descs[0].n_outer : 1;
+    prm.tpo = g.tiles_per_desc ? g.tiles_per_desc / outer_groups(g) : 1;
     prm.div_tpo = make_fastdiv(prm.tpo);
     prm.log2_ptr_align = ptr_align;
     prm.sums = sums;
     for (size_t i = 0; i < g.n_src; i++) prm.ptr[i] = const_cast<char *>(static_cast<const char *>(src[i]));
     for (size_t i = 0; i < g.n_dst; i++) prm.ptr[g.n_src + i] = static_cast<char *>(dst[i]);
     for (size_t i = g.n_src + g.n_dst; i < NPTR; i++) prm.ptr[i] = nullptr;
-    if (sums) {
+    if (g.ppt > 1) {
+        // multi-plane tiles: single-slot pools only, so the table is always in the smallest class
+        if (NPTR != 8 || sums) return fail(TC_ERR_INVALID_ARG, "internal: multi-plane tiles with a large table or checksums");
+        if constexpr (NPTR == 8) {
+            switch (mode) {
+            case kModeRun: tc_copy_kernel<NPTR, kModeRun, false, true><<<grid, Shape<kModeRun>::threads, 0, stream>>>(prm); break;
+            case kModeRows: tc_copy_kernel<NPTR, kModeRows, false, true><<<grid, Shape<kModeRows>::threads, 0, stream>>>(prm); break;
+            default: tc_copy_kernel<NPTR, kModeAny, false, true><<<grid, Shape<kModeAny>::threads, 0, stream>>>(prm); break;
+            }
+        }
+    } else if (sums) {
         if (mode == kModeRun) tc_copy_kernel<NPTR, kModeRun, true><<<grid, Shape<kModeRun>::threads, 0, stream>>>(prm);
         else tc_copy_kernel<NPTR, kModeRows, true><<<grid, Shape<kModeRows>::threads, 0, stream>>>(prm);
     } else

@@ -79,6 +79,10 @@ struct Group {
     bool stage_whole_host_pool = false; // staged MIXED group: the host side is a paged pool
     bool host_is_src = false;          // staged groups: direction (host -> device when true)
     uint32_t tiles_per_desc = 0;      // > 0: every descriptor owns exactly this many tile ids
+    // Planes per tile.  When one plane of a block is much smaller than a tile (few KV heads:
+    // 4-16 KiB), a tile takes ppt consecutive planes of its descriptor, each padded to
+    // 2^log2_unit bytes of the tile's byte space.  1: a tile is (part of) one plane.
+    uint32_t ppt = 1, log2_unit = 0;
     FastDiv div_tpd{0, 0};
     uint64_t n_tiles = 0;
     int64_t payload = 0;

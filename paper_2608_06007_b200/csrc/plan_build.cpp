@@ -209,12 +209,35 @@ static void lower_box(Group &g, Box b, uint32_t tile_bytes)
 // Assign tile ids.  A group whose descriptors all own (nearly) the same number of tiles is
 // "uniform": tile -> descriptor is a division and short descriptors simply own a few empty
 // tile ids.  Otherwise an explicit tile -> descriptor array is built.
-static int finish_group(Group &g)
+static int finish_group(Group &g, uint32_t tile_bytes)
 {
     if (g.descs.empty()) return TC_OK;
+    // Small planes: let a tile span several planes of its descriptor (see Group::ppt).  Needs one
+    // part per plane, planes reached by a byte stride (no table stepping) and a small table.
+    g.ppt = 1;
+    g.log2_unit = 0;
+    {
+        bool can = g.n_src + g.n_dst <= 8;
+        uint32_t max_unit = 0, min_outer = ~0u;
+        for (const Desc &d : g.descs) {
+            if (d.n_outer < 2 || d.tiles_per_outer != 1 || d.src_slot_step || d.dst_slot_step) can = false;
+            max_unit = std::max(max_unit, d.rows * d.run);
+            min_outer = std::min(min_outer, d.n_outer);
+        }
+        if (can && 2ull * max_unit <= tile_bytes) {
+            uint32_t lg = 9;  // units of at least 512 bytes
+            while ((1u << lg) < max_unit) lg++;
+            const uint32_t ppt = std::min({tile_bytes >> lg, min_outer, 64u});
+            if (ppt > 1) {
+                g.ppt = ppt;
+                g.log2_unit = lg;
+            }
+        }
+    }
+    auto outer_groups = [&](const Desc &d) { return (d.n_outer + g.ppt - 1) / g.ppt; };
     uint64_t total = 0, max_t = 0;
     for (const Desc &d : g.descs) {
-        uint64_t t = static_cast<uint64_t>(d.n_outer) * d.tiles_per_outer;
+        uint64_t t = static_cast<uint64_t>(outer_groups(d)) * d.tiles_per_outer;
         total += t;
         max_t = std::max(max_t, t);
     }
@@ -224,7 +247,7 @@ static int finish_group(Group &g)
         if (d.n_outer != g.descs[0].n_outer) same_shape = false;
     if (same_shape && padded < (1ull << 31) && total * 10 >= padded * 8) {
         // uniform: every descriptor is given max tiles_per_outer; extra parts are empty
-        uint32_t tpo = static_cast<uint32_t>(max_t / g.descs[0].n_outer);
+        uint32_t tpo = static_cast<uint32_t>(max_t / outer_groups(g.descs[0]));
         for (size_t i = 0; i < g.descs.size(); i++) {
             Desc &d = g.descs[i];
             d.tiles_per_outer = tpo;
@@ -236,6 +259,10 @@ static int finish_group(Group &g)
         g.n_tiles = padded;
         return TC_OK;
     }
+    g.ppt = 1;  // listed groups keep one plane per tile
+    g.log2_unit = 0;
+    total = 0;
+    for (const Desc &d : g.descs) total += static_cast<uint64_t>(d.n_outer) * d.tiles_per_outer;
     if (total >= (1ull << 31)) return fail(TC_ERR_INVALID_ARG, "plan has %llu tiles (limit 2^31)", (unsigned long long)total);
     g.tile_desc.resize(total);
     uint64_t t0 = 0;
@@ -829,7 +856,7 @@ int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
         const bool kv_kind = spec->kind != TC_WEIGHTS;
         if (kv_kind && !(spec->flags & TC_PLAN_STAGED) && spec->tuning.tile_order != 1)
             std::stable_sort(g.descs.begin(), g.descs.end(), [](const Desc &a, const Desc &b) { return a.dst_off < b.dst_off; });
-        if ((rc = finish_group(g))) return rc;
+        if ((rc = finish_group(g, tile_bytes))) return rc;
     }
     if ((spec->flags & TC_PLAN_SAME_POOL) && spec->kind != TC_KV_MIGRATE)
         return fail(TC_ERR_KIND, "TC_PLAN_SAME_POOL applies to TC_KV_MIGRATE plans only");

@@ -112,6 +112,79 @@ def test_pack_unpack_all_layouts(pool_l, packed_l, slots, tile):
     assert np.array_equal(fresh.result(), want_pool)
 
 
+@pytest.mark.parametrize("H,L", [(1, 5), (2, 3), (4, 6)])
+@pytest.mark.parametrize("pool_l,packed_l", list(itertools.product(LAYOUTS, LAYOUTS)))
+def test_few_kv_heads_several_planes_per_tile(H, L, pool_l, packed_l):
+    """Planes of 4-16 KiB (1, 2, 4 KV heads): a tile moves several planes of one block.  L is
+    chosen so that the last tile row of every block is only partly filled; ragged last blocks,
+    an empty request, block strides with padding, a pointer shifted by 8 bytes (narrow-vector
+    build), and staged windows whose plane ranges are not multiples of the planes per tile."""
+    rng = np.random.default_rng(40 + H)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=L, NB=70, B=16, H=H, D=128, E=2, T=(300, 16, 0, 37, 5, 512), pad_blocks=256)
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, pool_l, stride, planes_of(pool, L * 2), T, off, bt, packed_l, want, threads=8)
+    pl = tc.pool(pool_l, NB, 1, plane_stride=NB * stride, block_stride=stride)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_src=bt))
+    assert plan.descriptors(0)[0].planes_per_tile == min(8 // H, 2 * L)
+    d_pool = Guarded(pool.size, init=pool)
+    out = Guarded(want.size)
+    tc.tc_kv_pack(plan, [d_pool.ptr()], [out.ptr()])
+    assert np.array_equal(out.result(), want)
+    shifted = Guarded(want.size, shift=8)                      # 8-byte aligned destination: the narrow-vector build
+    tc.tc_kv_pack(plan, [d_pool.ptr()], [shifted.ptr()])
+    assert np.array_equal(shifted.result(), want)
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, pool_l, stride, planes_of(want_pool, L * 2), T, off, bt2, packed_l, want, threads=8)
+    plan2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_dst=bt2))
+    fresh = Guarded(pool.size)
+    tc.tc_kv_unpack(plan2, [out.ptr()], [fresh.ptr()])
+    assert np.array_equal(fresh.result(), want_pool)
+    want_mig = np.full_like(pool, 0xA5)
+    oracle.kv_migrate(shape, pool_l, stride, planes_of(pool, L * 2), pool_l, stride, planes_of(want_mig, L * 2), T, off, bt, bt2, threads=8)
+    mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl, T=T, bt_off=off, bt_src=bt, bt_dst=bt2, tuning=dict(tile_order=1)))
+    moved = Guarded(pool.size)
+    tc.tc_kv_pack(mig, [d_pool.ptr()], [moved.ptr()])
+    assert np.array_equal(moved.result(), want_mig)
+    # staged: the copy-engine path launches windows of planes
+    host = torch.full((want.size,), 0x77, dtype=torch.uint8).pin_memory()
+    sp = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_src=bt, flags=tc.TC_PLAN_STAGED))
+    su = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_dst=bt2, flags=tc.TC_PLAN_STAGED))
+    refill = Guarded(pool.size)
+    tc.tc_kv_pack(sp, [d_pool.ptr()], [host])
+    tc.tc_kv_unpack(su, [host], [refill.ptr()])
+    torch.cuda.synchronize()
+    assert np.array_equal(host.numpy(), want)
+    assert np.array_equal(refill.result(), want_pool)
+
+
+def test_staged_windows_cut_inside_a_tile_row_of_planes():
+    """Two KV heads, six planes, four planes per tile; one request of 184 MB is staged in windows
+    of two planes (30.7 MB each), so every window starts and ends inside a tile row."""
+    rng = np.random.default_rng(47)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=3, NB=3800, B=16, H=2, D=128, E=2, T=(60000, 100))
+    L = shape[0]
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, L * 2), T, off, bt, oracle.HND, want, threads=8)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride)
+    sp = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_src=bt, flags=tc.TC_PLAN_STAGED))
+    assert sp.descriptors(0)[0].planes_per_tile == 4
+    segs = sp.segments(0)
+    assert [(sg.outer0, sg.n_outer) for sg in segs[:3]] == [(0, 2), (2, 2), (4, 2)]
+    d_pool = dev(pool)
+    host = torch.full((want.size,), 0x77, dtype=torch.uint8).pin_memory()
+    tc.tc_kv_pack(sp, [d_pool], [host])
+    torch.cuda.synchronize()
+    assert np.array_equal(host.numpy(), want)
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(want_pool, L * 2), T, off, bt2, oracle.HND, want, threads=8)
+    su = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_dst=bt2, flags=tc.TC_PLAN_STAGED))
+    fresh = Guarded(pool.size)
+    tc.tc_kv_unpack(su, [host], [fresh.ptr()])
+    assert np.array_equal(fresh.result(), want_pool)
+
+
 @pytest.mark.parametrize("tune", [dict(tile_order=1), dict(ctas_per_sm=2), dict(max_ctas=7), dict(tile_bytes=65536), dict(tile_bytes=1024, ctas_per_sm=1, tile_order=1)])
 def test_tuning_knobs_change_the_schedule_not_the_bytes(tune):
     rng = np.random.default_rng(29)

@@ -504,6 +504,31 @@ def test_head_slice_and_layer_major_lowering_match_oracle(pool_l, packed_l, orde
     assert e.value.status == tc.TC_ERR_INVALID_ARG
 
 
+def test_small_planes_share_a_tile():
+    """Few KV heads: one plane of a block is 4-16 KiB, so a tile takes several planes of its
+    descriptor (planes_per_tile); pools with one pointer per plane keep one plane per tile."""
+    T = np.array([40, 16, 5], dtype=np.int64)
+    for H, want_ppt in ((1, 8), (2, 4), (4, 2), (8, 1)):
+        shape = (16, 16, H, 128, 2)                               # 32 planes of H * 4 KiB per block
+        off = np.concatenate([[0], np.cumsum((T + 15) // 16)])
+        bt = np.arange(off[-1], dtype=np.int32)
+        nb = int(off[-1])
+        chunk = 16 * H * 128 * 2
+        one = tc.pool(tc.TC_NHD, nb, 1, plane_stride=nb * chunk)
+        plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=one, dst_pool=one, T=T, bt_off=off, bt_src=bt, bt_dst=bt[::-1].copy(), flags=HOST))
+        ds, st = plan.descriptors(0), plan.stats()
+        assert all(d.planes_per_tile == want_ppt for d in ds)
+        assert st.n_tiles[0] == len(ds) * (32 // want_ppt) and st.payload_bytes[0] == int(T.sum()) * 32 * H * 256
+        per_plane = tc.pool(tc.TC_NHD, nb, 32)
+        plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=per_plane, dst_pool=per_plane, T=T, bt_off=off, bt_src=bt, bt_dst=bt[::-1].copy(), flags=HOST))
+        assert all(d.planes_per_tile == 1 for d in plan.descriptors(0))
+    # L = 3: six planes, tiles of four -> two tile rows per descriptor, the second one half full
+    shape = (3, 16, 2, 128, 2)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=tc.pool(tc.TC_NHD, 6, 1, plane_stride=6 * 8192), packed_layout=tc.TC_HND,
+                                        T=np.array([96]), bt_off=np.array([0, 6]), bt_src=np.arange(6, dtype=np.int32), flags=HOST))
+    assert plan.descriptors(0)[0].planes_per_tile == 4 and plan.stats().n_tiles[0] == 6 * 2
+
+
 def test_same_pool_compaction_lowering_and_its_overlap_check():
     """Defragmentation: the requests' blocks move to the low block ids of the same pool."""
     rng = np.random.default_rng(6)
