@@ -160,19 +160,27 @@ __device__ __forceinline__ void copy_rows(const Desc &d, const char *src, char *
 }
 
 // A tile of n_units consecutive planes of one descriptor (small planes, see Group::ppt).  The
-// tile's byte space gives every plane 2^log2_unit bytes, of which the first rows * run are real;
-// plane k sits k * outer bytes behind plane 0 on each side.  ROWS: decode rows inside a plane,
-// else every plane is one run.  src / dst point at row 0 of the tile's first plane.
-template <int LOGV, int U, int kThreads, bool ROWS>
-__device__ __forceinline__ void copy_multi(const Desc &d, const char *src, char *dst, uint32_t n_units, uint32_t log2_unit)
+// tile's byte space gives every plane 2^log2_unit bytes, of which the first rows * run are real.
+// Plane k of the tile starts at table[slot + (o + k) * slot_step] + off + (o + k) * outer on
+// each side: a byte stride for single-pointer pools, another table entry for pools with one
+// pointer per plane (a warp never straddles planes - they own at least 512 bytes of the byte
+// space - so that lookup has one index per warp).  ROWS: decode rows inside a plane, else
+// every plane is one run.  STEP: some pool of the group has one pointer per plane; without it
+// both base pointers are read once per tile.
+template <int LOGV, int U, int kThreads, bool ROWS, bool STEP, int NPTR>
+__device__ __forceinline__ void copy_multi(const Desc &d, const Params<NPTR> &prm, uint32_t o, uint32_t n_units)
 {
     using V = typename VecOf<LOGV>::type;
+    const uint32_t log2_unit = prm.log2_unit;
     const uint32_t unit_bytes = d.rows * d.run, mask = (1u << log2_unit) - 1;
     const uint32_t nbytes = n_units << log2_unit;
     const uint32_t run = d.run, n0 = d.n0;
     const FastDiv div_run = d.div_run, div_n0 = d.div_n0;
     const uint32_t ss0 = d.src_s0, ss1 = d.src_s1, ds0 = d.dst_s0, ds1 = d.dst_s1;
-    const long long src_outer = d.src_outer, dst_outer = d.dst_outer;
+    const long long src_outer = d.src_outer, dst_outer = d.dst_outer, src_off = d.src_off, dst_off = d.dst_off;
+    const uint32_t sslot = d.src_slot, dslot = d.dst_slot, sstep = d.src_slot_step, dstep = d.dst_slot_step;
+    const char *src_base = STEP ? nullptr : prm.ptr[sslot] + src_off;
+    char *dst_base = STEP ? nullptr : prm.ptr[dslot] + dst_off;
 #pragma unroll 1
     for (uint32_t base = threadIdx.x << LOGV; base < nbytes; base += (kThreads * U) << LOGV) {
         V val[U];
@@ -180,7 +188,7 @@ __device__ __forceinline__ void copy_multi(const Desc &d, const char *src, char 
 #pragma unroll
         for (int u = 0; u < U; u++) {
             const uint32_t byte = base + ((u * kThreads) << LOGV);
-            const uint32_t k = byte >> log2_unit, w = byte & mask;
+            const uint32_t k = o + (byte >> log2_unit), w = byte & mask;
             if (byte < nbytes && w < unit_bytes) {
                 uint32_t so = w;
                 doff[u] = w;
@@ -192,14 +200,14 @@ __device__ __forceinline__ void copy_multi(const Desc &d, const char *src, char 
                     doff[u] = i1 * ds1 + i0 * ds0 + col;
                     so = i1 * ss1 + i0 * ss0 + col;
                 }
-                val[u] = ld_stream<V>(src + k * src_outer + so);
+                val[u] = ld_stream<V>((STEP ? prm.ptr[sslot + k * sstep] + src_off : src_base) + k * src_outer + so);
             }
         }
 #pragma unroll
         for (int u = 0; u < U; u++) {
             const uint32_t byte = base + ((u * kThreads) << LOGV);
-            const uint32_t k = byte >> log2_unit, w = byte & mask;
-            if (byte < nbytes && w < unit_bytes) st_stream<V>(dst + k * dst_outer + doff[u], val[u]);
+            const uint32_t k = o + (byte >> log2_unit), w = byte & mask;
+            if (byte < nbytes && w < unit_bytes) st_stream<V>((STEP ? prm.ptr[dslot + k * dstep] + dst_off : dst_base) + k * dst_outer + doff[u], val[u]);
         }
     }
 }
@@ -223,7 +231,9 @@ __device__ __forceinline__ void copy_run16(const char *src, char *dst, uint32_t 
     }
 }
 
-template <int NPTR, int MODE, bool CHECK = false, bool MULTI = false>
+// MULTI: 0 one plane per tile; 1 several planes per tile, planes a byte stride apart; 2 the
+// same with a pool that has one pointer per plane.
+template <int NPTR, int MODE, bool CHECK = false, int MULTI = 0>
 __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) tc_copy_kernel(const __grid_constant__ Params<NPTR> prm)
 {
     constexpr int kThreads = Shape<MODE>::threads, kUnroll = Shape<MODE>::unroll;
@@ -278,19 +288,17 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
             const uint32_t o_end = prm.win_span ? prm.win_o_end : d.n_outer;
             if (o >= o_end) continue;
             const uint32_t n_units = min(prm.ppt, o_end - o);
-            const char *msrc = prm.ptr[d.src_slot] + d.src_off + o * d.src_outer;
-            char *mdst = prm.ptr[d.dst_slot] + d.dst_off + o * d.dst_outer;
             if (MODE == kModeRun) {
-                copy_multi<4, kUnroll, kThreads, false>(d, msrc, mdst, n_units, prm.log2_unit);
+                copy_multi<4, kUnroll, kThreads, false, MULTI == 2>(d, prm, o, n_units);
             } else if (MODE == kModeRows) {
-                copy_multi<4, kUnroll, kThreads, true>(d, msrc, mdst, n_units, prm.log2_unit);
+                copy_multi<4, kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units);
             } else {
                 switch (min(d.log2_align, prm.log2_ptr_align)) {
-                case 4: copy_multi<4, kUnroll, kThreads, true>(d, msrc, mdst, n_units, prm.log2_unit); break;
-                case 3: copy_multi<3, 2 * kUnroll, kThreads, true>(d, msrc, mdst, n_units, prm.log2_unit); break;
-                case 2: copy_multi<2, 2 * kUnroll, kThreads, true>(d, msrc, mdst, n_units, prm.log2_unit); break;
-                case 1: copy_multi<1, 2 * kUnroll, kThreads, true>(d, msrc, mdst, n_units, prm.log2_unit); break;
-                default: copy_multi<0, 2 * kUnroll, kThreads, true>(d, msrc, mdst, n_units, prm.log2_unit); break;
+                case 4: copy_multi<4, kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units); break;
+                case 3: copy_multi<3, 2 * kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units); break;
+                case 2: copy_multi<2, 2 * kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units); break;
+                case 1: copy_multi<1, 2 * kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units); break;
+                default: copy_multi<0, 2 * kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units); break;
                 }
             }
             continue;

@@ -114,13 +114,23 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     for (size_t i = 0; i < g.n_dst; i++) prm.ptr[g.n_src + i] = static_cast<char *>(dst[i]);
     for (size_t i = g.n_src + g.n_dst; i < NPTR; i++) prm.ptr[i] = nullptr;
     if (g.ppt > 1) {
-        // multi-plane tiles: single-slot pools only, so the table is always in the smallest class
-        if (NPTR != 8 || sums) return fail(TC_ERR_INVALID_ARG, "internal: multi-plane tiles with a large table or checksums");
-        if constexpr (NPTR == 8) {
-            switch (mode) {
-            case kModeRun: tc_copy_kernel<NPTR, kModeRun, false, true><<<grid, Shape<kModeRun>::threads, 0, stream>>>(prm); break;
-            case kModeRows: tc_copy_kernel<NPTR, kModeRows, false, true><<<grid, Shape<kModeRows>::threads, 0, stream>>>(prm); break;
-            default: tc_copy_kernel<NPTR, kModeAny, false, true><<<grid, Shape<kModeAny>::threads, 0, stream>>>(prm); break;
+        // multi-plane tiles: KV groups only (two pools of at most L*2 pointers each)
+        if (NPTR == TC_MAX_TABLE_SLOTS || sums) return fail(TC_ERR_INVALID_ARG, "internal: multi-plane tiles with a large table or checksums");
+        if constexpr (NPTR != TC_MAX_TABLE_SLOTS) {
+            bool step = false;  // some pool has one pointer per plane
+            for (const Desc &d : g.descs) step = step || d.src_slot_step || d.dst_slot_step;
+            if (step) {
+                switch (mode) {
+                case kModeRun: tc_copy_kernel<NPTR, kModeRun, false, 2><<<grid, Shape<kModeRun>::threads, 0, stream>>>(prm); break;
+                case kModeRows: tc_copy_kernel<NPTR, kModeRows, false, 2><<<grid, Shape<kModeRows>::threads, 0, stream>>>(prm); break;
+                default: tc_copy_kernel<NPTR, kModeAny, false, 2><<<grid, Shape<kModeAny>::threads, 0, stream>>>(prm); break;
+                }
+            } else {
+                switch (mode) {
+                case kModeRun: tc_copy_kernel<NPTR, kModeRun, false, 1><<<grid, Shape<kModeRun>::threads, 0, stream>>>(prm); break;
+                case kModeRows: tc_copy_kernel<NPTR, kModeRows, false, 1><<<grid, Shape<kModeRows>::threads, 0, stream>>>(prm); break;
+                default: tc_copy_kernel<NPTR, kModeAny, false, 1><<<grid, Shape<kModeAny>::threads, 0, stream>>>(prm); break;
+                }
             }
         }
     } else if (sums) {

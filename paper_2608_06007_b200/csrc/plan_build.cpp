@@ -213,14 +213,14 @@ static int finish_group(Group &g, uint32_t tile_bytes)
 {
     if (g.descs.empty()) return TC_OK;
     // Small planes: let a tile span several planes of its descriptor (see Group::ppt).  Needs one
-    // part per plane, planes reached by a byte stride (no table stepping) and a small table.
+    // part per plane and a pointer table of at most 400 entries (the kernel classes built for it).
     g.ppt = 1;
     g.log2_unit = 0;
     {
-        bool can = g.n_src + g.n_dst <= 8;
+        bool can = g.n_src + g.n_dst <= 400;
         uint32_t max_unit = 0, min_outer = ~0u;
         for (const Desc &d : g.descs) {
-            if (d.n_outer < 2 || d.tiles_per_outer != 1 || d.src_slot_step || d.dst_slot_step) can = false;
+            if (d.n_outer < 2 || d.tiles_per_outer != 1) can = false;
             max_unit = std::max(max_unit, d.rows * d.run);
             min_outer = std::min(min_outer, d.n_outer);
         }

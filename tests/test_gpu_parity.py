@@ -146,6 +146,21 @@ def test_few_kv_heads_several_planes_per_tile(H, L, pool_l, packed_l):
     moved = Guarded(pool.size)
     tc.tc_kv_pack(mig, [d_pool.ptr()], [moved.ptr()])
     assert np.array_equal(moved.result(), want_mig)
+    # the same pools addressed through one pointer per plane
+    per_plane = tc.pool(pool_l, NB, L * 2, block_stride=stride, slot_bytes=pool.size // (L * 2))
+    pp = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=per_plane, packed_layout=packed_l, T=T, bt_off=off, bt_src=bt))
+    assert pp.descriptors(0)[0].planes_per_tile == min(8 // H, 2 * L)
+    out2 = Guarded(want.size)
+    tc.tc_kv_pack(pp, pool_tables(d_pool, L * 2, "planes"), [out2.ptr()])
+    assert np.array_equal(out2.result(), want)
+    mp = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=per_plane, dst_pool=pl, T=T, bt_off=off, bt_src=bt, bt_dst=bt2))
+    moved2 = Guarded(pool.size)
+    tc.tc_kv_pack(mp, pool_tables(d_pool, L * 2, "planes"), [moved2.ptr()])
+    assert np.array_equal(moved2.result(), want_mig)
+    up2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=per_plane, packed_layout=packed_l, T=T, bt_off=off, bt_dst=bt2))
+    fresh2 = Guarded(pool.size)
+    tc.tc_kv_unpack(up2, [out.ptr()], pool_tables(fresh2, L * 2, "planes"))
+    assert np.array_equal(fresh2.result(), want_pool)
     # staged: the copy-engine path launches windows of planes
     host = torch.full((want.size,), 0x77, dtype=torch.uint8).pin_memory()
     sp = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_src=bt, flags=tc.TC_PLAN_STAGED))

@@ -506,7 +506,7 @@ def test_head_slice_and_layer_major_lowering_match_oracle(pool_l, packed_l, orde
 
 def test_small_planes_share_a_tile():
     """Few KV heads: one plane of a block is 4-16 KiB, so a tile takes several planes of its
-    descriptor (planes_per_tile); pools with one pointer per plane keep one plane per tile."""
+    descriptor (planes_per_tile), in pools with one pointer and in pools with a pointer per plane."""
     T = np.array([40, 16, 5], dtype=np.int64)
     for H, want_ppt in ((1, 8), (2, 4), (4, 2), (8, 1)):
         shape = (16, 16, H, 128, 2)                               # 32 planes of H * 4 KiB per block
@@ -521,7 +521,7 @@ def test_small_planes_share_a_tile():
         assert st.n_tiles[0] == len(ds) * (32 // want_ppt) and st.payload_bytes[0] == int(T.sum()) * 32 * H * 256
         per_plane = tc.pool(tc.TC_NHD, nb, 32)
         plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=per_plane, dst_pool=per_plane, T=T, bt_off=off, bt_src=bt, bt_dst=bt[::-1].copy(), flags=HOST))
-        assert all(d.planes_per_tile == 1 for d in plan.descriptors(0))
+        assert all(d.planes_per_tile == want_ppt for d in plan.descriptors(0))
     # L = 3: six planes, tiles of four -> two tile rows per descriptor, the second one half full
     shape = (3, 16, 2, 128, 2)
     plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=tc.pool(tc.TC_NHD, 6, 1, plane_stride=6 * 8192), packed_layout=tc.TC_HND,
