@@ -639,6 +639,7 @@ def test_random_geometries_on_the_device(seed):
     shift = int(rng.choice([0, 0, 0, E, 16]))
     tile = int(rng.choice([0, 0, 1024, 8192]))
     pool_l, other_l = int(rng.integers(0, 2)), int(rng.integers(0, 2))
+    slots = str(rng.choice(["planes", "one"]))             # one pointer per plane, or one pointer and a plane stride
     shape = (L, B, H, D, E)
     T = np.array(T, dtype=np.int64)
     off = np.concatenate([[0], np.cumsum((T + B - 1) // B)]).astype(np.int64)
@@ -648,20 +649,24 @@ def test_random_geometries_on_the_device(seed):
     bt = rng.permutation(NB)[:off[-1]].astype(np.int32)
     bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
     tune = dict(tile_bytes=tile) if tile else None
-    pl = tc.pool(pool_l, NB, L * 2, block_stride=stride, slot_bytes=NB * stride)
+    def mkpool(layout):
+        if slots == "planes":
+            return tc.pool(layout, NB, L * 2, block_stride=stride, slot_bytes=NB * stride)
+        return tc.pool(layout, NB, 1, plane_stride=NB * stride, block_stride=stride, slot_bytes=L * 2 * NB * stride)
+    pl = mkpool(pool_l)
     want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
     oracle.kv_pack(shape, pool_l, stride, planes_of(pool, L * 2), T, off, bt, other_l, want)
     d_pool = Guarded(pool.size, init=pool, shift=shift)
     out = Guarded(max(want.size, 1), shift=shift)
     plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=other_l, T=T, bt_off=off, bt_src=bt, tuning=tune))
-    tc.tc_kv_pack(plan, pool_tables(d_pool, L * 2, "planes"), [out.ptr()])
+    tc.tc_kv_pack(plan, pool_tables(d_pool, L * 2, slots), [out.ptr()])
     assert np.array_equal(out.result()[:want.size], want)
     want_pool = np.full_like(pool, 0xA5)
     oracle.kv_migrate(shape, pool_l, stride, planes_of(pool, L * 2), other_l, stride, planes_of(want_pool, L * 2), T, off, bt, bt2)
-    pl2 = tc.pool(other_l, NB, L * 2, block_stride=stride, slot_bytes=NB * stride)
+    pl2 = mkpool(other_l)
     mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl2, T=T, bt_off=off, bt_src=bt, bt_dst=bt2, tuning=tune))
     fresh = Guarded(pool.size, shift=shift)
-    tc.tc_kv_pack(mig, pool_tables(d_pool, L * 2, "planes"), pool_tables(fresh, L * 2, "planes"))
+    tc.tc_kv_pack(mig, pool_tables(d_pool, L * 2, slots), pool_tables(fresh, L * 2, slots))
     assert np.array_equal(fresh.result(), want_pool)
 
 
