@@ -245,7 +245,12 @@ typedef struct {
 
 /* Optional knobs; 0 everywhere = the library's defaults. */
 typedef struct {
-    int32_t tile_bytes;   /* target bytes per tile (one CTA iteration) */
+    int32_t tile_bytes;   /* target bytes per tile, the work of one CTA: a power of two in
+                             [512, 1 MiB], default 32 KiB (64 KiB for TC_PLAN_CHECKSUM plans).  A
+                             tile is a row range of one plane of one descriptor; it may reach
+                             1.5 x tile_bytes where that avoids a sliver, and it takes several
+                             consecutive planes of a KV block when one plane is at most half
+                             of tile_bytes (few KV heads). */
     int32_t ctas_per_sm;  /* > 0: a persistent grid-stride grid of this many CTAs per SM instead
                              of one CTA per tile */
     int32_t max_ctas;     /* > 0: cap on the grid (persistent grid-stride loop) */
