@@ -765,7 +765,7 @@ def kv_shapes(args, tc, torch, stream):
     K = wl.KVShape
     cases = [("8 KV heads (headline shape)", K(32, 16, 8, 128)), ("4 KV heads", K(28, 16, 4, 128)), ("2 KV heads", K(28, 16, 2, 128)),
              ("1 KV head", K(32, 16, 1, 128)), ("32 heads of 64", K(32, 16, 32, 64)), ("block 128", K(32, 128, 8, 128))]
-    for label, shape in cases[:2 if args.small else None]:
+    for label, shape in ([cases[1], cases[3]] if args.small else cases):
         s = shape.tuple
         NB = int(((1 if args.small else 8) << 30) // shape.block_bytes)
         WB = NB // 2
@@ -785,7 +785,7 @@ def kv_shapes(args, tc, torch, stream):
         res = {"plane_KiB": shape.chunk_bytes // 1024, "planes_per_tile": int(mig.descriptors(0)[0].planes_per_tile), "payload_bytes": payload}
         for name, fn in (("pack", lambda: tc.tc_kv_pack(pk, [poolA], [Q], sp)), ("unpack", lambda: tc.tc_kv_unpack(up, [Q], [poolB], sp)),
                          ("migrate", lambda: tc.tc_kv_pack(mig, [poolA], [poolB], sp))):
-            res["GBps_" + name] = 2 * payload / (b2b_ms(torch, stream, fn, reps=8, warm=3) * 1e-3) / GB
+            res["GBps_" + name] = 2 * payload / (b2b_ms(torch, stream, fn, reps=1 if args.small else 8, warm=1 if args.small else 3) * 1e-3) / GB
         out[label + f" L{shape.L} B{shape.B} H{shape.H} D{shape.D}"] = res
         for p_ in (pk, up, mig):
             p_.destroy()
@@ -802,6 +802,9 @@ def run_extras(args, tc, torch, stream):
     out = {}
     sp = stream.cuda_stream
     u8 = dict(dtype=torch.uint8, device="cuda")
+    if args.only_kv_shapes:  # profiler runs: just the KV geometries, a few GB on the device
+        out["rows a1-a3 on other KV geometries (8 GiB pools, first wave)"] = kv_shapes(args, tc, torch, stream)
+        return out
     # ---- configs[0]: 1.4 MB, launch-latency bound: microseconds and plans per second
     shape, NB1, src1, dst1 = wl.config1()
     pool1 = torch.empty(2 * NB1 * shape.chunk_bytes, **u8)
@@ -1014,6 +1017,7 @@ def main():
     ap.add_argument("--tile-bytes", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary workloads (configs[3], configs[4])")
+    ap.add_argument("--only-kv-shapes", action="store_true", help="of the secondary workloads run only the KV geometries (profiler captures)")
     ap.add_argument("--host-pool-blocks", type=int, default=8192, help="configs[4]: pinned host pool size in 2 MiB blocks")
     ap.add_argument("--burst-steps", type=int, default=10, help="configs[4]: scheduler steps timed (the workload has 200)")
     ap.add_argument("--cold-layers", type=int, default=8, help="cold-path extra: layers of the checkpoint written to a file (8: 4.0 GB)")
