@@ -53,8 +53,10 @@ extern "C" int tc_kv_pack_noalloc(const tc_plan_spec_t *spec, const void *const 
         return fail(TC_ERR_KIND, "tc_kv_pack_noalloc needs a PACK, MIGRATE or MIXED spec (kind %d given)", spec->kind);
     if (spec->deadline_ns && now_ns() > spec->deadline_ns) return fail(TC_ERR_DEADLINE, "deadline passed before the call");
     if (spec->flags & TC_PLAN_STAGED) return fail(TC_ERR_INVALID_ARG, "tc_kv_pack_noalloc does not stage: the staging ring is allocated device memory");
+    if (spec->flags & TC_PLAN_HOST_ONLY) return fail(TC_ERR_INVALID_ARG, "TC_PLAN_HOST_ONLY asks for a plan that is not executed; tc_kv_pack_noalloc always executes");
     tc_plan plan;  // lives on the host for the duration of this call only
     plan.kind = spec->kind;
+    plan.flags = spec->flags;
     plan.trace_id = spec->trace_id;
     plan.deadline_ns = spec->deadline_ns;
     plan.tuning = spec->tuning;
@@ -66,15 +68,17 @@ extern "C" int tc_kv_pack_noalloc(const tc_plan_spec_t *spec, const void *const 
     }
     if (rc != TC_OK) return rc;
     Group &g = plan.group[0];
+    // The device is resolved before anything else: execute() checks it, also for a request that
+    // moves nothing (R = 0, or every T_r = 0), which is a legal no-op returning TC_OK.
+    cudaError_t e = cudaGetDevice(&plan.device);
+    if (e != cudaSuccess) return cuda_fail(e, "querying the current device");
+    if (plan.device < 0 || plan.device >= kMaxDevices) return fail(TC_ERR_INVALID_ARG, "device ordinal %d is not supported", plan.device);
     if (g.n_tiles == 0) return execute(&plan, 0, src_bases, n_src, dst_bases, n_dst, stream);
     const size_t desc_bytes = g.descs.size() * sizeof(Desc);
     const size_t tile_bytes = g.tile_desc.size() * sizeof(uint32_t);
     if (desc_bytes + tile_bytes > TC_NOALLOC_SCRATCH_BYTES)
         return fail(TC_ERR_TOO_LARGE, "the call needs %zu bytes of descriptors and tiles; tc_kv_pack_noalloc holds at most %u: split the request or use tc_plan_create",
                     desc_bytes + tile_bytes, TC_NOALLOC_SCRATCH_BYTES);
-    cudaError_t e = cudaGetDevice(&plan.device);
-    if (e != cudaSuccess) return cuda_fail(e, "querying the current device");
-    if (plan.device < 0 || plan.device >= kMaxDevices) return fail(TC_ERR_INVALID_ARG, "device ordinal %d is not supported", plan.device);
     NoallocDevice dev;
     if ((rc = noalloc_setup(plan.device, &dev)) != TC_OK) return rc;
     plan.sm_count = dev.sm_count;

@@ -659,6 +659,7 @@ static int build_weights(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t til
     g.n_src = 1;
     g.n_dst = static_cast<size_t>(n_dst);
     std::vector<std::vector<Span>> spans(static_cast<size_t>(n_dst));
+    std::vector<uint8_t> verify_rows(static_cast<size_t>(n_dst), 0);  // slots that need the exact check
     std::vector<Box> boxes;
     boxes.reserve(static_cast<size_t>(w.n_tensors));
     for (int64_t i = 0; i < w.n_tensors; i++) {
@@ -716,6 +717,22 @@ static int build_weights(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t til
         if (slot_extent < 0) return fail(TC_ERR_INVALID_ARG, "tensor %lld: dst_bytes is required when a rule sets dst_off or dst_stride", (long long)i);
         if (hi > slot_extent) return fail(TC_ERR_BOUNDS, "tensor %lld: writes up to byte %lld of a %lld-byte destination", (long long)i, (long long)hi, (long long)slot_extent);
         spans[static_cast<size_t>(slot)].push_back(Span{rule.dst_off, hi, i});
+        if (!tight) {
+            // A tensor may also overlap ITSELF: rows or elements closer together than they are
+            // long.  Sufficient for disjointness: taken by ascending stride, every dimension
+            // steps over the whole extent of the dimensions inside it.  Strides that do not nest
+            // this way (interleavings) are decided by the exact check below.
+            std::pair<int64_t, int64_t> by_stride[4];
+            int nd = 0;
+            for (int m = 0; m < 4; m++)
+                if (ext[m] > 1) by_stride[nd++] = {dstr[m], ext[m]};
+            std::sort(by_stride, by_stride + nd);
+            int64_t inner = t.elem_bytes;
+            for (int k = 0; k < nd; k++) {
+                if (by_stride[k].first < inner) verify_rows[static_cast<size_t>(slot)] = 1;
+                inner += (by_stride[k].second - 1) * by_stride[k].first;
+            }
+        }
         Box b;
         b.run = t.elem_bytes;
         b.tag = static_cast<uint32_t>(i);
@@ -727,12 +744,13 @@ static int build_weights(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t til
         for (int m = 3; m >= 0; m--) b.dims.push_back(Dim{ext[m], sstr[m], dstr[m]});
         boxes.push_back(std::move(b));
     }
-    // exactly-once writes: bounding spans of one slot may not intersect.  (Interleaved strided
-    // destinations whose bounding spans intersect are checked row by row below.)
+    // exactly-once writes: bounding spans of one slot may not intersect and no tensor may overlap
+    // itself.  (Interleaved strided destinations, whose bounding spans intersect or whose strides
+    // do not nest, are checked row by row below.)
     for (size_t s = 0; s < spans.size(); s++) {
         auto &v = spans[s];
         std::sort(v.begin(), v.end(), [](const Span &a, const Span &b) { return a.lo < b.lo; });
-        bool clash = false;
+        bool clash = verify_rows[s] != 0;
         for (size_t k = 1; k < v.size(); k++)
             if (v[k].lo < v[k - 1].hi) clash = true;
         if (!clash) continue;

@@ -418,6 +418,45 @@ def test_weights_full_and_every_shard(variant):
                 assert np.array_equal(outs[i].result(), want[i]), (ck.names[i], world, rank)
 
 
+def test_tp_resharding_8_to_2_and_2_to_8_on_the_gpu():
+    """A checkpoint saved as W shard blobs, loaded at another TP degree.  8 -> 2: rank r' of 2
+    gathers four source shards into one buffer (dst_off / dst_stride windows, one plan per source
+    blob).  2 -> 8: rank r' of 8 takes a quarter of one source shard.  The expected bytes are the
+    oracle's direct shard of the FULL tensor at the new degree."""
+    rng = np.random.default_rng(8)
+    shp, E = (512, 768), 2                                 # rows of 1536 B; eighths are 192 B pieces
+    full = rng.integers(0, 256, shp[0] * shp[1] * E, dtype=np.uint8)
+    for dim in (0, 1):
+        def shard(rank, world):
+            out = np.zeros(full.size // world, dtype=np.uint8)
+            oracle.weights([0], [E], [[shp[0], shp[1], 1, 1]], [dim], rank, world, full, [out])
+            return out
+        sshape = lambda world: [shp[0] // world if dim == 0 else shp[0], shp[1] // world if dim == 1 else shp[1], 1, 1]
+        for r2 in range(2):                                # 8 -> 2
+            want = shard(r2, 2)
+            got = Guarded(want.size, fill=0xEE)
+            d2, s8 = sshape(2), sshape(8)
+            keep = []
+            for k in range(4):
+                src_blob = shard(4 * r2 + k, 8)
+                off = k * src_blob.size if dim == 0 else k * s8[1] * E
+                spec = tc.weights_spec([0], [src_blob.size], [E], [2], [s8], blob_bytes=src_blob.size, dst_slot=[0], dst_off=[off],
+                                       dst_stride=[[d2[1] * E, E, E, E]], n_dst=1, dst_bytes=[want.size], tuning=dict(tile_bytes=4096))
+                plan = tc.tc_plan_create(spec)
+                d_src = dev(src_blob)
+                tc.tc_weights_materialize(plan, d_src, [got.ptr()])
+                keep.append((plan, d_src))
+            assert np.array_equal(got.result(), want), (dim, r2)
+        for r8 in range(8):                                # 2 -> 8
+            src_blob = shard(r8 // 4, 2)
+            want = shard(r8, 8)
+            got = Guarded(want.size, fill=0xEE)
+            plan = tc.tc_plan_create(tc.weights_spec([0], [src_blob.size], [E], [2], [sshape(2)], split_dim=[dim], rank=r8 % 4, world=4,
+                                                     blob_bytes=src_blob.size, tuning=dict(tile_bytes=4096)))
+            tc.tc_weights_materialize(plan, dev(src_blob), [got.ptr()])
+            assert np.array_equal(got.result(), want), (dim, r8)
+
+
 def test_weights_from_a_pinned_blob_zero_copy_and_staged():
     ck = wl.llama_checkpoint(hidden=512, layers=3, q_heads=8, kv_heads=4, head_dim=64, mlp=2048, vocab=70000)   # 190 MB: several staging buffers
     blob = np.zeros(ck.nbytes_total, dtype=np.uint8)

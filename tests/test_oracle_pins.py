@@ -439,6 +439,49 @@ def test_layer_major_order_is_a_regrouping_of_request_major(packed_l):
     assert np.array_equal(pool2, pool3)
 
 
+@pytest.mark.parametrize("pool_l,packed_l", list(itertools.product([oracle.NHD, oracle.HND], repeat=2)))
+def test_layer_major_head_slice_is_a_regrouping_of_the_full_request_major_pack(pool_l, packed_l):
+    """Layer-major order and a head slice together, on NHD and HND pools.  The expected bytes are
+    cut out of the FULL request-major pack with numpy (slice the heads, then put plane p of every
+    request side by side), so the combined branch of the packed-address formula is checked
+    against the two options taken one at a time."""
+    rng = np.random.default_rng(16)
+    shape, NB, stride, pool, T, off, bt = random_case(rng, H=5, T=(6, 0, 9, 1, 13))
+    L, B, H, D, E = shape
+    planes = planes_of(pool, L * 2)
+    full = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, pool_l, stride, planes, T, off, bt, packed_l, full)
+    h0, hs = 2, 2
+    got = np.zeros(oracle.packed_nbytes(shape, T, hs), dtype=np.uint8)
+    cnt = np.zeros_like(got)
+    oracle.kv_pack(shape, pool_l, stride, planes, T, off, bt, packed_l, got, cnt,
+                   order=oracle.LAYER_MAJOR, head_begin=h0, head_count=hs)
+    assert (cnt == 1).all()
+    per_req, pos = [], 0
+    for t in T:
+        n = L * 2 * int(t) * H * D * E
+        reg = full[pos:pos + n]
+        pos += n
+        if packed_l == oracle.NHD:
+            per_req.append(reg.reshape(L * 2, int(t), H, D * E)[:, :, h0:h0 + hs].reshape(L * 2, -1))
+        else:
+            per_req.append(reg.reshape(L * 2, H, int(t), D * E)[:, h0:h0 + hs].reshape(L * 2, -1))
+    want = np.concatenate([np.concatenate([q[p] for q in per_req]) for p in range(L * 2)])
+    assert np.array_equal(got, want)
+    # unpack of that buffer writes exactly the sliced heads of the valid tokens, each byte once,
+    # and reading them back through the same table returns the buffer
+    pool2 = np.full_like(pool, 0xA5)
+    cnt2 = np.zeros_like(pool)
+    oracle.kv_unpack(shape, pool_l, stride, planes_of(pool2, L * 2), T, off, bt, packed_l, got, planes_of(cnt2, L * 2),
+                     order=oracle.LAYER_MAJOR, head_begin=h0, head_count=hs)
+    assert cnt2.sum() == got.size and cnt2.max() == 1 and (pool2[cnt2 == 0] == 0xA5).all()
+    assert np.array_equal(pool2[cnt2 == 1], pool[cnt2 == 1])
+    back = np.zeros_like(got)
+    oracle.kv_pack(shape, pool_l, stride, planes_of(pool2, L * 2), T, off, bt, packed_l, back,
+                   order=oracle.LAYER_MAJOR, head_begin=h0, head_count=hs)
+    assert np.array_equal(back, got)
+
+
 # ------------------------------------------------------------------ integrity checksum
 def test_checksum_shards_add_up_to_the_whole_and_replicas_equal_it():
     ck = small_checkpoint()

@@ -218,6 +218,41 @@ def test_weights_transform_into_fused_target():
     assert np.array_equal(target, want)
 
 
+def test_a_tensor_whose_own_destination_strides_overlap_is_refused():
+    """dst_stride can make one tensor overlap itself: rows closer together than they are long, or
+    elements closer than an element.  Those would write a destination byte twice with different
+    values; strides that interleave without colliding stay legal."""
+    blob = np.arange(4 * 8 * 2, dtype=np.uint8)
+    def create(stride, dst_bytes, shape=(4, 8)):
+        spec = tc.weights_spec([0], [shape[0] * shape[1] * 2], [2], [2], [[shape[0], shape[1], 1, 1]], blob_bytes=blob.size,
+                               dst_slot=[0], dst_off=[0], dst_stride=[stride], n_dst=1, dst_bytes=[dst_bytes], flags=HOST)
+        return tc.tc_plan_create(spec)
+    for stride in ([8, 2, 2, 2], [2, 2, 2, 2], [16, 1, 1, 1]):      # rows 8 B apart but 16 B long; rows 2 B apart; elements 1 B apart
+        with pytest.raises(tc.TensorCastError) as e:
+            create(stride, 256)
+        assert e.value.status == tc.TC_ERR_OVERLAP, stride
+    # a transpose (strides nest the other way round) and padded rows are fine
+    for stride, nbytes in (([2, 8, 2, 2], 64), ([32, 2, 2, 2], 128)):
+        plan = create(stride, nbytes)
+        out, cnt = np.zeros(nbytes, dtype=np.uint8), [np.zeros(nbytes, dtype=np.int32)]
+        run_descriptors(plan.descriptors(0), [blob], [out], cnt)
+        assert cnt[0].max() == 1 and cnt[0].sum() == 64
+    # strides that do not nest but never collide: element (i, j) of a [2, 3] tensor at 3i + 2j
+    plan = create([6, 4, 2, 2], 16, shape=(2, 3))
+    out, cnt = np.zeros(16, dtype=np.uint8), [np.zeros(16, dtype=np.int32)]
+    run_descriptors(plan.descriptors(0), [blob], [out], cnt)
+    assert cnt[0].max() == 1 and cnt[0].sum() == 12
+    src = blob[:12].view(np.uint16).reshape(2, 3)
+    got = out.view(np.uint16)
+    for i in range(2):
+        for j in range(3):
+            assert got[3 * i + 2 * j] == src[i, j]
+    # ... and the same shape with a collision: 2i + 2j puts (0, 1) on (1, 0)
+    with pytest.raises(tc.TensorCastError) as e:
+        create([4, 4, 2, 2], 16, shape=(2, 3))
+    assert e.value.status == tc.TC_ERR_OVERLAP
+
+
 def test_tp_resharding_8_to_2_and_2_to_8_by_composition_of_rules():
     """A checkpoint saved as W shard blobs, loaded at another TP degree W'.  8 -> 2: rank r' of 2
     concatenates four source shards along the split dim (dst_off / dst_stride windows, one plan
