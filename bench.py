@@ -794,6 +794,66 @@ def kv_shapes(args, tc, torch, stream):
     return out
 
 
+def misaligned(args, tc, torch, stream):
+    """Rows a1-a5 when source and destination are not 16-byte aligned: the same plans as the
+    headline rows (aligned geometry), run on base pointers shifted by 8 / 4 / 2 / 1 bytes - a
+    packed buffer or a blob that is a view at an odd offset of a larger allocation, a checkpoint
+    with a short lead pad.  'src' shifts only the source table (the two sides then differ in
+    alignment and every 16-byte store is assembled from two aligned loads), 'both' shifts both
+    sides by the same amount (heads and tails only)."""
+    sp = stream.cuda_stream
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    shape = wl.LLAMA3_8B_KV
+    s = shape.tuple
+    NB = int(((1 if args.small else 8) << 30) // shape.block_bytes)
+    WB = NB // 2
+    _, _, _, waves = wl.config2(NB=NB, R=256, wave_blocks=WB, NB_dst=WB, shape=shape)
+    src, dst = waves[0]
+    payload = int(src.T.sum()) * shape.token_bytes
+    rawA = torch.empty(NB * shape.block_bytes + 16, **u8)
+    wl.fill_torch(rawA, wl.SEED_BASE + 7)
+    rawB = torch.empty(WB * shape.block_bytes + 16, **u8)
+    rawQ = torch.empty(payload + 16, **u8)
+    plA = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=NB * shape.block_bytes)
+    plB = tc.pool(tc.TC_NHD, WB, 1, plane_stride=WB * shape.chunk_bytes, slot_bytes=WB * shape.block_bytes)
+    kw = dict(T=src.T, bt_off=src.bt_off)
+    pk = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, bt_src=src.bt, **kw))
+    up = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, bt_dst=dst.bt, **kw))
+    mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, s, src_pool=plA, dst_pool=plB, bt_src=src.bt, bt_dst=dst.bt, **kw))
+    ck = wl.llama_checkpoint(layers=1, vocab=16032) if args.small else wl.llama_checkpoint(layers=8, vocab=32064)
+    nbytes = [ck.nbytes(i) for i in range(ck.N)]
+    W = 8
+    sizes = [n // (W if ck.split_dim[i] >= 0 else 1) for i, n in enumerate(nbytes)]
+    blob = torch.empty(ck.nbytes_total + 16, **u8)
+    wl.fill_torch(blob, wl.SEED_BASE + 3, "normal")
+    dstw = torch.empty(ck.nbytes_total + 16, **u8)
+    starts_f = np.concatenate([[0], np.cumsum(nbytes)])[:-1]
+    starts_s = np.concatenate([[0], np.cumsum(sizes)])[:-1]
+    wf = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total))
+    ws = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, split_dim=ck.split_dim, rank=args.shard_rank, world=W, blob_bytes=ck.nbytes_total))
+    reps, warm = (1, 1) if args.small else (6, 2)
+    out = {"kv_payload_bytes": payload, "weights_bytes": ck.nbytes_total, "shard_bytes": sum(sizes)}
+    peak, _ = measured_peaks()
+    for label, a_src, a_dst in [("aligned", 0, 0)] + [(f"src+{a}", a, 0) for a in (8, 4, 2, 1)] + [("both+1", 1, 1), ("src+3 dst+9", 3, 9)]:
+        A, B = rawA.data_ptr(), rawB.data_ptr()
+        Q, bl, dw = rawQ.data_ptr(), blob.data_ptr(), dstw.data_ptr()
+        res = {}
+        for name, fn, moved in (
+                ("a1_pack", lambda: tc.tc_kv_pack(pk, [A + a_src], [Q + a_dst], sp), payload),
+                ("a2_unpack", lambda: tc.tc_kv_unpack(up, [Q + a_src], [B + a_dst], sp), payload),
+                ("a3_migrate", lambda: tc.tc_kv_pack(mig, [A + a_src], [B + a_dst], sp), payload),
+                ("a4_weights_full", lambda: tc.tc_weights_materialize(wf, bl + a_src, [dw + a_dst + int(o) for o in starts_f], sp), ck.nbytes_total),
+                ("a5_weights_shard", lambda: tc.tc_weights_materialize(ws, bl + a_src, [dw + a_dst + int(o) for o in starts_s], sp), sum(sizes))):
+            res[name] = 2 * moved / (b2b_ms(torch, stream, fn, reps=reps, warm=warm) * 1e-3) / GB
+        res["min_frac_of_measured_peak"] = min(res.values()) / peak
+        out[label] = res
+    for p_ in (pk, up, mig, wf, ws):
+        p_.destroy()
+    del rawA, rawB, rawQ, blob, dstw
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_extras(args, tc, torch, stream):
     """Secondary workloads, reported beside the headline: configs[3] (70B-shaped pool-to-pool
     migration, one wave) and configs[4] (prefix-reload burst: one mixed plan per scheduler step,
@@ -804,6 +864,9 @@ def run_extras(args, tc, torch, stream):
     u8 = dict(dtype=torch.uint8, device="cuda")
     if args.only_kv_shapes:  # profiler runs: just the KV geometries, a few GB on the device
         out["rows a1-a3 on other KV geometries (8 GiB pools, first wave)"] = kv_shapes(args, tc, torch, stream)
+        return out
+    if args.only_misaligned:
+        out["rows a1-a5 through misaligned base pointers (8 GiB pool, 4 GB checkpoint)"] = misaligned(args, tc, torch, stream)
         return out
     # ---- configs[0]: 1.4 MB, launch-latency bound: microseconds and plans per second
     shape, NB1, src1, dst1 = wl.config1()
@@ -888,6 +951,7 @@ def run_extras(args, tc, torch, stream):
     out["weights cold path: blob streamed from a file"] = cold_path(args, tc, torch, stream)
     out["transform_into: MoE expert stacking (Qwen3-30B-A3B-shaped layers)"] = moe_stacking(args, tc, torch, stream)
     out["rows a1-a3 on other KV geometries (8 GiB pools, first wave)"] = kv_shapes(args, tc, torch, stream)
+    out["rows a1-a5 through misaligned base pointers (8 GiB pool, 4 GB checkpoint)"] = misaligned(args, tc, torch, stream)
     # ---- configs[3]
     shape = wl.LLAMA3_70B_KV
     free, _ = torch.cuda.mem_get_info()
@@ -1018,6 +1082,7 @@ def main():
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary workloads (configs[3], configs[4])")
     ap.add_argument("--only-kv-shapes", action="store_true", help="of the secondary workloads run only the KV geometries (profiler captures)")
+    ap.add_argument("--only-misaligned", action="store_true", help="of the secondary workloads run only the misaligned-pointer rows")
     ap.add_argument("--host-pool-blocks", type=int, default=8192, help="configs[4]: pinned host pool size in 2 MiB blocks")
     ap.add_argument("--burst-steps", type=int, default=10, help="configs[4]: scheduler steps timed (the workload has 200)")
     ap.add_argument("--cold-layers", type=int, default=8, help="cold-path extra: layers of the checkpoint written to a file (8: 4.0 GB)")

@@ -458,6 +458,18 @@ TC_API int tc_plan_segments(const tc_plan_t *plan, int group, tc_segment_t *out,
  * allocate again. */
 TC_API int tc_trim(void);
 
+/* Flags a kernel of this library has set on the current device since the last call, then
+ * cleared (0 = none).  The execute calls cannot report what happens after the launch; the one
+ * condition a kernel can detect and survive is recorded here:
+ *   TC_DEVICE_BULK_WAIT_TIMEOUT  a CTA of the realigning path (misaligned geometry or pointers)
+ *       waited about a second for its asynchronous bulk copies into shared memory and gave up;
+ *       the CTA returned without storing, so the destination of that call is incomplete.  Not
+ *       expected to occur; the wait is bounded so that a failure cannot hang the device.
+ * flags: host pointer.  The call copies the word back and therefore waits for the device's
+ * previously enqueued work (it is a diagnostic, off the data path). */
+#define TC_DEVICE_BULK_WAIT_TIMEOUT 1u
+TC_API int tc_device_status(uint32_t *flags);
+
 /* Static string naming a status code. */
 TC_API const char *tc_strerror(int status);
 

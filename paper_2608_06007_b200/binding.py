@@ -27,6 +27,7 @@ TC_PLAN_CHECKSUM = 4
 TC_PLAN_SAME_POOL = 8
 TC_PLAN_STREAM = 16
 TC_MAX_TABLE_SLOTS = 4000
+TC_DEVICE_BULK_WAIT_TIMEOUT = 1
 
 
 class tc_kv_pool_t(C.Structure):
@@ -99,7 +100,7 @@ class tc_segment_t(C.Structure):
 EXPORTS = ("tc_plan_create", "tc_kv_pack", "tc_kv_unpack", "tc_weights_materialize",
            "tc_plan_destroy", "tc_plan_stats", "tc_plan_descriptors", "tc_strerror", "tc_last_error",
            "tc_kv_pack_noalloc", "tc_weights_materialize_checksum", "tc_trim",
-           "tc_weights_materialize_file", "tc_plan_segments")
+           "tc_weights_materialize_file", "tc_plan_segments", "tc_device_status")
 
 _lib = None
 
@@ -129,6 +130,8 @@ def load_library(path: str | None = None):
     lib.tc_weights_materialize_file.restype = C.c_int
     lib.tc_plan_segments.argtypes = [vp, C.c_int, vp, sz, C.POINTER(sz)]
     lib.tc_plan_segments.restype = C.c_int
+    lib.tc_device_status.argtypes = [C.POINTER(C.c_uint32)]
+    lib.tc_device_status.restype = C.c_int
     lib.tc_trim.argtypes = []
     lib.tc_trim.restype = C.c_int
     lib.tc_strerror.argtypes = [C.c_int]
@@ -360,6 +363,13 @@ def tc_plan_segments(plan: Plan, group: int = 0):
 def tc_trim() -> None:
     """Release the device memory the library caches between plans (plan-storage blocks, idle staging rings)."""
     _check(load_library().tc_trim())
+
+
+def tc_device_status() -> int:
+    """Flags kernels have set on the current device since the last call (0 = none); waits for the device."""
+    v = C.c_uint32()
+    _check(load_library().tc_device_status(C.byref(v)))
+    return int(v.value)
 
 
 def tc_plan_stats(plan: Plan) -> tc_plan_stats_t:

@@ -25,7 +25,7 @@ namespace tc {
 template <int MODE> struct Shape;
 template <> struct Shape<kModeRun> { static constexpr int threads = 256, unroll = 8, min_ctas = 3; };
 template <> struct Shape<kModeRows> { static constexpr int threads = 256, unroll = 8, min_ctas = 3; };
-template <> struct Shape<kModeAny> { static constexpr int threads = 256, unroll = 4, min_ctas = 2; };
+template <> struct Shape<kModeAny> { static constexpr int threads = 256, unroll = 4, min_ctas = 6; };
 
 template <int NPTR>
 struct Params {
@@ -44,6 +44,7 @@ struct Params {
     uint32_t win_o_end;         // first plane past the window
     uint32_t ppt, log2_unit;    // multi-plane tiles (MULTI builds): planes per tile, log2 of the padded plane
     uint32_t tile_base;         // first global tile id of this launch (tile-range segments)
+    uint32_t stage_bytes;       // dynamic shared memory of the launch (realigning path)
     unsigned long long *sums;   // checksum accumulators (checked builds only)
     char *ptr[NPTR];            // src table then dst table
 };
@@ -159,6 +160,362 @@ __device__ __forceinline__ void copy_rows(const Desc &d, const char *src, char *
     }
 }
 
+// Rows of a few bytes each (an element-granular scatter) at less than 16-byte alignment: vectors
+// as wide as the alignment allows, several in flight per thread.  Out of line, so that the four
+// widths do not weigh on the register allocation of the kernel's main paths.
+template <int U, int kThreads>
+__device__ __noinline__ void copy_rows_narrow(const Desc &d, const char *src, char *dst, uint32_t row0, uint32_t nrows, uint32_t align)
+{
+    switch (align) {
+    case 3: copy_rows<3, U, kThreads>(d, src, dst, row0, nrows); break;
+    case 2: copy_rows<2, 2 * U, kThreads>(d, src, dst, row0, nrows); break;
+    case 1: copy_rows<1, 2 * U, kThreads>(d, src, dst, row0, nrows); break;
+    default: copy_rows<0, 2 * U, kThreads>(d, src, dst, row0, nrows); break;
+    }
+}
+
+// ---- realigning path: rows whose source and destination are not both 16-byte aligned ---------
+// Alignment should cost a row its head and its tail, not the width of every access.  The CTA
+// first brings the 16-byte aligned source chunks that cover its rows into shared memory - one
+// bulk asynchronous copy (cp.async.bulk, completion on an mbarrier) per row, issued by one
+// thread, so loading costs neither registers nor instructions per byte - then walks the 16-byte
+// aligned DESTINATION chunks of every row: two aligned shared-memory loads and a funnel shift
+// give a chunk's 16 bytes whatever the difference between the two alignments is, and the chunk
+// leaves with one aligned 16-byte store.  Only the first and last chunk of a row can be
+// partial; they are stored in naturally aligned pieces of 8, 4, 2 and 1 bytes.  The source side
+// reads whole aligned 16-byte chunks, so up to 15 bytes before a row's first byte and after
+// its last one are read (never a chunk without a byte of the row, hence never another page);
+// nothing outside the row is ever written.
+// Tiles whose rows differ in alignment (a row pitch that is not a multiple of 16) load with
+// 16-byte cp.async per chunk instead and work out every chunk's own alignments.
+// The wait for the bulk copies is bounded: if it ever ran out, the CTA would record
+// kStatusBulkWaitTimeout in the device status word, wait once more for its copies, and return
+// without storing (the host reads the word with tc_device_status).
+__device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void *gptr)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr), "l"(gptr) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+
+// Bytes [sh, sh + 16) of the 32 bytes a | b.
+__device__ __forceinline__ uint4 shift_bytes(uint4 a, uint4 b, uint32_t sh)
+{
+    const bool w2 = sh & 8, w1 = sh & 4;
+    uint32_t b0 = w2 ? a.z : a.x, b1 = w2 ? a.w : a.y, b2 = w2 ? b.x : a.z, b3 = w2 ? b.y : a.w, b4 = w2 ? b.z : b.x, b5 = w2 ? b.w : b.y;
+    const uint32_t c0 = w1 ? b1 : b0, c1 = w1 ? b2 : b1, c2 = w1 ? b3 : b2, c3 = w1 ? b4 : b3, c4 = w1 ? b5 : b4;
+    const uint32_t bits = (sh & 3) * 8;
+    return make_uint4(__funnelshift_r(c0, c1, bits), __funnelshift_r(c1, c2, bits), __funnelshift_r(c2, c3, bits), __funnelshift_r(c3, c4, bits));
+}
+
+// Store bytes [lo, hi) of the 16-byte chunk v at the 16-byte aligned address p, in naturally
+// aligned pieces: ascending sizes up to the first boundary that fits, then descending sizes.
+__device__ __forceinline__ void store_partial(char *p, uint4 v, uint32_t lo, uint32_t hi)
+{
+    auto word = [&](uint32_t k) { const uint32_t i = k >> 2; return (i & 2) ? ((i & 1) ? v.w : v.z) : ((i & 1) ? v.y : v.x); };
+    auto put = [&](uint32_t k, uint32_t size) {
+        if (size == 8) *reinterpret_cast<uint2 *>(p + k) = k ? make_uint2(v.z, v.w) : make_uint2(v.x, v.y);
+        else if (size == 4) *reinterpret_cast<uint32_t *>(p + k) = word(k);
+        else if (size == 2) *reinterpret_cast<uint16_t *>(p + k) = static_cast<uint16_t>(word(k) >> ((k & 2) * 8));
+        else *reinterpret_cast<uint8_t *>(p + k) = static_cast<uint8_t>(word(k) >> ((k & 3) * 8));
+    };
+    uint32_t k = lo;
+#pragma unroll
+    for (uint32_t size = 1; size <= 8; size <<= 1)
+        if ((k & size) && k + size <= hi) { put(k, size); k += size; }
+#pragma unroll
+    for (uint32_t size = 8; size >= 1; size >>= 1)
+        if (k + size <= hi) { put(k, size); k += size; }
+}
+
+// Bytes [4 * WS + bits / 8, ... + 16) of the 32 bytes a | b, word shift known at compile time.
+template <int WS>
+__device__ __forceinline__ uint4 shift_words(uint4 a, uint4 b, uint32_t bits)
+{
+    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    return make_uint4(__funnelshift_r(w[WS], w[WS + 1], bits), __funnelshift_r(w[WS + 1], w[WS + 2], bits),
+                      __funnelshift_r(w[WS + 2], w[WS + 3], bits), __funnelshift_r(w[WS + 3], w[WS + 4], bits));
+}
+
+// Sticky error flags set by kernels (read and cleared by tc_device_status).
+enum : unsigned int { kStatusBulkWaitTimeout = 1u };
+__device__ unsigned int g_device_status = 0;
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// One potentially blocking test of a phase: the hardware may park the thread for up to about
+// `hint_ns` while the phase is incomplete, so a waiting thread does not compete for issue slots.
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t hint_ns)
+{
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
+    return done != 0;
+}
+// Bounded wait for a phase of the barrier: false if it did not complete within the limit
+// (a bulk copy takes microseconds; the limit is of the order of a second).
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t spin = 0; spin < (1u << 20); spin++) {
+        if (mbar_try_wait(bar, parity, 1000)) return true;
+        if (spin > 64) __nanosleep(1000);  // long past any normal completion: back off
+    }
+    return false;
+}
+// global -> shared bulk copy of `bytes` (a multiple of 16; both addresses 16-byte aligned) that
+// reports to the barrier.  The source is this GPU's memory, a peer's or mapped host memory;
+// no multicast.
+__device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void *gsrc, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_dst), "l"(gsrc), "r"(bytes), "r"(bar) : "memory");
+}
+
+// Geometry of one pass of the realigning path when every row of the tile has the same source
+// and the same destination alignment (all strides multiples of 16, the common case: a shifted
+// base pointer, a blob with a lead pad).  Chunk u = rr * units + c of the pass (row rr, chunk c
+// of the row's destination) finds its bytes in shared memory at data + 16 * u + delta,
+// delta = s_lo - d_lo.
+struct RealignPass {
+    const char *src;  // row 0 of the tile, plus the column offset
+    char *dst;
+    uint32_t row_base, n_rows;  // rows [row_base, row_base + n_rows) of the descriptor
+    uint32_t units, len;        // chunks per row in the unit space, bytes of the row (piece) that move
+    uint32_t s_lo, d_lo;        // source / destination address modulo 16
+};
+
+// One bulk copy per row: the aligned source chunks that hold the row's bytes.
+template <int kThreads>
+__device__ __forceinline__ void realign_load(const Desc &d, const RealignPass &p, uint32_t data_addr, uint32_t bar)
+{
+    const uint32_t n0 = d.n0, ss0 = d.src_s0, ss1 = d.src_s1;
+    const FastDiv div_n0 = d.div_n0;
+    const uint32_t row_bytes = ((p.s_lo + p.len + 15) >> 4) << 4;
+    const char *base = p.src - p.s_lo;
+    if (threadIdx.x == 0) mbar_expect_tx(bar, p.n_rows * row_bytes);
+    for (uint32_t rr = threadIdx.x; rr < p.n_rows; rr += kThreads) {
+        const uint32_t r = p.row_base + rr, i1 = fastdiv(r, div_n0), i0 = r - i1 * n0;
+        bulk_load(data_addr + 16 * rr * p.units, base + (i1 * ss1 + i0 * ss0), row_bytes, bar);
+    }
+}
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+// Whole destination chunks [c_begin, c_end) of every row of the pass.  data_addr: shared-memory
+// address of the staged rows.  Two thread mappings keep the loop body short:
+//   long rows   all threads walk the chunks of one row, kThreads at a time; the row is decoded
+//               once, outside the loop;
+//   short rows  (fewer chunks than threads) the CTA splits into groups of `units` threads; a
+//               thread keeps its chunk index and steps through the rows, one group apart.
+template <int WS, int kThreads>
+__device__ __forceinline__ void realign_store_full(const Desc &d, const RealignPass &p, uint32_t data_addr, uint32_t c_begin, uint32_t c_end)
+{
+    const uint32_t n0 = d.n0, ds0 = d.dst_s0, ds1 = d.dst_s1, units = p.units;
+    const FastDiv div_n0 = d.div_n0, div_units{d.units_mul, d.units_shift};
+    const int delta = static_cast<int>(p.s_lo) - static_cast<int>(p.d_lo);
+    const uint32_t bits = (static_cast<uint32_t>(delta) & 3) * 8;
+    const uint32_t shifted = data_addr + 16 * (delta >> 4);  // delta >> 4 is 0 or -1
+    char *base = p.dst - p.d_lo;
+    if (units >= kThreads) {
+        for (uint32_t rr = 0; rr < p.n_rows; rr++) {
+            const uint32_t r = p.row_base + rr, i1 = fastdiv(r, div_n0), i0 = r - i1 * n0;
+            uint32_t c = c_begin + threadIdx.x;
+            uint32_t at = shifted + 16 * (rr * units + c);
+            char *out = base + (i1 * ds1 + i0 * ds0) + 16 * static_cast<size_t>(c);
+#pragma unroll 2
+            for (; c < c_end; c += kThreads, at += 16 * kThreads, out += 16 * kThreads)
+                st_stream<uint4>(out, shift_words<WS>(lds128(at), lds128(at + 16), bits));
+        }
+    } else {
+        const uint32_t groups = fastdiv(kThreads, div_units);  // >= 1
+        const uint32_t g = fastdiv(threadIdx.x, div_units), c = threadIdx.x - g * units;
+        if (g >= groups || c < c_begin || c >= c_end) return;
+        uint32_t at = shifted + 16 * (g * units + c);
+        char *col = base + 16 * c;
+#pragma unroll 2
+        for (uint32_t rr = g; rr < p.n_rows; rr += groups, at += 16 * groups * units) {
+            const uint32_t r = p.row_base + rr, i1 = fastdiv(r, div_n0), i0 = r - i1 * n0;
+            st_stream<uint4>(col + (i1 * ds1 + i0 * ds0), shift_words<WS>(lds128(at), lds128(at + 16), bits));
+        }
+    }
+}
+
+// Bytes [0, t) of a and bytes [t, 16) of b.
+__device__ __forceinline__ uint4 merge_bytes(uint4 a, uint4 b, uint32_t t)
+{
+    auto pick = [&](uint32_t x, uint32_t y, uint32_t w) {
+        const int n = static_cast<int>(t) - static_cast<int>(4 * w);  // bytes of this word that come from a
+        const uint32_t mask = n >= 4 ? 0xffffffffu : n <= 0 ? 0u : (1u << (8 * n)) - 1;
+        return (x & mask) | (y & ~mask);
+    };
+    return make_uint4(pick(a.x, b.x, 0), pick(a.y, b.y, 1), pick(a.z, b.z, 2), pick(a.w, b.w, 3));
+}
+
+// The partial chunks of every row of the pass: a head of bytes [d_lo, 16) of chunk 0 and / or
+// a tail of bytes [0, t) of chunk c_last (or the bytes [d_lo, end) of a row that lies inside
+// its first chunk).  One thread per row.  Where the next row of the destination starts exactly
+// where this one ends (rows `adj` apart in the descriptor's row order, adjacent in memory), its
+// head and this row's tail fill one chunk between them: that chunk is assembled from both rows
+// and stored whole, instead of as up to eight small pieces.
+template <int WS, int kThreads>
+__device__ __forceinline__ void realign_store_edges(const Desc &d, const RealignPass &p, uint32_t data_addr, uint32_t c_last, uint32_t end)
+{
+    const uint32_t n0 = d.n0, ds0 = d.dst_s0, ds1 = d.dst_s1, units = p.units;
+    const FastDiv div_n0 = d.div_n0;
+    const int delta = static_cast<int>(p.s_lo) - static_cast<int>(p.d_lo);
+    const uint32_t bits = (static_cast<uint32_t>(delta) & 3) * 8;
+    const uint32_t shifted = data_addr + 16 * (delta >> 4);
+    char *base = p.dst - p.d_lo;
+    const bool one_chunk = c_last == 0;
+    const uint32_t t = end & 15;  // bytes of the tail
+    // rows adjacent in the destination: the whole row moves (no column pieces) and its length
+    // keeps the alignment, so that a tail of t bytes meets a head that starts at byte t = d_lo
+    uint32_t adj = 0;
+    if (!one_chunk && t && p.len == d.run && (d.run & 15) == 0) adj = (n0 > 1 && ds0 == d.run) ? 1 : (ds1 == d.run ? n0 : 0);
+    for (uint32_t rr = threadIdx.x; rr < p.n_rows; rr += kThreads) {
+        const uint32_t r = p.row_base + rr, i1 = fastdiv(r, div_n0), i0 = r - i1 * n0;
+        char *out = base + (i1 * ds1 + i0 * ds0);
+        const uint32_t row_at = shifted + 16 * rr * units;
+        const bool has_next = adj && (adj == 1 ? i0 + 1 < n0 : r + n0 < d.rows) && rr + adj < p.n_rows;
+        const bool has_prev = adj && (adj == 1 ? i0 >= 1 : r >= n0) && rr >= adj;
+        if ((p.d_lo || one_chunk) && !has_prev)
+            store_partial(out, shift_words<WS>(lds128(row_at), lds128(row_at + 16), bits), p.d_lo, one_chunk ? end : 16);
+        if (!one_chunk && t) {
+            const uint32_t at = row_at + 16 * c_last;
+            const uint4 tail = shift_words<WS>(lds128(at), lds128(at + 16), bits);
+            if (has_next) {
+                const uint32_t next_at = row_at + 16 * adj * units;
+                st_stream<uint4>(out + 16 * c_last, merge_bytes(tail, shift_words<WS>(lds128(next_at), lds128(next_at + 16), bits), t));
+            } else {
+                store_partial(out + 16 * c_last, tail, 0, t);
+            }
+        }
+    }
+}
+
+template <int WS, int kThreads>
+__device__ __forceinline__ void realign_store_all(const Desc &d, const RealignPass &p, uint32_t data)
+{
+    // chunk c of a row's destination covers row bytes [16c - d_lo, 16c - d_lo + 16)
+    const uint32_t end = p.d_lo + p.len;  // first byte past the row, counted from the row's first chunk
+    const uint32_t c_first = p.d_lo ? 1 : 0, c_last = end >> 4;  // whole chunks: [c_first, c_last)
+    if (c_last > c_first) realign_store_full<WS, kThreads>(d, p, data, c_first, c_last);
+    if (p.d_lo || (end & 15)) realign_store_edges<WS, kThreads>(d, p, data, c_last, end);
+}
+
+// The same for tiles whose rows differ in alignment (a row pitch that is not a multiple of 16):
+// every chunk works out its own row's alignments.  Out of line: a rare geometry.
+template <int kThreads>
+__device__ __noinline__ void realign_pass_mixed(const Desc &d, const char *src, char *dst, uint32_t row_base, uint32_t n_rows, uint32_t len, char *data)
+{
+    const uint32_t n0 = d.n0, ss0 = d.src_s0, ss1 = d.src_s1, ds0 = d.dst_s0, ds1 = d.dst_s1;
+    const FastDiv div_n0 = d.div_n0, div_units{d.units_mul, d.units_shift};
+    const uint32_t units = (min(d.run, kRealignColumn) + 30) >> 4;
+    const uint32_t data_addr = static_cast<uint32_t>(__cvta_generic_to_shared(data));
+    const uint32_t total = n_rows * units;
+    for (uint32_t u = threadIdx.x; u < total; u += kThreads) {
+        const uint32_t rr = fastdiv(u, div_units), c = u - rr * units;
+        const uint32_t r = row_base + rr, i1 = fastdiv(r, div_n0), i0 = r - i1 * n0;
+        const char *s = src + (i1 * ss1 + i0 * ss0);
+        const uintptr_t chunk = (reinterpret_cast<uintptr_t>(s) & ~uintptr_t(15)) + 16 * c;
+        if (chunk < reinterpret_cast<uintptr_t>(s) + len) cp_async16(data_addr + 16 * u, reinterpret_cast<const void *>(chunk));
+    }
+    cp_async_wait_all();
+    __syncthreads();
+    for (uint32_t u = threadIdx.x; u < total; u += kThreads) {
+        const uint32_t rr = fastdiv(u, div_units), c = u - rr * units;
+        const uint32_t r = row_base + rr, i1 = fastdiv(r, div_n0), i0 = r - i1 * n0;
+        const uint32_t s_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src + (i1 * ss1 + i0 * ss0))) & 15;
+        char *dp = dst + (i1 * ds1 + i0 * ds0);
+        const uint32_t d_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(dp)) & 15;
+        const int first = static_cast<int>(16 * c) - static_cast<int>(d_lo);  // row byte at the chunk's byte 0
+        const uint32_t lo = first < 0 ? static_cast<uint32_t>(-first) : 0;
+        const int left = static_cast<int>(len) - first;
+        if (left <= static_cast<int>(lo)) continue;
+        const uint32_t hi = left < 16 ? static_cast<uint32_t>(left) : 16;
+        const int q = static_cast<int>(s_lo) + first;  // the row's byte b sits at 16 * rr * units + s_lo + b; q >= -15
+        const char *at = data + 16 * (rr * units) + 16 * (q >> 4);
+        const uint4 a = *reinterpret_cast<const uint4 *>(at), b = *reinterpret_cast<const uint4 *>(at + 16);
+        const uint4 v = shift_bytes(a, b, static_cast<uint32_t>(q) & 15);
+        if (lo == 0 && hi == 16) st_stream<uint4>(dp + first, v);
+        else store_partial(dp + first, v, lo, hi);
+    }
+}
+
+// Rows [row0, row0 + nrows) of one outer index of descriptor d, any alignment; src / dst point
+// at row 0.  `stage` is the shared-memory staging area (16-byte aligned, stage_bytes long, of
+// which the first and last 16 are padding that neighbouring-chunk loads may touch): a pass
+// stages as many whole rows as fit, row rr in the `units` chunks from 16 * rr * units on,
+// starting at the row's first aligned source chunk.  A row longer than kRealignColumn is taken
+// in column pieces.  bar / phase: the CTA's mbarrier and the parity of its next phase.
+// Returns false if a bulk copy did not arrive in time (the caller returns from the kernel).
+template <int kThreads>
+__device__ __forceinline__ bool copy_rows_realign(const Desc &d, const char *src, char *dst, uint32_t row0, uint32_t nrows, char *stage, uint32_t stage_bytes,
+                                                  uint32_t bar, uint32_t &phase, uint32_t *wait_ok)
+{
+    const uint32_t run = d.run;
+    const uint32_t column = min(run, kRealignColumn);
+    const uint32_t units = (column + 30) >> 4;  // 16-byte chunks a row piece can touch, on either side
+    const uint32_t rows_per_pass = (stage_bytes - 32) / (units << 4);  // >= 1: the launch sizes the area for it
+    char *data = stage + 16;
+    const uint32_t data_addr = static_cast<uint32_t>(__cvta_generic_to_shared(data));
+    const bool same_alignment = ((d.src_s0 | d.src_s1 | d.dst_s0 | d.dst_s1) & 15) == 0;
+    for (uint32_t col0 = 0; col0 < run; col0 += column) {
+        const uint32_t len = min(column, run - col0);
+        for (uint32_t r0 = 0; r0 < nrows; r0 += rows_per_pass) {
+            const uint32_t n_rows = min(rows_per_pass, nrows - r0);
+            if (same_alignment) {
+                RealignPass p;
+                p.src = src + col0;
+                p.dst = dst + col0;
+                p.row_base = row0 + r0;
+                p.n_rows = n_rows;
+                p.units = units;
+                p.len = len;
+                p.s_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(p.src)) & 15;
+                p.d_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(p.dst)) & 15;
+                realign_load<kThreads>(d, p, data_addr, bar);
+                // one thread waits (bounded) and tells the others, so that the CTA stays together
+                if (threadIdx.x == 0) {
+                    bool ok = mbar_wait_bounded(bar, phase);
+                    if (!ok) {
+                        atomicOr(&g_device_status, kStatusBulkWaitTimeout);
+                        ok = mbar_wait_bounded(bar, phase);  // the copies still target this CTA's memory
+                        *wait_ok = 0;
+                    }
+                }
+                __syncthreads();
+                if (!*wait_ok) return false;
+                mbar_try_wait(bar, phase, 0);  // completed: every thread observes the phase itself
+                phase ^= 1;
+                switch (((p.s_lo - p.d_lo) & 15) >> 2) {
+                case 0: realign_store_all<0, kThreads>(d, p, data_addr); break;
+                case 1: realign_store_all<1, kThreads>(d, p, data_addr); break;
+                case 2: realign_store_all<2, kThreads>(d, p, data_addr); break;
+                default: realign_store_all<3, kThreads>(d, p, data_addr); break;
+                }
+            } else {
+                realign_pass_mixed<kThreads>(d, src + col0, dst + col0, row0 + r0, n_rows, len, data);
+            }
+            __syncthreads();
+        }
+    }
+    return true;
+}
+
 // A tile of n_units consecutive planes of one descriptor (small planes, see Group::ppt).  The
 // tile's byte space gives every plane 2^log2_unit bytes, of which the first rows * run are real.
 // Plane k of the tile starts at table[slot + (o + k) * slot_step] + off + (o + k) * outer on
@@ -234,10 +591,23 @@ __device__ __forceinline__ void copy_run16(const char *src, char *dst, uint32_t 
 // MULTI: 0 one plane per tile; 1 several planes per tile, planes a byte stride apart; 2 the
 // same with a pool that has one pointer per plane.
 template <int NPTR, int MODE, bool CHECK = false, int MULTI = 0>
-__global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) tc_copy_kernel(const __grid_constant__ Params<NPTR> prm)
+__global__ void __launch_bounds__(Shape<MODE>::threads, (MODE == kModeAny && MULTI) ? 2 : Shape<MODE>::min_ctas) tc_copy_kernel(const __grid_constant__ Params<NPTR> prm)
 {
     constexpr int kThreads = Shape<MODE>::threads, kUnroll = Shape<MODE>::unroll;
     __shared__ Desc sdesc[2];
+    extern __shared__ __align__(16) char stage[];  // the realigning path's staging area (kModeAny only)
+    __shared__ __align__(8) unsigned long long stage_bar;  // its mbarrier
+    __shared__ uint32_t stage_ok;
+    uint32_t bar = 0, phase = 0;
+    if (MODE == kModeAny && !MULTI) {
+        bar = static_cast<uint32_t>(__cvta_generic_to_shared(&stage_bar));
+        if (threadIdx.x == 0) {
+            mbar_init(bar, 1);
+            stage_ok = 1;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        // made visible to the CTA by the __syncthreads that follows the descriptor fetch below
+    }
     int buf = 0;
     for (uint32_t tile = blockIdx.x + prm.tile_base; tile < prm.n_tiles; tile += gridDim.x, buf ^= 1) {
         // tile id -> descriptor, plane o, part.  For uniform and windowed launches this needs
@@ -293,7 +663,7 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
             } else if (MODE == kModeRows) {
                 copy_multi<4, kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units);
             } else {
-                switch (min(d.log2_align, prm.log2_ptr_align)) {
+                switch (min(static_cast<uint32_t>(d.log2_align), prm.log2_ptr_align)) {
                 case 4: copy_multi<4, kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units); break;
                 case 3: copy_multi<3, 2 * kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units); break;
                 case 2: copy_multi<2, 2 * kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units); break;
@@ -331,13 +701,13 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
                 copy_rows<4, kUnroll, kThreads>(d, src, dst, row0, nrows);
             }
         } else {
-            switch (min(d.log2_align, prm.log2_ptr_align)) {
-            case 4: copy_rows<4, kUnroll, kThreads>(d, src, dst, row0, nrows); break;
-            // narrower vectors cost fewer registers each, so more of them can be in flight
-            case 3: copy_rows<3, 2 * kUnroll, kThreads>(d, src, dst, row0, nrows); break;
-            case 2: copy_rows<2, 2 * kUnroll, kThreads>(d, src, dst, row0, nrows); break;
-            case 1: copy_rows<1, 2 * kUnroll, kThreads>(d, src, dst, row0, nrows); break;
-            default: copy_rows<0, 2 * kUnroll, kThreads>(d, src, dst, row0, nrows); break;
+            const uint32_t align = min(static_cast<uint32_t>(d.log2_align), prm.log2_ptr_align);
+            if (align == 4) {
+                copy_rows<4, kUnroll, kThreads>(d, src, dst, row0, nrows);
+            } else if (d.run >= kRealignMinRun) {
+                if (!copy_rows_realign<kThreads>(d, src, dst, row0, nrows, stage, prm.stage_bytes, bar, phase, &stage_ok)) return;
+            } else {
+                copy_rows_narrow<kUnroll, kThreads>(d, src, dst, row0, nrows, align);
             }
         }
     }

@@ -296,6 +296,16 @@ extern "C" int tc_trim(void)
     return TC_OK;
 }
 
+extern "C" int tc_device_status(uint32_t *flags)
+{
+    clear_error();
+    if (!flags) return fail(TC_ERR_INVALID_ARG, "flags is NULL");
+    unsigned int v = 0;
+    const int rc = read_device_status(&v);
+    *flags = v;
+    return rc;
+}
+
 extern "C" int tc_plan_stats(const tc_plan_t *plan, tc_plan_stats_t *out)
 {
     clear_error();

@@ -35,6 +35,9 @@ uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *
 int launch_any(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s, const Segment *win,
                unsigned long long *sums = nullptr);
 
+// The current device's sticky status word (flags set by kernels); reading clears it.
+int read_device_status(unsigned int *out);
+
 // ---- staging.cu
 // Take / drop a reference on the device's staging rings (allocated on first use); *bytes
 // receives the device memory the rings hold.

@@ -21,7 +21,9 @@ template <int NPTR, int MODE>
 static int resident_ctas()
 {
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, tc_copy_kernel<NPTR, MODE>, Shape<MODE>::threads, 0) != cudaSuccess || n < 1) n = 1;
+    const size_t smem = MODE == kModeAny ? kRealignSmem : 0;
+    if (smem) cudaFuncSetAttribute(tc_copy_kernel<NPTR, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, tc_copy_kernel<NPTR, MODE>, Shape<MODE>::threads, smem) != cudaSuccess || n < 1) n = 1;
     return n;
 }
 
@@ -109,6 +111,7 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     prm.tpo = g.tiles_per_desc ? g.tiles_per_desc / outer_groups(g) : 1;
     prm.div_tpo = make_fastdiv(prm.tpo);
     prm.log2_ptr_align = ptr_align;
+    prm.stage_bytes = 0;
     prm.sums = sums;
     for (size_t i = 0; i < g.n_src; i++) prm.ptr[i] = const_cast<char *>(static_cast<const char *>(src[i]));
     for (size_t i = 0; i < g.n_dst; i++) prm.ptr[g.n_src + i] = static_cast<char *>(dst[i]);
@@ -140,11 +143,27 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     switch (mode) {
     case kModeRun: tc_copy_kernel<NPTR, kModeRun><<<grid, Shape<kModeRun>::threads, 0, stream>>>(prm); break;
     case kModeRows: tc_copy_kernel<NPTR, kModeRows><<<grid, Shape<kModeRows>::threads, 0, stream>>>(prm); break;
-    default: tc_copy_kernel<NPTR, kModeAny><<<grid, Shape<kModeAny>::threads, 0, stream>>>(prm); break;
+    default: {
+        // the realigning path stages rows in more dynamic shared memory than a kernel gets by
+        // default; the opt-in is per device and costs nothing to repeat
+        cudaError_t ea = cudaFuncSetAttribute(tc_copy_kernel<NPTR, kModeAny>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kRealignSmem));
+        if (ea != cudaSuccess) return cuda_fail(ea, "cudaFuncSetAttribute(dynamic shared memory)");
+        prm.stage_bytes = std::max<uint32_t>(g.realign_smem, 1024);
+        tc_copy_kernel<NPTR, kModeAny><<<grid, Shape<kModeAny>::threads, prm.stage_bytes, stream>>>(prm);
+        break;
+    }
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
     return TC_OK;
+}
+
+int read_device_status(unsigned int *out)
+{
+    unsigned int zero = 0;
+    cudaError_t e = cudaMemcpyFromSymbol(out, g_device_status, sizeof *out);
+    if (e == cudaSuccess && *out) e = cudaMemcpyToSymbol(g_device_status, &zero, sizeof zero);
+    return e == cudaSuccess ? TC_OK : cuda_fail(e, "reading the device status word");
 }
 
 int launch_any(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s, const Segment *win,

@@ -42,10 +42,13 @@ struct alignas(16) Desc {
     uint16_t src_slot, dst_slot, src_slot_step, dst_slot_step;
     FastDiv div_run;  // byte index inside a tile -> row
     uint32_t run, n0, rows, n_outer;
-    uint32_t rows_per_tile, tiles_per_outer, tile0, log2_align;
+    uint32_t rows_per_tile, tiles_per_outer, tile0;
+    uint16_t log2_align;
+    uint16_t units_shift; // with units_mul: FastDiv by the 16-byte units per row of the realigning
+                          // path, (min(run, kRealignColumn) + 30) / 16 (see copy_kernel.cuh)
     FastDiv div_n0, div_tpo;
     uint32_t tag;        // checksummed plans: which accumulator (tensor index) this box feeds
-    uint32_t pad;
+    uint32_t units_mul;
     int64_t csum_base;   // checksummed plans: src byte offset of the tensor's first byte
 };
 static_assert(sizeof(Desc) == 128, "Desc must stay 128 bytes");
@@ -87,6 +90,7 @@ struct Group {
     uint64_t n_tiles = 0;
     int64_t payload = 0;
     uint32_t log2_align = 4;
+    uint32_t realign_smem = 0;        // staging bytes one CTA of the realigning path needs for this group's largest tile
     size_t n_src = 0, n_dst = 0;      // table lengths the execute call must be given
     bool single_run_tiles = true;     // every tile is one contiguous run
     int resident_ctas[3] = {0, 0, 0}; // CTAs one SM holds, per executor build
@@ -129,5 +133,10 @@ constexpr uint32_t kDefaultTileBytes = 32768;
 constexpr int64_t kStageBytes = 64ll << 20;  // one staging buffer
 constexpr int kStageBuffers = 3;
 constexpr uint32_t kMaxTileBytes = 1u << 20;
+// Realigning path (misaligned geometry or pointers): shared memory one CTA stages a tile's rows
+// in, and the longest piece of a row it stages in one pass.
+constexpr uint32_t kRealignSmem = 52u << 10;
+constexpr uint32_t kRealignColumn = kRealignSmem - 64;
+constexpr uint32_t kRealignMinRun = 32;  // shorter rows take the narrow-vector loop instead
 
 }  // namespace tc

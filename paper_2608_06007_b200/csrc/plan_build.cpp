@@ -108,7 +108,10 @@ static void emit_desc(Group &g, const Box &b, int64_t run, const Dim *inner, con
     if (d.n0 > 1) a = std::min({a, ctz_cap(d.src_s0), ctz_cap(d.dst_s0)});
     if (n1 > 1) a = std::min({a, ctz_cap(d.src_s1), ctz_cap(d.dst_s1)});
     if (d.n_outer > 1) a = std::min({a, ctz_cap(d.src_outer), ctz_cap(d.dst_outer)});
-    d.log2_align = a;
+    d.log2_align = static_cast<uint16_t>(a);
+    const FastDiv units = make_fastdiv((std::min<uint32_t>(d.run, kRealignColumn) + 30) >> 4);
+    d.units_mul = units.mul;
+    d.units_shift = static_cast<uint16_t>(units.shift);
     d.tag = b.tag;
     d.csum_base = b.csum_base;
     g.log2_align = std::min(g.log2_align, a);
@@ -227,6 +230,13 @@ static void lower_box(Group &g, Box b, uint32_t tile_bytes)
 static int finish_group(Group &g, uint32_t tile_bytes)
 {
     if (g.descs.empty()) return TC_OK;
+    // Realigning path: one pass should hold a whole tile (every row in a slot of `units` 16-byte
+    // chunks, 32 bytes of padding), up to the size at which long rows go in column pieces.
+    for (const Desc &d : g.descs) {
+        const uint64_t units = (std::min<uint32_t>(d.run, kRealignColumn) + 30) >> 4;
+        const uint64_t need = std::min<uint64_t>(d.rows_per_tile, d.rows) * units * 16 + 32;
+        g.realign_smem = static_cast<uint32_t>(std::max<uint64_t>(g.realign_smem, std::min<uint64_t>(need, kRealignSmem)));
+    }
     // Small planes: let a tile span several planes of its descriptor (see Group::ppt).  Needs one
     // part per plane and a pointer table of at most 400 entries (the kernel classes built for it).
     g.ppt = 1;

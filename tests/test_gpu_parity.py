@@ -666,6 +666,81 @@ def test_weights_checksum_fused_with_the_copy():
     assert e.value.status == tc.TC_ERR_KIND
 
 
+# --------------------------------------------------------------------------- misaligned rows
+@pytest.mark.parametrize("cols,pitch,tile", [(100, 116, 0), (256, 256 + 16, 0), (33, 64, 1024), (5000, 5003, 0), (40000, 40000 + 7, 0), (70000, 70001, 65536)])
+def test_rows_at_every_source_and_destination_alignment(cols, pitch, tile):
+    """Rows of `cols` bytes whose source starts at blob offset ... + a and whose destination
+    starts at b inside its own slot, for a and b over all residues modulo 16 (a sample of the
+    256 pairs for the long rows).  Every slot is a guarded buffer, so a head or tail byte that
+    lands outside its row shows up either in the red zones or in the sentinel bytes between the
+    rows; pitch is not a multiple of 16 in most cases, so the rows of one tensor differ in
+    alignment as well."""
+    rng = np.random.default_rng(cols)
+    rows = 5 if cols < 1000 else 2
+    pairs = [(a, b) for a in range(16) for b in range(16)]
+    if cols >= 1000:
+        pairs = [pairs[i] for i in rng.permutation(256)[:40]] + [(0, 1), (1, 0), (15, 15), (8, 0), (3, 3)]
+    src_off, pos = [], 0
+    for a, b in pairs:
+        pos = (pos + 15) // 16 * 16 + a
+        src_off.append(pos)
+        pos += rows * cols
+    blob = rng.integers(0, 256, pos + 16, dtype=np.uint8)
+    N = len(pairs)
+    slot_bytes = [b + (rows - 1) * pitch + cols for a, b in pairs]
+    kw = dict(dst_off=[b for a, b in pairs], dst_stride=[[pitch, 1, 1, 1]] * N)
+    shapes = [[rows, cols, 1, 1]] * N
+    spec = tc.weights_spec(src_off, [rows * cols] * N, [1] * N, [2] * N, shapes, blob_bytes=blob.size, dst_slot=list(range(N)),
+                           n_dst=N, dst_bytes=slot_bytes, tuning=dict(tile_bytes=tile) if tile else None, **kw)
+    plan = tc.tc_plan_create(spec)
+    assert plan.stats().vec_bytes[0] == 1
+    want = [np.full(n, 0xEE, dtype=np.uint8) for n in slot_bytes]
+    oracle.weights(src_off, [1] * N, shapes, [-1] * N, 0, 1, blob, want, **kw)
+    d_blob = dev(blob)
+    for shift in (0, 1):                                      # destination buffers 16-byte aligned, then odd
+        outs = [Guarded(n, fill=0xEE, shift=shift) for n in slot_bytes]
+        tc.tc_weights_materialize(plan, d_blob, [o.ptr() for o in outs])
+        for k in range(N):
+            assert np.array_equal(outs[k].result(), want[k]), (pairs[k], shift)
+
+
+@pytest.mark.parametrize("shift_pool,shift_packed", [(0, 2), (2, 0), (6, 6), (1, 9), (8, 4)])
+def test_kv_pack_unpack_migrate_through_misaligned_pointers(shift_pool, shift_packed):
+    """Aligned geometry, misaligned base pointers: the pool and / or the packed buffer start at
+    an odd address (a view into a larger allocation).  Rows of 256 bytes (NHD <-> HND) and whole
+    32 KiB planes (same layout) both take the realigning path."""
+    rng = np.random.default_rng(77)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=40, B=16, H=8, D=64, E=2, T=(100, 16, 7, 333))
+    L, B, H, D, E = shape
+    planes = planes_of(pool, L * 2)
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride, slot_bytes=pool.size)
+    raw = torch.zeros(pool.size + 16, dtype=torch.uint8, device="cuda")
+    d_pool = raw[shift_pool:shift_pool + pool.size]
+    d_pool.copy_(dev(pool))
+    for packed_l in LAYOUTS:
+        want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+        oracle.kv_pack(shape, oracle.NHD, stride, planes, T, off, bt, packed_l, want)
+        packed = Guarded(want.size, shift=shift_packed)
+        plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_src=bt))
+        tc.tc_kv_pack(plan, [d_pool.data_ptr()], [packed.ptr()])
+        assert np.array_equal(packed.result(), want), packed_l
+        want_pool = np.full_like(pool, 0xA5)
+        oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(want_pool, L * 2), T, off, bt2, packed_l, want)
+        fresh = Guarded(pool.size, shift=shift_pool)
+        plan2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_dst=bt2))
+        tc.tc_kv_unpack(plan2, [packed.ptr()], [fresh.ptr()])
+        assert np.array_equal(fresh.result(), want_pool), packed_l
+    for dst_l in LAYOUTS:
+        pl2 = tc.pool(dst_l, NB, 1, plane_stride=NB * stride, slot_bytes=pool.size)
+        want_pool = np.full_like(pool, 0xA5)
+        oracle.kv_migrate(shape, oracle.NHD, stride, planes, dst_l, stride, planes_of(want_pool, L * 2), T, off, bt, bt2)
+        fresh = Guarded(pool.size, shift=shift_packed)
+        plan3 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl2, T=T, bt_off=off, bt_src=bt, bt_dst=bt2))
+        tc.tc_kv_pack(plan3, [d_pool.data_ptr()], [fresh.ptr()])
+        assert np.array_equal(fresh.result(), want_pool), dst_l
+
+
 # --------------------------------------------------------------------------- random geometries
 @pytest.mark.parametrize("seed", range(24))
 def test_random_geometries_on_the_device(seed):
