@@ -834,7 +834,19 @@ def misaligned(args, tc, torch, stream):
     reps, warm = (1, 1) if args.small else (6, 2)
     out = {"kv_payload_bytes": payload, "weights_bytes": ck.nbytes_total, "shard_bytes": sum(sizes)}
     peak, _ = measured_peaks()
-    for label, a_src, a_dst in [("aligned", 0, 0)] + [(f"src+{a}", a, 0) for a in (8, 4, 2, 1)] + [("both+1", 1, 1), ("src+3 dst+9", 3, 9)]:
+    auto = (pk, up, mig, wf, ws)
+    # the same plans forced onto the shared-memory path (bulk asynchronous copies in, 16-byte stores
+    # out), on aligned pointers: the A/B behind the choice of the register path for aligned geometry
+    smem = dict(copy_path=1)
+    staged = (tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, bt_src=src.bt, tuning=smem, **kw)),
+              tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, bt_dst=dst.bt, tuning=smem, **kw)),
+              tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, s, src_pool=plA, dst_pool=plB, bt_src=src.bt, bt_dst=dst.bt, tuning=smem, **kw)),
+              tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total, tuning=smem)),
+              tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, split_dim=ck.split_dim, rank=args.shard_rank, world=W,
+                                                blob_bytes=ck.nbytes_total, tuning=smem)))
+    cases = [("aligned", 0, 0, auto), ("aligned, through shared memory (tuning.copy_path = 1)", 0, 0, staged)]
+    cases += [(f"src+{a}", a, 0, auto) for a in (8, 4, 2, 1)] + [("both+1", 1, 1, auto), ("src+3 dst+9", 3, 9, auto)]
+    for label, a_src, a_dst, (pk, up, mig, wf, ws) in cases:
         A, B = rawA.data_ptr(), rawB.data_ptr()
         Q, bl, dw = rawQ.data_ptr(), blob.data_ptr(), dstw.data_ptr()
         res = {}
@@ -847,7 +859,7 @@ def misaligned(args, tc, torch, stream):
             res[name] = 2 * moved / (b2b_ms(torch, stream, fn, reps=reps, warm=warm) * 1e-3) / GB
         res["min_frac_of_measured_peak"] = min(res.values()) / peak
         out[label] = res
-    for p_ in (pk, up, mig, wf, ws):
+    for p_ in auto + staged:
         p_.destroy()
     del rawA, rawB, rawQ, blob, dstw
     torch.cuda.empty_cache()
@@ -866,7 +878,7 @@ def run_extras(args, tc, torch, stream):
         out["rows a1-a3 on other KV geometries (8 GiB pools, first wave)"] = kv_shapes(args, tc, torch, stream)
         return out
     if args.only_misaligned:
-        out["rows a1-a5 through misaligned base pointers (8 GiB pool, 4 GB checkpoint)"] = misaligned(args, tc, torch, stream)
+        out["rows a1-a5: copy paths and misaligned base pointers (8 GiB pool, 4 GB checkpoint)"] = misaligned(args, tc, torch, stream)
         return out
     # ---- configs[0]: 1.4 MB, launch-latency bound: microseconds and plans per second
     shape, NB1, src1, dst1 = wl.config1()
@@ -951,7 +963,7 @@ def run_extras(args, tc, torch, stream):
     out["weights cold path: blob streamed from a file"] = cold_path(args, tc, torch, stream)
     out["transform_into: MoE expert stacking (Qwen3-30B-A3B-shaped layers)"] = moe_stacking(args, tc, torch, stream)
     out["rows a1-a3 on other KV geometries (8 GiB pools, first wave)"] = kv_shapes(args, tc, torch, stream)
-    out["rows a1-a5 through misaligned base pointers (8 GiB pool, 4 GB checkpoint)"] = misaligned(args, tc, torch, stream)
+    out["rows a1-a5: copy paths and misaligned base pointers (8 GiB pool, 4 GB checkpoint)"] = misaligned(args, tc, torch, stream)
     # ---- configs[3]
     shape = wl.LLAMA3_70B_KV
     free, _ = torch.cuda.mem_get_info()

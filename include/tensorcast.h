@@ -257,6 +257,13 @@ typedef struct {
     int32_t tile_order;   /* 0 auto: KV groups run plane-major over descriptors sorted by
                              destination offset (ascending writes); 1: request / descriptor order
                              as given, planes of one block consecutively */
+    int32_t copy_path;    /* 0 auto: aligned geometry moves register to register (16-byte loads and
+                             stores), misaligned geometry through shared memory.  1: always
+                             through shared memory - bulk asynchronous copies (cp.async.bulk) bring
+                             a tile's rows in, 16-byte stores take them out - whatever the
+                             alignment; for comparing the two paths (groups with multi-plane
+                             tiles and checksummed executions keep the register path) */
+    int32_t reserved;     /* 0 */
 } tc_tuning_t;
 
 typedef struct {

@@ -67,7 +67,7 @@ class tc_weights_spec_t(C.Structure):
 
 class tc_tuning_t(C.Structure):
     _fields_ = [("tile_bytes", C.c_int32), ("ctas_per_sm", C.c_int32), ("max_ctas", C.c_int32),
-                ("tile_order", C.c_int32)]
+                ("tile_order", C.c_int32), ("copy_path", C.c_int32), ("reserved", C.c_int32)]
 
 
 class tc_plan_spec_t(C.Structure):

@@ -45,6 +45,7 @@ struct Params {
     uint32_t ppt, log2_unit;    // multi-plane tiles (MULTI builds): planes per tile, log2 of the padded plane
     uint32_t tile_base;         // first global tile id of this launch (tile-range segments)
     uint32_t stage_bytes;       // dynamic shared memory of the launch (realigning path)
+    uint32_t stage_always;      // take the shared-memory path for aligned tiles too (tuning.copy_path)
     unsigned long long *sums;   // checksum accumulators (checked builds only)
     char *ptr[NPTR];            // src table then dst table
 };
@@ -702,7 +703,7 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, (MODE == kModeAny && MUL
             }
         } else {
             const uint32_t align = min(static_cast<uint32_t>(d.log2_align), prm.log2_ptr_align);
-            if (align == 4) {
+            if (align == 4 && (!prm.stage_always || d.run < kRealignMinRun)) {
                 copy_rows<4, kUnroll, kThreads>(d, src, dst, row0, nrows);
             } else if (d.run >= kRealignMinRun) {
                 if (!copy_rows_realign<kThreads>(d, src, dst, row0, nrows, stage, prm.stage_bytes, bar, phase, &stage_ok)) return;

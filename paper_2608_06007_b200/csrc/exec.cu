@@ -322,7 +322,7 @@ extern "C" int tc_plan_stats(const tc_plan_t *plan, tc_plan_stats_t *out)
         out->vec_bytes[k] = 1 << g.log2_align;
         out->path[k] = g.n_tiles ? (g.segments.empty() ? 1 : 3) : 0;
         if (!g.segments.empty()) out->launches_per_execute = static_cast<int32_t>(g.segments.size());
-        out->grid[k] = g.n_tiles ? static_cast<int32_t>(grid_for(plan, g, mode_for(g, 4))) : 0;
+        out->grid[k] = g.n_tiles ? static_cast<int32_t>(grid_for(plan, g, mode_for(plan, g, 4))) : 0;
     }
     out->packed_bytes_required = plan->packed_required;
     out->device_bytes = plan->device_bytes;

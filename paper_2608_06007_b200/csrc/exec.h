@@ -26,7 +26,7 @@ int cuda_fail(cudaError_t e, const char *what);
 
 // ---- launch.cu
 // Which executor build a group needs, given the alignment shared by the call's base pointers.
-int mode_for(const Group &g, uint32_t ptr_align);
+int mode_for(const tc_plan *plan, const Group &g, uint32_t ptr_align, bool checksums = false);
 // CTAs of each build that one SM holds, for a pointer table of n_ptrs slots (cached).
 void resident_ctas_for(size_t n_ptrs, int out[3]);
 uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *win = nullptr);

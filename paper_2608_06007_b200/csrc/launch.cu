@@ -11,9 +11,10 @@
 namespace tc {
 
 // Which executor build a group needs, given the alignment shared by the call's base pointers.
-int mode_for(const Group &g, uint32_t ptr_align)
+int mode_for(const tc_plan *plan, const Group &g, uint32_t ptr_align, bool checksums)
 {
     if (g.log2_align < 4 || ptr_align < 4) return kModeAny;
+    if (plan->tuning.copy_path == 1 && g.ppt == 1 && !checksums) return kModeAny;  // staged through shared memory on request
     return g.single_run_tiles ? kModeRun : kModeRows;
 }
 
@@ -84,7 +85,7 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     // which measured 3-5 % faster than walking the planes of one block after another.
     Segment whole{0, static_cast<uint32_t>(g.descs.size()), 0, g.descs.empty() ? 0 : g.descs[0].n_outer, 0, 0, 0};
     if (!win && g.tiles_per_desc && !g.descs.empty() && g.descs[0].n_outer > 1 && plan->tuning.tile_order != 1) win = &whole;
-    const int mode = mode_for(g, ptr_align);
+    const int mode = mode_for(plan, g, ptr_align, sums != nullptr);
     if (sums && mode == kModeAny) return fail(TC_ERR_INVALID_ARG, "checksums need 16-byte aligned base pointers");
     const uint32_t grid = grid_for(plan, g, mode, win);
     Params<NPTR> prm;
@@ -112,6 +113,7 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     prm.div_tpo = make_fastdiv(prm.tpo);
     prm.log2_ptr_align = ptr_align;
     prm.stage_bytes = 0;
+    prm.stage_always = plan->tuning.copy_path == 1;
     prm.sums = sums;
     for (size_t i = 0; i < g.n_src; i++) prm.ptr[i] = const_cast<char *>(static_cast<const char *>(src[i]));
     for (size_t i = 0; i < g.n_dst; i++) prm.ptr[g.n_src + i] = static_cast<char *>(dst[i]);

@@ -741,6 +741,44 @@ def test_kv_pack_unpack_migrate_through_misaligned_pointers(shift_pool, shift_pa
         assert np.array_equal(fresh.result(), want_pool), dst_l
 
 
+def test_shared_memory_copy_path_on_aligned_geometry():
+    """tuning.copy_path = 1 sends aligned geometry through the shared-memory path too (it exists
+    to compare the two paths); the bytes must not depend on the path."""
+    rng = np.random.default_rng(78)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=40, B=16, H=8, D=64, E=2, T=(100, 16, 7, 333))
+    L, B, H, D, E = shape
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride, slot_bytes=pool.size)
+    d_pool = dev(pool)
+    smem = dict(copy_path=1)
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, L * 2), T, off, bt, oracle.HND, want)
+    packed = Guarded(want.size)
+    tc.tc_kv_pack(tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_src=bt, tuning=smem)),
+                  [d_pool], [packed.ptr()])
+    assert np.array_equal(packed.result(), want)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_migrate(shape, oracle.NHD, stride, planes_of(pool, L * 2), oracle.NHD, stride, planes_of(want_pool, L * 2), T, off, bt, bt2)
+    fresh = Guarded(pool.size)
+    tc.tc_kv_pack(tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl, T=T, bt_off=off, bt_src=bt, bt_dst=bt2, tuning=smem)),
+                  [d_pool], [fresh.ptr()])
+    assert np.array_equal(fresh.result(), want_pool)
+    ck = small_checkpoint()
+    blob = np.zeros(ck.nbytes_total, dtype=np.uint8)
+    wl.fill_np(blob, 5, "normal")
+    sizes = [ck.nbytes(i) // (4 if ck.split_dim[i] >= 0 else 1) for i in range(ck.N)]
+    want_w = [np.zeros(n, dtype=np.uint8) for n in sizes]
+    oracle.weights(ck.byte_off, ck.E, ck.shapes, ck.split_dim, 2, 4, blob, want_w)
+    outs = [Guarded(n, fill=0xEE) for n in sizes]
+    tc.tc_weights_materialize(tc.tc_plan_create(ck_spec(ck, split_dim=ck.split_dim, rank=2, world=4, tuning=smem)), dev(blob), [o.ptr() for o in outs])
+    for i in range(ck.N):
+        assert np.array_equal(outs[i].result(), want_w[i]), ck.names[i]
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_plan_create(ck_spec(ck, tuning=dict(copy_path=7)))
+    assert e.value.status == tc.TC_ERR_INVALID_ARG
+    assert tc.tc_device_status() == 0
+
+
 # --------------------------------------------------------------------------- random geometries
 @pytest.mark.parametrize("seed", range(24))
 def test_random_geometries_on_the_device(seed):
