@@ -37,6 +37,40 @@ import workloads as wl  # noqa: E402
 GB = 1e9
 
 
+def mem_available() -> int:
+    try:
+        return int(next(l for l in open("/proc/meminfo") if l.startswith("MemAvailable")).split()[1]) * 1024
+    except Exception:
+        return 64 << 30
+
+
+class PinnedArena:
+    """One pinned host allocation for the whole run, carved into the buffers its parts need one
+    after the other (pinning 100 GB takes the better part of a minute; doing it once is the point)."""
+
+    def __init__(self, torch, nbytes: int):
+        t0 = time.perf_counter()
+        self.buf = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+        self.seconds = time.perf_counter() - t0
+        self.used = 0
+
+    def reset(self):
+        self.used = 0
+
+    def take(self, nbytes: int):
+        lo = (self.used + 4095) // 4096 * 4096
+        assert lo + nbytes <= self.buf.numel(), "pinned arena too small"
+        self.used = lo + nbytes
+        return self.buf[lo:lo + nbytes]
+
+
+def burst_host_blocks(args, avail: int, world: int = 1) -> int:
+    """configs[4]: blocks of the pinned host pool - min(262144, half of MemAvailable / 2 MiB)."""
+    if args.host_pool_blocks > 0:
+        return args.host_pool_blocks
+    return min(262144, int(0.5 * avail / world) // wl.LLAMA3_8B_KV.block_bytes)
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -51,38 +85,55 @@ def measured_peaks():
 # clocks
 # --------------------------------------------------------------------------------------
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs.  The sampler is
+    started ahead of the region (nvidia-smi takes a moment to come up) and every sample is stamped
+    on arrival; stop() keeps the samples that arrived between mark_begin() and mark_end()."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
         self.index, self.proc, self.lines = index, None, []
+        self.t0 = self.t1 = None
 
-    def start(self):
+    def start(self, wait_s: float = 3.0):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
                                           "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True, bufsize=1)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
+            t = time.time()
+            while not self.lines and time.time() - t < wait_s:   # until the first sample is in
+                time.sleep(0.02)
         except Exception:
             self.proc = None
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
+
+    def mark_begin(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        self.t1 = time.time()
 
     def stop(self):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        if self.t1 is not None:
+            time.sleep(max(0.0, 0.15 - (time.time() - self.t1)))   # the sample in flight when the region ended
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
+        t0 = self.t0 if self.t0 is not None else 0.0
+        t1 = (self.t1 if self.t1 is not None else time.time()) + 0.15
+        inside = [ln for ts, ln in self.lines if t0 <= ts <= t1]
         sm, mx, reasons = [], [], set()
-        for ln in self.lines:
+        for ln in inside:
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 7:
                 continue
@@ -96,36 +147,47 @@ class ClockSampler:
                     reasons.add(name)
         busy = [c for c in sm if c > 500] or sm
         return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "samples_outside_the_timed_region": len(self.lines) - len(inside)}
 
 
 # --------------------------------------------------------------------------------------
 # CPU oracle leg (cpu_baseline / --impl reference)
 # --------------------------------------------------------------------------------------
 class OracleSample:
-    """The oracle, as it stands, on a bounded sample of the same workload: the requests of
-    wave 0 of a scaled-down pool (`sample_blocks` blocks) packed NHD -> HND and unpacked again
-    through an independent block table.  run() returns (GB/s in read+write bytes, seconds)."""
+    """The oracle, as it stands, on a bounded sample of the same workload, all five rows of the step:
+      a1 + a2  kv_pack NHD -> HND and kv_unpack through an independent block table,
+      a3       kv_migrate pool to pool,
+               (the first requests of the Llama-3-8B KV workload that fit `sample_blocks` blocks)
+      a4 + a5  weights full and the 1-of-8 shard of one decoder layer of the checkpoint (9 tensors,
+               436 MB, dim-0 slabs and dim-1 strided slices like the whole),
+    split over `threads` host threads by request / tensor, plus a1 + a2 on the first requests
+    (`single_blocks` blocks) with ONE thread.  Bytes are counted like the GPU metric: read + written."""
 
-    def __init__(self, sample_blocks: int, threads: int):
+    def __init__(self, sample_blocks: int, threads: int, single_blocks: int = 96):
         import oracle
-        self.oracle, self.threads = oracle, threads
+        self.oracle = oracle
         self.shape = shape = wl.LLAMA3_8B_KV
         NBs = sample_blocks
-        # the first requests of the workload, in order, that fit the sample's block budget
         T_all = wl.config2()[2]
-        keep, used = [], 0
-        for t in T_all:
-            n = (int(t) + shape.B - 1) // shape.B
-            if used + n <= NBs:
-                keep.append(int(t))
-                used += n
-        T = np.array(keep, dtype=np.int64)
-        off = np.concatenate([[0], np.cumsum((T + shape.B - 1) // shape.B)]).astype(np.int64)
-        rng = np.random.default_rng(wl.SEED_BASE + 20)
-        self.src = wl.KVRequests(T, off, rng.permutation(NBs)[:off[-1]].astype(np.int32))
-        self.dst = wl.KVRequests(T, off, rng.permutation(NBs)[:off[-1]].astype(np.int32))
-        self.threads = threads = max(1, min(threads, len(T)))
+
+        def first_requests(budget):
+            keep, used = [], 0
+            for t in T_all:
+                n = (int(t) + shape.B - 1) // shape.B
+                if used + n <= budget:
+                    keep.append(int(t))
+                    used += n
+            return np.array(keep, dtype=np.int64)
+
+        def requests(T, seed):
+            off = np.concatenate([[0], np.cumsum((T + shape.B - 1) // shape.B)]).astype(np.int64)
+            rng = np.random.default_rng(seed)
+            return (wl.KVRequests(T, off, rng.permutation(NBs)[:off[-1]].astype(np.int32)),
+                    wl.KVRequests(T, off, rng.permutation(NBs)[:off[-1]].astype(np.int32)))
+
+        self.src, self.dst = requests(first_requests(NBs), wl.SEED_BASE + 20)
+        self.src1, self.dst1 = requests(first_requests(min(single_blocks, NBs)), wl.SEED_BASE + 21)
+        self.threads = max(1, min(threads, len(self.src.T)))
         pool = np.zeros(NBs * shape.block_bytes, dtype=np.uint8)
         try:
             import torch
@@ -146,28 +208,70 @@ class OracleSample:
         pool2.fill(0)            # touch the pages now: page faults are not part of the oracle's time
         self.packed.fill(0)
         self.planes2 = [pool2[p * per:(p + 1) * per] for p in range(shape.L * 2)]
-        self.desc = (f"oracle kv_pack NHD->HND + kv_unpack of {len(self.src.T)} requests / {self.src.n_blocks} blocks "
-                     f"({self.packed.size / GB:.2f} GB payload) of the Llama-3-8B KV workload, {threads} threads")
+        # one decoder layer of the checkpoint, at its offsets inside a blob that holds just that layer
+        ck = wl.config3()
+        ids = [i for i, n in enumerate(ck.names) if n.startswith("layers.0.")]
+        base = int(ck.byte_off[ids[0]])
+        self.w_off = [int(ck.byte_off[i]) - base for i in ids]
+        self.w_E, self.w_shapes, self.w_split = ck.E[ids], ck.shapes[ids], ck.split_dim[ids]
+        self.w_bytes = [ck.nbytes(i) for i in ids]
+        self.blob = np.zeros(sum(self.w_bytes), dtype=np.uint8)
+        wl.fill_np(self.blob[:1 << 24], wl.SEED_BASE + 3, "normal")   # contents are opaque to the loops
+        self.w_full = [np.zeros(n, dtype=np.uint8) for n in self.w_bytes]
+        self.w_shard = [np.zeros(n // (8 if sd >= 0 else 1), dtype=np.uint8) for n, sd in zip(self.w_bytes, self.w_split)]
+        self.single_bytes = oracle.packed_nbytes(shape.tuple, self.src1.T)
+        self.desc = (f"oracle on {self.threads} threads: kv_pack NHD->HND + kv_unpack + kv_migrate of {len(self.src.T)} requests / "
+                     f"{self.src.n_blocks} blocks ({self.packed.size / GB:.2f} GB payload) of the Llama-3-8B KV workload, weights full + "
+                     f"1-of-8 shard of one decoder layer ({self.blob.size / GB:.2f} GB); 1 thread: kv_pack + kv_unpack of "
+                     f"{len(self.src1.T)} requests / {self.src1.n_blocks} blocks ({self.single_bytes / GB:.2f} GB payload)")
 
-    def run(self):
-        o, s, src, dst = self.oracle, self.shape, self.src, self.dst
-        t0 = time.perf_counter()
-        o.kv_pack(s.tuple, o.NHD, s.chunk_bytes, self.planes, src.T, src.bt_off, src.bt, o.HND, self.packed, threads=self.threads)
-        o.kv_unpack(s.tuple, o.NHD, s.chunk_bytes, self.planes2, dst.T, dst.bt_off, dst.bt, o.HND, self.packed, threads=self.threads)
-        dt = time.perf_counter() - t0
-        return 2 * 2 * self.packed.size / dt / GB, dt
+    def run(self, single_thread: bool = True):
+        """Returns (GB/s over all rows on `threads` threads, seconds of that part, per-part GB/s)."""
+        o, s, src, dst, th = self.oracle, self.shape, self.src, self.dst, self.threads
+        parts, clock = {}, time.perf_counter
+        t0 = clock()
+        o.kv_pack(s.tuple, o.NHD, s.chunk_bytes, self.planes, src.T, src.bt_off, src.bt, o.HND, self.packed, threads=th)
+        o.kv_unpack(s.tuple, o.NHD, s.chunk_bytes, self.planes2, dst.T, dst.bt_off, dst.bt, o.HND, self.packed, threads=th)
+        t1 = clock()
+        o.kv_migrate(s.tuple, o.NHD, s.chunk_bytes, self.planes, o.NHD, s.chunk_bytes, self.planes2, src.T, src.bt_off, src.bt, dst.bt, threads=th)
+        t2 = clock()
+        o.weights(self.w_off, self.w_E, self.w_shapes, np.full(len(self.w_off), -1), 0, 1, self.blob, self.w_full, threads=th)
+        t3 = clock()
+        o.weights(self.w_off, self.w_E, self.w_shapes, self.w_split, 0, 8, self.blob, self.w_shard, threads=th)
+        t4 = clock()
+        kv, wf, wsh = self.packed.size, self.blob.size, sum(a.size for a in self.w_shard)
+        parts["a1_a2_kv_pack_unpack"] = 2 * 2 * kv / (t1 - t0) / GB
+        parts["a3_kv_migrate"] = 2 * kv / (t2 - t1) / GB
+        parts["a4_weights_full"] = 2 * wf / (t3 - t2) / GB
+        parts["a5_weights_shard"] = 2 * wsh / (t4 - t3) / GB
+        total = 2 * (3 * kv + wf + wsh)
+        if single_thread:
+            src1, dst1 = self.src1, self.dst1
+            t5 = clock()
+            o.kv_pack(s.tuple, o.NHD, s.chunk_bytes, self.planes, src1.T, src1.bt_off, src1.bt, o.HND, self.packed, threads=1)
+            o.kv_unpack(s.tuple, o.NHD, s.chunk_bytes, self.planes2, dst1.T, dst1.bt_off, dst1.bt, o.HND, self.packed, threads=1)
+            parts["a1_a2_kv_pack_unpack_1_thread"] = 2 * 2 * self.single_bytes / (clock() - t5) / GB
+        return total / (t4 - t0) / GB, t4 - t0, parts
 
 
 def run_reference(args):
-    """`--impl reference`: the oracle is the reference arm of this tier."""
+    """`--impl reference`: the oracle is the reference arm of this tier.  The sample of a step is
+    sized from a short calibration so that warm-up plus timed steps end within a few minutes."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     threads = os.cpu_count() or 1
-    sample = OracleSample(args.oracle_blocks, threads)
+    blocks = args.oracle_blocks
+    probe = OracleSample(min(64, blocks), threads)
+    _, dt, _ = probe.run(single_thread=False)
+    per_block = dt / max(1, probe.src.n_blocks)          # the layer of weights rides along: an overestimate
+    budget_s = 150.0 / max(1, args.steps + args.warmup)
+    blocks = int(max(32, min(blocks, budget_s / per_block)))
+    del probe
+    sample = OracleSample(blocks, threads)
     vals, dts = [], []
     for i in range(args.warmup + args.steps):
-        v, dt = sample.run()
+        v, dt, _ = sample.run(single_thread=False)
         if i >= args.warmup:
             vals.append(v)
             dts.append(dt)
@@ -274,10 +378,10 @@ def run_ours(args):
     # the CPU baseline goes first, while the host's memory is still unfragmented (the 50+ GB of
     # pinned buffers allocated and freed below slow the oracle down 3-4x if it runs after them)
     threads = os.cpu_count() or 1
-    cpu_v, cpu_desc = None, "skipped"
+    cpu_v, cpu_desc, cpu_parts = None, "skipped", None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sample = OracleSample(args.oracle_blocks, threads)
-        cpu_v, _ = sample.run()
+        cpu_v, _, cpu_parts = sample.run()
         cpu_desc, threads = sample.desc, sample.threads
         del sample
     free, total = torch.cuda.mem_get_info()
@@ -321,7 +425,6 @@ def run_ours(args):
     host_tune = dict(tune)
     if args.host_ctas:
         host_tune["max_ctas"] = args.host_ctas
-    host_flags = 0 if args.host_path == "zerocopy" else tc.TC_PLAN_STAGED
     t_plan0 = time.perf_counter()
     plans = []
     for src, dst in waves:
@@ -330,16 +433,34 @@ def run_ours(args):
             pack=tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, packed_bytes=Q.numel(), bt_src=src.bt, tuning=tune or None, **kw)),
             unpack=tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, packed_bytes=Q.numel(), bt_dst=dst.bt, tuning=tune or None, **kw)),
             migrate=tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, s, src_pool=plA, dst_pool=plB, bt_src=src.bt, bt_dst=dst.bt, tuning=tune or None, **kw)),
-            pack_h=tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, packed_bytes=Q.numel(), bt_src=src.bt, tuning=host_tune or None, flags=host_flags, **kw)),
-            unpack_h=tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, packed_bytes=Q.numel(), bt_dst=dst.bt, tuning=host_tune or None, flags=host_flags, **kw)),
-            payload=int(src.T.sum()) * shape.token_bytes))
+            src=src, dst=dst, payload=int(src.T.sum()) * shape.token_bytes))
     nbytes = [ck.nbytes(i) for i in range(ck.N)]
     mk_w = lambda tn, **kw: tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, blob_bytes=ck.nbytes_total, tuning=tn or None, **kw))
     w_full, w_shard = mk_w(tune), mk_w(tune, split_dim=ck.split_dim, rank=args.shard_rank, world=W)
-    w_full_h = mk_w(host_tune, flags=host_flags)
-    w_shard_h = mk_w(host_tune, split_dim=ck.split_dim, rank=args.shard_rank, world=W, flags=host_flags)
     plan_ms = 1e3 * (time.perf_counter() - t_plan0)
-    n_plans = 5 * len(waves) + 4
+    n_plans = 3 * len(waves) + 2
+
+    def host_plans(path):
+        """The same calls with the packed buffer and the blob in pinned host memory: plans for the
+        staged path (copy engines + staging rings) or the zero-copy path (kernel loads / stores)."""
+        flags = tc.TC_PLAN_STAGED if path == "staged" else 0
+        hp = dict(kv=[], path=path)
+        for p in plans:
+            kw = dict(T=p["src"].T, bt_off=p["src"].bt_off, tuning=host_tune or None, flags=flags, packed_layout=tc.TC_HND, packed_bytes=Q.numel())
+            hp["kv"].append((tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, bt_src=p["src"].bt, **kw)),
+                             tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, bt_dst=p["dst"].bt, **kw)), p["payload"]))
+        hp["w_full"] = mk_w(host_tune, flags=flags)
+        hp["w_shard"] = mk_w(host_tune, split_dim=ck.split_dim, rank=args.shard_rank, world=W, flags=flags)
+        hp["launches"] = (sum(a.stats().launches_per_execute + b.stats().launches_per_execute for a, b, _ in hp["kv"])
+                          + hp["w_full"].stats().launches_per_execute + hp["w_shard"].stats().launches_per_execute)
+        return hp
+
+    def drop_host_plans(hp):
+        for a, b, _ in hp["kv"]:
+            a.destroy()
+            b.destroy()
+        hp["w_full"].destroy()
+        hp["w_shard"].destroy()
 
     rows = {k: Row(k, m) for k, m in (("a1_kv_pack", "rows"), ("a2_kv_unpack", "rows"), ("a3_kv_migrate", "run"),
                                       ("a4_weights_full", "run"), ("a5_weights_shard", "rows"))}
@@ -367,13 +488,14 @@ def run_ours(args):
 
     barrier = ranks.barrier
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     with torch.cuda.stream(stream):
         for _ in range(args.warmup):
             step([])
         barrier()
-        sampler = ClockSampler(local)
-        if rank == 0:
-            sampler.start()
+        sampler.mark_begin()
         ev_all = []
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0.record(stream)
@@ -383,6 +505,7 @@ def run_ours(args):
             ev_all.append(ev)
         t1.record(stream)
         barrier()
+        sampler.mark_end()
         clocks = sampler.stop() if rank == 0 else None
     total_ms = t0.elapsed_time(t1)
     for ev in ev_all:
@@ -393,8 +516,6 @@ def run_ours(args):
             rows[k].ms.append(v)
     step_bytes = sum(r.bytes for r in rows.values())
     launches_per_step = sum(r.launches for r in rows.values())
-    e2e_launches = (sum(p["pack_h"].stats().launches_per_execute + p["unpack_h"].stats().launches_per_execute for p in plans)
-                    + w_full_h.stats().launches_per_execute + w_shard_h.stats().launches_per_execute)
     total_ms = ranks.max_ms(total_ms)
     value = world * step_bytes * args.steps / (total_ms * 1e-3) / GB
 
@@ -416,28 +537,37 @@ def run_ours(args):
 
     # ---------------- e2e: packed buffer and blob in pinned host memory --------------------
     e2e = None
+    e2e_all = {}
     e2e_skipped = None
+    avail = mem_available()
+    want_extras = not args.no_extras and world == 1
+    burst_bytes = 0
+    if want_extras and (args.extras == "all" or "config4" in args.extras.split(",")) and not args.only_kv_shapes and not args.only_misaligned:
+        burst_bytes = burst_host_blocks(args, avail) * shape.block_bytes
+    can_duplex = False
     if not args.no_e2e:
         # pinned host memory is per process: N ranks on one node share the node's RAM
-        try:
-            avail = int(next(l for l in open("/proc/meminfo") if l.startswith("MemAvailable")).split()[1]) * 1024
-        except Exception:
-            avail = 64 << 30
         budget = 0.6 * avail / world
         need_duplex, need_serial = 2 * max_packed + ck.nbytes_total, max_packed + ck.nbytes_total
-        if args.e2e_schedule == "duplex" and need_duplex > budget:
-            args.e2e_schedule = "serial"
+        can_duplex = need_duplex <= budget
         if need_serial > budget:
             e2e_skipped = (f"skipped: {need_serial / GB:.0f} GB of pinned host memory per rank needed, "
                            f"{budget / GB:.0f} GB available per rank with {world} ranks on this node")
+    e2e_bytes = 0 if (args.no_e2e or e2e_skipped) else ((2 if can_duplex else 1) * max_packed + ck.nbytes_total + (1 << 20))
+    arena = PinnedArena(torch, max(e2e_bytes, burst_bytes)) if max(e2e_bytes, burst_bytes) else None
+    args.pinned_arena = arena
     if not args.no_e2e and e2e_skipped is None:
-        Qh = torch.empty(max_packed, dtype=torch.uint8).pin_memory()
-        blob_h = torch.empty(ck.nbytes_total, dtype=torch.uint8).pin_memory()
+        Qh = arena.take(max_packed)
+        Qh2 = arena.take(max_packed) if can_duplex else Qh
+        blob_h = arena.take(ck.nbytes_total)
         blob_h.copy_(blob)
-        probe = torch.empty(4096, dtype=torch.uint8).pin_memory()
+        probe = torch.empty(4096, dtype=torch.uint8, pin_memory=True)
+        stream_u = torch.cuda.Stream()
+        ev_fork, ev_join = torch.cuda.Event(), torch.cuda.Event()
         torch.cuda.synchronize()
+        n_c = min(Qh.numel(), 4 << 30)
 
-        def ceiling(fn, nbytes):  # cudaMemcpyAsync on the same pinned allocation, best of 3
+        def ceiling(fn, nbytes):  # cudaMemcpyAsync on the same pinned allocation, best of 4
             best = 1e9
             for _ in range(4):
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -448,99 +578,108 @@ def run_ours(args):
                 best = min(best, a.elapsed_time(b))
             return nbytes / (best * 1e-3) / GB
 
-        with torch.cuda.stream(stream):
-            n_c = min(Qh.numel(), 4 << 30)
-            ceil_h2d = ceiling(lambda: Q[:n_c].copy_(Qh[:n_c], non_blocking=True), n_c)
-            ceil_d2h = ceiling(lambda: Qh[:n_c].copy_(Q[:n_c], non_blocking=True), n_c)
-
-        duplex = args.e2e_schedule == "duplex"
-        Qh2 = torch.empty(max_packed, dtype=torch.uint8).pin_memory() if duplex else Qh
-        Qhs = (Qh, Qh2)
-        stream_u = torch.cuda.Stream() if duplex else stream
-        su = stream_u.cuda_stream
-        ev_packed = [torch.cuda.Event() for _ in range(2)]
-        ev_unpacked = [torch.cuda.Event() for _ in range(2)]
-        ev_fork, ev_join = torch.cuda.Event(), torch.cuda.Event()
-
-        def bidir_ceiling():  # both directions at once with cudaMemcpyAsync, GB/s summed
-            n_c = min(Qh.numel(), 4 << 30)
-            best = 1e9
-            for _ in range(3):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream)
-                ev_fork.record(stream)
-                stream_u.wait_event(ev_fork)
-                Qh[:n_c].copy_(Q[:n_c], non_blocking=True)
-                with torch.cuda.stream(stream_u):
-                    poolB[:n_c].copy_(Qh2[:n_c], non_blocking=True)
-                    ev_join.record(stream_u)
-                stream.wait_event(ev_join)
-                b.record(stream)
-                torch.cuda.synchronize()
-                best = min(best, a.elapsed_time(b))
-            return 2 * n_c / (best * 1e-3) / GB
-
-        def e2e_step():
-            """Offload every wave to pinned host memory and reload it into the second pool; load the
-            weights from the pinned blob.  duplex: the link is full duplex, so wave k+1 is offloaded
-            (stream) while wave k is reloaded (stream_u), through two host buffers."""
-            h2d = d2h = 0
+        def both_ways():  # both directions at once with cudaMemcpyAsync
             ev_fork.record(stream)
             stream_u.wait_event(ev_fork)
-            tc.tc_weights_materialize(w_full_h, blob_h, full_ptrs, su)
-            tc.tc_weights_materialize(w_shard_h, blob_h, shard_ptrs, su)
-            h2d += sum(full_sizes) + sum(shard_sizes)
-            for k, p in enumerate(plans):
-                i = k % 2 if duplex else 0
-                if k >= (2 if duplex else 1):
-                    stream.wait_event(ev_unpacked[i])                    # the host buffer is free again
-                tc.tc_kv_pack(p["pack_h"], [poolA], [Qhs[i]], sp)        # offload (device -> host)
-                ev_packed[i].record(stream)
-                stream_u.wait_event(ev_packed[i])
-                tc.tc_kv_unpack(p["unpack_h"], [Qhs[i]], [poolB], su)    # reload (host -> device)
-                ev_unpacked[i].record(stream_u)
-                d2h += p["payload"]
-                h2d += p["payload"]
+            Qh[:n_c].copy_(Q[:n_c], non_blocking=True)
             with torch.cuda.stream(stream_u):
-                probe.copy_(dst_full[-4096:], non_blocking=True)         # read a result back
+                poolB[:n_c].copy_(Qh2[:n_c], non_blocking=True)
                 ev_join.record(stream_u)
             stream.wait_event(ev_join)
-            d2h += 4096
-            return h2d, d2h
 
         with torch.cuda.stream(stream):
-            ceil_bidir = bidir_ceiling() if duplex else None
-            for _ in range(args.e2e_warmup):
-                e2e_step()
-            barrier()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            for _ in range(args.e2e_steps):
-                h2d, d2h = e2e_step()
-            b.record(stream)
-            barrier()
-        e_ms = a.elapsed_time(b)
-        e_ms = ranks.max_ms(e_ms)
-        # same byte convention as `value`: every payload byte is read once and written once
-        e2e = {"value": world * 2 * (h2d + d2h - 4096) * args.e2e_steps / (e_ms * 1e-3) / GB, "unit": "GB/s",
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
-               "ms_per_step": e_ms / args.e2e_steps,
-               "host_link_GBps": world * (h2d + d2h) * args.e2e_steps / (e_ms * 1e-3) / GB,
-               "host_link_ceiling_GBps": {"h2d_cudaMemcpyAsync": ceil_h2d, "d2h_cudaMemcpyAsync": ceil_d2h,
-                                          "both_directions_at_once_summed": ceil_bidir},
-               "host_link_frac_of_ceiling": (h2d + d2h) * args.e2e_steps / (e_ms * 1e-3) / GB /
-                                            (ceil_bidir if duplex else (h2d + d2h) / (h2d / ceil_h2d + d2h / ceil_d2h)),
-               "kv_host_path": args.host_path, "schedule": args.e2e_schedule,
-               "note": "packed KV buffer and weight blob in pinned host memory. staged: copy engines + device staging rings + "
-                       "D2D kernel (the TP shard's strided slices stay zero copy); zerocopy: kernel loads/stores on host memory"}
-        del Qh, Qh2, Qhs, blob_h
+            ceil_h2d = ceiling(lambda: Q[:n_c].copy_(Qh[:n_c], non_blocking=True), n_c)
+            ceil_d2h = ceiling(lambda: Qh[:n_c].copy_(Q[:n_c], non_blocking=True), n_c)
+            ceil_bidir = ceiling(both_ways, 2 * n_c) if can_duplex else None
+        ceilings = {"h2d_cudaMemcpyAsync": ceil_h2d, "d2h_cudaMemcpyAsync": ceil_d2h, "both_directions_at_once_summed": ceil_bidir}
+
+        def run_e2e(hp, duplex, steps, warmup):
+            """Offload every wave to pinned host memory and reload it into the second pool; load the
+            weights from the pinned blob; read a result back.  duplex: the link is full duplex, so wave
+            k+1 is offloaded (stream) while wave k is reloaded (stream_u), through two host buffers."""
+            Qhs = (Qh, Qh2)
+            su = stream_u.cuda_stream if duplex else sp
+            s_u = stream_u if duplex else stream
+            ev_packed = [torch.cuda.Event() for _ in range(2)]
+            ev_unpacked = [torch.cuda.Event() for _ in range(2)]
+
+            def one_step():
+                h2d = d2h = 0
+                ev_fork.record(stream)
+                s_u.wait_event(ev_fork)
+                tc.tc_weights_materialize(hp["w_full"], blob_h, full_ptrs, su)
+                tc.tc_weights_materialize(hp["w_shard"], blob_h, shard_ptrs, su)
+                h2d += sum(full_sizes) + sum(shard_sizes)
+                for k, (pack_h, unpack_h, payload) in enumerate(hp["kv"]):
+                    i = k % 2 if duplex else 0
+                    if k >= (2 if duplex else 1):
+                        stream.wait_event(ev_unpacked[i])                 # the host buffer is free again
+                    tc.tc_kv_pack(pack_h, [poolA], [Qhs[i]], sp)         # offload (device -> host)
+                    ev_packed[i].record(stream)
+                    s_u.wait_event(ev_packed[i])
+                    tc.tc_kv_unpack(unpack_h, [Qhs[i]], [poolB], su)     # reload (host -> device)
+                    ev_unpacked[i].record(s_u)
+                    d2h += payload
+                    h2d += payload
+                with torch.cuda.stream(s_u):
+                    probe.copy_(dst_full[-4096:], non_blocking=True)      # read a result back
+                    ev_join.record(s_u)
+                stream.wait_event(ev_join)
+                d2h += 4096
+                return h2d, d2h
+
+            with torch.cuda.stream(stream):
+                for _ in range(warmup):
+                    one_step()
+                barrier()
+                marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+                marks[0].record(stream)
+                for k in range(steps):
+                    h2d, d2h = one_step()
+                    marks[k + 1].record(stream)
+                barrier()
+            per_step = [marks[k].elapsed_time(marks[k + 1]) for k in range(steps)]
+            e_ms = ranks.max_ms(marks[0].elapsed_time(marks[steps]))
+            link = world * (h2d + d2h) * steps / (e_ms * 1e-3) / GB
+            serial_ceiling = (h2d + d2h) / (h2d / ceil_h2d + d2h / ceil_d2h)
+            # same byte convention as `value`: every payload byte is read once and written once
+            return {"value": world * 2 * (h2d + d2h - 4096) * steps / (e_ms * 1e-3) / GB, "unit": "GB/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": steps, "warmup": warmup,
+                    "ms_per_step": e_ms / steps, "ms_per_step_median": statistics.median(per_step),
+                    "ms_per_step_min_max": [min(per_step), max(per_step)],
+                    "host_link_GBps": link, "host_link_ceiling_GBps": ceilings,
+                    "host_link_frac_of_ceiling": link / world / (ceil_bidir if duplex else serial_ceiling),
+                    "ceiling_used": "both_directions_at_once_summed" if duplex else "serial mix of the one-direction ceilings",
+                    "kv_host_path": hp["path"], "schedule": "duplex" if duplex else "serial", "gpu_launches_per_step": hp["launches"]}
+
+        want_duplex = args.e2e_schedule == "duplex" and can_duplex
+        runs = [("staged", want_duplex)] if args.host_path == "staged" else []
+        runs += [("zerocopy", False), ("zerocopy", True)] if can_duplex else [("zerocopy", False)]
+        if args.host_path == "zerocopy":
+            runs = [r for r in runs if r[0] == "zerocopy"]
+        made = {}
+        for path, duplex in runs:
+            if path not in made:
+                made[path] = host_plans(path)
+            key = f"{path}_{'duplex' if duplex else 'serial'}"
+            e2e_all[key] = run_e2e(made[path], duplex, args.e2e_steps, args.e2e_warmup)
+        for hp in made.values():
+            drop_host_plans(hp)
+        best = max(e2e_all, key=lambda k: e2e_all[k]["host_link_GBps"])
+        e2e = dict(e2e_all[best])
+        e2e["note"] = ("the fastest of the host paths measured in this run (all of them under e2e_paths). Packed KV buffer and "
+                       "weight blob in pinned host memory. staged: copy engines + device staging rings + D2D kernel (the TP "
+                       "shard's strided slices stay zero copy); zerocopy: kernel loads / stores on host memory; host_link_GBps "
+                       "counts every byte once, in its direction; `value` counts it read and written like the device metric")
+        del Qh, Qh2, blob_h
+        arena.reset()
 
     extras = None
-    if not args.no_extras and world == 1:
+    if want_extras:
         for p in plans:
-            for k in ("pack", "unpack", "migrate", "pack_h", "unpack_h"):
+            for k in ("pack", "unpack", "migrate"):
                 p[k].destroy()
-        for w in (w_full, w_shard, w_full_h, w_shard_h):
+        for w in (w_full, w_shard):
             w.destroy()
         del poolA, poolB, Q, blob, dst_full, dst_shard, plans
         torch.cuda.empty_cache()
@@ -587,9 +726,10 @@ def run_ours(args):
                    "parallelism": "replicas only" if world > 1 else "1 GPU", "plans": n_plans, "plan_create_ms_total": plan_ms},
         "clocks": clocks, "e2e": e2e if e2e is not None else ({"value": None, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0, "note": e2e_skipped or "skipped (--no-e2e)"}),
         "gpu_launches": launches_per_step * args.steps,
-        "e2e_gpu_launches_per_step": e2e_launches,
+        "e2e_zerocopy": e2e_all.get("zerocopy_duplex") or e2e_all.get("zerocopy_serial"),
+        "e2e_paths": e2e_all or None,
         "roofline": roofline, "rows": per_row, "other_workloads": extras,
-        "cpu_baseline": {"value": cpu_v, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": cpu_desc},
+        "cpu_baseline": {"value": cpu_v, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": cpu_desc, "parts_GBps": cpu_parts},
     }
     print(json.dumps(line))
     ranks.close()
@@ -627,7 +767,7 @@ def cold_path(args, tc, torch, stream):
         return {"skipped": f"no room for a {ck.nbytes_total} byte file under {root}"}
     blob = torch.empty(ck.nbytes_total, dtype=torch.uint8, device="cuda")
     wl.fill_torch(blob, wl.SEED_BASE + 3, "normal")
-    host = torch.empty(ck.nbytes_total, dtype=torch.uint8).pin_memory()
+    host = torch.empty(ck.nbytes_total, dtype=torch.uint8, pin_memory=True)
     host.copy_(blob)
     header = 4096 + 8 * ck.N
     fdw, path = tempfile.mkstemp(prefix="tc_cold_", suffix=".bin", dir=root)
@@ -866,20 +1006,9 @@ def misaligned(args, tc, torch, stream):
     return out
 
 
-def run_extras(args, tc, torch, stream):
-    """Secondary workloads, reported beside the headline: configs[3] (70B-shaped pool-to-pool
-    migration, one wave) and configs[4] (prefix-reload burst: one mixed plan per scheduler step,
-    created and executed inside the timed region, both directions concurrently over the host
-    link with zero-copy kernels)."""
-    out = {}
+def extra_config0(args, tc, torch, stream, out):
     sp = stream.cuda_stream
     u8 = dict(dtype=torch.uint8, device="cuda")
-    if args.only_kv_shapes:  # profiler runs: just the KV geometries, a few GB on the device
-        out["rows a1-a3 on other KV geometries (8 GiB pools, first wave)"] = kv_shapes(args, tc, torch, stream)
-        return out
-    if args.only_misaligned:
-        out["rows a1-a5: copy paths and misaligned base pointers (8 GiB pool, 4 GB checkpoint)"] = misaligned(args, tc, torch, stream)
-        return out
     # ---- configs[0]: 1.4 MB, launch-latency bound: microseconds and plans per second
     shape, NB1, src1, dst1 = wl.config1()
     pool1 = torch.empty(2 * NB1 * shape.chunk_bytes, **u8)
@@ -929,6 +1058,11 @@ def run_extras(args, tc, torch, stream):
         "us_per_pack_plus_unpack_stream": us_pair, "us_per_pack_plus_unpack_cuda_graph": us_pair_graph,
         "plans_per_s_create_execute_sync_destroy": 400 / wall, "payload_bytes": packed1.numel()}
     del pool1, fresh1, packed1
+
+
+def extra_weights(args, tc, torch, stream, out):
+    sp = stream.cuda_stream
+    u8 = dict(dtype=torch.uint8, device="cuda")
     # ---- configs[2] again, with the integrity checksum folded into the copy
     ck = wl.config3() if not args.small else wl.llama_checkpoint(layers=1, vocab=16032)
     blob = torch.empty(ck.nbytes_total, **u8)
@@ -960,44 +1094,57 @@ def run_extras(args, tc, torch, stream):
         "payload_bytes": sum(sizes), "GBps_per_rank": per_rank}
     del blob, dstw
     torch.cuda.empty_cache()
-    out["weights cold path: blob streamed from a file"] = cold_path(args, tc, torch, stream)
-    out["transform_into: MoE expert stacking (Qwen3-30B-A3B-shaped layers)"] = moe_stacking(args, tc, torch, stream)
-    out["rows a1-a3 on other KV geometries (8 GiB pools, first wave)"] = kv_shapes(args, tc, torch, stream)
-    out["rows a1-a5: copy paths and misaligned base pointers (8 GiB pool, 4 GB checkpoint)"] = misaligned(args, tc, torch, stream)
-    # ---- configs[3]
+
+
+def extra_config3(args, tc, torch, stream, out):
+    """configs[3]: Llama-3-70B-shaped KV migration between two pools on the GPU.  The workload has
+    about 35 waves of <= 4096 blocks; five of them are timed - the first, the last and three seeded
+    ones in between - each with its own plan (created outside the timed launches)."""
+    sp = stream.cuda_stream
+    u8 = dict(dtype=torch.uint8, device="cuda")
     shape = wl.LLAMA3_70B_KV
     free, _ = torch.cuda.mem_get_info()
     NB = 4096
     while 2 * NB * shape.block_bytes > 0.8 * free:
         NB //= 2
-    _, _, _, waves = wl.config4(NB=NB, max_waves=1)
-    src, dst = waves[0]
+    _, _, _, waves = wl.config4(NB=NB)
+    if args.small:
+        waves = waves[:1]
+    pick = sorted({0, len(waves) - 1, *[int(x) for x in np.random.default_rng(wl.SEED_BASE + 40).choice(len(waves), size=min(3, len(waves)), replace=False)]})
     A = torch.empty(NB * shape.block_bytes, **u8)
     A.fill_(7)
     B = torch.empty(NB * shape.block_bytes, **u8)
     B.fill_(9)
     pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=A.numel())
-    torch.cuda.synchronize()  # the fills above are still running; plan upload would wait for them
-    t0 = time.perf_counter()
-    mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape.tuple, src_pool=pl, dst_pool=pl, T=src.T, bt_off=src.bt_off, bt_src=src.bt, bt_dst=dst.bt))
-    create_ms = 1e3 * (time.perf_counter() - t0)
-    payload = int(src.T.sum()) * shape.token_bytes
-    ms_mig = b2b_ms(torch, stream, lambda: tc.tc_kv_pack(mig, [A], [B], sp), reps=3)
-    out["configs[3] 70B KV migrate (one wave)"] = {
-        "pool_blocks": NB, "requests": len(src.T), "blocks": src.n_blocks, "payload_bytes": payload,
-        "GBps": 2 * payload / (ms_mig * 1e-3) / GB, "ms": ms_mig, "plan_create_ms": create_ms}
-    mig.destroy()
-    # the same wave into an HND pool (layout transform fused into the migration) ...
     pl_hnd = tc.pool(tc.TC_HND, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=A.numel())
-    mig_t = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape.tuple, src_pool=pl, dst_pool=pl_hnd, T=src.T, bt_off=src.bt_off, bt_src=src.bt, bt_dst=dst.bt))
-
-    def timed(fn):
-        return b2b_ms(torch, stream, fn, reps=3)
-    ms_t = timed(lambda: tc.tc_kv_pack(mig_t, [A], [B], sp))
-    mig_t.destroy()
-    out["configs[3] 70B KV migrate (one wave)"]["GBps_into_an_HND_pool"] = 2 * payload / (ms_t * 1e-3) / GB
-    # ... and, for comparison, unfused: pack into a device buffer, then unpack (twice the traffic).
-    # The buffer takes what memory is left, so only the first requests that fit take part.
+    torch.cuda.synchronize()  # the fills above are still running; plan upload would wait for them
+    per_wave, create, tot_bytes, tot_ms, tot_ms_t = [], [], 0, 0.0, 0.0
+    for w in pick:
+        src, dst = waves[w]
+        kw = dict(T=src.T, bt_off=src.bt_off, bt_src=src.bt, bt_dst=dst.bt)
+        t0 = time.perf_counter()
+        mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape.tuple, src_pool=pl, dst_pool=pl, **kw))
+        create.append(1e3 * (time.perf_counter() - t0))
+        mig_t = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape.tuple, src_pool=pl, dst_pool=pl_hnd, **kw))
+        payload = int(src.T.sum()) * shape.token_bytes
+        ms = b2b_ms(torch, stream, lambda: tc.tc_kv_pack(mig, [A], [B], sp), reps=3)
+        ms_t = b2b_ms(torch, stream, lambda: tc.tc_kv_pack(mig_t, [A], [B], sp), reps=3)
+        per_wave.append({"wave": w, "requests": len(src.T), "blocks": src.n_blocks, "payload_bytes": payload, "ms": ms,
+                         "GBps": 2 * payload / (ms * 1e-3) / GB, "GBps_into_an_HND_pool": 2 * payload / (ms_t * 1e-3) / GB})
+        tot_bytes += payload
+        tot_ms += ms
+        tot_ms_t += ms_t
+        mig.destroy()
+        mig_t.destroy()
+    peak, _ = measured_peaks()
+    res = {"pool_blocks": NB, "waves_in_workload": len(waves), "waves_timed": pick, "payload_bytes": tot_bytes,
+           "GBps": 2 * tot_bytes / (tot_ms * 1e-3) / GB, "frac_of_measured_peak": 2 * tot_bytes / (tot_ms * 1e-3) / GB / peak,
+           "GBps_into_an_HND_pool": 2 * tot_bytes / (tot_ms_t * 1e-3) / GB, "ms_total": tot_ms,
+           "plan_create_ms": statistics.mean(create), "per_wave": per_wave}
+    out["configs[3] 70B KV migrate (first, last and three seeded waves)"] = res
+    # for comparison, unfused: pack into a device buffer, then unpack (twice the traffic).  The
+    # buffer takes what memory is left, so only the first requests of wave 0 that fit take part.
+    src, dst = waves[0]
     free, _ = torch.cuda.mem_get_info()
     budget = int(0.8 * free)
     k = int(np.searchsorted(np.cumsum(src.T) * shape.token_bytes, budget, side="right"))
@@ -1009,58 +1156,179 @@ def run_extras(args, tc, torch, stream):
         pk = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape.tuple, src_pool=pl, packed_layout=tc.TC_NHD, T=Tk, bt_off=offk, bt_src=src.bt[:nblk]))
         up = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape.tuple, dst_pool=pl, packed_layout=tc.TC_NHD, T=Tk, bt_off=offk, bt_dst=dst.bt[:nblk]))
         fused = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape.tuple, src_pool=pl, dst_pool=pl, T=Tk, bt_off=offk, bt_src=src.bt[:nblk], bt_dst=dst.bt[:nblk]))
-        ms_two = timed(lambda: (tc.tc_kv_pack(pk, [A], [Q], sp), tc.tc_kv_unpack(up, [Q], [B], sp)))
-        ms_one = timed(lambda: tc.tc_kv_pack(fused, [A], [B], sp))
-        out["configs[3] 70B KV migrate (one wave)"]["fused_vs_pack_then_unpack"] = {
-            "requests": k, "payload_bytes": part, "ms_fused_migrate": ms_one, "ms_pack_then_unpack_through_a_device_buffer": ms_two}
+        ms_two = b2b_ms(torch, stream, lambda: (tc.tc_kv_pack(pk, [A], [Q], sp), tc.tc_kv_unpack(up, [Q], [B], sp)), reps=3)
+        ms_one = b2b_ms(torch, stream, lambda: tc.tc_kv_pack(fused, [A], [B], sp), reps=3)
+        res["fused_vs_pack_then_unpack"] = {"requests": k, "payload_bytes": part, "ms_fused_migrate": ms_one,
+                                            "ms_pack_then_unpack_through_a_device_buffer": ms_two}
         for p_ in (pk, up, fused):
             p_.destroy()
         del Q
     del A, B
     torch.cuda.empty_cache()
-    # ---- configs[4]
+
+
+def extra_config4(args, tc, torch, stream, out):
+    """configs[4]: multi-turn prefix-reload burst.  512 sessions; every scheduler step reloads
+    about 6 100 cached 2 MiB pages from a paged pinned host pool into scattered device blocks and
+    offloads about 1 280 new blocks, one MIXED plan per step (created, executed on two streams,
+    synchronised and destroyed inside the timed region), 200 steps.  The ceilings it is held
+    against are cudaMemcpyAsync on the burst's own pinned pool, measured here: one direction
+    alone and both directions at once."""
+    sp = stream.cuda_stream
+    u8 = dict(dtype=torch.uint8, device="cuda")
     shape = wl.LLAMA3_8B_KV
-    NBd, NBh, n_steps = 20000, args.host_pool_blocks, args.burst_steps
+    NBd, n_steps = 20000, args.burst_steps
+    arena = getattr(args, "pinned_arena", None)
+    rule = burst_host_blocks(args, mem_available() + (arena.buf.numel() if arena else 0))
+    NBh = min(rule, arena.buf.numel() // shape.block_bytes) if arena else rule
     dev = torch.empty(NBd * shape.block_bytes, **u8)
     dev.fill_(3)
-    host = torch.empty(NBh * shape.block_bytes, dtype=torch.uint8).pin_memory()
+    if arena is None:
+        arena = PinnedArena(torch, NBh * shape.block_bytes)
+    arena.reset()
+    host = arena.take(NBh * shape.block_bytes)
+    pin_s = arena.seconds
     dev_pool = tc.pool(tc.TC_NHD, NBd, 1, plane_stride=NBd * shape.chunk_bytes, slot_bytes=dev.numel())
     host_pool = tc.pool(tc.TC_HND, NBh, 1, plane_stride=shape.chunk_bytes, block_stride=shape.block_bytes, slot_bytes=host.numel())
     s2 = torch.cuda.Stream()
-    create, h2d, d2h = [], 0, 0
-    steps = list(wl.config5(NB_dev=NBd, NB_host=NBh, steps=n_steps + 1))
-    torch.cuda.synchronize()
-    t_all = None
-    for i, st in enumerate(steps):
-        if i == 1:  # step 0 is the warm-up
+    # ceilings: contiguous cudaMemcpyAsync on this pool, 4 GiB, best of 3
+    n_c = min(host.numel() // 2, 4 << 30)
+    fork, join = torch.cuda.Event(), torch.cuda.Event()
+
+    def best_of(fn, nbytes, reps=3):
+        best = 1e9
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(stream):
+                a.record(stream)
+                fn()
+                b.record(stream)
             torch.cuda.synchronize()
-            t_all = time.perf_counter()
-        t0 = time.perf_counter()
-        plan = tc.tc_plan_create(tc.kv_spec(
-            tc.TC_KV_MIXED, shape.tuple, src_pool=dev_pool, dst_pool=host_pool,
-            T=st.offload_T, bt_off=st.offload_off, bt_src=st.offload_dev, bt_dst=st.offload_host,
-            reload=dict(T=st.reload_T, bt_off=st.reload_off, bt_src=st.reload_host, bt_dst=st.reload_dev),
-            flags=0 if args.host_path == "zerocopy" else tc.TC_PLAN_STAGED))
-        if i >= 1:
-            create.append(1e3 * (time.perf_counter() - t0))
-            h2d += int(st.reload_T.sum()) * shape.token_bytes
-            d2h += int(st.offload_T.sum()) * shape.token_bytes
-        # the short offload is enqueued first: the reload's ~6 000 page copies fill the driver's
-        # stream queue, so whatever is enqueued after it only starts when it is nearly done
-        tc.tc_kv_pack(plan, [dev], [host], s2.cuda_stream)
-        tc.tc_kv_unpack(plan, [host], [dev], sp)
-        torch.cuda.synchronize()   # a scheduler step ends when both directions have landed
-        plan.destroy()
-    wall = time.perf_counter() - t_all
-    out["configs[4] prefix-reload burst (mixed plan per step)"] = {
-        "steps": n_steps, "sessions": 512, "host_pool_blocks": NBh, "device_pool_blocks": NBd,
-        "plans_per_s": n_steps / wall, "ms_per_step_wall": 1e3 * wall / n_steps, "plan_create_ms": statistics.mean(create),
-        "h2d_GBps": h2d / wall / GB, "d2h_GBps": d2h / wall / GB, "link_GBps_both_directions": (h2d + d2h) / wall / GB,
-        "h2d_bytes_per_step": h2d // n_steps, "d2h_bytes_per_step": d2h // n_steps,
-        "host_path": args.host_path,
-        "note": "wall clock over create + execute + synchronise of every step; reload and offload run concurrently on two streams"}
+            best = min(best, a.elapsed_time(b))
+        return nbytes / (best * 1e-3) / GB
+
+    dup = {}
+
+    def both():  # each direction timed on its own stream while the other runs
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        fork.record(stream)
+        s2.wait_event(fork)
+        ev[0].record(stream)
+        dev[:n_c].copy_(host[:n_c], non_blocking=True)
+        ev[1].record(stream)
+        with torch.cuda.stream(s2):
+            ev[2].record(s2)
+            host[n_c:2 * n_c].copy_(dev[n_c:2 * n_c], non_blocking=True)
+            ev[3].record(s2)
+            join.record(s2)
+        stream.wait_event(join)
+        dup["ev"] = ev
+
+    ceil_h2d = best_of(lambda: dev[:n_c].copy_(host[:n_c], non_blocking=True), n_c)
+    ceil_d2h = best_of(lambda: host[:n_c].copy_(dev[:n_c], non_blocking=True), n_c)
+    ceil_both = best_of(both, 2 * n_c)
+    # rates of the two directions while both are busy (from the last repetition: the shorter copy ends
+    # first, so these are lower bounds of the contended rates)
+    dup_h2d = n_c / (dup["ev"][0].elapsed_time(dup["ev"][1]) * 1e-3) / GB
+    dup_d2h = n_c / (dup["ev"][2].elapsed_time(dup["ev"][3]) * 1e-3) / GB
+
+    def ideal_ms(h2d_bytes, d2h_bytes):
+        """The shortest a step can take at cudaMemcpyAsync rates on contiguous memory: both directions
+        run together at their contended rates until the shorter one is done, the rest runs alone."""
+        t_h, t_d = h2d_bytes / (dup_h2d * GB), d2h_bytes / (dup_d2h * GB)
+        if t_d <= t_h:
+            return 1e3 * (t_d + (h2d_bytes - dup_h2d * GB * t_d) / (ceil_h2d * GB))
+        return 1e3 * (t_h + (d2h_bytes - dup_d2h * GB * t_h) / (ceil_d2h * GB))
+
+    paths = ["staged", "mixed", "zerocopy"] if args.burst_paths == "all" else [args.burst_paths]
+    results = {}
+    for path in paths:
+        # a comparison path runs a tenth of the steps; the reported one runs them all
+        steps_here = n_steps if path == paths[0] else max(2, n_steps // 10)
+        create, h2d, d2h = [], 0, 0
+        flags = {"staged": tc.TC_PLAN_STAGED, "mixed": tc.TC_PLAN_STAGED | tc.TC_PLAN_OFFLOAD_ZERO_COPY, "zerocopy": 0}[path]
+        torch.cuda.synchronize()
+        t_all = None
+        dev_ms = []
+        all_steps = list(wl.config5(NB_dev=NBd, NB_host=NBh, steps=steps_here + 1))  # drawn before the clock starts
+        for i, st in enumerate(all_steps):
+            if i == 1:  # step 0 is the warm-up
+                torch.cuda.synchronize()
+                t_all = time.perf_counter()
+            t0 = time.perf_counter()
+            plan = tc.tc_plan_create(tc.kv_spec(
+                tc.TC_KV_MIXED, shape.tuple, src_pool=dev_pool, dst_pool=host_pool,
+                T=st.offload_T, bt_off=st.offload_off, bt_src=st.offload_dev, bt_dst=st.offload_host,
+                reload=dict(T=st.reload_T, bt_off=st.reload_off, bt_src=st.reload_host, bt_dst=st.reload_dev), flags=flags))
+            if i >= 1:
+                create.append(1e3 * (time.perf_counter() - t0))
+                h2d += int(st.reload_T.sum()) * shape.token_bytes
+                d2h += int(st.offload_T.sum()) * shape.token_bytes
+            # the short offload is enqueued first: the reload's ~6 000 page copies fill the driver's
+            # stream queue, so whatever is enqueued after it only starts when it is nearly done
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            ev[2].record(s2)
+            tc.tc_kv_pack(plan, [dev], [host], s2.cuda_stream)
+            ev[3].record(s2)
+            ev[0].record(stream)
+            tc.tc_kv_unpack(plan, [host], [dev], sp)
+            ev[1].record(stream)
+            torch.cuda.synchronize()   # a scheduler step ends when both directions have landed
+            plan.destroy()
+            if i >= 1:
+                dev_ms.append((ev[0].elapsed_time(ev[1]), ev[2].elapsed_time(ev[3])))
+        wall = time.perf_counter() - t_all
+        ideal = ideal_ms(h2d / steps_here, d2h / steps_here)
+        results[path] = {
+            "steps": steps_here, "plans_per_s": steps_here / wall, "ms_per_step_wall": 1e3 * wall / steps_here, "plan_create_ms": statistics.mean(create),
+            "h2d_GBps": h2d / wall / GB, "d2h_GBps": d2h / wall / GB, "link_GBps_both_directions": (h2d + d2h) / wall / GB,
+            "h2d_bytes_per_step": h2d // steps_here, "d2h_bytes_per_step": d2h // steps_here,
+            # the reload is the long leg of every step (5x the offload's bytes): the step cannot end before
+            # h2d bytes / H2D ceiling; with the offload sharing the link, before h2d bytes / duplex share
+            "device_ms_per_step_reload_stream": statistics.mean(x[0] for x in dev_ms), "device_ms_per_step_offload_stream": statistics.mean(x[1] for x in dev_ms),
+            "ideal_ms_per_step_at_contiguous_cudaMemcpyAsync_rates": ideal, "frac_of_ideal_schedule": ideal / (1e3 * wall / steps_here),
+            "h2d_frac_of_one_direction_ceiling": h2d / wall / GB / ceil_h2d,
+            "h2d_frac_of_its_share_of_the_both_directions_ceiling": h2d / wall / GB / (ceil_both / 2),
+            "d2h_frac_of_one_direction_ceiling": d2h / wall / GB / ceil_d2h}
+    first = dict(results[paths[0]])
+    first.update({
+        "sessions": 512, "host_pool_blocks": NBh, "host_pool_rule_min_262144_half_MemAvailable": rule, "host_pool_GB": NBh * shape.block_bytes / GB,
+        "pin_seconds": pin_s, "device_pool_blocks": NBd, "host_path": paths[0],
+        "ceilings_GBps_cudaMemcpyAsync_on_this_pool": {"h2d": ceil_h2d, "d2h": ceil_d2h, "both_directions_at_once_summed": ceil_both,
+                                                       "h2d_while_d2h_runs": dup_h2d, "d2h_while_h2d_runs": dup_d2h},
+        "other_host_paths_on_a_tenth_of_the_steps": {k: v for k, v in results.items() if k != paths[0]} or None,
+        "note": "wall clock over create + execute + synchronise + destroy of every step; reload and offload run concurrently on two "
+                "streams. staged: host pages travel one cudaMemcpyAsync each through the staging rings; mixed: the reload is staged, "
+                "the offload stores straight into the host pool from the kernel; zerocopy: kernel loads and stores both ways"})
+    out["configs[4] prefix-reload burst (mixed plan per step)"] = first
     del dev, host
     torch.cuda.empty_cache()
+
+
+EXTRAS = [
+    ("config0", extra_config0),
+    ("weights", extra_weights),
+    ("cold_path", lambda a, tc, torch, st, out: out.__setitem__("weights cold path: blob streamed from a file", cold_path(a, tc, torch, st))),
+    ("moe", lambda a, tc, torch, st, out: out.__setitem__("transform_into: MoE expert stacking (Qwen3-30B-A3B-shaped layers)", moe_stacking(a, tc, torch, st))),
+    ("kv_shapes", lambda a, tc, torch, st, out: out.__setitem__("rows a1-a3 on other KV geometries (8 GiB pools, first wave)", kv_shapes(a, tc, torch, st))),
+    ("misaligned", lambda a, tc, torch, st, out: out.__setitem__("rows a1-a5: copy paths and misaligned base pointers (8 GiB pool, 4 GB checkpoint)", misaligned(a, tc, torch, st))),
+    ("config3", extra_config3),
+    ("config4", extra_config4),
+]
+
+
+def run_extras(args, tc, torch, stream):
+    """Secondary workloads, reported beside the headline (`--extras a,b` runs only the named ones)."""
+    want = None if args.extras == "all" else set(args.extras.split(","))
+    if args.only_kv_shapes:  # profiler runs: just the KV geometries, a few GB on the device
+        want = {"kv_shapes"}
+    if args.only_misaligned:
+        want = {"misaligned"}
+    out = {}
+    for name, fn in EXTRAS:
+        if want is None or name in want:
+            fn(args, tc, torch, stream, out)
+            torch.cuda.empty_cache()
     return out
 
 
@@ -1070,6 +1338,18 @@ def traffic_per_launch(algorithmic_bytes: float) -> float:
     writes = payload less the ~50 MB of dirty lines still in L2 at kernel end."""
     payload = algorithmic_bytes / 2
     return 1.0002 * payload + max(payload - 50.7e6, 0.0)
+
+
+def spawn_ranks(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start the N ranks ourselves (one process per
+    GPU through torch.distributed.run on this node) with the same arguments; rank 0 prints the line."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -1087,16 +1367,18 @@ def main():
     ap.add_argument("--dry-run", action="store_true", help="CPU-only check of the multi-rank plumbing (gloo)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiler runs)")
-    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--e2e-warmup", type=int, default=1)
-    ap.add_argument("--oracle-blocks", type=int, default=1536)
+    ap.add_argument("--oracle-blocks", type=int, default=1024)
     ap.add_argument("--tile-bytes", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary workloads (configs[3], configs[4])")
     ap.add_argument("--only-kv-shapes", action="store_true", help="of the secondary workloads run only the KV geometries (profiler captures)")
     ap.add_argument("--only-misaligned", action="store_true", help="of the secondary workloads run only the misaligned-pointer rows")
-    ap.add_argument("--host-pool-blocks", type=int, default=8192, help="configs[4]: pinned host pool size in 2 MiB blocks")
-    ap.add_argument("--burst-steps", type=int, default=10, help="configs[4]: scheduler steps timed (the workload has 200)")
+    ap.add_argument("--extras", default="all", help="secondary workloads to run: all, or a comma list of " + ",".join(n for n, _ in EXTRAS))
+    ap.add_argument("--host-pool-blocks", type=int, default=0, help="configs[4]: pinned host pool size in 2 MiB blocks (0: min(262144, half of MemAvailable))")
+    ap.add_argument("--burst-steps", type=int, default=200, help="configs[4]: scheduler steps timed (the workload has 200)")
+    ap.add_argument("--burst-paths", default="staged", choices=["staged", "mixed", "zerocopy", "all"], help="configs[4]: host path (all: the first in full, the others on a tenth of the steps)")
     ap.add_argument("--cold-layers", type=int, default=8, help="cold-path extra: layers of the checkpoint written to a file (8: 4.0 GB)")
     ap.add_argument("--moe-layers", type=int, default=8, help="expert-stacking extra: layers of the MoE checkpoint (8: 11 GB)")
     ap.add_argument("--host-ctas", type=int, default=0)
@@ -1104,6 +1386,8 @@ def main():
     ap.add_argument("--e2e-schedule", default="duplex", choices=["duplex", "serial"],
                     help="duplex: offload wave k+1 while wave k reloads (two streams, two host buffers)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        sys.exit(spawn_ranks(args.gpus))
     if args.dry_run:
         run_dry(args)
     elif args.impl == "reference":

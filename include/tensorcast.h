@@ -156,6 +156,11 @@ enum {
                                16-byte aligned geometry and tensors that start on 4-byte
                                boundaries of the blob (TC_ERR_INVALID_ARG otherwise).  Such
                                plans default to 64 KiB tiles (tuning.tile_bytes overrides). */
+    TC_PLAN_OFFLOAD_ZERO_COPY = 32u, /* staged TC_KV_MIXED plans: stage only the reload group
+                               (host pages -> copy engine -> staging ring -> kernel); the offload
+                               group stores into the host pool straight from the kernel.  Kernel
+                               stores to host memory keep their speed while the other direction of
+                               the link is busy, and the copy engines then serve one direction only */
     TC_PLAN_STREAM = 16u    /* TC_WEIGHTS: the blob is streamed chunk by chunk, from a file
                                (tc_weights_materialize_file) or from pinned host memory
                                (tc_weights_materialize), through the staging ring.  Unlike

@@ -26,6 +26,7 @@ TC_PLAN_STAGED = 2
 TC_PLAN_CHECKSUM = 4
 TC_PLAN_SAME_POOL = 8
 TC_PLAN_STREAM = 16
+TC_PLAN_OFFLOAD_ZERO_COPY = 32
 TC_MAX_TABLE_SLOTS = 4000
 TC_DEVICE_BULK_WAIT_TIMEOUT = 1
 

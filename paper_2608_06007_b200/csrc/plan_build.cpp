@@ -633,10 +633,15 @@ static int build_kv(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t tile_byt
             tc_kv_group_t off_v = kv.group, rel_v = kv.reload;
             off_v.bt_dst = virt.data();
             rel_v.bt_src = virt.data();
-            lower_kv_group(g0, kv, off_v, &sp, &ring, 0, tile_bytes);
+            if (spec->flags & TC_PLAN_OFFLOAD_ZERO_COPY) {  // only the reload travels through the ring
+                lower_kv_group(g0, kv, kv.group, &sp, &dp, 0, tile_bytes);
+            } else {
+                lower_kv_group(g0, kv, off_v, &sp, &ring, 0, tile_bytes);
+                g0.stage_whole_host_pool = true;
+                stage_pages(g0, kv.group.bt_dst, n_off, slots, page, dp.block_stride);
+            }
             lower_kv_group(g1, kv, rel_v, &ring, &sp, 0, tile_bytes);
-            g0.stage_whole_host_pool = g1.stage_whole_host_pool = true;
-            stage_pages(g0, kv.group.bt_dst, n_off, slots, page, dp.block_stride);
+            g1.stage_whole_host_pool = true;
             stage_pages(g1, kv.reload.bt_src, n_rel, slots, page, dp.block_stride);
         } else {
             lower_kv_group(g0, kv, kv.group, &sp, &dp, 0, tile_bytes);
@@ -908,6 +913,8 @@ int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
     if ((spec->flags & TC_PLAN_CHECKSUM) && spec->kind != TC_WEIGHTS)
         return fail(TC_ERR_KIND, "TC_PLAN_CHECKSUM applies to TC_WEIGHTS plans only");
     plan->group[1].host_is_src = true;  // UNPACK / reload read the host side
+    if ((spec->flags & TC_PLAN_OFFLOAD_ZERO_COPY) && (spec->kind != TC_KV_MIXED || !(spec->flags & TC_PLAN_STAGED)))
+        return fail(TC_ERR_KIND, "TC_PLAN_OFFLOAD_ZERO_COPY applies to staged TC_KV_MIXED plans only");
     if ((spec->flags & TC_PLAN_STREAM) && spec->kind != TC_WEIGHTS)
         return fail(TC_ERR_KIND, "TC_PLAN_STREAM applies to TC_WEIGHTS plans only");
     if (spec->flags & (TC_PLAN_STAGED | TC_PLAN_STREAM)) {

@@ -41,3 +41,15 @@ def test_single_process_dry_run():
     assert out.returncode == 0, out.stderr[-2000:]
     j = json.loads(out.stdout.strip().splitlines()[-1])
     assert j["n_gpus"] == 1 and abs(j["value"] - 1e9 / 0.100 / 1e9) < 1e-9
+
+
+def test_plain_invocation_with_gpus_2_starts_its_own_two_ranks():
+    """`python bench.py --gpus 2` as the driver calls it, without a launcher around it."""
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run", "--steps", "4", "--warmup", "3"],
+                         capture_output=True, text=True, timeout=240, cwd=ROOT,
+                         env={k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")})
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, out.stdout
+    j = json.loads(lines[0])
+    assert j["n_gpus"] == 2 and abs(j["ms_per_step"] - 150.0) < 1e-9

@@ -307,7 +307,7 @@ def test_same_pool_compaction_in_place():
     assert np.array_equal(buf.result(), want)
 
 
-@pytest.mark.parametrize("flags", [0, tc.TC_PLAN_STAGED])
+@pytest.mark.parametrize("flags", [0, tc.TC_PLAN_STAGED, tc.TC_PLAN_STAGED | tc.TC_PLAN_OFFLOAD_ZERO_COPY])
 def test_mixed_plan_offload_and_reload_through_pinned_host_pool(flags):
     """Device NHD pool <-> pinned page-first HND host pool, both directions of one plan on two
     streams; the kernels store into / load from host memory directly."""
@@ -331,7 +331,7 @@ def test_mixed_plan_offload_and_reload_through_pinned_host_pool(flags):
                       T=step.offload_T, bt_off=step.offload_off, bt_src=step.offload_dev, bt_dst=step.offload_host,
                       reload=dict(T=step.reload_T, bt_off=step.reload_off, bt_src=step.reload_host, bt_dst=step.reload_dev), flags=flags)
     plan = tc.tc_plan_create(spec)
-    assert plan.stats().path[0] == (3 if flags else 1) and plan.stats().path[1] == (3 if flags else 1)
+    assert plan.stats().path[0] == (3 if flags == tc.TC_PLAN_STAGED else 1) and plan.stats().path[1] == (3 if flags else 1)
     s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
     torch.cuda.synchronize()
     tc.tc_kv_pack(plan, [d_dev], [h_host], stream=s1)
