@@ -161,6 +161,10 @@ enum {
                                group stores into the host pool straight from the kernel.  Kernel
                                stores to host memory keep their speed while the other direction of
                                the link is busy, and the copy engines then serve one direction only */
+    TC_PLAN_TRACE = 64u,    /* record a pair of CUDA events around every execution of the plan, so that
+                               tc_plan_stats can report the device time of the last one (the
+                               call context's tracing hook, Sec. 3.2).  Two event records per
+                               call; executions of one traced plan should not overlap */
     TC_PLAN_STREAM = 16u    /* TC_WEIGHTS: the blob is streamed chunk by chunk, from a file
                                (tc_weights_materialize_file) or from pinned host memory
                                (tc_weights_materialize), through the staging ring.  Unlike
@@ -421,6 +425,10 @@ typedef struct {
     int32_t path[2];               /* 1 direct (zero copy when a buffer is host memory),
                                       3 staged through the copy engines */
     int32_t grid[2];               /* CTAs launched per execution */
+    double last_device_us[2];      /* TC_PLAN_TRACE plans: device time of the group's most recent
+                                      execution, event to event on the caller's stream; -1 when the
+                                      group has not run yet or its last run has not finished (the
+                                      query never blocks); 0 for untraced plans */
 } tc_plan_stats_t;
 
 /* Fill *out (host pointer) with the plan's figures. */

@@ -27,6 +27,7 @@ TC_PLAN_CHECKSUM = 4
 TC_PLAN_SAME_POOL = 8
 TC_PLAN_STREAM = 16
 TC_PLAN_OFFLOAD_ZERO_COPY = 32
+TC_PLAN_TRACE = 64
 TC_MAX_TABLE_SLOTS = 4000
 TC_DEVICE_BULK_WAIT_TIMEOUT = 1
 
@@ -82,7 +83,8 @@ class tc_plan_stats_t(C.Structure):
                 ("n_descriptors", C.c_int64 * 2), ("n_tiles", C.c_int64 * 2),
                 ("payload_bytes", C.c_int64 * 2), ("packed_bytes_required", C.c_int64),
                 ("device_bytes", C.c_int64), ("vec_bytes", C.c_int32 * 2),
-                ("launches_per_execute", C.c_int32), ("path", C.c_int32 * 2), ("grid", C.c_int32 * 2)]
+                ("launches_per_execute", C.c_int32), ("path", C.c_int32 * 2), ("grid", C.c_int32 * 2),
+                ("last_device_us", C.c_double * 2)]
 
 
 class tc_descriptor_t(C.Structure):

@@ -78,6 +78,11 @@ void block_free(int device, void *ptr, size_t bytes)
 
 static void free_plan_storage(tc_plan *plan)
 {
+    for (auto &pair : plan->trace_ev)
+        for (void *&ev : pair) {
+            if (ev) cudaEventDestroy(static_cast<cudaEvent_t>(ev));
+            ev = nullptr;
+        }
     block_free(plan->device, plan->d_storage, plan->d_storage_bytes);
     plan->d_storage = nullptr;
     for (int k = 0; k < 2; k++) plan->group[k].d_descs = nullptr, plan->group[k].d_tile_desc = nullptr;
@@ -170,9 +175,20 @@ int execute(const tc_plan *plan, int gi, const void *const *src, size_t n_src, v
     if (!file && (rc = check_addressable(src, n_src, "source")) != TC_OK) return rc;
     if ((rc = check_addressable(const_cast<const void *const *>(dst), n_dst, "destination")) != TC_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (file) return execute_streamed(plan, g, file->fd, file->offset, dst, ptr_align, s, sums);
-    if (!g.segments.empty()) return execute_staged(plan, g, src, dst, ptr_align, s, sums);
-    return launch_any(plan, g, src, dst, ptr_align, s, nullptr, sums);
+    const bool trace = plan->trace_ev[gi][0] != nullptr;
+    if (trace) {
+        cudaError_t e = cudaEventRecord(static_cast<cudaEvent_t>(plan->trace_ev[gi][0]), s);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord(trace)");
+    }
+    if (file) rc = execute_streamed(plan, g, file->fd, file->offset, dst, ptr_align, s, sums);
+    else if (!g.segments.empty()) rc = execute_staged(plan, g, src, dst, ptr_align, s, sums);
+    else rc = launch_any(plan, g, src, dst, ptr_align, s, nullptr, sums);
+    if (trace && rc == TC_OK) {
+        cudaError_t e = cudaEventRecord(static_cast<cudaEvent_t>(plan->trace_ev[gi][1]), s);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord(trace)");
+        plan->traced_once[gi] = true;
+    }
+    return rc;
 }
 
 }  // namespace tc
@@ -212,6 +228,14 @@ extern "C" int tc_plan_create(const tc_plan_spec_t *spec, tc_plan_t **out)
             }
         }
         if (rc == TC_OK) rc = upload_plan(plan);
+        if (rc == TC_OK && (spec->flags & TC_PLAN_TRACE))
+            for (auto &pair : plan->trace_ev)
+                for (void *&ev : pair) {
+                    cudaEvent_t made = nullptr;
+                    cudaError_t e2 = cudaEventCreate(&made);
+                    if (e2 != cudaSuccess && rc == TC_OK) rc = cuda_fail(e2, "cudaEventCreate(trace)");
+                    ev = made;
+                }
         for (int k = 0; k < 2 && rc == TC_OK; k++)
             if (plan->group[k].n_tiles) resident_ctas_for(plan->group[k].n_src + plan->group[k].n_dst, plan->group[k].resident_ctas);
     }
@@ -323,6 +347,14 @@ extern "C" int tc_plan_stats(const tc_plan_t *plan, tc_plan_stats_t *out)
         out->path[k] = g.n_tiles ? (g.segments.empty() ? 1 : 3) : 0;
         if (!g.segments.empty()) out->launches_per_execute = static_cast<int32_t>(g.segments.size());
         out->grid[k] = g.n_tiles ? static_cast<int32_t>(grid_for(plan, g, mode_for(plan, g, 4))) : 0;
+        if (plan->trace_ev[k][0]) {
+            float ms = 0.f;
+            out->last_device_us[k] = -1.0;
+            if (plan->traced_once[k] && cudaEventElapsedTime(&ms, static_cast<cudaEvent_t>(plan->trace_ev[k][0]), static_cast<cudaEvent_t>(plan->trace_ev[k][1])) == cudaSuccess)
+                out->last_device_us[k] = 1e3 * ms;
+            else
+                cudaGetLastError();  // cudaErrorNotReady is the expected answer while the run is in flight
+        }
     }
     out->packed_bytes_required = plan->packed_required;
     out->device_bytes = plan->device_bytes;

@@ -116,6 +116,8 @@ struct tc_plan {
     bool checksummed = false;  // built with TC_PLAN_CHECKSUM
     int64_t n_sums = 0;        // accumulators a checksummed execution fills
     bool staged = false;  // holds a reference on the device's staging ring
+    void *trace_ev[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};  // TC_PLAN_TRACE: cudaEvent_t begin / end per group
+    mutable bool traced_once[2] = {false, false};
     tc::Group group[2];
 };
 

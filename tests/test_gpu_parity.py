@@ -666,6 +666,69 @@ def test_weights_checksum_fused_with_the_copy():
     assert e.value.status == tc.TC_ERR_KIND
 
 
+def test_traced_plan_reports_the_device_time_of_its_last_execution():
+    shape = wl.KVShape(L=4, B=16, H=8, D=128, E=2)
+    NB = 512
+    T = np.array([NB * shape.B], dtype=np.int64)
+    off = np.array([0, NB], dtype=np.int64)
+    bt = np.random.default_rng(5).permutation(NB).astype(np.int32)
+    pool = torch.zeros(NB * shape.block_bytes, dtype=torch.uint8, device="cuda")
+    out = torch.zeros(NB * shape.block_bytes, dtype=torch.uint8, device="cuda")
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=pool.numel())
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape.tuple, src_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_src=bt,
+                                        flags=tc.TC_PLAN_TRACE, trace_id=77))
+    assert plan.stats().last_device_us[0] == -1.0            # not run yet
+    stream = torch.cuda.Stream()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    tc.tc_kv_pack(plan, [pool], [out], stream.cuda_stream)
+    b.record(stream)
+    stream.synchronize()
+    st = plan.stats()
+    outer_us = 1e3 * a.elapsed_time(b)
+    assert st.trace_id == 77 and 0 < st.last_device_us[0] <= outer_us + 1.0   # 1 GiB moved: hundreds of microseconds
+    assert st.last_device_us[0] > 0.5 * outer_us
+    untraced = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape.tuple, src_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_src=bt))
+    assert untraced.stats().last_device_us[0] == 0.0
+
+
+# --------------------------------------------------------------------------- another GPU's memory
+@pytest.mark.skipif(torch.cuda.is_available() and torch.cuda.device_count() < 2, reason="needs two GPUs with peer access")
+def test_pack_and_migrate_from_a_pool_on_another_gpu():
+    """Cross-GPU migration: the source pool lives on device 1, the plan and the destination on
+    device 0.  A table entry is then a peer pointer; every CTA moves its own tile with plain loads
+    over NVLink (no bulk or multicast copy is involved: the geometry is aligned, so the register
+    path runs).  Compared with the oracle like any other pack / migrate."""
+    if not torch.cuda.can_device_access_peer(0, 1):
+        pytest.skip("devices 0 and 1 have no peer access")
+    rng = np.random.default_rng(91)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=48, B=16, H=8, D=128, E=2, T=(100, 16, 7, 333))
+    L = shape[0]
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    remote = torch.from_numpy(pool).to("cuda:1")           # the other engine's pool
+    torch.cuda.synchronize(1)
+    torch.cuda.set_device(0)
+    x = torch.empty(16, dtype=torch.uint8, device="cuda:0")
+    x.copy_(remote[:16])                                   # torch enables peer access between the two devices here
+    torch.cuda.synchronize(0)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride, slot_bytes=pool.size)
+    for packed_l in LAYOUTS:
+        want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+        oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, L * 2), T, off, bt, packed_l, want)
+        packed = Guarded(want.size)
+        plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_src=bt))
+        tc.tc_kv_pack(plan, [remote.data_ptr()], [packed.ptr()])
+        assert np.array_equal(packed.result(), want), packed_l
+    for dst_l in LAYOUTS:
+        pl2 = tc.pool(dst_l, NB, 1, plane_stride=NB * stride, slot_bytes=pool.size)
+        want_pool = np.full_like(pool, 0xA5)
+        oracle.kv_migrate(shape, oracle.NHD, stride, planes_of(pool, L * 2), dst_l, stride, planes_of(want_pool, L * 2), T, off, bt, bt2)
+        fresh = Guarded(pool.size)
+        plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl2, T=T, bt_off=off, bt_src=bt, bt_dst=bt2))
+        tc.tc_kv_pack(plan, [remote.data_ptr()], [fresh.ptr()])
+        assert np.array_equal(fresh.result(), want_pool), dst_l
+
+
 # --------------------------------------------------------------------------- misaligned rows
 @pytest.mark.parametrize("cols,pitch,tile", [(100, 116, 0), (256, 256 + 16, 0), (33, 64, 1024), (5000, 5003, 0), (40000, 40000 + 7, 0), (70000, 70001, 65536)])
 def test_rows_at_every_source_and_destination_alignment(cols, pitch, tile):
