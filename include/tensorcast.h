@@ -46,8 +46,9 @@
  * addressable addresses: device memory, pinned host memory mapped into the device's
  * address space (cudaHostAlloc / cudaHostRegister under unified addressing), which the kernel
  * then reads or writes directly over the host link (zero copy), or another GPU's memory once
- * peer access is enabled (every CTA then moves its own tile with plain loads and stores over
- * NVLink; the library issues no multicast or bulk-tensor copy).  Pageable host memory is not
+ * peer access is enabled (every CTA then moves its own tile over NVLink with plain loads and
+ * stores - misaligned geometry: with per-CTA bulk asynchronous loads into its shared memory;
+ * the library issues no multicast copy of any kind).  Pageable host memory is not
  * addressable by the device: the execute calls refuse it (TC_ERR_INVALID_ARG) instead of
  * letting a kernel fault.  The tables themselves, the
  * spec and every array it points to are HOST memory.
@@ -143,8 +144,10 @@ enum {
                                exits.  Groups that cannot be staged (strided slices of a blob,
                                partial blocks of a paged pool) stay zero copy.  Layer-major
                                packed buffers are cut into runs of whole planes, in layer
-                               order.  Staged executions are serialised with one another
-                               by the library while they are enqueued. */
+                               order.  While they are being enqueued, staged executions in the
+                               same direction on the same device wait for one another (the
+                               ring is theirs in turn); other devices and the other direction
+                               are not held up. */
     TC_PLAN_SAME_POOL = 8u, /* TC_KV_MIGRATE inside ONE pool (compaction / defragmentation): the
                                caller will pass the same table as source and destination.
                                src_pool and dst_pool must describe the same geometry, and no
@@ -360,7 +363,7 @@ TC_API int tc_weights_materialize_checksum(const tc_plan_t *plan, const void *bl
  * Reading runs up to two chunks ahead of transfer and scatter.
  * The call RETURNS when the last chunk has been read and enqueued, so unlike the other entry
  * points it blocks for about the time the storage reads take; device work completes on
- * `stream` as usual.  Calls are serialised with one another.
+ * `stream` as usual.  Calls on one device are serialised with one another.
  * Errors: everything tc_weights_materialize checks, before the first read; TC_ERR_KIND for a
  * plan without TC_PLAN_STREAM; TC_ERR_IO when a read fails or the file ends early - chunks
  * before the failing one have been enqueued and will still complete, the destination tensors

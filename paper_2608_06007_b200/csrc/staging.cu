@@ -28,6 +28,7 @@ struct StageRing {
     cudaEvent_t ready[kStageBuffers] = {}, freed[kStageBuffers] = {};
     bool freed_recorded[kStageBuffers] = {};
     cudaStream_t copy = nullptr;
+    cudaEvent_t entry = nullptr;  // orders the ring's copy stream behind the caller's stream
     uint64_t next = 0;
 };
 // Pinned host buffers that file chunks are read into (tc_weights_materialize_file).
@@ -41,11 +42,18 @@ struct HostRing {
 struct StageArena {
     StageRing ring[2];
     HostRing host;
-    cudaEvent_t entry = nullptr;
     int refs = 0;
 };
 static StageArena g_stage[kMaxDevices];
-static pthread_mutex_t g_stage_mu = PTHREAD_MUTEX_INITIALIZER;
+// Locks are per device and per ring, plus one per device for file streaming: staged calls on
+// different GPUs of one process, or in the two directions of one GPU, do not queue behind one
+// another on the host.  Whoever needs both rings (allocation, trimming) takes ring 0 first.
+struct DeviceLocks {
+    pthread_mutex_t ring[2] = {PTHREAD_MUTEX_INITIALIZER, PTHREAD_MUTEX_INITIALIZER}, file = PTHREAD_MUTEX_INITIALIZER;
+    void lock_both() { pthread_mutex_lock(&ring[0]); pthread_mutex_lock(&ring[1]); }
+    void unlock_both() { pthread_mutex_unlock(&ring[1]); pthread_mutex_unlock(&ring[0]); }
+};
+static DeviceLocks g_locks[kMaxDevices];
 
 static void stage_free(StageArena &a)
 {
@@ -56,25 +64,26 @@ static void stage_free(StageArena &a)
             if (r.freed[b]) cudaEventDestroy(r.freed[b]);
         }
         if (r.copy) cudaStreamDestroy(r.copy);
+        if (r.entry) cudaEventDestroy(r.entry);
     }
     for (int b = 0; b < kHostBuffers; b++) {
         if (a.host.buf[b]) cudaFreeHost(a.host.buf[b]);
         if (a.host.freed[b]) cudaEventDestroy(a.host.freed[b]);
     }
-    if (a.entry) cudaEventDestroy(a.entry);
     a = StageArena();
 }
 
 int stage_acquire(int device, int64_t *bytes)
 {
     if (device < 0 || device >= kMaxDevices) return fail(TC_ERR_INVALID_ARG, "device ordinal %d is not supported", device);
-    pthread_mutex_lock(&g_stage_mu);
+    g_locks[device].lock_both();
     StageArena &a = g_stage[device];
     int rc = TC_OK;
     if (a.refs == 0) {
         a.refs = 1;  // the library's own reference: keeps the rings alive between plans
-        cudaError_t e = cudaEventCreateWithFlags(&a.entry, cudaEventDisableTiming);
+        cudaError_t e = cudaSuccess;
         for (StageRing &r : a.ring) {
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&r.entry, cudaEventDisableTiming);
             if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&r.copy, cudaStreamNonBlocking);
             for (int b = 0; b < kStageBuffers && e == cudaSuccess; b++) {
                 e = cudaMalloc(&r.buf[b], kStageBytes);
@@ -91,7 +100,7 @@ int stage_acquire(int device, int64_t *bytes)
         a.refs++;
         *bytes = 2 * kStageBytes * kStageBuffers;
     }
-    pthread_mutex_unlock(&g_stage_mu);
+    g_locks[device].unlock_both();
     return rc;
 }
 
@@ -100,10 +109,10 @@ int stage_acquire(int device, int64_t *bytes)
 void stage_release(int device)
 {
     if (device < 0 || device >= kMaxDevices) return;
-    pthread_mutex_lock(&g_stage_mu);
+    g_locks[device].lock_both();
     StageArena &a = g_stage[device];
     if (a.refs > 1) a.refs--;  // the last reference is never dropped: the rings stay until exit
-    pthread_mutex_unlock(&g_stage_mu);
+    g_locks[device].unlock_both();
 }
 
 #define TC_TRY(call, what)                                   \
@@ -124,9 +133,10 @@ int execute_staged(const tc_plan *plan, const Group &g, const void *const *src, 
     const bool to_device = g.host_is_src;
     StageRing &r = a.ring[to_device ? 1 : 0];
     int rc = TC_OK;
-    pthread_mutex_lock(&g_stage_mu);
-    TC_TRY(cudaEventRecord(a.entry, s), "cudaEventRecord");
-    TC_TRY(cudaStreamWaitEvent(r.copy, a.entry, 0), "cudaStreamWaitEvent");
+    pthread_mutex_t *mu = &g_locks[plan->device].ring[to_device ? 1 : 0];
+    pthread_mutex_lock(mu);
+    TC_TRY(cudaEventRecord(r.entry, s), "cudaEventRecord");
+    TC_TRY(cudaStreamWaitEvent(r.copy, r.entry, 0), "cudaStreamWaitEvent");
     for (const Segment &seg : g.segments) {
         const int b = static_cast<int>(r.next++ % kStageBuffers);
         char *shifted = r.buf[b] - seg.shift;
@@ -158,12 +168,11 @@ int execute_staged(const tc_plan *plan, const Group &g, const void *const *src, 
         for (int b = 0; b < kStageBuffers; b++)
             if (r.freed_recorded[b]) TC_TRY(cudaStreamWaitEvent(s, r.freed[b], 0), "cudaStreamWaitEvent");
 out:
-    pthread_mutex_unlock(&g_stage_mu);
+    pthread_mutex_unlock(mu);
     return rc;
 }
 
 // ---- cold path: file -> pinned host ring -> staging ring -> kernel ---------------------------
-static pthread_mutex_t g_file_mu = PTHREAD_MUTEX_INITIALIZER;  // one file stream per process at a time
 
 // Reader threads of one tc_weights_materialize_file call.  Every chunk of the plan is a job of
 // 1 MiB pieces; the caller opens jobs in order as pinned buffers become free, the readers take
@@ -299,12 +308,13 @@ int execute_streamed(const tc_plan *plan, const Group &g, int fd, int64_t file_o
     HostRing &h = a.host;
     const size_t n = g.segments.size();
     int rc = TC_OK;
-    pthread_mutex_lock(&g_file_mu);
-    pthread_mutex_lock(&g_stage_mu);
+    pthread_mutex_t *mu = &g_locks[plan->device].ring[1], *file_mu = &g_locks[plan->device].file;
+    pthread_mutex_lock(file_mu);  // one file stream per device at a time (they share the pinned buffers)
+    pthread_mutex_lock(mu);
     rc = host_ring_acquire(h);
-    pthread_mutex_unlock(&g_stage_mu);
+    pthread_mutex_unlock(mu);
     if (rc != TC_OK) {
-        pthread_mutex_unlock(&g_file_mu);
+        pthread_mutex_unlock(file_mu);
         return rc;
     }
     {
@@ -336,7 +346,7 @@ int execute_streamed(const tc_plan *plan, const Group &g, int fd, int64_t file_o
                 break;
             }
             const int hb = host_buf(i);
-            pthread_mutex_lock(&g_stage_mu);
+            pthread_mutex_lock(mu);
             {
                 const int b = static_cast<int>(r.next++ % kStageBuffers);
                 char *shifted = r.buf[b] - seg.shift;
@@ -353,24 +363,26 @@ int execute_streamed(const tc_plan *plan, const Group &g, int fd, int64_t file_o
                 r.freed_recorded[b] = true;
             }
         out:
-            pthread_mutex_unlock(&g_stage_mu);
+            pthread_mutex_unlock(mu);
         }
     }  // the pool's destructor stops and joins the readers
-    pthread_mutex_unlock(&g_file_mu);
+    pthread_mutex_unlock(file_mu);
     return rc;
 }
 #undef TC_TRY
 
 void stage_trim()
 {
-    pthread_mutex_lock(&g_stage_mu);
-    for (StageArena &a : g_stage)
+    for (int device = 0; device < kMaxDevices; device++) {
+        g_locks[device].lock_both();
+        StageArena &a = g_stage[device];
         if (a.refs == 1) {  // only the library's own reference is left
             for (StageRing &r : a.ring)
                 if (r.copy) cudaStreamSynchronize(r.copy);
             stage_free(a);
         }
-    pthread_mutex_unlock(&g_stage_mu);
+        g_locks[device].unlock_both();
+    }
 }
 
 }  // namespace tc

@@ -66,6 +66,151 @@ def run_tile_range(descs, tile0, n_tiles, src_tables, dst_tables, dst_counts=Non
                         dst_counts[d.dst_slot + o * d.dst_slot_step][b:b + d.run_bytes] += 1
 
 
+def run_multiplane_tiles(descs, n_tiles, src_tables, dst_tables, dst_counts=None, threads=256, vec=16):
+    """Walk a uniform group whose tiles take several planes of a descriptor (planes_per_tile > 1)
+    tile id by tile id, with the index arithmetic of the kernel's multi-plane path: tile ->
+    (descriptor, first plane); inside the tile every plane owns 2^log2_unit bytes of a byte space
+    that `threads` lanes cross `vec` bytes at a time; byte -> (plane, row, column).  Every access is
+    bounds-checked; lanes past a plane's real bytes or past the descriptor's last plane stay idle."""
+    ppt = descs[0].planes_per_tile
+    assert ppt > 1
+    unit_max = max(d.rows * d.run_bytes for d in descs)
+    log2_unit = 9
+    while (1 << log2_unit) < unit_max:
+        log2_unit += 1
+    mask = (1 << log2_unit) - 1
+    groups = -(-descs[0].n_outer // ppt)
+    tiles_per_desc = groups * descs[0].tiles_per_outer
+    assert n_tiles == tiles_per_desc * len(descs) and all(d.tiles_per_outer == 1 for d in descs)
+    for tile in range(n_tiles):
+        di, t = divmod(tile, tiles_per_desc)
+        d = descs[di]
+        assert d.tile0 == di * tiles_per_desc
+        o = t * ppt
+        if o >= d.n_outer:
+            continue
+        n_units = min(ppt, d.n_outer - o)
+        unit_bytes = d.rows * d.run_bytes
+        for byte in range(0, n_units << log2_unit, vec):          # lane order does not matter on the CPU
+            k, w = o + (byte >> log2_unit), byte & mask
+            if w >= unit_bytes:
+                continue
+            assert w + vec <= unit_bytes, "a vector straddles the end of a plane"
+            r, col = divmod(w, d.run_bytes)
+            i1, i0 = divmod(r, d.n0)
+            a = d.src_off + k * d.src_outer + i1 * d.src_s1 + i0 * d.src_s0 + col
+            b = d.dst_off + k * d.dst_outer + i1 * d.dst_s1 + i0 * d.dst_s0 + col
+            s_ = src_tables[d.src_slot + k * d.src_slot_step]
+            t_ = dst_tables[d.dst_slot + k * d.dst_slot_step]
+            assert 0 <= a and a + vec <= s_.size, "multi-plane tile reads outside its source slot"
+            assert 0 <= b and b + vec <= t_.size, "multi-plane tile writes outside its destination slot"
+            t_[b:b + vec] = s_[a:a + vec]
+            if dst_counts is not None:
+                dst_counts[d.dst_slot + k * d.dst_slot_step][b:b + vec] += 1
+
+
+class _Mem:
+    """A flat buffer placed at a virtual address, so that a model can reason about alignment.
+    Reads of whole aligned 16-byte chunks may reach up to 15 bytes outside the buffer (the
+    kernel's realigning path does that, staying inside chunks that hold a byte it needs); those
+    bytes read as 0xCC.  Writes outside the buffer are errors."""
+
+    def __init__(self, arr, va):
+        self.a, self.va = arr, va
+
+    def read16(self, addr):
+        assert addr % 16 == 0
+        lo = addr - self.va
+        out = np.full(16, 0xCC, dtype=np.uint8)
+        a, b = max(lo, 0), min(lo + 16, self.a.size)
+        assert a < b, "an aligned chunk with no byte of the buffer was read"
+        out[a - lo:b - lo] = self.a[a:b]
+        return out
+
+    def write(self, addr, data, cnt=None):
+        lo = addr - self.va
+        assert 0 <= lo and lo + len(data) <= self.a.size, "write outside the destination"
+        self.a[lo:lo + len(data)] = data
+        if cnt is not None:
+            cnt[lo:lo + len(data)] += 1
+
+
+def run_realign_tile(d, o, part, src, dst, cnt, smem_bytes=52 << 10, threads=256):
+    """The realigning path of the kernel (rows whose source and destination are not both
+    16-byte aligned, all strides multiples of 16), replayed for tile (outer o, part) of
+    descriptor d on _Mem buffers: per pass, one aligned bulk load per row into a staging array,
+    then aligned 16-byte destination chunks assembled from two staged chunks, partial first /
+    last chunks in aligned pieces, and the chunk that two destination-adjacent rows share
+    stored once.  Same quantities and formulas as the CUDA code; every staged byte that is
+    consumed must have been loaded, every destination byte is counted."""
+    column_max = smem_bytes - 64
+    row0 = part * d.rows_per_tile
+    nrows = min(d.rows_per_tile, d.rows - row0)
+    run = d.run_bytes
+    column = min(run, column_max)
+    units = (column + 30) >> 4
+    rows_per_pass = (smem_bytes - 32) // (units << 4)
+    assert rows_per_pass >= 1 and all(x % 16 == 0 for x in (d.src_s0, d.src_s1, d.dst_s0, d.dst_s1))
+    src0 = src.va + d.src_off + o * d.src_outer
+    dst0 = dst.va + d.dst_off + o * d.dst_outer
+    rowoff = lambda r, s0, s1: (r // d.n0) * s1 + (r % d.n0) * s0
+    for col0 in range(0, run, column):
+        length = min(column, run - col0)
+        for r0 in range(0, nrows, rows_per_pass):
+            n_rows = min(rows_per_pass, nrows - r0)
+            row_base = row0 + r0
+            s_lo, d_lo = (src0 + col0) % 16, (dst0 + col0) % 16
+            stage = np.full(smem_bytes, 0xDD, dtype=np.uint8)
+            loaded = np.zeros(smem_bytes, dtype=bool)
+            data = 16
+            row_bytes = ((s_lo + length + 15) >> 4) << 4
+            for rr in range(n_rows):                          # one bulk copy per row
+                g = src0 + col0 - s_lo + rowoff(row_base + rr, d.src_s0, d.src_s1)
+                at = data + 16 * rr * units
+                assert at + row_bytes <= smem_bytes - 16
+                for c in range(row_bytes // 16):
+                    stage[at + 16 * c:at + 16 * c + 16] = src.read16(g + 16 * c)
+                    loaded[at + 16 * c:at + 16 * c + 16] = True
+            delta = s_lo - d_lo
+            sh, shifted = delta % 16, data + 16 * (delta >> 4)
+            end = d_lo + length
+            c_first, c_last = (1 if d_lo else 0), end >> 4
+
+            def chunk(u, lo, hi):
+                at = shifted + 16 * u + sh
+                assert 0 <= shifted + 16 * u and shifted + 16 * u + 32 <= smem_bytes, "staging read outside the area"
+                assert loaded[at + lo:at + hi].all(), "a staged byte that was never loaded is consumed"
+                return stage[at:at + 16].copy()
+
+            def out_addr(rr, c):
+                return dst0 + col0 - d_lo + rowoff(row_base + rr, d.dst_s0, d.dst_s1) + 16 * c
+
+            for rr in range(n_rows):                          # whole chunks (either thread mapping covers exactly these)
+                for c in range(c_first, c_last):
+                    dst.write(out_addr(rr, c), chunk(rr * units + c, 0, 16), cnt)
+            one_chunk, t = c_last == 0, end & 15
+            if not (d_lo or t):
+                continue
+            adj = 0
+            if not one_chunk and t and length == run and run % 16 == 0:
+                adj = 1 if (d.n0 > 1 and d.dst_s0 == run) else (d.n0 if d.dst_s1 == run else 0)
+            for rr in range(n_rows):                          # partial chunks, one thread per row
+                r = row_base + rr
+                i0 = r % d.n0
+                has_next = bool(adj) and (i0 + 1 < d.n0 if adj == 1 else r + d.n0 < d.rows) and rr + adj < n_rows
+                has_prev = bool(adj) and (i0 >= 1 if adj == 1 else r >= d.n0) and rr >= adj
+                if (d_lo or one_chunk) and not has_prev:
+                    hi = end if one_chunk else 16
+                    dst.write(out_addr(rr, 0) + d_lo, chunk(rr * units, d_lo, hi)[d_lo:hi], cnt)
+                if not one_chunk and t:
+                    tail = chunk(rr * units + c_last, 0, t)
+                    if has_next:
+                        head = chunk((rr + adj) * units, t, 16)
+                        dst.write(out_addr(rr, c_last), np.concatenate([tail[:t], head[t:]]), cnt)
+                    else:
+                        dst.write(out_addr(rr, c_last), tail[:t], cnt)
+
+
 def planes_of(pool, n_planes):
     per = pool.size // n_planes
     return [pool[i * per:(i + 1) * per] for i in range(n_planes)]

@@ -564,6 +564,73 @@ def test_small_planes_share_a_tile():
     assert plan.descriptors(0)[0].planes_per_tile == 4 and plan.stats().n_tiles[0] == 6 * 2
 
 
+@pytest.mark.parametrize("H,L,slots", [(1, 4, "one"), (2, 3, "planes"), (4, 2, "one"), (2, 16, "planes")])
+@pytest.mark.parametrize("dst_l", [tc.TC_NHD, tc.TC_HND])
+def test_multi_plane_tile_walk_matches_the_oracle(H, L, slots, dst_l):
+    """The tile -> (descriptor, planes) -> byte -> (plane, row, column) arithmetic of tiles that
+    take several small planes, replayed on the CPU with bounds checks and write counts, for pools
+    with one pointer and with one pointer per plane, ragged last blocks, and a plane count that
+    the planes per tile do not divide (L = 3)."""
+    from helpers import run_multiplane_tiles
+    rng = np.random.default_rng(60 + H + L)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=L, NB=14, B=16, H=H, D=128, E=2, T=(37, 16, 5, 48))
+    planes = L * 2
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    n_slots = planes if slots == "planes" else 1
+    kw = {} if slots == "planes" else dict(plane_stride=NB * stride)
+    src_pool = tc.pool(tc.TC_NHD, NB, n_slots, **kw)
+    dst_pool = tc.pool(dst_l, NB, n_slots, **kw)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=src_pool, dst_pool=dst_pool, T=T, bt_off=off, bt_src=bt, bt_dst=bt2, flags=HOST))
+    ds = plan.descriptors(0)
+    assert ds[0].planes_per_tile > 1
+    want = np.full_like(pool, 0xA5)
+    oracle.kv_migrate(shape, oracle.NHD, stride, planes_of(pool, planes), dst_l, stride, planes_of(want, planes), T, off, bt, bt2)
+    got = np.full_like(pool, 0xA5)
+    cnt = np.zeros(pool.size, dtype=np.int32)
+    tables = (lambda a: planes_of(a, planes)) if slots == "planes" else (lambda a: [a])
+    run_multiplane_tiles(ds, plan.stats().n_tiles[0], tables(pool), tables(got), tables(cnt))
+    assert np.array_equal(got, want)
+    assert cnt.max() == 1 and cnt.sum() == int(T.sum()) * planes * H * 256
+
+
+@pytest.mark.parametrize("a,b", [(0, 1), (1, 0), (15, 15), (8, 4), (3, 9), (5, 5)])
+def test_realigning_path_arithmetic_on_the_cpu(a, b):
+    """Base pointers at addresses = a / b modulo 16 under aligned geometry: the chunk, shift,
+    head / tail and shared-boundary-chunk arithmetic of the realigning path, replayed on the CPU
+    for KV pack (256-byte rows, destination rows adjacent along tokens), unpack, a same-layout
+    migration (whole-plane runs), and a staging area small enough to force several passes and
+    column pieces.  Each destination byte must be written once, with the oracle's value."""
+    from helpers import _Mem, run_realign_tile
+    rng = np.random.default_rng(70 + a + b)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=1, NB=10, B=16, H=4, D=64, E=2, T=(37, 16, 5))
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride)
+    packed_n = oracle.packed_nbytes(shape, T)
+    cases = []
+    want = np.zeros(packed_n, dtype=np.uint8)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, 2), T, off, bt, oracle.HND, want)
+    cases.append((tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_src=bt, flags=HOST), 0, pool, want, 0))
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(want_pool, 2), T, off, bt2, oracle.HND, want)
+    cases.append((tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_dst=bt2, flags=HOST), 1, want, want_pool, 0xA5))
+    want_mig = np.full_like(pool, 0xA5)
+    oracle.kv_migrate(shape, oracle.NHD, stride, planes_of(pool, 2), oracle.NHD, stride, planes_of(want_mig, 2), T, off, bt, bt2)
+    cases.append((tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl, T=T, bt_off=off, bt_src=bt, bt_dst=bt2, flags=HOST), 0, pool, want_mig, 0xA5))
+    for spec, group, source, expect, fill in cases:
+        plan = tc.tc_plan_create(spec)
+        for smem in (52 << 10, 1360, 592):                    # one pass per tile; five 256-byte rows per pass; column pieces
+            got = np.full(expect.size, fill, dtype=np.uint8)
+            cnt = np.zeros(expect.size, dtype=np.int32)
+            src, dst = _Mem(source, 4096 + a), _Mem(got, 1 << 20 | b)
+            for d in plan.descriptors(group):
+                for o in range(d.n_outer):
+                    for part in range(d.tiles_per_outer):
+                        if part * d.rows_per_tile < d.rows:
+                            run_realign_tile(d, o, part, src, dst, cnt, smem_bytes=smem)
+            assert np.array_equal(got, expect), (spec.kind, smem)
+            assert cnt.max() == 1 and cnt.sum() == int(T.sum()) * 2 * 4 * 128, (spec.kind, smem)
+
+
 def test_same_pool_compaction_lowering_and_its_overlap_check():
     """Defragmentation: the requests' blocks move to the low block ids of the same pool."""
     rng = np.random.default_rng(6)
