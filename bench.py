@@ -1003,6 +1003,39 @@ def misaligned(args, tc, torch, stream):
         p_.destroy()
     del rawA, rawB, rawQ, blob, dstw
     torch.cuda.empty_cache()
+    # few KV heads (planes of 8 KiB, four to a tile) through misaligned pointers
+    shape = wl.KVShape(28, 16, 2, 128)
+    s = shape.tuple
+    NB = int(((1 if args.small else 4) << 30) // shape.block_bytes)
+    WB = NB // 2
+    _, _, _, waves = wl.config2(NB=NB, R=256, wave_blocks=WB, NB_dst=WB, shape=shape)
+    src, dst = waves[0]
+    payload = int(src.T.sum()) * shape.token_bytes
+    rawA = torch.empty(NB * shape.block_bytes + 16, **u8)
+    wl.fill_torch(rawA, wl.SEED_BASE + 7)
+    rawB = torch.empty(WB * shape.block_bytes + 16, **u8)
+    rawQ = torch.empty(payload + 16, **u8)
+    plA = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=NB * shape.block_bytes)
+    plB = tc.pool(tc.TC_NHD, WB, 1, plane_stride=WB * shape.chunk_bytes, slot_bytes=WB * shape.block_bytes)
+    kw = dict(T=src.T, bt_off=src.bt_off)
+    pk = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, bt_src=src.bt, **kw))
+    up = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, bt_dst=dst.bt, **kw))
+    mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, s, src_pool=plA, dst_pool=plB, bt_src=src.bt, bt_dst=dst.bt, **kw))
+    few = {"kv_payload_bytes": payload, "planes_per_tile": int(mig.descriptors(0)[0].planes_per_tile)}
+    A, B, Q = rawA.data_ptr(), rawB.data_ptr(), rawQ.data_ptr()
+    for label, a_src, a_dst in (("aligned", 0, 0), ("src+2", 2, 0), ("both+1", 1, 1)):
+        res = {}
+        for name, fn in (("a1_pack", lambda: tc.tc_kv_pack(pk, [A + a_src], [Q + a_dst], sp)),
+                         ("a2_unpack", lambda: tc.tc_kv_unpack(up, [Q + a_src], [B + a_dst], sp)),
+                         ("a3_migrate", lambda: tc.tc_kv_pack(mig, [A + a_src], [B + a_dst], sp))):
+            res[name] = 2 * payload / (b2b_ms(torch, stream, fn, reps=reps, warm=warm) * 1e-3) / GB
+        res["min_frac_of_measured_peak"] = min(res.values()) / peak
+        few[label] = res
+    out["2 KV heads (L28 B16 H2 D128, 4 GiB pool)"] = few
+    for p_ in (pk, up, mig):
+        p_.destroy()
+    del rawA, rawB, rawQ
+    torch.cuda.empty_cache()
     return out
 
 

@@ -293,15 +293,19 @@ struct RealignPass {
     uint32_t s_lo, d_lo;        // source / destination address modulo 16
 };
 
-// One bulk copy per row: the aligned source chunks that hold the row's bytes.
-template <int kThreads>
+// Bytes one row of the pass brings in: the aligned source chunks that hold the row's bytes.
+__device__ __forceinline__ uint32_t realign_row_bytes(const RealignPass &p) { return ((p.s_lo + p.len + 15) >> 4) << 4; }
+
+// One bulk copy per row.  EXPECT: also announce the pass's bytes to the barrier (a caller that
+// loads several passes' worth at once announces their sum itself).
+template <int kThreads, bool EXPECT = true>
 __device__ __forceinline__ void realign_load(const Desc &d, const RealignPass &p, uint32_t data_addr, uint32_t bar)
 {
     const uint32_t n0 = d.n0, ss0 = d.src_s0, ss1 = d.src_s1;
     const FastDiv div_n0 = d.div_n0;
-    const uint32_t row_bytes = ((p.s_lo + p.len + 15) >> 4) << 4;
+    const uint32_t row_bytes = realign_row_bytes(p);
     const char *base = p.src - p.s_lo;
-    if (threadIdx.x == 0) mbar_expect_tx(bar, p.n_rows * row_bytes);
+    if (EXPECT && threadIdx.x == 0) mbar_expect_tx(bar, p.n_rows * row_bytes);
     for (uint32_t rr = threadIdx.x; rr < p.n_rows; rr += kThreads) {
         const uint32_t r = p.row_base + rr, i1 = fastdiv(r, div_n0), i0 = r - i1 * n0;
         bulk_load(data_addr + 16 * rr * p.units, base + (i1 * ss1 + i0 * ss0), row_bytes, bar);
@@ -415,6 +419,37 @@ __device__ __forceinline__ void realign_store_all(const Desc &d, const RealignPa
     const uint32_t c_first = p.d_lo ? 1 : 0, c_last = end >> 4;  // whole chunks: [c_first, c_last)
     if (c_last > c_first) realign_store_full<WS, kThreads>(d, p, data, c_first, c_last);
     if (p.d_lo || (end & 15)) realign_store_edges<WS, kThreads>(d, p, data, c_last, end);
+}
+
+// Wait for the bulk copies of the current phase.  One thread waits (bounded) and tells the
+// others, so that the CTA stays together; false: the copies did not arrive in time, the status
+// word says so, and the caller returns from the kernel.
+__device__ __forceinline__ bool realign_wait(uint32_t bar, uint32_t &phase, uint32_t *wait_ok)
+{
+    if (threadIdx.x == 0) {
+        bool ok = mbar_wait_bounded(bar, phase);
+        if (!ok) {
+            atomicOr(&g_device_status, kStatusBulkWaitTimeout);
+            ok = mbar_wait_bounded(bar, phase);  // the copies still target this CTA's memory
+            *wait_ok = 0;
+        }
+    }
+    __syncthreads();
+    if (!*wait_ok) return false;
+    mbar_try_wait(bar, phase, 0);  // completed: every thread observes the phase itself
+    phase ^= 1;
+    return true;
+}
+
+template <int kThreads>
+__device__ __forceinline__ void realign_store_dispatch(const Desc &d, const RealignPass &p, uint32_t data_addr)
+{
+    switch (((p.s_lo - p.d_lo) & 15) >> 2) {
+    case 0: realign_store_all<0, kThreads>(d, p, data_addr); break;
+    case 1: realign_store_all<1, kThreads>(d, p, data_addr); break;
+    case 2: realign_store_all<2, kThreads>(d, p, data_addr); break;
+    default: realign_store_all<3, kThreads>(d, p, data_addr); break;
+    }
 }
 
 // The same for tiles whose rows differ in alignment (a row pitch that is not a multiple of 16):
@@ -589,10 +624,63 @@ __device__ __forceinline__ void copy_run16(const char *src, char *dst, uint32_t 
     }
 }
 
+// A multi-plane tile (planes o .. o + n_units of descriptor d) on the realigning path: the rows
+// of all its planes are staged in one pass - plane j in its own region of the staging area, one
+// bulk copy per row - and stored plane by plane; planes may differ in alignment (a pointer per
+// plane).  False: not applicable to this tile (rows of a few bytes, rows that differ in alignment,
+// a staging area too small), the caller takes the narrow-vector loop; `alive` false: give up.
+template <int kThreads, bool STEP, int NPTR>
+__device__ __forceinline__ bool copy_multi_realign(const Desc &d, const Params<NPTR> &prm, uint32_t o, uint32_t n_units, char *stage,
+                                                   uint32_t bar, uint32_t &phase, uint32_t *wait_ok, bool &alive)
+{
+    const uint32_t units = (d.run + 30) >> 4, plane_stage = d.rows * units * 16;
+    if (d.run < kRealignMinRun || d.run > kRealignColumn || ((d.src_s0 | d.src_s1 | d.dst_s0 | d.dst_s1) & 15) || n_units * plane_stage + 32 > prm.stage_bytes)
+        return false;
+    const uint32_t data_addr = static_cast<uint32_t>(__cvta_generic_to_shared(stage + 16));
+    auto plane = [&](uint32_t j) {
+        const uint32_t k = o + j;
+        RealignPass p;
+        p.src = prm.ptr[d.src_slot + (STEP ? k * d.src_slot_step : 0)] + d.src_off + k * d.src_outer;
+        p.dst = prm.ptr[d.dst_slot + (STEP ? k * d.dst_slot_step : 0)] + d.dst_off + k * d.dst_outer;
+        p.row_base = 0;
+        p.n_rows = d.rows;
+        p.units = units;
+        p.len = d.run;
+        p.s_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(p.src)) & 15;
+        p.d_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(p.dst)) & 15;
+        return p;
+    };
+    if (threadIdx.x == 0) {
+        uint32_t bytes = 0;
+        for (uint32_t j = 0; j < n_units; j++) bytes += d.rows * realign_row_bytes(plane(j));
+        mbar_expect_tx(bar, bytes);
+    }
+    for (uint32_t j = 0; j < n_units; j++) realign_load<kThreads, false>(d, plane(j), data_addr + j * plane_stage, bar);
+    if (!realign_wait(bar, phase, wait_ok)) {
+        alive = false;
+        return true;
+    }
+    for (uint32_t j = 0; j < n_units; j++) realign_store_dispatch<kThreads>(d, plane(j), data_addr + j * plane_stage);
+    __syncthreads();
+    return true;
+}
+
+// The narrow-vector loops of a multi-plane tile, out of line like copy_rows_narrow.
+template <int U, int kThreads, bool STEP, int NPTR>
+__device__ __noinline__ void copy_multi_narrow(const Desc &d, const Params<NPTR> &prm, uint32_t o, uint32_t n_units, uint32_t align)
+{
+    switch (align) {
+    case 3: copy_multi<3, U, kThreads, true, STEP>(d, prm, o, n_units); break;
+    case 2: copy_multi<2, U, kThreads, true, STEP>(d, prm, o, n_units); break;
+    case 1: copy_multi<1, U, kThreads, true, STEP>(d, prm, o, n_units); break;
+    default: copy_multi<0, U, kThreads, true, STEP>(d, prm, o, n_units); break;
+    }
+}
+
 // MULTI: 0 one plane per tile; 1 several planes per tile, planes a byte stride apart; 2 the
 // same with a pool that has one pointer per plane.
 template <int NPTR, int MODE, bool CHECK = false, int MULTI = 0>
-__global__ void __launch_bounds__(Shape<MODE>::threads, (MODE == kModeAny && MULTI) ? 2 : Shape<MODE>::min_ctas) tc_copy_kernel(const __grid_constant__ Params<NPTR> prm)
+__global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) tc_copy_kernel(const __grid_constant__ Params<NPTR> prm)
 {
     constexpr int kThreads = Shape<MODE>::threads, kUnroll = Shape<MODE>::unroll;
     __shared__ Desc sdesc[2];
@@ -600,7 +688,7 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, (MODE == kModeAny && MUL
     __shared__ __align__(8) unsigned long long stage_bar;  // its mbarrier
     __shared__ uint32_t stage_ok;
     uint32_t bar = 0, phase = 0;
-    if (MODE == kModeAny && !MULTI) {
+    if (MODE == kModeAny) {
         bar = static_cast<uint32_t>(__cvta_generic_to_shared(&stage_bar));
         if (threadIdx.x == 0) {
             mbar_init(bar, 1);
@@ -664,13 +752,12 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, (MODE == kModeAny && MUL
             } else if (MODE == kModeRows) {
                 copy_multi<4, kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units);
             } else {
-                switch (min(static_cast<uint32_t>(d.log2_align), prm.log2_ptr_align)) {
-                case 4: copy_multi<4, kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units); break;
-                case 3: copy_multi<3, 2 * kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units); break;
-                case 2: copy_multi<2, 2 * kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units); break;
-                case 1: copy_multi<1, 2 * kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units); break;
-                default: copy_multi<0, 2 * kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units); break;
-                }
+                const uint32_t align = min(static_cast<uint32_t>(d.log2_align), prm.log2_ptr_align);
+                bool alive = true;
+                if (align == 4) copy_multi<4, kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units);
+                else if (!copy_multi_realign<kThreads, MULTI == 2>(d, prm, o, n_units, stage, bar, phase, &stage_ok, alive))
+                    copy_multi_narrow<2 * kUnroll, kThreads, MULTI == 2>(d, prm, o, n_units, align);
+                if (!alive) return;
             }
             continue;
         }

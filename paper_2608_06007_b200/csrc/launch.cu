@@ -118,6 +118,12 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     for (size_t i = 0; i < g.n_src; i++) prm.ptr[i] = const_cast<char *>(static_cast<const char *>(src[i]));
     for (size_t i = 0; i < g.n_dst; i++) prm.ptr[g.n_src + i] = static_cast<char *>(dst[i]);
     for (size_t i = g.n_src + g.n_dst; i < NPTR; i++) prm.ptr[i] = nullptr;
+    // the realigning path stages rows in more dynamic shared memory than a kernel gets by
+    // default; the opt-in is per device and costs nothing to repeat
+    auto with_stage = [&](auto kernel) {
+        prm.stage_bytes = std::max<uint32_t>(g.realign_smem, 1024);
+        return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kRealignSmem));
+    };
     if (g.ppt > 1) {
         // multi-plane tiles: KV groups only (two pools of at most L*2 pointers each)
         if (NPTR == TC_MAX_TABLE_SLOTS || sums) return fail(TC_ERR_INVALID_ARG, "internal: multi-plane tiles with a large table or checksums");
@@ -128,13 +134,19 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
                 switch (mode) {
                 case kModeRun: tc_copy_kernel<NPTR, kModeRun, false, 2><<<grid, Shape<kModeRun>::threads, 0, stream>>>(prm); break;
                 case kModeRows: tc_copy_kernel<NPTR, kModeRows, false, 2><<<grid, Shape<kModeRows>::threads, 0, stream>>>(prm); break;
-                default: tc_copy_kernel<NPTR, kModeAny, false, 2><<<grid, Shape<kModeAny>::threads, 0, stream>>>(prm); break;
+                default:
+                    if (cudaError_t ea = with_stage(tc_copy_kernel<NPTR, kModeAny, false, 2>); ea != cudaSuccess) return cuda_fail(ea, "cudaFuncSetAttribute(dynamic shared memory)");
+                    tc_copy_kernel<NPTR, kModeAny, false, 2><<<grid, Shape<kModeAny>::threads, prm.stage_bytes, stream>>>(prm);
+                    break;
                 }
             } else {
                 switch (mode) {
                 case kModeRun: tc_copy_kernel<NPTR, kModeRun, false, 1><<<grid, Shape<kModeRun>::threads, 0, stream>>>(prm); break;
                 case kModeRows: tc_copy_kernel<NPTR, kModeRows, false, 1><<<grid, Shape<kModeRows>::threads, 0, stream>>>(prm); break;
-                default: tc_copy_kernel<NPTR, kModeAny, false, 1><<<grid, Shape<kModeAny>::threads, 0, stream>>>(prm); break;
+                default:
+                    if (cudaError_t ea = with_stage(tc_copy_kernel<NPTR, kModeAny, false, 1>); ea != cudaSuccess) return cuda_fail(ea, "cudaFuncSetAttribute(dynamic shared memory)");
+                    tc_copy_kernel<NPTR, kModeAny, false, 1><<<grid, Shape<kModeAny>::threads, prm.stage_bytes, stream>>>(prm);
+                    break;
                 }
             }
         }
@@ -145,15 +157,10 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     switch (mode) {
     case kModeRun: tc_copy_kernel<NPTR, kModeRun><<<grid, Shape<kModeRun>::threads, 0, stream>>>(prm); break;
     case kModeRows: tc_copy_kernel<NPTR, kModeRows><<<grid, Shape<kModeRows>::threads, 0, stream>>>(prm); break;
-    default: {
-        // the realigning path stages rows in more dynamic shared memory than a kernel gets by
-        // default; the opt-in is per device and costs nothing to repeat
-        cudaError_t ea = cudaFuncSetAttribute(tc_copy_kernel<NPTR, kModeAny>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kRealignSmem));
-        if (ea != cudaSuccess) return cuda_fail(ea, "cudaFuncSetAttribute(dynamic shared memory)");
-        prm.stage_bytes = std::max<uint32_t>(g.realign_smem, 1024);
+    default:
+        if (cudaError_t ea = with_stage(tc_copy_kernel<NPTR, kModeAny>); ea != cudaSuccess) return cuda_fail(ea, "cudaFuncSetAttribute(dynamic shared memory)");
         tc_copy_kernel<NPTR, kModeAny><<<grid, Shape<kModeAny>::threads, prm.stage_bytes, stream>>>(prm);
         break;
-    }
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "kernel launch");

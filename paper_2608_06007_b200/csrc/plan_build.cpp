@@ -230,13 +230,6 @@ static void lower_box(Group &g, Box b, uint32_t tile_bytes)
 static int finish_group(Group &g, uint32_t tile_bytes)
 {
     if (g.descs.empty()) return TC_OK;
-    // Realigning path: one pass should hold a whole tile (every row in a slot of `units` 16-byte
-    // chunks, 32 bytes of padding), up to the size at which long rows go in column pieces.
-    for (const Desc &d : g.descs) {
-        const uint64_t units = (std::min<uint32_t>(d.run, kRealignColumn) + 30) >> 4;
-        const uint64_t need = std::min<uint64_t>(d.rows_per_tile, d.rows) * units * 16 + 32;
-        g.realign_smem = static_cast<uint32_t>(std::max<uint64_t>(g.realign_smem, std::min<uint64_t>(need, kRealignSmem)));
-    }
     // Small planes: let a tile span several planes of its descriptor (see Group::ppt).  Needs one
     // part per plane and a pointer table of at most 400 entries (the kernel classes built for it).
     g.ppt = 1;
@@ -259,6 +252,18 @@ static int finish_group(Group &g, uint32_t tile_bytes)
             }
         }
     }
+    // Realigning path: one pass should hold a whole tile (every row in a slot of `units` 16-byte
+    // chunks, all planes of a multi-plane tile, 32 bytes of padding), up to the size at which long
+    // rows go in column pieces.
+    auto realign_need = [&](uint32_t ppt) {
+        uint64_t most = 0;
+        for (const Desc &d : g.descs) {
+            const uint64_t units = (std::min<uint32_t>(d.run, kRealignColumn) + 30) >> 4;
+            most = std::max<uint64_t>(most, std::min<uint64_t>(d.rows_per_tile, d.rows) * units * 16 * ppt + 32);
+        }
+        return static_cast<uint32_t>(std::min<uint64_t>(most, kRealignSmem));
+    };
+    g.realign_smem = realign_need(g.ppt);
     auto outer_groups = [&](const Desc &d) { return (d.n_outer + g.ppt - 1) / g.ppt; };
     uint64_t total = 0, max_t = 0;
     for (const Desc &d : g.descs) {
@@ -286,6 +291,7 @@ static int finish_group(Group &g, uint32_t tile_bytes)
     }
     g.ppt = 1;  // listed groups keep one plane per tile
     g.log2_unit = 0;
+    g.realign_smem = realign_need(1);
     total = 0;
     for (const Desc &d : g.descs) total += static_cast<uint64_t>(d.n_outer) * d.tiles_per_outer;
     if (total >= (1ull << 31)) return fail(TC_ERR_INVALID_ARG, "plan has %llu tiles (limit 2^31)", (unsigned long long)total);

@@ -767,41 +767,47 @@ def test_rows_at_every_source_and_destination_alignment(cols, pitch, tile):
             assert np.array_equal(outs[k].result(), want[k]), (pairs[k], shift)
 
 
+@pytest.mark.parametrize("D,slots", [(128, "one"), (64, "one"), (32, "planes")])
 @pytest.mark.parametrize("shift_pool,shift_packed", [(0, 2), (2, 0), (6, 6), (1, 9), (8, 4)])
-def test_kv_pack_unpack_migrate_through_misaligned_pointers(shift_pool, shift_packed):
+def test_kv_pack_unpack_migrate_through_misaligned_pointers(shift_pool, shift_packed, D, slots):
     """Aligned geometry, misaligned base pointers: the pool and / or the packed buffer start at
-    an odd address (a view into a larger allocation).  Rows of 256 bytes (NHD <-> HND) and whole
-    32 KiB planes (same layout) both take the realigning path."""
+    an odd address (a view into a larger allocation).  Rows of D * 2 bytes (NHD <-> HND) and whole
+    planes (same layout) both take the realigning path; with D = 64 and 32 a plane is small enough
+    for tiles of two and four planes, in a pool with one pointer or a pointer per plane."""
     rng = np.random.default_rng(77)
-    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=40, B=16, H=8, D=64, E=2, T=(100, 16, 7, 333))
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=40, B=16, H=8, D=D, E=2, T=(100, 16, 7, 333))
     L, B, H, D, E = shape
     planes = planes_of(pool, L * 2)
     bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
-    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride, slot_bytes=pool.size)
+    n_slots = L * 2 if slots == "planes" else 1
+    pl = tc.pool(tc.TC_NHD, NB, n_slots, plane_stride=0 if slots == "planes" else NB * stride, slot_bytes=pool.size // n_slots)
     raw = torch.zeros(pool.size + 16, dtype=torch.uint8, device="cuda")
     d_pool = raw[shift_pool:shift_pool + pool.size]
     d_pool.copy_(dev(pool))
+    per = pool.size // (L * 2)
+    table = lambda base: [base + p * per for p in range(L * 2)] if slots == "planes" else [base]
     for packed_l in LAYOUTS:
         want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
         oracle.kv_pack(shape, oracle.NHD, stride, planes, T, off, bt, packed_l, want)
         packed = Guarded(want.size, shift=shift_packed)
         plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_src=bt))
-        tc.tc_kv_pack(plan, [d_pool.data_ptr()], [packed.ptr()])
+        tc.tc_kv_pack(plan, table(d_pool.data_ptr()), [packed.ptr()])
         assert np.array_equal(packed.result(), want), packed_l
         want_pool = np.full_like(pool, 0xA5)
         oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(want_pool, L * 2), T, off, bt2, packed_l, want)
         fresh = Guarded(pool.size, shift=shift_pool)
         plan2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=packed_l, T=T, bt_off=off, bt_dst=bt2))
-        tc.tc_kv_unpack(plan2, [packed.ptr()], [fresh.ptr()])
+        tc.tc_kv_unpack(plan2, [packed.ptr()], table(fresh.ptr()))
         assert np.array_equal(fresh.result(), want_pool), packed_l
     for dst_l in LAYOUTS:
-        pl2 = tc.pool(dst_l, NB, 1, plane_stride=NB * stride, slot_bytes=pool.size)
+        pl2 = tc.pool(dst_l, NB, n_slots, plane_stride=0 if slots == "planes" else NB * stride, slot_bytes=pool.size // n_slots)
         want_pool = np.full_like(pool, 0xA5)
         oracle.kv_migrate(shape, oracle.NHD, stride, planes, dst_l, stride, planes_of(want_pool, L * 2), T, off, bt, bt2)
         fresh = Guarded(pool.size, shift=shift_packed)
         plan3 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl2, T=T, bt_off=off, bt_src=bt, bt_dst=bt2))
-        tc.tc_kv_pack(plan3, [d_pool.data_ptr()], [fresh.ptr()])
+        tc.tc_kv_pack(plan3, table(d_pool.data_ptr()), table(fresh.ptr()))
         assert np.array_equal(fresh.result(), want_pool), dst_l
+    assert tc.tc_device_status() == 0
 
 
 def test_shared_memory_copy_path_on_aligned_geometry():
