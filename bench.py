@@ -1273,7 +1273,7 @@ def extra_config4(args, tc, torch, stream, out):
             return 1e3 * (t_d + (h2d_bytes - dup_h2d * GB * t_d) / (ceil_h2d * GB))
         return 1e3 * (t_h + (d2h_bytes - dup_d2h * GB * t_h) / (ceil_d2h * GB))
 
-    paths = ["staged", "mixed", "zerocopy"] if args.burst_paths == "all" else [args.burst_paths]
+    paths = ["zerocopy", "staged", "mixed"] if args.burst_paths == "all" else [args.burst_paths]
     results = {}
     for path in paths:
         # a comparison path runs a tenth of the steps; the reported one runs them all
@@ -1331,8 +1331,9 @@ def extra_config4(args, tc, torch, stream, out):
                                                        "h2d_while_d2h_runs": dup_h2d, "d2h_while_h2d_runs": dup_d2h},
         "other_host_paths_on_a_tenth_of_the_steps": {k: v for k, v in results.items() if k != paths[0]} or None,
         "note": "wall clock over create + execute + synchronise + destroy of every step; reload and offload run concurrently on two "
-                "streams. staged: host pages travel one cudaMemcpyAsync each through the staging rings; mixed: the reload is staged, "
-                "the offload stores straight into the host pool from the kernel; zerocopy: kernel loads and stores both ways"})
+                "streams. zerocopy: the kernel loads pages from and stores pages into the pinned host pool itself (one CTA per SM); "
+                "staged: host pages travel one cudaMemcpyAsync each through the staging rings; mixed: the reload is staged, the "
+                "offload stores straight into the host pool from the kernel"})
     out["configs[4] prefix-reload burst (mixed plan per step)"] = first
     del dev, host
     torch.cuda.empty_cache()
@@ -1411,7 +1412,8 @@ def main():
     ap.add_argument("--extras", default="all", help="secondary workloads to run: all, or a comma list of " + ",".join(n for n, _ in EXTRAS))
     ap.add_argument("--host-pool-blocks", type=int, default=0, help="configs[4]: pinned host pool size in 2 MiB blocks (0: min(262144, half of MemAvailable))")
     ap.add_argument("--burst-steps", type=int, default=200, help="configs[4]: scheduler steps timed (the workload has 200)")
-    ap.add_argument("--burst-paths", default="staged", choices=["staged", "mixed", "zerocopy", "all"], help="configs[4]: host path (all: the first in full, the others on a tenth of the steps)")
+    ap.add_argument("--burst-paths", default="all", choices=["staged", "mixed", "zerocopy", "all"],
+                    help="configs[4]: host path (all: zerocopy over all the steps, staged and mixed on a tenth of them)")
     ap.add_argument("--cold-layers", type=int, default=8, help="cold-path extra: layers of the checkpoint written to a file (8: 4.0 GB)")
     ap.add_argument("--moe-layers", type=int, default=8, help="expert-stacking extra: layers of the MoE checkpoint (8: 11 GB)")
     ap.add_argument("--host-ctas", type=int, default=0)

@@ -265,7 +265,10 @@ typedef struct {
                              of tile_bytes (few KV heads). */
     int32_t ctas_per_sm;  /* > 0: a persistent grid-stride grid of this many CTAs per SM instead
                              of one CTA per tile */
-    int32_t max_ctas;     /* > 0: cap on the grid (persistent grid-stride loop) */
+    int32_t max_ctas;     /* > 0: cap on the grid (persistent grid-stride loop).  When a table entry
+                             of an execute call is pinned host memory and neither this nor
+                             ctas_per_sm is set, the grid is capped at one CTA per SM: few
+                             long-lived CTAs serve the host link better than one CTA per tile */
     int32_t tile_order;   /* 0 auto: KV groups run plane-major over descriptors sorted by
                              destination offset (ascending writes); 1: request / descriptor order
                              as given, planes of one block consecutively */

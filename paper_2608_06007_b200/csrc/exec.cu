@@ -127,7 +127,7 @@ static int upload_plan(tc_plan *plan)
 // memory that is pinned and mapped.  Plain pageable host memory would make the kernel fault, so
 // it is refused here, on the host.  Every entry is checked (a fraction of a microsecond each):
 // one unchecked pageable pointer would be a GPU fault.
-static int check_addressable(const void *const *table, size_t n, const char *what)
+static int check_addressable(const void *const *table, size_t n, const char *what, bool *host_memory)
 {
     for (size_t i = 0; i < n; i++) {
         cudaPointerAttributes attr;
@@ -138,6 +138,7 @@ static int check_addressable(const void *const *table, size_t n, const char *wha
         }
         if (attr.type == cudaMemoryTypeUnregistered)
             return fail(TC_ERR_INVALID_ARG, "%s table entry %zu (%p) is pageable host memory: pin it (cudaHostAlloc / cudaHostRegister) or use device memory", what, i, table[i]);
+        if (attr.type == cudaMemoryTypeHost) *host_memory = true;
     }
     return TC_OK;
 }
@@ -172,8 +173,9 @@ int execute(const tc_plan *plan, int gi, const void *const *src, size_t n_src, v
         ptr_align = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(dst[i]) | 16));
     }
     int rc;
-    if (!file && (rc = check_addressable(src, n_src, "source")) != TC_OK) return rc;
-    if ((rc = check_addressable(const_cast<const void *const *>(dst), n_dst, "destination")) != TC_OK) return rc;
+    bool host_memory = false;  // some table entry is pinned host memory: the kernel works over the host link
+    if (!file && (rc = check_addressable(src, n_src, "source", &host_memory)) != TC_OK) return rc;
+    if ((rc = check_addressable(const_cast<const void *const *>(dst), n_dst, "destination", &host_memory)) != TC_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool trace = plan->trace_ev[gi][0] != nullptr;
     if (trace) {
@@ -182,7 +184,7 @@ int execute(const tc_plan *plan, int gi, const void *const *src, size_t n_src, v
     }
     if (file) rc = execute_streamed(plan, g, file->fd, file->offset, dst, ptr_align, s, sums);
     else if (!g.segments.empty()) rc = execute_staged(plan, g, src, dst, ptr_align, s, sums);
-    else rc = launch_any(plan, g, src, dst, ptr_align, s, nullptr, sums);
+    else rc = launch_any(plan, g, src, dst, ptr_align, s, nullptr, sums, host_memory);
     if (trace && rc == TC_OK) {
         cudaError_t e = cudaEventRecord(static_cast<cudaEvent_t>(plan->trace_ev[gi][1]), s);
         if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord(trace)");

@@ -29,11 +29,11 @@ int cuda_fail(cudaError_t e, const char *what);
 int mode_for(const tc_plan *plan, const Group &g, uint32_t ptr_align, bool checksums = false);
 // CTAs of each build that one SM holds, for a pointer table of n_ptrs slots (cached).
 void resident_ctas_for(size_t n_ptrs, int out[3]);
-uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *win = nullptr);
+uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *win = nullptr, bool over_host_link = false);
 // Launch group g (or the window / tile range `win` of it) on stream s.  sums: checksum
 // accumulators or null.
 int launch_any(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s, const Segment *win,
-               unsigned long long *sums = nullptr);
+               unsigned long long *sums = nullptr, bool over_host_link = false);
 
 // The current device's sticky status word (flags set by kernels); reading clears it.
 int read_device_status(unsigned int *out);

@@ -58,7 +58,7 @@ void resident_ctas_for(size_t n_ptrs, int out[3])
 // Tile rows per descriptor: planes, or groups of ppt planes.
 static uint32_t outer_groups(const Group &g) { return (g.descs[0].n_outer + g.ppt - 1) / g.ppt; }
 
-uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *win)
+uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *win, bool over_host_link)
 {
     // Default: one CTA per tile.  The hardware block scheduler then balances the tiles over the
     // SMs and de-phases the CTAs' load and store bursts, which measured faster than a
@@ -72,12 +72,18 @@ uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *
         grid = std::min<uint64_t>(grid, static_cast<uint64_t>(plan->sm_count > 0 ? plan->sm_count : 148) * per_sm);
     }
     if (plan->tuning.max_ctas > 0) grid = std::min<uint64_t>(grid, plan->tuning.max_ctas);
+    // Over the host link (a table entry is pinned host memory) a persistent grid of one CTA per SM
+    // is the default: with both directions of the link busy, 64 to 148 CTAs moved 72 GB/s where one
+    // CTA per tile (tens of thousands of short-lived CTAs) moved 42 to 53 and 16 CTAs 60; one
+    // direction alone does not care (51-52 GB/s either way).
+    else if (over_host_link && plan->tuning.ctas_per_sm <= 0)
+        grid = std::min<uint64_t>(grid, plan->sm_count > 0 ? plan->sm_count : 148);
     return static_cast<uint32_t>(grid);
 }
 
 template <int NPTR>
 static int launch(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t stream,
-                  const Segment *win = nullptr, unsigned long long *sums = nullptr)
+                  const Segment *win, unsigned long long *sums, bool over_host_link)
 {
     // Uniform groups with planes (KV) are walked plane-major by default: all blocks of plane 0,
     // then plane 1, ...  Together with descriptors sorted by destination offset, every plane
@@ -87,7 +93,7 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     if (!win && g.tiles_per_desc && !g.descs.empty() && g.descs[0].n_outer > 1 && plan->tuning.tile_order != 1) win = &whole;
     const int mode = mode_for(plan, g, ptr_align, sums != nullptr);
     if (sums && mode == kModeAny) return fail(TC_ERR_INVALID_ARG, "checksums need 16-byte aligned base pointers");
-    const uint32_t grid = grid_for(plan, g, mode, win);
+    const uint32_t grid = grid_for(plan, g, mode, win, over_host_link);
     Params<NPTR> prm;
     prm.descs = g.d_descs;
     prm.tile_desc = g.d_tile_desc;
@@ -176,12 +182,12 @@ int read_device_status(unsigned int *out)
 }
 
 int launch_any(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s, const Segment *win,
-               unsigned long long *sums)
+               unsigned long long *sums, bool over_host_link)
 {
     const size_t n = g.n_src + g.n_dst;
-    if (n <= 8) return launch<8>(plan, g, src, dst, ptr_align, s, win, sums);
-    if (n <= 400) return launch<400>(plan, g, src, dst, ptr_align, s, win, sums);
-    return launch<TC_MAX_TABLE_SLOTS>(plan, g, src, dst, ptr_align, s, win, sums);
+    if (n <= 8) return launch<8>(plan, g, src, dst, ptr_align, s, win, sums, over_host_link);
+    if (n <= 400) return launch<400>(plan, g, src, dst, ptr_align, s, win, sums, over_host_link);
+    return launch<TC_MAX_TABLE_SLOTS>(plan, g, src, dst, ptr_align, s, win, sums, over_host_link);
 }
 
 }  // namespace tc
