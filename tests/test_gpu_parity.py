@@ -363,6 +363,34 @@ def test_pack_to_pinned_host_hnd_and_reload():
     assert np.array_equal(fresh.result(), want_pool)
 
 
+def test_zero_copy_offload_and_reload_through_a_misaligned_pinned_buffer():
+    """The packed buffer is a view at an odd offset of a pinned host allocation: the realigning
+    path then stores to and bulk-loads from host memory over the link."""
+    rng = np.random.default_rng(26)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=64, B=16, H=8, D=128, E=2, T=(300, 16, 45))
+    L = shape[0]
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, L * 2), T, off, bt, oracle.HND, want)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride)
+    raw = torch.full((want.size + 64,), 0x3C, dtype=torch.uint8).pin_memory()
+    for shift in (2, 9):
+        raw.fill_(0x3C)
+        host = raw[shift:shift + want.size]
+        plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_src=bt))
+        tc.tc_kv_pack(plan, [dev(pool)], [host.data_ptr()])
+        torch.cuda.synchronize()
+        assert np.array_equal(host.numpy(), want)
+        assert bool((raw[:shift] == 0x3C).all()) and bool((raw[shift + want.size:] == 0x3C).all())
+        bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+        want_pool = np.full_like(pool, 0xA5)
+        oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(want_pool, L * 2), T, off, bt2, oracle.HND, want)
+        plan2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_dst=bt2))
+        fresh = Guarded(pool.size)
+        tc.tc_kv_unpack(plan2, [host.data_ptr()], [fresh.ptr()])
+        assert np.array_equal(fresh.result(), want_pool)
+    assert tc.tc_device_status() == 0
+
+
 @pytest.mark.parametrize("packed_l", LAYOUTS)
 @pytest.mark.parametrize("order", [tc.TC_REQUEST_MAJOR, tc.TC_LAYER_MAJOR])
 def test_staged_offload_and_reload_through_the_copy_engines(packed_l, order):
