@@ -425,6 +425,8 @@ def run_ours(args):
     host_tune = dict(tune)
     if args.host_ctas:
         host_tune["max_ctas"] = args.host_ctas
+    if args.host_copy_path:
+        host_tune["copy_path"] = args.host_copy_path
     t_plan0 = time.perf_counter()
     plans = []
     for src, dst in waves:
@@ -1417,6 +1419,7 @@ def main():
     ap.add_argument("--cold-layers", type=int, default=8, help="cold-path extra: layers of the checkpoint written to a file (8: 4.0 GB)")
     ap.add_argument("--moe-layers", type=int, default=8, help="expert-stacking extra: layers of the MoE checkpoint (8: 11 GB)")
     ap.add_argument("--host-ctas", type=int, default=0)
+    ap.add_argument("--host-copy-path", type=int, default=0, help="tuning.copy_path of the e2e plans (1: through shared memory, bulk copies)")
     ap.add_argument("--host-path", default="staged", choices=["staged", "zerocopy"])
     ap.add_argument("--e2e-schedule", default="duplex", choices=["duplex", "serial"],
                     help="duplex: offload wave k+1 while wave k reloads (two streams, two host buffers)")
