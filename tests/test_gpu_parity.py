@@ -919,9 +919,11 @@ def test_random_geometries_on_the_device(seed):
     assert np.array_equal(fresh.result(), want_pool)
 
 
-def test_execute_calls_can_be_captured_in_a_cuda_graph_and_replayed():
+@pytest.mark.parametrize("shift", [0, 2])
+def test_execute_calls_can_be_captured_in_a_cuda_graph_and_replayed(shift):
     """Launch-bound use (config 1 moves 1.4 MB): pack + unpack captured once, replayed many
-    times; every replay reproduces the oracle's bytes (re-execution is idempotent)."""
+    times; every replay reproduces the oracle's bytes (re-execution is idempotent).  With the
+    packed buffer at a misaligned address the captured kernels are the realigning build."""
     shape, NB, src, dst = wl.config1()
     s = shape.tuple
     pool = np.zeros(2 * NB * shape.chunk_bytes, dtype=np.uint8)
@@ -933,7 +935,8 @@ def test_execute_calls_can_be_captured_in_a_cuda_graph_and_replayed():
     pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=pool.size)
     pack = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=pl, packed_layout=tc.TC_HND, T=src.T, bt_off=src.bt_off, bt_src=src.bt))
     unpack = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=pl, packed_layout=tc.TC_HND, T=dst.T, bt_off=dst.bt_off, bt_dst=dst.bt))
-    d_pool, packed, fresh = dev(pool), torch.zeros(want.size, dtype=torch.uint8, device="cuda"), Guarded(pool.size)
+    d_pool, fresh = dev(pool), Guarded(pool.size)
+    packed = torch.zeros(want.size + 16, dtype=torch.uint8, device="cuda")[shift:shift + want.size]
     side = torch.cuda.Stream()
     graph = torch.cuda.CUDAGraph()
     torch.cuda.synchronize()
