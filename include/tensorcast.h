@@ -496,6 +496,13 @@ TC_API int tc_trim(void);
 #define TC_DEVICE_BULK_WAIT_TIMEOUT 1u
 TC_API int tc_device_status(uint32_t *flags);
 
+/* Self-test of that bounded wait: launches one small kernel on `stream` that waits on a barrier
+ * nothing will ever arrive at.  The wait gives up after a few milliseconds, the kernel sets
+ * TC_DEVICE_BULK_WAIT_TIMEOUT exactly as the copy kernel would and returns normally; the next
+ * tc_device_status reports (and clears) the flag.  It shows that a wait which cannot complete ends
+ * with a status instead of a hung device. */
+TC_API int tc_selftest_wait_timeout(void *stream);
+
 /* Static string naming a status code. */
 TC_API const char *tc_strerror(int status);
 

@@ -103,7 +103,7 @@ class tc_segment_t(C.Structure):
 EXPORTS = ("tc_plan_create", "tc_kv_pack", "tc_kv_unpack", "tc_weights_materialize",
            "tc_plan_destroy", "tc_plan_stats", "tc_plan_descriptors", "tc_strerror", "tc_last_error",
            "tc_kv_pack_noalloc", "tc_weights_materialize_checksum", "tc_trim",
-           "tc_weights_materialize_file", "tc_plan_segments", "tc_device_status")
+           "tc_weights_materialize_file", "tc_plan_segments", "tc_device_status", "tc_selftest_wait_timeout")
 
 _lib = None
 
@@ -135,6 +135,8 @@ def load_library(path: str | None = None):
     lib.tc_plan_segments.restype = C.c_int
     lib.tc_device_status.argtypes = [C.POINTER(C.c_uint32)]
     lib.tc_device_status.restype = C.c_int
+    lib.tc_selftest_wait_timeout.argtypes = [vp]
+    lib.tc_selftest_wait_timeout.restype = C.c_int
     lib.tc_trim.argtypes = []
     lib.tc_trim.restype = C.c_int
     lib.tc_strerror.argtypes = [C.c_int]
@@ -373,6 +375,12 @@ def tc_device_status() -> int:
     v = C.c_uint32()
     _check(load_library().tc_device_status(C.byref(v)))
     return int(v.value)
+
+
+def tc_selftest_wait_timeout(stream=None) -> None:
+    """Run the self-test of the bounded device-side wait: afterwards tc_device_status() reports
+    TC_DEVICE_BULK_WAIT_TIMEOUT once."""
+    _check(load_library().tc_selftest_wait_timeout(_stream(stream)))
 
 
 def tc_plan_stats(plan: Plan) -> tc_plan_stats_t:

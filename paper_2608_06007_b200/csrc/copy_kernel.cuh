@@ -263,14 +263,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uin
 }
 // Bounded wait for a phase of the barrier: false if it did not complete within the limit
 // (a bulk copy takes microseconds; the limit is of the order of a second).
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = 1u << 20)
 {
-    for (uint32_t spin = 0; spin < (1u << 20); spin++) {
+    for (uint32_t spin = 0; spin < limit; spin++) {
         if (mbar_try_wait(bar, parity, 1000)) return true;
         if (spin > 64) __nanosleep(1000);  // long past any normal completion: back off
     }
     return false;
 }
+// Self-test of the bounded wait: a barrier that nothing ever arrives at.  The wait runs out after
+// `limit` tries (milliseconds), the thread records the flag exactly as the copy kernel would, and
+// the kernel returns normally; no copy is in flight, so there is nothing else to wait for.
+__global__ void tc_wait_timeout_probe(uint32_t limit)
+{
+    __shared__ __align__(8) unsigned long long probe_bar;
+    if (threadIdx.x != 0) return;
+    const uint32_t bar = static_cast<uint32_t>(__cvta_generic_to_shared(&probe_bar));
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait_bounded(bar, 0, limit)) atomicOr(&g_device_status, kStatusBulkWaitTimeout);
+}
+
 // global -> shared bulk copy of `bytes` (a multiple of 16; both addresses 16-byte aligned) that
 // reports to the barrier.  The source is this GPU's memory, a peer's or mapped host memory;
 // no multicast.

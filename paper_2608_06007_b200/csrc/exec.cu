@@ -332,6 +332,12 @@ extern "C" int tc_device_status(uint32_t *flags)
     return rc;
 }
 
+extern "C" int tc_selftest_wait_timeout(void *stream)
+{
+    clear_error();
+    return launch_wait_timeout_probe(static_cast<cudaStream_t>(stream));
+}
+
 extern "C" int tc_plan_stats(const tc_plan_t *plan, tc_plan_stats_t *out)
 {
     clear_error();

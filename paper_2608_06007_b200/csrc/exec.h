@@ -38,6 +38,9 @@ int launch_any(const tc_plan *plan, const Group &g, const void *const *src, void
 // The current device's sticky status word (flags set by kernels); reading clears it.
 int read_device_status(unsigned int *out);
 
+// Launch the self-test of the bounded wait (see tc_selftest_wait_timeout).
+int launch_wait_timeout_probe(cudaStream_t s);
+
 // ---- staging.cu
 // Take / drop a reference on the device's staging rings (allocated on first use); *bytes
 // receives the device memory the rings hold.

@@ -181,6 +181,13 @@ int read_device_status(unsigned int *out)
     return e == cudaSuccess ? TC_OK : cuda_fail(e, "reading the device status word");
 }
 
+int launch_wait_timeout_probe(cudaStream_t s)
+{
+    tc_wait_timeout_probe<<<1, 32, 0, s>>>(256);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? TC_OK : cuda_fail(e, "kernel launch");
+}
+
 int launch_any(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s, const Segment *win,
                unsigned long long *sums, bool over_host_link)
 {

@@ -694,6 +694,19 @@ def test_weights_checksum_fused_with_the_copy():
     assert e.value.status == tc.TC_ERR_KIND
 
 
+def test_a_wait_that_cannot_complete_ends_with_a_status_word_not_a_hang():
+    """The realigning build waits for its bulk copies with a bound.  The self-test waits on a
+    barrier nothing arrives at: the wait runs out, the kernel returns normally, the status word
+    carries the flag once, and the device keeps working."""
+    assert tc.tc_device_status() == 0
+    tc.tc_selftest_wait_timeout()
+    torch.cuda.synchronize()
+    assert tc.tc_device_status() == tc.TC_DEVICE_BULK_WAIT_TIMEOUT
+    assert tc.tc_device_status() == 0                       # reading cleared it
+    x = torch.arange(1024, device="cuda")
+    assert int(x.sum().item()) == 1023 * 512                # the context is alive and well
+
+
 def test_traced_plan_reports_the_device_time_of_its_last_execution():
     shape = wl.KVShape(L=4, B=16, H=8, D=128, E=2)
     NB = 512
@@ -714,8 +727,8 @@ def test_traced_plan_reports_the_device_time_of_its_last_execution():
     stream.synchronize()
     st = plan.stats()
     outer_us = 1e3 * a.elapsed_time(b)
-    assert st.trace_id == 77 and 0 < st.last_device_us[0] <= outer_us + 1.0   # 1 GiB moved: hundreds of microseconds
-    assert st.last_device_us[0] > 0.5 * outer_us
+    assert st.trace_id == 77 and st.last_device_us[0] <= outer_us + 1.0
+    assert st.last_device_us[0] > 2 * pool.numel() / 8e12 * 1e6   # 128 MiB read and written cannot beat 8 TB/s
     untraced = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape.tuple, src_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_src=bt))
     assert untraced.stats().last_device_us[0] == 0.0
 
