@@ -932,6 +932,56 @@ def test_random_geometries_on_the_device(seed):
     assert np.array_equal(fresh.result(), want_pool)
 
 
+@pytest.mark.parametrize("seed", range(32))
+def test_random_misaligned_geometries_on_the_device(seed):
+    """Random shapes, every buffer at its own random address modulo 16, rows of D * E bytes that
+    are or are not multiples of 16 (same alignment in every row, or a different one per row), block
+    strides with odd padding: pack, unpack and migrate against the oracle, destinations guarded."""
+    rng = np.random.default_rng(2000 + seed)
+    L, B, H = int(rng.integers(1, 4)), int(rng.choice([1, 4, 16, 32])), int(rng.integers(1, 9))
+    D, E = int(rng.choice([16, 20, 33, 64, 100, 128, 192])), int(rng.choice([1, 2, 4]))
+    R = int(rng.integers(1, 6))
+    T = np.array([int(rng.choice([0, 1, B, B + 1, 3 * B - 1, 9 * B, 12 * B + B // 2])) for _ in range(R)], dtype=np.int64)
+    pad = int(rng.choice([0, 0, E, 16, 48]))
+    s_pool, s_out, s_dst = (int(x) for x in rng.integers(0, 16, 3))
+    tile = int(rng.choice([0, 0, 2048, 8192]))
+    pool_l, other_l = int(rng.integers(0, 2)), int(rng.integers(0, 2))
+    slots = str(rng.choice(["planes", "one"]))
+    shape = (L, B, H, D, E)
+    off = np.concatenate([[0], np.cumsum((T + B - 1) // B)]).astype(np.int64)
+    NB = int(off[-1]) + 2
+    stride = B * H * D * E + pad
+    pool = rng.integers(0, 256, L * 2 * NB * stride, dtype=np.uint8)
+    bt = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    tune = dict(tile_bytes=tile) if tile else None
+    def mkpool(layout):
+        if slots == "planes":
+            return tc.pool(layout, NB, L * 2, block_stride=stride, slot_bytes=NB * stride)
+        return tc.pool(layout, NB, 1, plane_stride=NB * stride, block_stride=stride, slot_bytes=L * 2 * NB * stride)
+    pl, pl2 = mkpool(pool_l), mkpool(other_l)
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, pool_l, stride, planes_of(pool, L * 2), T, off, bt, other_l, want)
+    d_pool = Guarded(pool.size, init=pool, shift=s_pool)
+    out = Guarded(max(want.size, 1), shift=s_out)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=other_l, T=T, bt_off=off, bt_src=bt, tuning=tune))
+    tc.tc_kv_pack(plan, pool_tables(d_pool, L * 2, slots), [out.ptr()])
+    assert np.array_equal(out.result()[:want.size], want)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, pool_l, stride, planes_of(want_pool, L * 2), T, off, bt2, other_l, want)
+    fresh = Guarded(pool.size, shift=s_dst)
+    plan2 = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=other_l, T=T, bt_off=off, bt_dst=bt2, tuning=tune))
+    tc.tc_kv_unpack(plan2, [out.ptr()], pool_tables(fresh, L * 2, slots))
+    assert np.array_equal(fresh.result(), want_pool)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_migrate(shape, pool_l, stride, planes_of(pool, L * 2), other_l, stride, planes_of(want_pool, L * 2), T, off, bt, bt2)
+    mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl2, T=T, bt_off=off, bt_src=bt, bt_dst=bt2, tuning=tune))
+    fresh = Guarded(pool.size, shift=s_dst)
+    tc.tc_kv_pack(mig, pool_tables(d_pool, L * 2, slots), pool_tables(fresh, L * 2, slots))
+    assert np.array_equal(fresh.result(), want_pool)
+    assert tc.tc_device_status() == 0
+
+
 @pytest.mark.parametrize("shift", [0, 2])
 def test_execute_calls_can_be_captured_in_a_cuda_graph_and_replayed(shift):
     """Launch-bound use (config 1 moves 1.4 MB): pack + unpack captured once, replayed many
