@@ -1038,6 +1038,37 @@ def misaligned(args, tc, torch, stream):
         p_.destroy()
     del rawA, rawB, rawQ
     torch.cuda.empty_cache()
+    # rows whose length is not a multiple of 16 (head_dim 100 / 66 / 65 in 2-byte elements): aligned
+    # pointers, but every row of a tile has its own alignment
+    odd = {}
+    for D in (100,) if args.small else (100, 66, 65):
+        shape = wl.KVShape(32, 16, 8, D, 2)
+        s = shape.tuple
+        NB = int(((1 if args.small else 4) << 30) // shape.block_bytes)
+        WB = NB // 2
+        _, _, _, waves = wl.config2(NB=NB, R=256, wave_blocks=WB, NB_dst=WB, shape=shape)
+        src, dst = waves[0]
+        payload = int(src.T.sum()) * shape.token_bytes
+        A = torch.empty(NB * shape.block_bytes, **u8)
+        B = torch.empty(WB * shape.block_bytes, **u8)
+        Q = torch.empty(payload, **u8)
+        plA = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * shape.chunk_bytes, slot_bytes=A.numel())
+        plB = tc.pool(tc.TC_NHD, WB, 1, plane_stride=WB * shape.chunk_bytes, slot_bytes=B.numel())
+        kw = dict(T=src.T, bt_off=src.bt_off)
+        pk = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, s, src_pool=plA, packed_layout=tc.TC_HND, bt_src=src.bt, **kw))
+        up = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_UNPACK, s, dst_pool=plB, packed_layout=tc.TC_HND, bt_dst=dst.bt, **kw))
+        mig = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIGRATE, s, src_pool=plA, dst_pool=plB, bt_src=src.bt, bt_dst=dst.bt, **kw))
+        res = {"alignment_of_the_geometry_bytes": int(pk.stats().vec_bytes[0])}
+        for name, fn in (("a1_pack", lambda: tc.tc_kv_pack(pk, [A], [Q], sp)), ("a2_unpack", lambda: tc.tc_kv_unpack(up, [Q], [B], sp)),
+                         ("a3_migrate", lambda: tc.tc_kv_pack(mig, [A], [B], sp))):
+            res[name] = 2 * payload / (b2b_ms(torch, stream, fn, reps=reps, warm=warm) * 1e-3) / GB
+        odd[f"rows of {2 * D} bytes"] = res
+        for p_ in (pk, up, mig):
+            p_.destroy()
+        del A, B, Q
+        torch.cuda.empty_cache()
+    out["row length not a multiple of 16 (L32 B16 H8, 4 GiB pool, aligned pointers)"] = odd
+    torch.cuda.empty_cache()
     return out
 
 

@@ -466,42 +466,76 @@ __device__ __forceinline__ void realign_store_dispatch(const Desc &d, const Real
 }
 
 // The same for tiles whose rows differ in alignment (a row pitch that is not a multiple of 16):
-// every chunk works out its own row's alignments.  Out of line: a rare geometry.
+// one bulk copy per row as well - every row announces its own byte count, the sum reaches the
+// barrier through a shared-memory counter - and every chunk works out its own row's alignments.
+// Out of line: a rare geometry.  False: the copies did not arrive in time (see realign_wait).
 template <int kThreads>
-__device__ __noinline__ void realign_pass_mixed(const Desc &d, const char *src, char *dst, uint32_t row_base, uint32_t n_rows, uint32_t len, char *data)
+__device__ __noinline__ bool realign_pass_mixed(const Desc &d, const char *src, char *dst, uint32_t row_base, uint32_t n_rows, uint32_t len, char *data,
+                                                uint32_t bar, uint32_t phase, uint32_t *wait_ok, uint32_t *tx_total)
 {
     const uint32_t n0 = d.n0, ss0 = d.src_s0, ss1 = d.src_s1, ds0 = d.dst_s0, ds1 = d.dst_s1;
     const FastDiv div_n0 = d.div_n0, div_units{d.units_mul, d.units_shift};
     const uint32_t units = (min(d.run, kRealignColumn) + 30) >> 4;
     const uint32_t data_addr = static_cast<uint32_t>(__cvta_generic_to_shared(data));
     const uint32_t total = n_rows * units;
-    for (uint32_t u = threadIdx.x; u < total; u += kThreads) {
-        const uint32_t rr = fastdiv(u, div_units), c = u - rr * units;
+    if (threadIdx.x == 0) *tx_total = 0;
+    __syncthreads();
+    uint32_t mine = 0;
+    for (uint32_t rr = threadIdx.x; rr < n_rows; rr += kThreads) {
         const uint32_t r = row_base + rr, i1 = fastdiv(r, div_n0), i0 = r - i1 * n0;
         const char *s = src + (i1 * ss1 + i0 * ss0);
-        const uintptr_t chunk = (reinterpret_cast<uintptr_t>(s) & ~uintptr_t(15)) + 16 * c;
-        if (chunk < reinterpret_cast<uintptr_t>(s) + len) cp_async16(data_addr + 16 * u, reinterpret_cast<const void *>(chunk));
+        const uint32_t s_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(s)) & 15;
+        const uint32_t bytes = ((s_lo + len + 15) >> 4) << 4;
+        bulk_load(data_addr + 16 * rr * units, s - s_lo, bytes, bar);
+        mine += bytes;
     }
-    cp_async_wait_all();
+    if (mine) atomicAdd(tx_total, mine);
     __syncthreads();
+    // the copies may complete before their bytes are announced (the count runs negative for a
+    // moment); the phase cannot end before the one arrival that comes with the announcement
+    if (threadIdx.x == 0) mbar_expect_tx(bar, *tx_total);
+    if (!realign_wait(bar, phase, wait_ok)) return false;  // the caller flips its own copy of the phase
+    // whole chunks first, in one loop without the partial-store code; a chunk knows from its row's
+    // destination alignment whether it is whole
     for (uint32_t u = threadIdx.x; u < total; u += kThreads) {
         const uint32_t rr = fastdiv(u, div_units), c = u - rr * units;
         const uint32_t r = row_base + rr, i1 = fastdiv(r, div_n0), i0 = r - i1 * n0;
-        const uint32_t s_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src + (i1 * ss1 + i0 * ss0))) & 15;
         char *dp = dst + (i1 * ds1 + i0 * ds0);
         const uint32_t d_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(dp)) & 15;
         const int first = static_cast<int>(16 * c) - static_cast<int>(d_lo);  // row byte at the chunk's byte 0
-        const uint32_t lo = first < 0 ? static_cast<uint32_t>(-first) : 0;
-        const int left = static_cast<int>(len) - first;
-        if (left <= static_cast<int>(lo)) continue;
-        const uint32_t hi = left < 16 ? static_cast<uint32_t>(left) : 16;
-        const int q = static_cast<int>(s_lo) + first;  // the row's byte b sits at 16 * rr * units + s_lo + b; q >= -15
-        const char *at = data + 16 * (rr * units) + 16 * (q >> 4);
-        const uint4 a = *reinterpret_cast<const uint4 *>(at), b = *reinterpret_cast<const uint4 *>(at + 16);
-        const uint4 v = shift_bytes(a, b, static_cast<uint32_t>(q) & 15);
-        if (lo == 0 && hi == 16) st_stream<uint4>(dp + first, v);
-        else store_partial(dp + first, v, lo, hi);
+        if (first < 0 || first + 16 > static_cast<int>(len)) continue;
+        const uint32_t s_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src + (i1 * ss1 + i0 * ss0))) & 15;
+        const uint32_t q = s_lo + first;  // the row's byte b sits at 16 * rr * units + s_lo + b
+        const uint32_t at = data_addr + 16 * (rr * units) + 16 * (q >> 4);
+        st_stream<uint4>(dp + first, shift_bytes(lds128(at), lds128(at + 16), q & 15));
     }
+    // then the partial first and last chunk of every row: one thread per (row, end).  (Storing
+    // the chunk that two destination-adjacent rows share once, as the same-alignment path does,
+    // measured no faster here.)
+    for (uint32_t item = threadIdx.x; item < 2 * n_rows; item += kThreads) {
+        const uint32_t rr = item >> 1;
+        const uint32_t r = row_base + rr, i1 = fastdiv(r, div_n0), i0 = r - i1 * n0;
+        char *dp = dst + (i1 * ds1 + i0 * ds0);
+        const uint32_t d_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(dp)) & 15;
+        const uint32_t end = d_lo + len;  // first byte past the row, counted from its first chunk
+        uint32_t c, lo, hi;
+        if (item & 1) {  // tail: chunk end / 16, unless the row ends on a boundary or lies in one chunk
+            c = end >> 4;
+            lo = 0;
+            hi = end & 15;
+            if (c == 0 || hi == 0) continue;
+        } else {         // head: chunk 0, unless it is whole
+            c = 0;
+            lo = d_lo;
+            hi = min(end, 16u);
+            if (lo == 0 && hi == 16) continue;
+        }
+        const uint32_t s_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src + (i1 * ss1 + i0 * ss0))) & 15;
+        const int q = static_cast<int>(s_lo) + static_cast<int>(16 * c) - static_cast<int>(d_lo);  // >= -15
+        const uint32_t at = data_addr + 16 * (rr * units) + 16 * (q >> 4);
+        store_partial(dp - d_lo + 16 * c, shift_bytes(lds128(at), lds128(at + 16), static_cast<uint32_t>(q) & 15), lo, hi);
+    }
+    return true;
 }
 
 // Rows [row0, row0 + nrows) of one outer index of descriptor d, any alignment; src / dst point
@@ -557,7 +591,8 @@ __device__ __forceinline__ bool copy_rows_realign(const Desc &d, const char *src
                 default: realign_store_all<3, kThreads>(d, p, data_addr); break;
                 }
             } else {
-                realign_pass_mixed<kThreads>(d, src + col0, dst + col0, row0 + r0, n_rows, len, data);
+                if (!realign_pass_mixed<kThreads>(d, src + col0, dst + col0, row0 + r0, n_rows, len, data, bar, phase, wait_ok, wait_ok + 1)) return false;
+                phase ^= 1;
             }
             __syncthreads();
         }
@@ -699,13 +734,13 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
     __shared__ Desc sdesc[2];
     extern __shared__ __align__(16) char stage[];  // the realigning path's staging area (kModeAny only)
     __shared__ __align__(8) unsigned long long stage_bar;  // its mbarrier
-    __shared__ uint32_t stage_ok;
+    __shared__ uint32_t stage_ok[2];  // [0] the bulk copies arrived, [1] byte counter of the mixed-alignment path
     uint32_t bar = 0, phase = 0;
     if (MODE == kModeAny) {
         bar = static_cast<uint32_t>(__cvta_generic_to_shared(&stage_bar));
         if (threadIdx.x == 0) {
             mbar_init(bar, 1);
-            stage_ok = 1;
+            stage_ok[0] = 1;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
         // made visible to the CTA by the __syncthreads that follows the descriptor fetch below
@@ -768,7 +803,7 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
                 const uint32_t align = min(static_cast<uint32_t>(d.log2_align), prm.log2_ptr_align);
                 bool alive = true;
                 if (align == 4) copy_multi<4, kUnroll, kThreads, true, MULTI == 2>(d, prm, o, n_units);
-                else if (!copy_multi_realign<kThreads, MULTI == 2>(d, prm, o, n_units, stage, bar, phase, &stage_ok, alive))
+                else if (!copy_multi_realign<kThreads, MULTI == 2>(d, prm, o, n_units, stage, bar, phase, stage_ok, alive))
                     copy_multi_narrow<2 * kUnroll, kThreads, MULTI == 2>(d, prm, o, n_units, align);
                 if (!alive) return;
             }
@@ -806,7 +841,7 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
             if (align == 4 && (!prm.stage_always || d.run < kRealignMinRun)) {
                 copy_rows<4, kUnroll, kThreads>(d, src, dst, row0, nrows);
             } else if (d.run >= kRealignMinRun) {
-                if (!copy_rows_realign<kThreads>(d, src, dst, row0, nrows, stage, prm.stage_bytes, bar, phase, &stage_ok)) return;
+                if (!copy_rows_realign<kThreads>(d, src, dst, row0, nrows, stage, prm.stage_bytes, bar, phase, stage_ok)) return;
             } else {
                 copy_rows_narrow<kUnroll, kThreads>(d, src, dst, row0, nrows, align);
             }
