@@ -332,27 +332,52 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
     return v;
 }
 
+// A pass over several planes of one descriptor (multi-plane tiles): row rr of the pass is row
+// rr % rows of plane rr / rows, and plane j's destination (its address rounded down to 16) is
+// dst[j], an array in shared memory.  All planes of such a pass share one alignment.
+struct PlaneSet {
+    uint32_t rows, magic;            // rows per plane; ceil(2^32 / rows) for the division (rows > 1)
+    const unsigned long long *dst;   // per plane: destination of row 0, chunk 0
+};
+
+// Destination of chunk 0 of row rr of the pass, and the row's index inside its descriptor.
+template <bool PLANES>
+__device__ __forceinline__ char *realign_row(const Desc &d, const RealignPass &p, const PlaneSet *ps, uint32_t rr, uint32_t &r)
+{
+    char *base;
+    if (PLANES) {
+        const uint32_t j = ps->rows > 1 ? __umulhi(rr, ps->magic) : rr;
+        r = rr - j * ps->rows;
+        base = reinterpret_cast<char *>(ps->dst[j]);
+    } else {
+        r = p.row_base + rr;
+        base = p.dst - p.d_lo;
+    }
+    const uint32_t i1 = fastdiv(r, d.div_n0), i0 = r - i1 * d.n0;
+    return base + (i1 * d.dst_s1 + i0 * d.dst_s0);
+}
+
 // Whole destination chunks [c_begin, c_end) of every row of the pass.  data_addr: shared-memory
 // address of the staged rows.  Two thread mappings keep the loop body short:
 //   long rows   all threads walk the chunks of one row, kThreads at a time; the row is decoded
 //               once, outside the loop;
 //   short rows  (fewer chunks than threads) the CTA splits into groups of `units` threads; a
 //               thread keeps its chunk index and steps through the rows, one group apart.
-template <int WS, int kThreads>
-__device__ __forceinline__ void realign_store_full(const Desc &d, const RealignPass &p, uint32_t data_addr, uint32_t c_begin, uint32_t c_end)
+template <int WS, int kThreads, bool PLANES = false>
+__device__ __forceinline__ void realign_store_full(const Desc &d, const RealignPass &p, uint32_t data_addr, uint32_t c_begin, uint32_t c_end,
+                                                   const PlaneSet *ps = nullptr)
 {
-    const uint32_t n0 = d.n0, ds0 = d.dst_s0, ds1 = d.dst_s1, units = p.units;
-    const FastDiv div_n0 = d.div_n0, div_units{d.units_mul, d.units_shift};
+    const uint32_t units = p.units;
+    const FastDiv div_units{d.units_mul, d.units_shift};
     const int delta = static_cast<int>(p.s_lo) - static_cast<int>(p.d_lo);
     const uint32_t bits = (static_cast<uint32_t>(delta) & 3) * 8;
     const uint32_t shifted = data_addr + 16 * (delta >> 4);  // delta >> 4 is 0 or -1
-    char *base = p.dst - p.d_lo;
+    uint32_t r;
     if (units >= kThreads) {
         for (uint32_t rr = 0; rr < p.n_rows; rr++) {
-            const uint32_t r = p.row_base + rr, i1 = fastdiv(r, div_n0), i0 = r - i1 * n0;
             uint32_t c = c_begin + threadIdx.x;
             uint32_t at = shifted + 16 * (rr * units + c);
-            char *out = base + (i1 * ds1 + i0 * ds0) + 16 * static_cast<size_t>(c);
+            char *out = realign_row<PLANES>(d, p, ps, rr, r) + 16 * static_cast<size_t>(c);
 #pragma unroll 2
             for (; c < c_end; c += kThreads, at += 16 * kThreads, out += 16 * kThreads)
                 st_stream<uint4>(out, shift_words<WS>(lds128(at), lds128(at + 16), bits));
@@ -362,12 +387,9 @@ __device__ __forceinline__ void realign_store_full(const Desc &d, const RealignP
         const uint32_t g = fastdiv(threadIdx.x, div_units), c = threadIdx.x - g * units;
         if (g >= groups || c < c_begin || c >= c_end) return;
         uint32_t at = shifted + 16 * (g * units + c);
-        char *col = base + 16 * c;
 #pragma unroll 2
-        for (uint32_t rr = g; rr < p.n_rows; rr += groups, at += 16 * groups * units) {
-            const uint32_t r = p.row_base + rr, i1 = fastdiv(r, div_n0), i0 = r - i1 * n0;
-            st_stream<uint4>(col + (i1 * ds1 + i0 * ds0), shift_words<WS>(lds128(at), lds128(at + 16), bits));
-        }
+        for (uint32_t rr = g; rr < p.n_rows; rr += groups, at += 16 * groups * units)
+            st_stream<uint4>(realign_row<PLANES>(d, p, ps, rr, r) + 16 * c, shift_words<WS>(lds128(at), lds128(at + 16), bits));
     }
 }
 
@@ -388,27 +410,29 @@ __device__ __forceinline__ uint4 merge_bytes(uint4 a, uint4 b, uint32_t t)
 // where this one ends (rows `adj` apart in the descriptor's row order, adjacent in memory), its
 // head and this row's tail fill one chunk between them: that chunk is assembled from both rows
 // and stored whole, instead of as up to eight small pieces.
-template <int WS, int kThreads>
-__device__ __forceinline__ void realign_store_edges(const Desc &d, const RealignPass &p, uint32_t data_addr, uint32_t c_last, uint32_t end)
+template <int WS, int kThreads, bool PLANES = false>
+__device__ __forceinline__ void realign_store_edges(const Desc &d, const RealignPass &p, uint32_t data_addr, uint32_t c_last, uint32_t end,
+                                                    const PlaneSet *ps = nullptr)
 {
     const uint32_t n0 = d.n0, ds0 = d.dst_s0, ds1 = d.dst_s1, units = p.units;
-    const FastDiv div_n0 = d.div_n0;
     const int delta = static_cast<int>(p.s_lo) - static_cast<int>(p.d_lo);
     const uint32_t bits = (static_cast<uint32_t>(delta) & 3) * 8;
     const uint32_t shifted = data_addr + 16 * (delta >> 4);
-    char *base = p.dst - p.d_lo;
     const bool one_chunk = c_last == 0;
     const uint32_t t = end & 15;  // bytes of the tail
     // rows adjacent in the destination: the whole row moves (no column pieces) and its length
     // keeps the alignment, so that a tail of t bytes meets a head that starts at byte t = d_lo
     uint32_t adj = 0;
     if (!one_chunk && t && p.len == d.run && (d.run & 15) == 0) adj = (n0 > 1 && ds0 == d.run) ? 1 : (ds1 == d.run ? n0 : 0);
+    // rows of the descriptor that the pass holds of the row's plane: [first, first + count)
+    const uint32_t first = PLANES ? 0 : p.row_base, count = PLANES ? ps->rows : p.n_rows;
     for (uint32_t rr = threadIdx.x; rr < p.n_rows; rr += kThreads) {
-        const uint32_t r = p.row_base + rr, i1 = fastdiv(r, div_n0), i0 = r - i1 * n0;
-        char *out = base + (i1 * ds1 + i0 * ds0);
+        uint32_t r;
+        char *out = realign_row<PLANES>(d, p, ps, rr, r);
+        const uint32_t i0 = r - fastdiv(r, d.div_n0) * n0;
         const uint32_t row_at = shifted + 16 * rr * units;
-        const bool has_next = adj && (adj == 1 ? i0 + 1 < n0 : r + n0 < d.rows) && rr + adj < p.n_rows;
-        const bool has_prev = adj && (adj == 1 ? i0 >= 1 : r >= n0) && rr >= adj;
+        const bool has_next = adj && (adj == 1 ? i0 + 1 < n0 : r + n0 < d.rows) && r + adj < first + count;
+        const bool has_prev = adj && (adj == 1 ? i0 >= 1 : r >= n0) && r >= first + adj;
         if ((p.d_lo || one_chunk) && !has_prev)
             store_partial(out, shift_words<WS>(lds128(row_at), lds128(row_at + 16), bits), p.d_lo, one_chunk ? end : 16);
         if (!one_chunk && t) {
@@ -424,14 +448,14 @@ __device__ __forceinline__ void realign_store_edges(const Desc &d, const Realign
     }
 }
 
-template <int WS, int kThreads>
-__device__ __forceinline__ void realign_store_all(const Desc &d, const RealignPass &p, uint32_t data)
+template <int WS, int kThreads, bool PLANES = false>
+__device__ __forceinline__ void realign_store_all(const Desc &d, const RealignPass &p, uint32_t data, const PlaneSet *ps = nullptr)
 {
     // chunk c of a row's destination covers row bytes [16c - d_lo, 16c - d_lo + 16)
     const uint32_t end = p.d_lo + p.len;  // first byte past the row, counted from the row's first chunk
     const uint32_t c_first = p.d_lo ? 1 : 0, c_last = end >> 4;  // whole chunks: [c_first, c_last)
-    if (c_last > c_first) realign_store_full<WS, kThreads>(d, p, data, c_first, c_last);
-    if (p.d_lo || (end & 15)) realign_store_edges<WS, kThreads>(d, p, data, c_last, end);
+    if (c_last > c_first) realign_store_full<WS, kThreads, PLANES>(d, p, data, c_first, c_last, ps);
+    if (p.d_lo || (end & 15)) realign_store_edges<WS, kThreads, PLANES>(d, p, data, c_last, end, ps);
 }
 
 // Wait for the bulk copies of the current phase.  One thread waits (bounded) and tells the
@@ -454,14 +478,14 @@ __device__ __forceinline__ bool realign_wait(uint32_t bar, uint32_t &phase, uint
     return true;
 }
 
-template <int kThreads>
-__device__ __forceinline__ void realign_store_dispatch(const Desc &d, const RealignPass &p, uint32_t data_addr)
+template <int kThreads, bool PLANES = false>
+__device__ __forceinline__ void realign_store_dispatch(const Desc &d, const RealignPass &p, uint32_t data_addr, const PlaneSet *ps = nullptr)
 {
     switch (((p.s_lo - p.d_lo) & 15) >> 2) {
-    case 0: realign_store_all<0, kThreads>(d, p, data_addr); break;
-    case 1: realign_store_all<1, kThreads>(d, p, data_addr); break;
-    case 2: realign_store_all<2, kThreads>(d, p, data_addr); break;
-    default: realign_store_all<3, kThreads>(d, p, data_addr); break;
+    case 0: realign_store_all<0, kThreads, PLANES>(d, p, data_addr, ps); break;
+    case 1: realign_store_all<1, kThreads, PLANES>(d, p, data_addr, ps); break;
+    case 2: realign_store_all<2, kThreads, PLANES>(d, p, data_addr, ps); break;
+    default: realign_store_all<3, kThreads, PLANES>(d, p, data_addr, ps); break;
     }
 }
 
@@ -698,17 +722,49 @@ __device__ __forceinline__ bool copy_multi_realign(const Desc &d, const Params<N
         p.d_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(p.dst)) & 15;
         return p;
     };
+    // per plane: where its destination starts (rounded down to 16), and whether every plane has
+    // the alignment of plane 0 on both sides, so that one pass of the store loops can serve all
+    __shared__ unsigned long long plane_dst[64];
+    __shared__ uint32_t same_alignment;
+    uint32_t *same = &same_alignment;
     if (threadIdx.x == 0) {
-        uint32_t bytes = 0;
-        for (uint32_t j = 0; j < n_units; j++) bytes += d.rows * realign_row_bytes(plane(j));
+        uint32_t bytes = 0, ok = 1;
+        const RealignPass p0 = plane(0);
+        for (uint32_t j = 0; j < n_units; j++) {
+            const RealignPass pj = plane(j);
+            bytes += d.rows * realign_row_bytes(pj);
+            plane_dst[j] = reinterpret_cast<unsigned long long>(pj.dst - pj.d_lo);
+            ok &= pj.s_lo == p0.s_lo && pj.d_lo == p0.d_lo;
+        }
+        same_alignment = ok;
         mbar_expect_tx(bar, bytes);
     }
-    for (uint32_t j = 0; j < n_units; j++) realign_load<kThreads, false>(d, plane(j), data_addr + j * plane_stage, bar);
+    if (d.rows >= kThreads) {
+        for (uint32_t j = 0; j < n_units; j++) realign_load<kThreads, false>(d, plane(j), data_addr + j * plane_stage, bar);
+    } else {  // few rows per plane: one thread per row of the tile, whatever its plane
+        const uint32_t magic = d.rows > 1 ? 0xffffffffu / d.rows + 1 : 0;
+        for (uint32_t rr = threadIdx.x; rr < n_units * d.rows; rr += kThreads) {
+            const uint32_t j = d.rows > 1 ? __umulhi(rr, magic) : rr, r = rr - j * d.rows;
+            const RealignPass pj = plane(j);
+            const uint32_t i1 = fastdiv(r, d.div_n0), i0 = r - i1 * d.n0;
+            bulk_load(data_addr + 16 * rr * units, pj.src - pj.s_lo + (i1 * d.src_s1 + i0 * d.src_s0), realign_row_bytes(pj), bar);
+        }
+    }
     if (!realign_wait(bar, phase, wait_ok)) {
         alive = false;
         return true;
     }
-    for (uint32_t j = 0; j < n_units; j++) realign_store_dispatch<kThreads>(d, plane(j), data_addr + j * plane_stage);
+    if (*same) {  // one pass of the store loops over the rows of all planes
+        RealignPass all = plane(0);
+        all.n_rows = n_units * d.rows;
+        PlaneSet ps;
+        ps.rows = d.rows;
+        ps.magic = d.rows > 1 ? 0xffffffffu / d.rows + 1 : 0;
+        ps.dst = plane_dst;
+        realign_store_dispatch<kThreads, true>(d, all, data_addr, &ps);
+    } else {
+        for (uint32_t j = 0; j < n_units; j++) realign_store_dispatch<kThreads>(d, plane(j), data_addr + j * plane_stage);
+    }
     __syncthreads();
     return true;
 }
