@@ -375,7 +375,9 @@ __device__ __forceinline__ void realign_store_full(const Desc &d, const RealignP
     uint32_t r;
     if (units >= kThreads) {
         for (uint32_t rr = 0; rr < p.n_rows; rr++) {
-            uint32_t c = c_begin + threadIdx.x;
+            // a thread's chunks are threadIdx.x + k * kThreads whatever c_begin is, so that a warp's
+            // 512 bytes keep to whole 128-byte lines of the destination
+            uint32_t c = threadIdx.x < c_begin ? threadIdx.x + kThreads : threadIdx.x;
             uint32_t at = shifted + 16 * (rr * units + c);
             char *out = realign_row<PLANES>(d, p, ps, rr, r) + 16 * static_cast<size_t>(c);
 #pragma unroll 2
