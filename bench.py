@@ -1325,7 +1325,8 @@ def extra_config4(args, tc, torch, stream, out):
             plan = tc.tc_plan_create(tc.kv_spec(
                 tc.TC_KV_MIXED, shape.tuple, src_pool=dev_pool, dst_pool=host_pool,
                 T=st.offload_T, bt_off=st.offload_off, bt_src=st.offload_dev, bt_dst=st.offload_host,
-                reload=dict(T=st.reload_T, bt_off=st.reload_off, bt_src=st.reload_host, bt_dst=st.reload_dev), flags=flags))
+                reload=dict(T=st.reload_T, bt_off=st.reload_off, bt_src=st.reload_host, bt_dst=st.reload_dev), flags=flags,
+                tuning=dict(max_ctas=args.host_ctas) if args.host_ctas else None))
             if i >= 1:
                 create.append(1e3 * (time.perf_counter() - t0))
                 h2d += int(st.reload_T.sum()) * shape.token_bytes
