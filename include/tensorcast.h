@@ -435,7 +435,8 @@ typedef struct {
     int64_t payload_bytes[2];      /* bytes moved by one execution of each group */
     int64_t packed_bytes_required; /* PACK / UNPACK: sum of L*2*T_r*H*D*E */
     int64_t device_bytes;          /* plan storage held on the device */
-    int32_t vec_bytes[2];          /* widest access the geometry allows (pointers may narrow it) */
+    int32_t vec_bytes[2];          /* alignment the geometry guarantees, in bytes, up to 16; below 16 - or
+                                      with less aligned base pointers - the realigning path runs */
     int32_t launches_per_execute;  /* kernels one execute call launches (1; one per segment for
                                       staged plans) */
     int32_t path[2];               /* 1 direct (zero copy when a buffer is host memory),
