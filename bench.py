@@ -665,6 +665,15 @@ def run_ours(args):
                 made[path] = host_plans(path)
             key = f"{path}_{'duplex' if duplex else 'serial'}"
             e2e_all[key] = run_e2e(made[path], duplex, args.e2e_steps, args.e2e_warmup)
+        if can_duplex and "staged" in made and "zerocopy" in made and args.e2e_schedule == "duplex":
+            # the offload by kernel stores straight into pinned memory (they keep their speed while the
+            # other direction is busy), the reload and the weights through the copy engines
+            st, zc = made["staged"], made["zerocopy"]
+            mix = dict(kv=[(z[0], s_[1], s_[2]) for z, s_ in zip(zc["kv"], st["kv"])], path="offload zerocopy, reload staged",
+                       w_full=st["w_full"], w_shard=st["w_shard"])
+            mix["launches"] = (sum(a.stats().launches_per_execute + b.stats().launches_per_execute for a, b, _ in mix["kv"])
+                               + st["w_full"].stats().launches_per_execute + st["w_shard"].stats().launches_per_execute)
+            e2e_all["offload_zerocopy_reload_staged_duplex"] = run_e2e(mix, True, args.e2e_steps, args.e2e_warmup)
         for hp in made.values():
             drop_host_plans(hp)
         best = max(e2e_all, key=lambda k: e2e_all[k]["host_link_GBps"])
