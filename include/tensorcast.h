@@ -48,7 +48,7 @@
  * then reads or writes directly over the host link (zero copy), or another GPU's memory once
  * peer access is enabled (every CTA then moves its own tile over NVLink with plain loads and
  * stores - misaligned geometry: with per-CTA bulk asynchronous loads into its shared memory;
- * the library issues no multicast copy of any kind).  Pageable host memory is not
+ * every copy lands in the issuing CTA's own shared memory or registers).  Pageable host memory is not
  * addressable by the device: the execute calls refuse it (TC_ERR_INVALID_ARG) instead of
  * letting a kernel fault.  The tables themselves, the
  * spec and every array it points to are HOST memory.

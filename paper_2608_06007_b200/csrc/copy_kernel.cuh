@@ -187,20 +187,11 @@ __device__ __noinline__ void copy_rows_narrow(const Desc &d, const char *src, ch
 // reads whole aligned 16-byte chunks, so up to 15 bytes before a row's first byte and after
 // its last one are read (never a chunk without a byte of the row, hence never another page);
 // nothing outside the row is ever written.
-// Tiles whose rows differ in alignment (a row pitch that is not a multiple of 16) load with
-// 16-byte cp.async per chunk instead and work out every chunk's own alignments.
+// Tiles whose rows differ in alignment (a row pitch that is not a multiple of 16) load the same
+// way and work out every chunk's own alignments at run time.
 // The wait for the bulk copies is bounded: if it ever ran out, the CTA would record
 // kStatusBulkWaitTimeout in the device status word, wait once more for its copies, and return
 // without storing (the host reads the word with tc_device_status).
-__device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void *gptr)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr), "l"(gptr) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all()
-{
-    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-}
-
 // Bytes [sh, sh + 16) of the 32 bytes a | b.
 __device__ __forceinline__ uint4 shift_bytes(uint4 a, uint4 b, uint32_t sh)
 {
@@ -285,8 +276,8 @@ __global__ void tc_wait_timeout_probe(uint32_t limit)
 }
 
 // global -> shared bulk copy of `bytes` (a multiple of 16; both addresses 16-byte aligned) that
-// reports to the barrier.  The source is this GPU's memory, a peer's or mapped host memory;
-// no multicast.
+// reports to the barrier.  The source is this GPU's memory, a peer's or mapped host memory; the
+// copy lands in the issuing CTA's own shared memory only.
 __device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void *gsrc, uint32_t bytes, uint32_t bar)
 {
     asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"

@@ -738,7 +738,7 @@ def test_traced_plan_reports_the_device_time_of_its_last_execution():
 def test_pack_and_migrate_from_a_pool_on_another_gpu():
     """Cross-GPU migration: the source pool lives on device 1, the plan and the destination on
     device 0.  A table entry is then a peer pointer; every CTA moves its own tile with plain loads
-    over NVLink (no bulk or multicast copy is involved: the geometry is aligned, so the register
+    over NVLink (no bulk copy is involved: the geometry is aligned, so the register
     path runs).  Compared with the oracle like any other pack / migrate."""
     if not torch.cuda.can_device_access_peer(0, 1):
         pytest.skip("devices 0 and 1 have no peer access")
