@@ -211,6 +211,62 @@ def run_realign_tile(d, o, part, src, dst, cnt, smem_bytes=52 << 10, threads=256
                         dst.write(out_addr(rr, c_last), tail[:t], cnt)
 
 
+def run_realign_tile_mixed(d, o, part, src, dst, cnt, smem_bytes=52 << 10):
+    """The realigning path for rows that differ in alignment (a row pitch that is not a multiple
+    of 16), replayed like run_realign_tile: one aligned bulk load per row, then every whole
+    destination chunk from its own row's two alignments, then each row's partial first and last
+    chunk."""
+    column_max = smem_bytes - 64
+    row0 = part * d.rows_per_tile
+    nrows = min(d.rows_per_tile, d.rows - row0)
+    run = d.run_bytes
+    column = min(run, column_max)
+    units = (column + 30) >> 4
+    rows_per_pass = (smem_bytes - 32) // (units << 4)
+    src0 = src.va + d.src_off + o * d.src_outer
+    dst0 = dst.va + d.dst_off + o * d.dst_outer
+    rowoff = lambda r, s0, s1: (r // d.n0) * s1 + (r % d.n0) * s0
+    data = 16
+    for col0 in range(0, run, column):
+        length = min(column, run - col0)
+        for r0 in range(0, nrows, rows_per_pass):
+            n_rows = min(rows_per_pass, nrows - r0)
+            stage = np.full(smem_bytes, 0xDD, dtype=np.uint8)
+            loaded = np.zeros(smem_bytes, dtype=bool)
+            for rr in range(n_rows):
+                s = src0 + col0 + rowoff(row0 + r0 + rr, d.src_s0, d.src_s1)
+                s_lo = s % 16
+                nbytes = ((s_lo + length + 15) >> 4) << 4
+                at = data + 16 * rr * units
+                assert nbytes <= units * 16 and at + nbytes <= smem_bytes - 16
+                for c in range(nbytes // 16):
+                    stage[at + 16 * c:at + 16 * c + 16] = src.read16(s - s_lo + 16 * c)
+                    loaded[at + 16 * c:at + 16 * c + 16] = True
+
+            def chunk(rr, q, lo, hi):                         # 16 bytes that start q bytes into row rr's staged chunks
+                at = data + 16 * rr * units + q
+                assert data - 16 <= at - (q % 16) and at - (q % 16) + 32 <= smem_bytes, "staging read outside the area"
+                assert loaded[at + lo:at + hi].all(), "a staged byte that was never loaded is consumed"
+                return stage[at:at + 16].copy()
+
+            for rr in range(n_rows):
+                s = src0 + col0 + rowoff(row0 + r0 + rr, d.src_s0, d.src_s1)
+                dp = dst0 + col0 + rowoff(row0 + r0 + rr, d.dst_s0, d.dst_s1)
+                s_lo, d_lo = s % 16, dp % 16
+                end = d_lo + length
+                for c in range(units):                        # whole chunks
+                    first = 16 * c - d_lo
+                    if first < 0 or first + 16 > length:
+                        continue
+                    dst.write(dp + first, chunk(rr, s_lo + first, 0, 16), cnt)
+                if not (d_lo == 0 and min(end, 16) == 16):    # head
+                    hi = min(end, 16)
+                    dst.write(dp, chunk(rr, s_lo - d_lo, d_lo, hi)[d_lo:hi], cnt)
+                c, t = end >> 4, end & 15                     # tail
+                if c and t:
+                    dst.write(dp - d_lo + 16 * c, chunk(rr, s_lo + 16 * c - d_lo, 0, t)[:t], cnt)
+
+
 def planes_of(pool, n_planes):
     per = pool.size // n_planes
     return [pool[i * per:(i + 1) * per] for i in range(n_planes)]

@@ -631,6 +631,39 @@ def test_realigning_path_arithmetic_on_the_cpu(a, b):
             assert cnt.max() == 1 and cnt.sum() == int(T.sum()) * 2 * 4 * 128, (spec.kind, smem)
 
 
+@pytest.mark.parametrize("D,E,a,b", [(40, 1, 0, 0), (50, 2, 3, 0), (33, 1, 7, 12), (36, 1, 0, 5), (100, 2, 1, 1)])
+def test_realigning_path_arithmetic_for_rows_that_differ_in_alignment(D, E, a, b):
+    """Rows of D * E bytes, not a multiple of 16: every row of a tile has its own source and
+    destination alignment.  Pack, unpack and a same-layout migration replayed on the CPU with
+    the kernel's per-chunk arithmetic, one pass and several passes per tile."""
+    from helpers import _Mem, run_realign_tile_mixed
+    rng = np.random.default_rng(80 + D + a)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=1, NB=8, B=8, H=3, D=D, E=E, T=(19, 8, 3))
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride)
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, 2), T, off, bt, oracle.HND, want)
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(want_pool, 2), T, off, bt2, oracle.HND, want)
+    cases = [(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_src=bt, flags=HOST), 0, pool, want, 0),
+             (tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_dst=bt2, flags=HOST), 1, want, want_pool, 0xA5)]
+    for spec, group, source, expect, fill in cases:
+        plan = tc.tc_plan_create(spec)
+        for smem in (52 << 10, 704):
+            got = np.full(expect.size, fill, dtype=np.uint8)
+            cnt = np.zeros(expect.size, dtype=np.int32)
+            src, dst = _Mem(source, 4096 + a), _Mem(got, 1 << 20 | b)
+            for d in plan.descriptors(group):
+                if d.run_bytes < 32:
+                    pytest.skip("rows this short take the narrow-vector loop")
+                for o in range(d.n_outer):
+                    for part in range(d.tiles_per_outer):
+                        if part * d.rows_per_tile < d.rows:
+                            run_realign_tile_mixed(d, o, part, src, dst, cnt, smem_bytes=smem)
+            assert np.array_equal(got, expect), (spec.kind, smem)
+            assert cnt.max() == 1 and cnt.sum() == int(T.sum()) * 2 * 3 * D * E, (spec.kind, smem)
+
+
 def test_same_pool_compaction_lowering_and_its_overlap_check():
     """Defragmentation: the requests' blocks move to the low block ids of the same pool."""
     rng = np.random.default_rng(6)
