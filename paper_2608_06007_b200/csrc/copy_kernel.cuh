@@ -403,6 +403,7 @@ __device__ __forceinline__ uint4 merge_bytes(uint4 a, uint4 b, uint32_t t)
 // where this one ends (rows `adj` apart in the descriptor's row order, adjacent in memory), its
 // head and this row's tail fill one chunk between them: that chunk is assembled from both rows
 // and stored whole, instead of as up to eight small pieces.
+
 template <int WS, int kThreads, bool PLANES = false>
 __device__ __forceinline__ void realign_store_edges(const Desc &d, const RealignPass &p, uint32_t data_addr, uint32_t c_last, uint32_t end,
                                                     const PlaneSet *ps = nullptr)
@@ -441,6 +442,32 @@ __device__ __forceinline__ void realign_store_edges(const Desc &d, const Realign
     }
 }
 
+// Long rows (few per tile, down to one 32 KiB run): one thread per BYTE of the heads and tails,
+// all at once.  A single thread walking the pieces of a head and a tail at the end of the tile
+// is a latency the whole CTA waits for (a misaligned destination cost long rows 4-6 % that way).
+// Short rows have too many ends for byte stores (128 rows of 256 bytes: half the speed) and
+// keep the per-row loop of realign_store_edges.
+constexpr uint32_t kByteEdgeMinRow = 1024;
+template <int kThreads>
+__device__ __forceinline__ void realign_store_edge_bytes(const Desc &d, const RealignPass &p, uint32_t data_addr, uint32_t c_last, uint32_t end)
+{
+    const bool one_chunk = c_last == 0;
+    const uint32_t t = end & 15, units = p.units;
+    for (uint32_t item = threadIdx.x; item < p.n_rows * 32; item += kThreads) {
+        const uint32_t rr = item >> 5, k = item & 31;
+        // k < 16: byte k of the row's first chunk; else byte k - 16 of its last chunk
+        const bool is_tail = k >= 16;
+        const bool valid = is_tail ? (!one_chunk && k - 16 < t) : (k >= p.d_lo && k < min(end, 16u) && (p.d_lo || one_chunk));
+        if (!valid) continue;
+        uint32_t r;
+        char *out = realign_row<false>(d, p, nullptr, rr, r);
+        const uint32_t byte = is_tail ? 16 * c_last + (k - 16) : k;  // position in the row's chunk space
+        uint32_t v;
+        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(data_addr + 16 * rr * units + p.s_lo + byte - p.d_lo));
+        out[byte] = static_cast<char>(v);
+    }
+}
+
 template <int WS, int kThreads, bool PLANES = false>
 __device__ __forceinline__ void realign_store_all(const Desc &d, const RealignPass &p, uint32_t data, const PlaneSet *ps = nullptr)
 {
@@ -448,7 +475,10 @@ __device__ __forceinline__ void realign_store_all(const Desc &d, const RealignPa
     const uint32_t end = p.d_lo + p.len;  // first byte past the row, counted from the row's first chunk
     const uint32_t c_first = p.d_lo ? 1 : 0, c_last = end >> 4;  // whole chunks: [c_first, c_last)
     if (c_last > c_first) realign_store_full<WS, kThreads, PLANES>(d, p, data, c_first, c_last, ps);
-    if (p.d_lo || (end & 15)) realign_store_edges<WS, kThreads, PLANES>(d, p, data, c_last, end, ps);
+    if (p.d_lo || (end & 15)) {
+        if (!PLANES && p.len >= kByteEdgeMinRow) realign_store_edge_bytes<kThreads>(d, p, data, c_last, end);
+        else realign_store_edges<WS, kThreads, PLANES>(d, p, data, c_last, end, ps);
+    }
 }
 
 // Wait for the bulk copies of the current phase.  One thread waits (bounded) and tells the

@@ -191,6 +191,18 @@ def run_realign_tile(d, o, part, src, dst, cnt, smem_bytes=52 << 10, threads=256
             one_chunk, t = c_last == 0, end & 15
             if not (d_lo or t):
                 continue
+            if length >= 1024:                                # long rows: heads and tails byte by byte, a thread each
+                for rr in range(n_rows):
+                    for k in range(32):
+                        is_tail = k >= 16
+                        valid = (not one_chunk and k - 16 < t) if is_tail else (d_lo <= k < min(end, 16) and bool(d_lo or one_chunk))
+                        if not valid:
+                            continue
+                        byte = 16 * c_last + (k - 16) if is_tail else k
+                        at = data + 16 * rr * units + s_lo + byte - d_lo
+                        assert loaded[at], "a staged byte that was never loaded is consumed"
+                        dst.write(out_addr(rr, 0) + byte, stage[at:at + 1], cnt)
+                continue
             adj = 0
             if not one_chunk and t and length == run and run % 16 == 0:
                 adj = 1 if (d.n0 > 1 and d.dst_s0 == run) else (d.n0 if d.dst_s1 == run else 0)
