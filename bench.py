@@ -580,20 +580,42 @@ def run_ours(args):
                 best = min(best, a.elapsed_time(b))
             return nbytes / (best * 1e-3) / GB
 
-        def both_ways():  # both directions at once with cudaMemcpyAsync
+        dup_ev = {}
+
+        def both_ways():  # both directions at once with cudaMemcpyAsync, each timed on its own stream
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
             ev_fork.record(stream)
             stream_u.wait_event(ev_fork)
+            ev[0].record(stream)
             Qh[:n_c].copy_(Q[:n_c], non_blocking=True)
+            ev[1].record(stream)
             with torch.cuda.stream(stream_u):
+                ev[2].record(stream_u)
                 poolB[:n_c].copy_(Qh2[:n_c], non_blocking=True)
+                ev[3].record(stream_u)
                 ev_join.record(stream_u)
             stream.wait_event(ev_join)
+            dup_ev["ev"] = ev
 
         with torch.cuda.stream(stream):
             ceil_h2d = ceiling(lambda: Q[:n_c].copy_(Qh[:n_c], non_blocking=True), n_c)
             ceil_d2h = ceiling(lambda: Qh[:n_c].copy_(Q[:n_c], non_blocking=True), n_c)
             ceil_bidir = ceiling(both_ways, 2 * n_c) if can_duplex else None
         ceilings = {"h2d_cudaMemcpyAsync": ceil_h2d, "d2h_cudaMemcpyAsync": ceil_d2h, "both_directions_at_once_summed": ceil_bidir}
+        dup_h2d = dup_d2h = None
+        if can_duplex:  # the rate of each direction while the other is busy (last repetition)
+            dup_d2h = n_c / (dup_ev["ev"][0].elapsed_time(dup_ev["ev"][1]) * 1e-3) / GB
+            dup_h2d = n_c / (dup_ev["ev"][2].elapsed_time(dup_ev["ev"][3]) * 1e-3) / GB
+            ceilings.update({"h2d_while_d2h_runs": dup_h2d, "d2h_while_h2d_runs": dup_d2h})
+
+        def ideal_ms(h2d_bytes, d2h_bytes):
+            """The shortest a step can take at cudaMemcpyAsync rates on contiguous buffers: both directions
+            run together at their contended rates until the shorter one is done, the rest runs alone (a
+            step moves more bytes to the device than back: the weights only travel one way)."""
+            t_h, t_d = h2d_bytes / (dup_h2d * GB), d2h_bytes / (dup_d2h * GB)
+            if t_d <= t_h:
+                return 1e3 * (t_d + (h2d_bytes - dup_h2d * GB * t_d) / (ceil_h2d * GB))
+            return 1e3 * (t_h + (d2h_bytes - dup_d2h * GB * t_h) / (ceil_d2h * GB))
 
         def run_e2e(hp, duplex, steps, warmup):
             """Offload every wave to pinned host memory and reload it into the second pool; load the
@@ -652,6 +674,7 @@ def run_ours(args):
                     "host_link_GBps": link, "host_link_ceiling_GBps": ceilings,
                     "host_link_frac_of_ceiling": link / world / (ceil_bidir if duplex else serial_ceiling),
                     "ceiling_used": "both_directions_at_once_summed" if duplex else "serial mix of the one-direction ceilings",
+                    "frac_of_ideal_schedule": (ideal_ms(h2d, d2h) / (e_ms / steps)) if duplex else None,
                     "kv_host_path": hp["path"], "schedule": "duplex" if duplex else "serial", "gpu_launches_per_step": hp["launches"]}
 
         want_duplex = args.e2e_schedule == "duplex" and can_duplex
