@@ -178,6 +178,14 @@ enum {
                                tc_plan_stats can report the device time of the last one (the
                                call context's tracing hook, Sec. 3.2).  Two event records per
                                call; executions of one traced plan should not overlap */
+    TC_PLAN_DEBUG_BOUNDS = 128u, /* debugging aid (the pool's memory checker tools are not always at hand):
+                               the plan also keeps, on the device, the byte extent of every table
+                               slot as the spec declares it.  Before every execution a small
+                               kernel holds the descriptors AS UPLOADED against those extents; an
+                               access outside sets TC_DEVICE_OUT_OF_BOUNDS in the device status
+                               word and the copy kernel that follows returns without touching
+                               memory (it never traps).  tc_plan_check_device runs the checker
+                               alone.  Not for staged or streamed plans */
     TC_PLAN_STREAM = 16u    /* TC_WEIGHTS: the blob is streamed chunk by chunk, from a file
                                (tc_weights_materialize_file) or from pinned host memory
                                (tc_weights_materialize), through the staging ring.  Unlike
@@ -505,7 +513,18 @@ TC_API int tc_trim(void);
  * flags: host pointer.  The call copies the word back and therefore waits for the device's
  * previously enqueued work (it is a diagnostic, off the data path). */
 #define TC_DEVICE_BULK_WAIT_TIMEOUT 1u
+#define TC_DEVICE_OUT_OF_BOUNDS 2u /* the bounds checker of a TC_PLAN_DEBUG_BOUNDS plan found a descriptor that
+                                      reaches outside its table slot; copy kernels of such plans return
+                                      without copying while the flag is set (read it to clear it) */
 TC_API int tc_device_status(uint32_t *flags);
+
+/* Run only the device-side bounds checker of a TC_PLAN_DEBUG_BOUNDS plan on `stream`: every
+ * descriptor of both groups, as it sits in device memory, against the declared extent of its
+ * table slots less `shrink` bytes.  shrink = 0 is the real check (a plan that tc_plan_create
+ * accepted passes it); a positive shrink pretends every slot is that much smaller and shows the
+ * checker firing (tests use it: a plan that uses its slots to the last byte must then raise
+ * TC_DEVICE_OUT_OF_BOUNDS).  Nothing is copied.  The verdict arrives through tc_device_status. */
+TC_API int tc_plan_check_device(const tc_plan_t *plan, int64_t shrink, void *stream);
 
 /* Self-test of that bounded wait: launches one small kernel on `stream` that waits on a barrier
  * nothing will ever arrive at.  The wait gives up after a few milliseconds, the kernel sets

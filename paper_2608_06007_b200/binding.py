@@ -28,8 +28,10 @@ TC_PLAN_SAME_POOL = 8
 TC_PLAN_STREAM = 16
 TC_PLAN_OFFLOAD_ZERO_COPY = 32
 TC_PLAN_TRACE = 64
+TC_PLAN_DEBUG_BOUNDS = 128
 TC_MAX_TABLE_SLOTS = 4000
 TC_DEVICE_BULK_WAIT_TIMEOUT = 1
+TC_DEVICE_OUT_OF_BOUNDS = 2
 
 
 class tc_kv_pool_t(C.Structure):
@@ -103,7 +105,7 @@ class tc_segment_t(C.Structure):
 EXPORTS = ("tc_plan_create", "tc_kv_pack", "tc_kv_unpack", "tc_weights_materialize",
            "tc_plan_destroy", "tc_plan_stats", "tc_plan_descriptors", "tc_strerror", "tc_last_error",
            "tc_kv_pack_noalloc", "tc_weights_materialize_checksum", "tc_trim",
-           "tc_weights_materialize_file", "tc_plan_segments", "tc_device_status", "tc_selftest_wait_timeout")
+           "tc_weights_materialize_file", "tc_plan_segments", "tc_device_status", "tc_selftest_wait_timeout", "tc_plan_check_device")
 
 _lib = None
 
@@ -135,6 +137,8 @@ def load_library(path: str | None = None):
     lib.tc_plan_segments.restype = C.c_int
     lib.tc_device_status.argtypes = [C.POINTER(C.c_uint32)]
     lib.tc_device_status.restype = C.c_int
+    lib.tc_plan_check_device.argtypes = [vp, C.c_int64, vp]
+    lib.tc_plan_check_device.restype = C.c_int
     lib.tc_selftest_wait_timeout.argtypes = [vp]
     lib.tc_selftest_wait_timeout.restype = C.c_int
     lib.tc_trim.argtypes = []
@@ -375,6 +379,12 @@ def tc_device_status() -> int:
     v = C.c_uint32()
     _check(load_library().tc_device_status(C.byref(v)))
     return int(v.value)
+
+
+def tc_plan_check_device(plan: Plan, shrink: int = 0, stream=None) -> None:
+    """Run the device-side bounds checker of a TC_PLAN_DEBUG_BOUNDS plan (slot extents less
+    `shrink` bytes); the verdict arrives through tc_device_status()."""
+    _check(load_library().tc_plan_check_device(plan.handle, int(shrink), _stream(stream)))
 
 
 def tc_selftest_wait_timeout(stream=None) -> None:

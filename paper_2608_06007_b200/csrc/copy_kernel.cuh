@@ -46,6 +46,7 @@ struct Params {
     uint32_t tile_base;         // first global tile id of this launch (tile-range segments)
     uint32_t stage_bytes;       // dynamic shared memory of the launch (realigning path)
     uint32_t stage_always;      // take the shared-memory path for aligned tiles too (tuning.copy_path)
+    uint32_t debug_bounds;      // the plan's bounds checker ran just before: copy nothing if it raised its flag
     unsigned long long *sums;   // checksum accumulators (checked builds only)
     char *ptr[NPTR];            // src table then dst table
 };
@@ -232,7 +233,7 @@ __device__ __forceinline__ uint4 shift_words(uint4 a, uint4 b, uint32_t bits)
 }
 
 // Sticky error flags set by kernels (read and cleared by tc_device_status).
-enum : unsigned int { kStatusBulkWaitTimeout = 1u };
+enum : unsigned int { kStatusBulkWaitTimeout = 1u, kStatusOutOfBounds = 2u };
 __device__ unsigned int g_device_status = 0;
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
@@ -804,6 +805,34 @@ __device__ __noinline__ void copy_multi_narrow(const Desc &d, const Params<NPTR>
     }
 }
 
+// Debugging aid (TC_PLAN_DEBUG_BOUNDS): one thread per (descriptor, outer index) works out the
+// first and last byte the descriptor touches on each side and holds them against the declared
+// extent of the table slot (less `shrink`, for the self-test).  A violation sets a flag; nothing
+// traps, nothing is dereferenced.
+__global__ void tc_bounds_check_kernel(const Desc *descs, uint32_t n_descs, const long long *extents, long long shrink)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_descs) return;
+    const Desc d = descs[i];
+    bool bad = d.n0 == 0 || d.rows == 0 || d.run == 0;
+    if (!bad) {
+        // strides are unsigned: the farthest row is the last one, or the last of the row before
+        const uint32_t last = d.rows - 1, i1 = last / d.n0, i0 = last - i1 * d.n0;
+        long long s_far = static_cast<long long>(i1) * d.src_s1 + static_cast<long long>(i0) * d.src_s0;
+        long long d_far = static_cast<long long>(i1) * d.dst_s1 + static_cast<long long>(i0) * d.dst_s0;
+        if (i1) {
+            s_far = max(s_far, static_cast<long long>(i1 - 1) * d.src_s1 + static_cast<long long>(d.n0 - 1) * d.src_s0);
+            d_far = max(d_far, static_cast<long long>(i1 - 1) * d.dst_s1 + static_cast<long long>(d.n0 - 1) * d.dst_s0);
+        }
+        for (uint32_t o = 0; o < d.n_outer && !bad; o++) {
+            const long long s_lo = d.src_off + static_cast<long long>(o) * d.src_outer, d_lo = d.dst_off + static_cast<long long>(o) * d.dst_outer;
+            const long long s_ext = extents[d.src_slot + o * d.src_slot_step] - shrink, d_ext = extents[d.dst_slot + o * d.dst_slot_step] - shrink;
+            bad = s_lo < 0 || d_lo < 0 || s_lo + s_far + d.run > s_ext || d_lo + d_far + d.run > d_ext;
+        }
+    }
+    if (bad) atomicOr(&g_device_status, kStatusOutOfBounds);
+}
+
 // MULTI: 0 one plane per tile; 1 several planes per tile, planes a byte stride apart; 2 the
 // same with a pool that has one pointer per plane.
 template <int NPTR, int MODE, bool CHECK = false, int MULTI = 0>
@@ -824,6 +853,8 @@ __global__ void __launch_bounds__(Shape<MODE>::threads, Shape<MODE>::min_ctas) t
         }
         // made visible to the CTA by the __syncthreads that follows the descriptor fetch below
     }
+    // a debug-checked plan whose checker has raised its flag copies nothing
+    if (prm.debug_bounds && (*static_cast<volatile unsigned int *>(&g_device_status) & kStatusOutOfBounds)) return;
     int buf = 0;
     for (uint32_t tile = blockIdx.x + prm.tile_base; tile < prm.n_tiles; tile += gridDim.x, buf ^= 1) {
         // tile id -> descriptor, plane o, part.  For uniform and windowed launches this needs

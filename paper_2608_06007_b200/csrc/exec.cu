@@ -85,7 +85,7 @@ static void free_plan_storage(tc_plan *plan)
         }
     block_free(plan->device, plan->d_storage, plan->d_storage_bytes);
     plan->d_storage = nullptr;
-    for (int k = 0; k < 2; k++) plan->group[k].d_descs = nullptr, plan->group[k].d_tile_desc = nullptr;
+    for (int k = 0; k < 2; k++) plan->group[k].d_descs = nullptr, plan->group[k].d_tile_desc = nullptr, plan->group[k].d_extents = nullptr;
 }
 
 // One allocation and one copy per plan: [g0 descriptors | g0 tiles | g1 descriptors | g1 tiles],
@@ -93,12 +93,14 @@ static void free_plan_storage(tc_plan *plan)
 static int upload_plan(tc_plan *plan)
 {
     auto pad = [](size_t n) { return (n + 255) & ~size_t(255); };
-    size_t off[4], total = 0;
+    size_t off[4], ext_off[2], total = 0;
     for (int k = 0; k < 2; k++) {
         off[2 * k] = total;
         total += pad(plan->group[k].descs.size() * sizeof(Desc));
         off[2 * k + 1] = total;
         total += pad(plan->group[k].tile_desc.size() * sizeof(uint32_t));
+        ext_off[k] = total;
+        total += pad(plan->group[k].extents.size() * sizeof(int64_t));
     }
     if (total == 0) return TC_OK;
     std::vector<unsigned char> image(total);
@@ -106,6 +108,7 @@ static int upload_plan(tc_plan *plan)
         const Group &g = plan->group[k];
         if (!g.descs.empty()) memcpy(image.data() + off[2 * k], g.descs.data(), g.descs.size() * sizeof(Desc));
         if (!g.tile_desc.empty()) memcpy(image.data() + off[2 * k + 1], g.tile_desc.data(), g.tile_desc.size() * sizeof(uint32_t));
+        if (!g.extents.empty()) memcpy(image.data() + ext_off[k], g.extents.data(), g.extents.size() * sizeof(int64_t));
     }
     cudaError_t e = block_alloc(plan->device, total, &plan->d_storage, &plan->d_storage_bytes);
     if (e != cudaSuccess) {
@@ -119,6 +122,7 @@ static int upload_plan(tc_plan *plan)
         Group &g = plan->group[k];
         if (!g.descs.empty()) g.d_descs = reinterpret_cast<Desc *>(base + off[2 * k]);
         if (!g.tile_desc.empty()) g.d_tile_desc = reinterpret_cast<uint32_t *>(base + off[2 * k + 1]);
+        if (!g.extents.empty()) g.d_extents = reinterpret_cast<int64_t *>(base + ext_off[k]);
     }
     return TC_OK;
 }
@@ -182,6 +186,7 @@ int execute(const tc_plan *plan, int gi, const void *const *src, size_t n_src, v
         cudaError_t e = cudaEventRecord(static_cast<cudaEvent_t>(plan->trace_ev[gi][0]), s);
         if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord(trace)");
     }
+    if (g.d_extents && (rc = launch_bounds_check(g, 0, s)) != TC_OK) return rc;  // TC_PLAN_DEBUG_BOUNDS
     if (file) rc = execute_streamed(plan, g, file->fd, file->offset, dst, ptr_align, s, sums);
     else if (!g.segments.empty()) rc = execute_staged(plan, g, src, dst, ptr_align, s, sums);
     else rc = launch_any(plan, g, src, dst, ptr_align, s, nullptr, sums, host_memory);
@@ -330,6 +335,25 @@ extern "C" int tc_device_status(uint32_t *flags)
     const int rc = read_device_status(&v);
     *flags = v;
     return rc;
+}
+
+extern "C" int tc_plan_check_device(const tc_plan_t *plan, int64_t shrink, void *stream)
+{
+    clear_error();
+    if (!plan) return fail(TC_ERR_INVALID_ARG, "plan is NULL");
+    if (!(plan->flags & TC_PLAN_DEBUG_BOUNDS) || (plan->flags & TC_PLAN_HOST_ONLY))
+        return fail(TC_ERR_KIND, "tc_plan_check_device needs an executable plan created with TC_PLAN_DEBUG_BOUNDS");
+    if (shrink < 0) return fail(TC_ERR_INVALID_ARG, "shrink %lld < 0", (long long)shrink);
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess || current != plan->device)
+        return fail(TC_ERR_INVALID_ARG, "the plan lives on device %d but device %d is current", plan->device, current);
+    for (int k = 0; k < 2; k++) {
+        const Group &g = plan->group[k];
+        if (g.descs.empty()) continue;
+        const int rc = launch_bounds_check(g, shrink, static_cast<cudaStream_t>(stream));
+        if (rc != TC_OK) return rc;
+    }
+    return TC_OK;
 }
 
 extern "C" int tc_selftest_wait_timeout(void *stream)

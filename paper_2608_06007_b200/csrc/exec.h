@@ -38,6 +38,10 @@ int launch_any(const tc_plan *plan, const Group &g, const void *const *src, void
 // The current device's sticky status word (flags set by kernels); reading clears it.
 int read_device_status(unsigned int *out);
 
+// TC_PLAN_DEBUG_BOUNDS: check group g's uploaded descriptors against its slot extents less
+// `shrink` bytes; a violation sets the out-of-bounds flag of the device status word.
+int launch_bounds_check(const Group &g, int64_t shrink, cudaStream_t s);
+
 // Launch the self-test of the bounded wait (see tc_selftest_wait_timeout).
 int launch_wait_timeout_probe(cudaStream_t s);
 

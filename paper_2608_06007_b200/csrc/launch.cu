@@ -120,6 +120,7 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     prm.log2_ptr_align = ptr_align;
     prm.stage_bytes = 0;
     prm.stage_always = plan->tuning.copy_path == 1;
+    prm.debug_bounds = g.d_extents != nullptr;
     prm.sums = sums;
     for (size_t i = 0; i < g.n_src; i++) prm.ptr[i] = const_cast<char *>(static_cast<const char *>(src[i]));
     for (size_t i = 0; i < g.n_dst; i++) prm.ptr[g.n_src + i] = static_cast<char *>(dst[i]);
@@ -179,6 +180,15 @@ int read_device_status(unsigned int *out)
     cudaError_t e = cudaMemcpyFromSymbol(out, g_device_status, sizeof *out);
     if (e == cudaSuccess && *out) e = cudaMemcpyToSymbol(g_device_status, &zero, sizeof zero);
     return e == cudaSuccess ? TC_OK : cuda_fail(e, "reading the device status word");
+}
+
+int launch_bounds_check(const Group &g, int64_t shrink, cudaStream_t s)
+{
+    const uint32_t n = static_cast<uint32_t>(g.descs.size());
+    if (n == 0 || !g.d_extents) return TC_OK;
+    tc_bounds_check_kernel<<<(n + 255) / 256, 256, 0, s>>>(g.d_descs, n, reinterpret_cast<const long long *>(g.d_extents), shrink);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? TC_OK : cuda_fail(e, "kernel launch");
 }
 
 int launch_wait_timeout_probe(cudaStream_t s)

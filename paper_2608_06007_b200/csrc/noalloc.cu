@@ -54,6 +54,7 @@ extern "C" int tc_kv_pack_noalloc(const tc_plan_spec_t *spec, const void *const 
     if (spec->deadline_ns && now_ns() > spec->deadline_ns) return fail(TC_ERR_DEADLINE, "deadline passed before the call");
     if (spec->flags & TC_PLAN_STAGED) return fail(TC_ERR_INVALID_ARG, "tc_kv_pack_noalloc does not stage: the staging ring is allocated device memory");
     if (spec->flags & TC_PLAN_HOST_ONLY) return fail(TC_ERR_INVALID_ARG, "TC_PLAN_HOST_ONLY asks for a plan that is not executed; tc_kv_pack_noalloc always executes");
+    if (spec->flags & TC_PLAN_DEBUG_BOUNDS) return fail(TC_ERR_INVALID_ARG, "TC_PLAN_DEBUG_BOUNDS keeps slot extents in allocated device memory; tc_kv_pack_noalloc allocates none");
     tc_plan plan;  // lives on the host for the duration of this call only
     plan.kind = spec->kind;
     plan.flags = spec->flags;

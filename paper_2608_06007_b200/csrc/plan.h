@@ -79,6 +79,7 @@ struct Group {
     std::vector<RequestSpan> requests; // KV groups with a packed side
     std::vector<Segment> segments;    // staged plans only
     std::vector<StageCopy> copies;    // staged plans only
+    std::vector<int64_t> extents;     // TC_PLAN_DEBUG_BOUNDS: byte extent of every table slot (src slots, then dst slots)
     bool stage_whole_host_pool = false; // staged MIXED group: the host side is a paged pool
     bool host_is_src = false;          // staged groups: direction (host -> device when true)
     uint32_t tiles_per_desc = 0;      // > 0: every descriptor owns exactly this many tile ids
@@ -97,6 +98,7 @@ struct Group {
     // device copies (null for host-only plans and empty groups)
     Desc *d_descs = nullptr;
     uint32_t *d_tile_desc = nullptr;
+    int64_t *d_extents = nullptr;
 };
 
 }  // namespace tc

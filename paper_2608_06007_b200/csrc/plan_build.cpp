@@ -658,6 +658,22 @@ static int build_kv(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t tile_byt
         g1.n_src = kv.dst_pool.n_slots;
         g1.n_dst = kv.src_pool.n_slots;
     }
+    if (spec->flags & TC_PLAN_DEBUG_BOUNDS) {
+        // what every table slot is declared to hold: the device-side checker holds the uploaded
+        // descriptors against these numbers
+        auto pool_extent = [](const tc_kv_pool_t &p, const PoolView &v) { return p.slot_bytes ? p.slot_bytes : v.slot_need; };
+        const int64_t packed = kv.packed_bytes ? kv.packed_bytes : plan->packed_required;
+        auto fill = [&](Group &g, bool src_pool_side, bool dst_pool_side, const tc_kv_pool_t &spool, const PoolView &sv, const tc_kv_pool_t &dpool, const PoolView &dv) {
+            g.extents.assign(g.n_src, src_pool_side ? pool_extent(spool, sv) : packed);
+            g.extents.insert(g.extents.end(), g.n_dst, dst_pool_side ? pool_extent(dpool, dv) : packed);
+        };
+        if (kind == TC_KV_PACK) fill(g0, true, false, kv.src_pool, sp, kv.dst_pool, dp);
+        else if (kind == TC_KV_UNPACK) fill(g1, false, true, kv.src_pool, sp, kv.dst_pool, dp);
+        else {
+            fill(g0, true, true, kv.src_pool, sp, kv.dst_pool, dp);
+            if (kind == TC_KV_MIXED) fill(g1, true, true, kv.dst_pool, dp, kv.src_pool, sp);
+        }
+    }
     return TC_OK;
 }
 
@@ -796,6 +812,13 @@ static int build_weights(const tc_plan_spec_t *spec, tc_plan *plan, uint32_t til
     }
     for (const Box &b : boxes) lower_box(g, b, tile_bytes);
     g.host_is_src = true;
+    if (spec->flags & TC_PLAN_DEBUG_BOUNDS) {
+        g.extents.assign(1, w.blob_bytes);
+        g.extents.resize(1 + static_cast<size_t>(n_dst), 0);
+        for (size_t slot = 0; slot < spans.size(); slot++)
+            for (const Span &sp_ : spans[slot])
+                g.extents[1 + slot] = w.dst_bytes ? w.dst_bytes[slot] : std::max(g.extents[1 + slot], sp_.hi);
+    }
     if (spec->flags & TC_PLAN_CHECKSUM) {
         // checksums are sums over aligned 4-byte words of each tensor: every run must be made of
         // whole words and every access must be 16-byte aligned
@@ -921,6 +944,8 @@ int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
     plan->group[1].host_is_src = true;  // UNPACK / reload read the host side
     if ((spec->flags & TC_PLAN_OFFLOAD_ZERO_COPY) && (spec->kind != TC_KV_MIXED || !(spec->flags & TC_PLAN_STAGED)))
         return fail(TC_ERR_KIND, "TC_PLAN_OFFLOAD_ZERO_COPY applies to staged TC_KV_MIXED plans only");
+    if ((spec->flags & TC_PLAN_DEBUG_BOUNDS) && (spec->flags & (TC_PLAN_STAGED | TC_PLAN_STREAM)))
+        return fail(TC_ERR_INVALID_ARG, "TC_PLAN_DEBUG_BOUNDS checks plans that run directly, not staged or streamed ones");
     if ((spec->flags & TC_PLAN_STREAM) && spec->kind != TC_WEIGHTS)
         return fail(TC_ERR_KIND, "TC_PLAN_STREAM applies to TC_WEIGHTS plans only");
     if (spec->flags & (TC_PLAN_STAGED | TC_PLAN_STREAM)) {

@@ -707,6 +707,67 @@ def test_a_wait_that_cannot_complete_ends_with_a_status_word_not_a_hang():
     assert int(x.sum().item()) == 1023 * 512                # the context is alive and well
 
 
+def test_debug_plans_check_their_descriptors_on_the_device_and_skip_the_copy_when_out_of_bounds():
+    """TC_PLAN_DEBUG_BOUNDS: a small kernel holds the uploaded descriptors against the slot extents
+    before each execution.  A valid plan passes (and copies the right bytes); with every slot
+    pretended one byte smaller a plan that fills its packed buffer to the last byte must raise
+    TC_DEVICE_OUT_OF_BOUNDS, and while the flag stands the copy kernel copies nothing.  Nothing
+    traps and the context stays usable."""
+    rng = np.random.default_rng(31)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=40, B=16, H=8, D=64, E=2, T=(100, 16, 7, 333))
+    L = shape[0]
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride, slot_bytes=pool.size)
+    d_pool = dev(pool)
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, L * 2), T, off, bt, oracle.HND, want)
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_src=bt,
+                                        packed_bytes=want.size, flags=tc.TC_PLAN_DEBUG_BOUNDS))
+    assert tc.tc_device_status() == 0
+    packed = Guarded(want.size)
+    tc.tc_kv_pack(plan, [d_pool], [packed.ptr()])
+    assert np.array_equal(packed.result(), want)
+    assert tc.tc_device_status() == 0
+    tc.tc_plan_check_device(plan, 0)
+    torch.cuda.synchronize()
+    assert tc.tc_device_status() == 0
+    tc.tc_plan_check_device(plan, 1)                          # every slot one byte smaller
+    untouched = Guarded(want.size, fill=0xEE)
+    tc.tc_kv_pack(plan, [d_pool], [untouched.ptr()])          # the flag stands: nothing is copied
+    assert (untouched.result() == 0xEE).all()
+    assert tc.tc_device_status() == tc.TC_DEVICE_OUT_OF_BOUNDS
+    assert tc.tc_device_status() == 0                         # reading cleared it
+    tc.tc_kv_pack(plan, [d_pool], [untouched.ptr()])
+    assert np.array_equal(untouched.result(), want)
+    # unpack (group 1), migrate and weights plans pass their own check too
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    for spec in (tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_dst=bt2, flags=tc.TC_PLAN_DEBUG_BOUNDS),
+                 tc.kv_spec(tc.TC_KV_MIGRATE, shape, src_pool=pl, dst_pool=pl, T=T, bt_off=off, bt_src=bt, bt_dst=bt2, flags=tc.TC_PLAN_DEBUG_BOUNDS)):
+        p2 = tc.tc_plan_create(spec)
+        tc.tc_plan_check_device(p2, 0)
+        assert tc.tc_device_status() == 0
+        tc.tc_plan_check_device(p2, pool.size)                # no slot left at all
+        assert tc.tc_device_status() == tc.TC_DEVICE_OUT_OF_BOUNDS
+    ck = small_checkpoint()
+    blob = np.zeros(ck.nbytes_total, dtype=np.uint8)
+    wl.fill_np(blob, 5, "normal")
+    sizes = [ck.nbytes(i) // (4 if ck.split_dim[i] >= 0 else 1) for i in range(ck.N)]
+    want_w = [np.zeros(n, dtype=np.uint8) for n in sizes]
+    oracle.weights(ck.byte_off, ck.E, ck.shapes, ck.split_dim, 2, 4, blob, want_w)
+    outs = [Guarded(n, fill=0xEE) for n in sizes]
+    wplan = tc.tc_plan_create(ck_spec(ck, split_dim=ck.split_dim, rank=2, world=4, flags=tc.TC_PLAN_DEBUG_BOUNDS))
+    tc.tc_weights_materialize(wplan, dev(blob), [o.ptr() for o in outs])
+    for i in range(ck.N):
+        assert np.array_equal(outs[i].result(), want_w[i]), ck.names[i]
+    assert tc.tc_device_status() == 0
+    tc.tc_plan_check_device(wplan, 1)
+    assert tc.tc_device_status() == tc.TC_DEVICE_OUT_OF_BOUNDS
+    with pytest.raises(tc.TensorCastError) as e:              # only plans made for it carry the extents
+        tc.tc_plan_check_device(tc.tc_plan_create(ck_spec(ck)), 0)
+    assert e.value.status == tc.TC_ERR_KIND
+    x = torch.arange(1024, device="cuda")
+    assert int(x.sum().item()) == 1023 * 512
+
+
 def test_traced_plan_reports_the_device_time_of_its_last_execution():
     shape = wl.KVShape(L=4, B=16, H=8, D=128, E=2)
     NB = 512

@@ -507,6 +507,21 @@ def test_stream_flag_limits():
     assert e.value.status == tc.TC_ERR_KIND
 
 
+def test_debug_bounds_flag_limits():
+    shape = (1, 4, 2, 8, 2)
+    pl = tc.pool(tc.TC_NHD, 4, 1, plane_stride=4 * 4 * 2 * 8 * 2)
+    kw = dict(src_pool=pl, bt_src=np.arange(2, dtype=np.int32), T=np.array([8]), bt_off=np.array([0, 2]))
+    plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, flags=HOST | tc.TC_PLAN_DEBUG_BOUNDS, **kw))
+    plain = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, flags=HOST, **kw))
+    assert plan.stats().n_tiles[:] == plain.stats().n_tiles[:]  # the flag changes nothing in the lowering
+    with pytest.raises(tc.TensorCastError) as e:              # a host-only plan has nothing on a device to check
+        tc.tc_plan_check_device(plan, 0)
+    assert e.value.status == tc.TC_ERR_KIND
+    with pytest.raises(tc.TensorCastError) as e:
+        tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, flags=HOST | tc.TC_PLAN_DEBUG_BOUNDS | tc.TC_PLAN_STAGED, **kw))
+    assert e.value.status == tc.TC_ERR_INVALID_ARG and "DEBUG_BOUNDS" in str(e.value)
+
+
 @pytest.mark.parametrize("pool_l,packed_l", list(itertools.product(LAYOUTS, LAYOUTS)))
 @pytest.mark.parametrize("order", [tc.TC_REQUEST_MAJOR, tc.TC_LAYER_MAJOR])
 def test_head_slice_and_layer_major_lowering_match_oracle(pool_l, packed_l, order):
