@@ -586,6 +586,131 @@ __device__ __noinline__ bool realign_pass_mixed(const Desc &d, const char *src, 
     return true;
 }
 
+// Rows that are ADJACENT IN THE DESTINATION (tokens of one head in a head-major buffer, heads of
+// one token in a token-major block, the rows of a dim-1 weight slice) are staged in destination
+// order, back to back, so that a group of them is one long row for the store loop: one row
+// decode per group, heads and tails only at the ends of a group.  With a misaligned source a row
+// occupies [s_lo, s_lo + run) of its run + 16 covering bytes, and the next row's data begins in
+// the chunk that holds this row's last s_lo bytes: the whole chunks of a row arrive by bulk copy,
+// the chunk two rows share is put together by one thread from the two aligned source chunks.
+// Geometry of the tile in the descriptor's row order k -> (i1, i0) = (k / n0, k % n0):
+//   across  rows a step of n0 apart are adjacent (dst_s1 == run): the tile must hold whole
+//           i1-columns, group g = i0, position i1; the groups are dst_s0 apart, and when that
+//           equals a group's length the whole tile is one group;
+//   along   rows one apart are adjacent (dst_s0 == run), the tile lies inside one i1 or the i1
+//           are adjacent too: one group, position = row.
+// Rows of at least kJoinMinRun bytes in groups of at least kThreads chunks only.  Short rows (the
+// 256-byte head rows of a KV block) measured slower this way than in their own slots (pack / unpack
+// with the source misaligned 5.9 / 5.6 against 6.3 / 6.4 TB/s: one more bulk copy and one merge
+// per row, and a store loop entered once per group, cost more instructions than the per-row
+// loop's heads and tails); rows of 1 KiB and more gain 3-4 % with a misaligned destination.
+// Returns 1 done, 0 not this geometry (nothing touched), -1 the bulk copies did not arrive.
+template <int WS, int kThreads>
+__device__ __forceinline__ void realign_store_joined(char *dst0, uint32_t vstride, uint32_t groups, uint32_t units, uint32_t len, uint32_t s_lo, uint32_t d_lo,
+                                                     uint32_t data_addr)
+{
+    const uint32_t end = d_lo + len, c_first = d_lo ? 1 : 0, c_last = end >> 4, t = end & 15;
+    const int delta = static_cast<int>(s_lo) - static_cast<int>(d_lo);
+    const uint32_t bits = (static_cast<uint32_t>(delta) & 3) * 8;
+    const uint32_t shifted = data_addr + 16 * (delta >> 4);
+    for (uint32_t g = 0; g < groups; g++) {
+        uint32_t c = threadIdx.x < c_first ? threadIdx.x + kThreads : threadIdx.x;
+        uint32_t at = shifted + 16 * (g * units + c);
+        char *out = dst0 + static_cast<size_t>(g) * vstride + 16 * static_cast<size_t>(c);
+#pragma unroll 2
+        for (; c < c_last; c += kThreads, at += 16 * kThreads, out += 16 * kThreads)
+            st_stream<uint4>(out, shift_words<WS>(lds128(at), lds128(at + 16), bits));
+    }
+    if (d_lo || t) {  // one thread per byte of the groups' heads and tails
+        for (uint32_t item = threadIdx.x; item < groups * 32; item += kThreads) {
+            const uint32_t g = item >> 5, k = item & 31;
+            const bool is_tail = k >= 16;
+            if (is_tail ? k - 16 >= t : (k < d_lo || !d_lo)) continue;
+            const uint32_t byte = is_tail ? 16 * c_last + (k - 16) : k;
+            uint32_t v;
+            asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(data_addr + 16 * g * units + s_lo + byte - d_lo));
+            dst0[static_cast<size_t>(g) * vstride + byte] = static_cast<char>(v);
+        }
+    }
+}
+
+template <int kThreads>
+__device__ __forceinline__ int realign_tile_joined(const Desc &d, const char *src, char *dst, uint32_t row0, uint32_t nrows, uint32_t data_addr, uint32_t stage_bytes,
+                                                   uint32_t bar, uint32_t &phase, uint32_t *wait_ok)
+{
+    const uint32_t run = d.run, n0 = d.n0;
+    if ((run & 15) || run < kJoinMinRun || run > kRealignColumn || nrows < 2) return 0;
+    const uint32_t j1 = fastdiv(row0, d.div_n0), j0 = row0 - j1 * n0;  // the tile's first row
+    bool across = false;
+    uint32_t groups = 1, glen = nrows, vstride = 0, cols = 0;  // cols: i1-columns of the tile
+    if (d.dst_s1 == run) {
+        cols = fastdiv(nrows, d.div_n0);
+        if (j0 || cols * n0 != nrows) return 0;
+        across = true;
+        if (n0 > 1 && d.dst_s0 != cols * run) groups = n0, glen = cols, vstride = d.dst_s0;
+    } else if (n0 > 1 && d.dst_s0 == run) {
+        if (j0 + nrows > n0 && d.dst_s1 != n0 * run) return 0;
+    } else {
+        return 0;
+    }
+    const uint32_t len = glen * run, units = (len + 30) >> 4;
+    const uint32_t side = data_addr + groups * (units << 4) + 16;  // 16 bytes per row: the chunk that holds its last bytes
+    if (glen < 2 || units < kThreads || groups * (units << 4) + 48 + 16 * (nrows + 1) > stage_bytes) return 0;
+    const char *s0 = src + (j1 * d.src_s1 + j0 * d.src_s0);
+    char *d0 = dst + (j1 * d.dst_s1 + j0 * d.dst_s0);
+    const uint32_t s_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(s0)) & 15;
+    const uint32_t d_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(d0)) & 15;
+    if (threadIdx.x == 0) mbar_expect_tx(bar, nrows * (s_lo ? run + 16 : run));
+    // row rr of the tile -> group g, position pos in it, place q among all staged rows
+    auto place = [&](uint32_t rr, uint32_t &i1, uint32_t &i0, uint32_t &g, uint32_t &pos) {
+        const uint32_t r = row0 + rr;
+        i1 = fastdiv(r, d.div_n0);
+        i0 = r - i1 * n0;
+        g = 0;
+        pos = rr;
+        if (across) {
+            if (groups > 1) g = i0, pos = i1 - j1;
+            else pos = i0 * cols + (i1 - j1);
+        }
+    };
+    for (uint32_t rr = threadIdx.x; rr < nrows; rr += kThreads) {
+        uint32_t i1, i0, g, pos;
+        place(rr, i1, i0, g, pos);
+        const char *row = src + (i1 * d.src_s1 + i0 * d.src_s0) - s_lo;  // its first aligned chunk
+        const uint32_t at = data_addr + 16 * g * units + pos * run;
+        if (!s_lo || pos + 1 == glen) {
+            bulk_load(at, row, s_lo ? run + 16 : run, bar);
+        } else {
+            // the chunk with the row's last s_lo bytes would land on the next row's first chunk
+            bulk_load(at, row, run, bar);
+            bulk_load(side + 16 * (g * glen + pos + 1), row + run, 16, bar);
+        }
+    }
+    if (!realign_wait(bar, phase, wait_ok)) return -1;
+    if (s_lo) {
+        for (uint32_t rr = threadIdx.x; rr < nrows; rr += kThreads) {
+            uint32_t i1, i0, g, pos;
+            place(rr, i1, i0, g, pos);
+            if (pos == 0) continue;
+            const uint32_t at = data_addr + 16 * g * units + pos * run;
+            const uint4 v = merge_bytes(lds128(side + 16 * (g * glen + pos)), lds128(at), s_lo);
+            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(at), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+        }
+        __syncthreads();
+    }
+    char *out0 = d0 - d_lo;
+    switch (((s_lo - d_lo) & 15) >> 2) {
+    case 0: realign_store_joined<0, kThreads>(out0, vstride, groups, units, len, s_lo, d_lo, data_addr); break;
+    case 1: realign_store_joined<1, kThreads>(out0, vstride, groups, units, len, s_lo, d_lo, data_addr); break;
+    case 2: realign_store_joined<2, kThreads>(out0, vstride, groups, units, len, s_lo, d_lo, data_addr); break;
+    default: realign_store_joined<3, kThreads>(out0, vstride, groups, units, len, s_lo, d_lo, data_addr); break;
+    }
+    // the next tile's bulk copies overwrite chunks this one wrote with ordinary stores
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+    return 1;
+}
+
 // Rows [row0, row0 + nrows) of one outer index of descriptor d, any alignment; src / dst point
 // at row 0.  `stage` is the shared-memory staging area (16-byte aligned, stage_bytes long, of
 // which the first and last 16 are padding that neighbouring-chunk loads may touch): a pass
@@ -604,6 +729,10 @@ __device__ __forceinline__ bool copy_rows_realign(const Desc &d, const char *src
     char *data = stage + 16;
     const uint32_t data_addr = static_cast<uint32_t>(__cvta_generic_to_shared(data));
     const bool same_alignment = ((d.src_s0 | d.src_s1 | d.dst_s0 | d.dst_s1) & 15) == 0;
+    if (same_alignment) {
+        const int joined = realign_tile_joined<kThreads>(d, src, dst, row0, nrows, data_addr, stage_bytes, bar, phase, wait_ok);
+        if (joined) return joined > 0;
+    }
     for (uint32_t col0 = 0; col0 < run; col0 += column) {
         const uint32_t len = min(column, run - col0);
         for (uint32_t r0 = 0; r0 < nrows; r0 += rows_per_pass) {

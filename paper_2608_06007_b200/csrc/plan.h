@@ -142,5 +142,6 @@ constexpr uint32_t kMaxTileBytes = 1u << 20;
 constexpr uint32_t kRealignSmem = 52u << 10;
 constexpr uint32_t kRealignColumn = kRealignSmem - 64;
 constexpr uint32_t kRealignMinRun = 32;  // shorter rows take the narrow-vector loop instead
+constexpr uint32_t kJoinMinRun = 1024;   // rows at least this long are staged back to back where the destination has them so
 
 }  // namespace tc

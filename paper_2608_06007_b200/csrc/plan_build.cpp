@@ -259,7 +259,12 @@ static int finish_group(Group &g, uint32_t tile_bytes)
         uint64_t most = 0;
         for (const Desc &d : g.descs) {
             const uint64_t units = (std::min<uint32_t>(d.run, kRealignColumn) + 30) >> 4;
-            most = std::max<uint64_t>(most, std::min<uint64_t>(d.rows_per_tile, d.rows) * units * 16 * ppt + 32);
+            const uint64_t rows = std::min<uint64_t>(d.rows_per_tile, d.rows);
+            most = std::max<uint64_t>(most, rows * units * 16 * ppt + 32);
+            // rows adjacent in the destination are staged back to back, one group per destination
+            // run (16 bytes of slack each), plus one 16-byte side chunk per row
+            if (ppt == 1 && (d.run & 15) == 0 && d.run >= kJoinMinRun && d.run <= kRealignColumn && (d.dst_s1 == d.run || d.dst_s0 == d.run))
+                most = std::max<uint64_t>(most, rows * d.run + 16 * std::min<uint64_t>(d.n0, rows) + 16 * (rows + 1) + 64);
         }
         return static_cast<uint32_t>(std::min<uint64_t>(most, kRealignSmem));
     };

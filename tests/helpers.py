@@ -135,6 +135,110 @@ class _Mem:
             cnt[lo:lo + len(data)] += 1
 
 
+JOIN_MIN_RUN = 1024
+
+
+def run_realign_tile_joined(d, o, part, src, dst, cnt, smem_bytes=52 << 10, threads=256):
+    """The realigning path's back-to-back staging of rows that are adjacent in the destination
+    (rows of at least JOIN_MIN_RUN bytes), replayed like run_realign_tile.  Returns False,
+    touching nothing, for a tile the kernel would not take this way.  Per row one bulk load of
+    its whole chunks to its place in its group, one of the chunk that holds its last s_lo bytes
+    to a side array (unless it is the last of its group), then a merge of that side chunk into
+    the next row's first chunk; the groups are then stored as long rows: whole chunks, heads and
+    tails byte by byte."""
+    run, n0 = d.run_bytes, d.n0
+    row0 = part * d.rows_per_tile
+    nrows = min(d.rows_per_tile, d.rows - row0)
+    if run % 16 or run < JOIN_MIN_RUN or run > smem_bytes - 64 or nrows < 2:
+        return False
+    j1, j0 = divmod(row0, n0)
+    across, groups, glen, vstride, cols = False, 1, nrows, 0, 0
+    if d.dst_s1 == run:
+        cols = nrows // n0
+        if j0 or cols * n0 != nrows:
+            return False
+        across = True
+        if n0 > 1 and d.dst_s0 != cols * run:
+            groups, glen, vstride = n0, cols, d.dst_s0
+    elif n0 > 1 and d.dst_s0 == run:
+        if j0 + nrows > n0 and d.dst_s1 != n0 * run:
+            return False
+    else:
+        return False
+    length = glen * run
+    units = (length + 30) >> 4
+    data = 16
+    side = data + groups * (units << 4) + 16
+    if glen < 2 or units < threads or groups * (units << 4) + 48 + 16 * (nrows + 1) > smem_bytes:
+        return False
+    src0 = src.va + d.src_off + o * d.src_outer
+    dst0 = dst.va + d.dst_off + o * d.dst_outer
+    s_first = src0 + j1 * d.src_s1 + j0 * d.src_s0
+    d_first = dst0 + j1 * d.dst_s1 + j0 * d.dst_s0
+    s_lo, d_lo = s_first % 16, d_first % 16
+    stage = np.full(smem_bytes, 0xDD, dtype=np.uint8)
+    loaded = np.zeros(smem_bytes, dtype=bool)
+
+    def place(rr):
+        i1, i0 = divmod(row0 + rr, n0)
+        g, pos = 0, rr
+        if across:
+            g, pos = (i0, i1 - j1) if groups > 1 else (0, i0 * cols + (i1 - j1))
+        return i1, i0, g, pos
+
+    def bulk(at, gaddr, nbytes):
+        assert at % 16 == 0 and gaddr % 16 == 0 and nbytes % 16 == 0 and nbytes > 0 and at + nbytes <= smem_bytes
+        for c in range(nbytes // 16):
+            assert not loaded[at + 16 * c], "two bulk copies land on one staged chunk"
+            stage[at + 16 * c:at + 16 * c + 16] = src.read16(gaddr + 16 * c)
+            loaded[at + 16 * c:at + 16 * c + 16] = True
+
+    announced = nrows * (run + 16 if s_lo else run)
+    arrived = 0
+    for rr in range(nrows):
+        i1, i0, g, pos = place(rr)
+        row = src0 + i1 * d.src_s1 + i0 * d.src_s0 - s_lo
+        at = data + 16 * g * units + pos * run
+        if not s_lo or pos + 1 == glen:
+            n = run + 16 if s_lo else run
+            bulk(at, row, n)
+            arrived += n
+        else:
+            bulk(at, row, run)
+            bulk(side + 16 * (g * glen + pos + 1), row + run, 16)
+            arrived += run + 16
+    assert arrived == announced, "the barrier's byte count"
+    if s_lo:
+        for rr in range(nrows):
+            _, _, g, pos = place(rr)
+            if pos == 0:
+                continue
+            at = data + 16 * g * units + pos * run
+            sd = side + 16 * (g * glen + pos)
+            assert loaded[sd:sd + 16].all() and loaded[at:at + 16].all()
+            stage[at:at + s_lo] = stage[sd:sd + s_lo]
+    delta = s_lo - d_lo
+    sh, shifted = delta % 16, data + 16 * (delta >> 4)
+    end = d_lo + length
+    c_first, c_last, t = (1 if d_lo else 0), end >> 4, end & 15
+    out0 = d_first - d_lo
+    for g in range(groups):
+        for c in range(c_first, c_last):
+            at = shifted + 16 * (g * units + c)
+            assert 0 <= at and at + 32 <= smem_bytes, "staging read outside the area"
+            assert loaded[at + sh:at + sh + 16].all(), "a staged byte that was never loaded is consumed"
+            dst.write(out0 + g * vstride + 16 * c, stage[at + sh:at + sh + 16].copy(), cnt)
+        for k in range(32):
+            is_tail = k >= 16
+            if (k - 16 >= t) if is_tail else (k < d_lo or not d_lo):
+                continue
+            byte = 16 * c_last + (k - 16) if is_tail else k
+            at = data + 16 * g * units + s_lo + byte - d_lo
+            assert loaded[at], "a staged byte that was never loaded is consumed"
+            dst.write(out0 + g * vstride + byte, stage[at:at + 1], cnt)
+    return True
+
+
 def run_realign_tile(d, o, part, src, dst, cnt, smem_bytes=52 << 10, threads=256):
     """The realigning path of the kernel (rows whose source and destination are not both
     16-byte aligned, all strides multiples of 16), replayed for tile (outer o, part) of
@@ -143,6 +247,9 @@ def run_realign_tile(d, o, part, src, dst, cnt, smem_bytes=52 << 10, threads=256
     last chunks in aligned pieces, and the chunk that two destination-adjacent rows share
     stored once.  Same quantities and formulas as the CUDA code; every staged byte that is
     consumed must have been loaded, every destination byte is counted."""
+    assert all(x % 16 == 0 for x in (d.src_s0, d.src_s1, d.dst_s0, d.dst_s1))
+    if run_realign_tile_joined(d, o, part, src, dst, cnt, smem_bytes, threads):
+        return "joined"
     column_max = smem_bytes - 64
     row0 = part * d.rows_per_tile
     nrows = min(d.rows_per_tile, d.rows - row0)
@@ -150,7 +257,7 @@ def run_realign_tile(d, o, part, src, dst, cnt, smem_bytes=52 << 10, threads=256
     column = min(run, column_max)
     units = (column + 30) >> 4
     rows_per_pass = (smem_bytes - 32) // (units << 4)
-    assert rows_per_pass >= 1 and all(x % 16 == 0 for x in (d.src_s0, d.src_s1, d.dst_s0, d.dst_s1))
+    assert rows_per_pass >= 1
     src0 = src.va + d.src_off + o * d.src_outer
     dst0 = dst.va + d.dst_off + o * d.dst_outer
     rowoff = lambda r, s0, s1: (r // d.n0) * s1 + (r % d.n0) * s0

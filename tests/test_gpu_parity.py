@@ -869,15 +869,41 @@ def test_rows_at_every_source_and_destination_alignment(cols, pitch, tile):
             assert np.array_equal(outs[k].result(), want[k]), (pairs[k], shift)
 
 
-@pytest.mark.parametrize("D,slots", [(128, "one"), (64, "one"), (32, "planes")])
+@pytest.mark.parametrize("a,b", [(0, 1), (2, 0), (15, 15), (8, 4), (3, 9), (0, 0)])
+def test_dim1_weight_slices_with_long_rows_through_misaligned_pointers(a, b):
+    """Row-parallel shards of [rows, cols] matrices: strided source rows of 1-3.5 KiB that are
+    adjacent in the destination, the blob starting a bytes and the outputs b bytes off a 16-byte
+    boundary.  Such rows are staged back to back and stored as one long destination run."""
+    rng = np.random.default_rng(60 + a + b)
+    shapes = [[96, 4096, 1, 1], [40, 7168, 1, 1], [33, 2048, 1, 1], [5, 8192, 1, 1]]
+    nbytes = [2 * r * c for r, c, _, _ in shapes]
+    byte_off = np.concatenate([[0], np.cumsum(nbytes)[:-1]]).tolist()
+    total = int(sum(nbytes))
+    blob = rng.integers(0, 256, total, dtype=np.uint8)
+    raw = torch.zeros(total + 16, dtype=torch.uint8, device="cuda")
+    raw[a:a + total].copy_(dev(blob))
+    for world, rank in ((4, 1), (8, 7), (2, 0)):
+        want = [np.zeros(n // world, dtype=np.uint8) for n in nbytes]
+        oracle.weights(byte_off, [2] * 4, shapes, [1] * 4, rank, world, blob, want)
+        plan = tc.tc_plan_create(tc.weights_spec(byte_off, nbytes, [2] * 4, [2] * 4, shapes, split_dim=[1] * 4, rank=rank, world=world, blob_bytes=total))
+        outs = [Guarded(n // world, fill=0xEE, shift=b) for n in nbytes]
+        tc.tc_weights_materialize(plan, raw[a:].data_ptr(), [o.ptr() for o in outs])
+        for i in range(4):
+            assert np.array_equal(outs[i].result(), want[i]), (i, world, rank)
+    assert tc.tc_device_status() == 0
+
+
+@pytest.mark.parametrize("H,D,E,slots", [(8, 128, 2, "one"), (8, 64, 2, "one"), (8, 32, 2, "planes"), (8, 512, 2, "one"), (2, 512, 2, "one"), (4, 256, 4, "one")])
 @pytest.mark.parametrize("shift_pool,shift_packed", [(0, 2), (2, 0), (6, 6), (1, 9), (8, 4)])
-def test_kv_pack_unpack_migrate_through_misaligned_pointers(shift_pool, shift_packed, D, slots):
+def test_kv_pack_unpack_migrate_through_misaligned_pointers(shift_pool, shift_packed, H, D, E, slots):
     """Aligned geometry, misaligned base pointers: the pool and / or the packed buffer start at
-    an odd address (a view into a larger allocation).  Rows of D * 2 bytes (NHD <-> HND) and whole
+    an odd address (a view into a larger allocation).  Rows of D * E bytes (NHD <-> HND) and whole
     planes (same layout) both take the realigning path; with D = 64 and 32 a plane is small enough
-    for tiles of two and four planes, in a pool with one pointer or a pointer per plane."""
+    for tiles of two and four planes, in a pool with one pointer or a pointer per plane; rows of
+    1 KiB are staged back to back where the destination has them adjacent (a head's tokens, a
+    token's heads)."""
     rng = np.random.default_rng(77)
-    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=40, B=16, H=8, D=D, E=2, T=(100, 16, 7, 333))
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=40, B=16, H=H, D=D, E=E, T=(100, 16, 7, 333))
     L, B, H, D, E = shape
     planes = planes_of(pool, L * 2)
     bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)

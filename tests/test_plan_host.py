@@ -646,6 +646,46 @@ def test_realigning_path_arithmetic_on_the_cpu(a, b):
             assert cnt.max() == 1 and cnt.sum() == int(T.sum()) * 2 * 4 * 128, (spec.kind, smem)
 
 
+@pytest.mark.parametrize("a,b", [(0, 1), (1, 0), (15, 15), (8, 4), (3, 9)])
+def test_realigning_path_stages_long_destination_adjacent_rows_back_to_back(a, b):
+    """Rows of 1 KiB: pack (groups of a head's tokens, one per head), unpack (the whole tile is
+    one destination run) and a dim-1 weight slice (strided source rows, contiguous destination)
+    take the back-to-back staging: no two bulk copies share a staged chunk, the barrier's byte
+    count adds up, every consumed byte was loaded, every destination byte is written once with
+    the oracle's value.  Ragged last tiles and a small staging area fall back to per-row slots."""
+    from helpers import _Mem, run_realign_tile
+    rng = np.random.default_rng(90 + a + b)
+    shape, NB, stride, pool, T, off, bt = kv_case(rng, L=1, NB=10, B=8, H=4, D=256, E=4, T=(19, 8, 5, 24))
+    bt2 = rng.permutation(NB)[:off[-1]].astype(np.int32)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride)
+    want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+    oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, 2), T, off, bt, oracle.HND, want)
+    cases = [(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_src=bt, flags=HOST), 0, pool, want, 0)]
+    want_pool = np.full_like(pool, 0xA5)
+    oracle.kv_unpack(shape, oracle.NHD, stride, planes_of(want_pool, 2), T, off, bt2, oracle.HND, want)
+    cases.append((tc.kv_spec(tc.TC_KV_UNPACK, shape, dst_pool=pl, packed_layout=tc.TC_HND, T=T, bt_off=off, bt_dst=bt2, flags=HOST), 1, want, want_pool, 0xA5))
+    # a [96, 4096] fp16 matrix split 4 ways along dim 1: 96 rows of 2 KiB, 8 KiB apart in the blob
+    blob = rng.integers(0, 256, 96 * 8192, dtype=np.uint8)
+    want_w = [np.zeros(96 * 2048, dtype=np.uint8)]
+    oracle.weights([0], [2], [[96, 4096, 1, 1]], [1], 1, 4, blob, want_w)
+    cases.append((tc.weights_spec([0], [blob.size], [2], [2], [[96, 4096, 1, 1]], split_dim=[1], rank=1, world=4, blob_bytes=blob.size, flags=HOST), 0, blob, want_w[0], 0))
+    for spec, group, source, expect, fill in cases:
+        plan = tc.tc_plan_create(spec)
+        for smem in (52 << 10, 6000):
+            got = np.full(expect.size, fill, dtype=np.uint8)
+            cnt = np.zeros(expect.size, dtype=np.int32)
+            src, dst = _Mem(source, 4096 + a), _Mem(got, 1 << 20 | b)
+            how = []
+            for d in plan.descriptors(group):
+                for o in range(d.n_outer):
+                    for part in range(d.tiles_per_outer):
+                        if part * d.rows_per_tile < d.rows:
+                            how.append(run_realign_tile(d, o, part, src, dst, cnt, smem_bytes=smem))
+            assert np.array_equal(got, expect), (spec.kind, smem)
+            assert cnt.max() == 1
+            assert ("joined" in how) == (smem > 6000), (spec.kind, smem, how)
+
+
 @pytest.mark.parametrize("D,E,a,b", [(40, 1, 0, 0), (50, 2, 3, 0), (33, 1, 7, 12), (36, 1, 0, 5), (100, 2, 1, 1)])
 def test_realigning_path_arithmetic_for_rows_that_differ_in_alignment(D, E, a, b):
     """Rows of D * E bytes, not a multiple of 16: every row of a tile has its own source and
