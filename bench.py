@@ -1372,7 +1372,11 @@ def extra_config4(args, tc, torch, stream, out):
             ev[0].record(stream)
             tc.tc_kv_unpack(plan, [host], [dev], sp)
             ev[1].record(stream)
-            torch.cuda.synchronize()   # a scheduler step ends when both directions have landed
+            try:
+                torch.cuda.synchronize()   # a scheduler step ends when both directions have landed
+            except Exception as e:         # say which step of which path it was
+                raise RuntimeError(f"configs[4] burst: host path {path!r}, step {i} of {steps_here}, {len(st.reload_dev)} reload and "
+                                   f"{len(st.offload_dev)} offload blocks") from e
             plan.destroy()
             if i >= 1:
                 dev_ms.append((ev[0].elapsed_time(ev[1]), ev[2].elapsed_time(ev[3])))

@@ -62,6 +62,26 @@ cudaError_t block_alloc(int device, size_t nb, void **out, size_t *got)
     return cudaMalloc(out, want);
 }
 
+// Plans are uploaded on a stream of the library's own, one per device, and the upload is waited
+// for: a copy from pageable host memory may return once the bytes sit in the driver's staging
+// buffer, before they have reached the device, and a kernel the caller then launches on a
+// non-blocking stream would not wait for it (it would read whatever plan used the block before).
+cudaStream_t g_upload_stream[kMaxDevices] = {};
+
+cudaError_t upload_stream_for(int device, cudaStream_t *out)
+{
+    if (device < 0 || device >= kMaxDevices) {  // no private stream: the legacy stream, waited for as well
+        *out = cudaStreamLegacy;
+        return cudaSuccess;
+    }
+    cudaError_t e = cudaSuccess;
+    pthread_mutex_lock(&g_block_mu);
+    if (!g_upload_stream[device]) e = cudaStreamCreateWithFlags(&g_upload_stream[device], cudaStreamNonBlocking);
+    *out = g_upload_stream[device];
+    pthread_mutex_unlock(&g_block_mu);
+    return e;
+}
+
 void block_free(int device, void *ptr, size_t bytes)
 {
     if (!ptr) return;
@@ -115,7 +135,10 @@ static int upload_plan(tc_plan *plan)
         plan->d_storage = nullptr;
         return e == cudaErrorMemoryAllocation ? fail(TC_ERR_OOM, "device allocation of %zu plan bytes failed", total) : cuda_fail(e, "cudaMalloc");
     }
-    if ((e = cudaMemcpy(plan->d_storage, image.data(), total, cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(e, "cudaMemcpy(plan)");
+    cudaStream_t up;
+    if ((e = upload_stream_for(plan->device, &up)) != cudaSuccess) return cuda_fail(e, "cudaStreamCreate(plan upload)");
+    if ((e = cudaMemcpyAsync(plan->d_storage, image.data(), total, cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync(plan)");
+    if ((e = cudaStreamSynchronize(up)) != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize(plan upload)");
     plan->device_bytes += static_cast<int64_t>(plan->d_storage_bytes);
     char *base = static_cast<char *>(plan->d_storage);
     for (int k = 0; k < 2; k++) {
