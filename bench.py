@@ -774,7 +774,9 @@ def b2b_ms(torch, stream, fn, reps=5, warm=2):
     behind `warm` untimed ones that are still running when the first event is enqueued.  The host
     side of a call (marshalling the pointer table, checks, the launch itself) then overlaps the GPU
     work of the call before it; with a synchronise before every timed launch a short kernel would be
-    charged for the time the idle GPU waits for the host."""
+    charged for the time the idle GPU waits for the host.  Whatever other streams still run (the
+    fill of a fresh pool on the default stream) is waited for first: plan creation does not."""
+    torch.cuda.synchronize()
     with torch.cuda.stream(stream):
         for _ in range(warm):
             fn()
@@ -1281,6 +1283,7 @@ def extra_config4(args, tc, torch, stream, out):
     NBh = min(rule, arena.buf.numel() // shape.block_bytes) if arena else rule
     dev = torch.empty(NBd * shape.block_bytes, **u8)
     dev.fill_(3)
+    torch.cuda.synchronize()
     if arena is None:
         arena = PinnedArena(torch, NBh * shape.block_bytes)
     arena.reset()

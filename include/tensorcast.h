@@ -318,6 +318,10 @@ typedef struct tc_plan tc_plan_t;
  * Validate `spec` on the host, lower it to descriptors and tiles, upload them to the current
  * CUDA device (unless TC_PLAN_HOST_ONLY) and return an immutable plan in *out.
  * spec, out: host pointers.  On error *out = NULL and nothing stays allocated.
+ * The upload runs on a stream of the library's own and has completed when the call returns, so
+ * the plan may be executed on any stream at once.  The call orders itself against NO stream of
+ * the caller: it neither waits for work already enqueued (a buffer still being filled on another
+ * stream is the caller's to wait for) nor makes later work wait.
  */
 TC_API int tc_plan_create(const tc_plan_spec_t *spec, tc_plan_t **out);
 

@@ -1124,6 +1124,7 @@ def test_concurrent_threads_create_execute_destroy():
             lay = LAYOUTS[k % 2]
             out = torch.zeros(wants[lay].size, dtype=torch.uint8, device="cuda")
             host = torch.zeros(wants[lay].size, dtype=torch.uint8).pin_memory()
+            torch.cuda.synchronize()                         # `out` was zeroed on the default stream
             for it in range(25):
                 flags = tc.TC_PLAN_STAGED if (it + k) % 3 == 0 else 0
                 plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=lay, T=T, bt_off=off, bt_src=bt, flags=flags))

@@ -40,8 +40,9 @@ def test_noalloc_pack_matches_planned_pack_on_two_calls_in_a_row():
     for make, pool, nbytes in cases:
         want = torch.full((nbytes,), 0x11, dtype=torch.uint8, device="cuda")
         plan = tc.tc_plan_create(make())
-        tc.tc_kv_pack(plan, [pool], [want], stream.cuda_stream)
         got = torch.full((nbytes + 512,), 0x22, dtype=torch.uint8, device="cuda")
+        torch.cuda.synchronize()                           # the fills ran on the default stream
+        tc.tc_kv_pack(plan, [pool], [want], stream.cuda_stream)
         spec, keep = make()
         tc.tc_kv_pack_noalloc(spec, [pool], [got], stream.cuda_stream)
         stream.synchronize()
@@ -54,6 +55,7 @@ def test_noalloc_calls_leave_free_device_memory_unchanged():
     make, pool, nbytes = _case(33, tc.TC_HND, (100, 64, 7))
     got = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
     tc.tc_kv_pack_noalloc(make()[0], [pool], [got], stream.cuda_stream)   # first call on the device: resolves the scratch address
     stream.synchronize()
     free0 = torch.cuda.mem_get_info()[0]
@@ -100,9 +102,11 @@ def test_noalloc_runs_migrate_specs_and_ragged_geometries():
         make = lambda: tc.kv_spec(tc.TC_KV_MIGRATE, shape.tuple, src_pool=pl, dst_pool=dst_pool, T=T, bt_off=off, bt_src=bt_s, bt_dst=bt_d)
         want = torch.full_like(src, 0xA5)
         plan = tc.tc_plan_create(make())
+        torch.cuda.synchronize()                           # the fills ran on the default stream
         tc.tc_kv_pack(plan, [src], [want], stream.cuda_stream)
         for _ in range(2):
             got = torch.full_like(src, 0xA5)
+            torch.cuda.synchronize()
             spec, keep = make()
             tc.tc_kv_pack_noalloc(spec, [src], [got], stream.cuda_stream)
             stream.synchronize()
