@@ -1102,6 +1102,35 @@ def test_execute_calls_can_be_captured_in_a_cuda_graph_and_replayed(shift):
         assert np.array_equal(fresh.result(), want_pool)
 
 
+def test_a_plan_can_run_on_a_non_blocking_stream_the_moment_it_is_created():
+    """Plans of 2 000 descriptors (a 256 KB upload) created, executed at once on a non-blocking
+    stream and destroyed, two geometries taking turns so that each inherits the other's storage
+    block: the upload must have landed when tc_plan_create returns, whatever stream runs next."""
+    rng = np.random.default_rng(41)
+    shape, NB, stride, pool, _, _, _ = kv_case(rng, L=1, NB=2400, B=4, H=1, D=8, E=2, T=(4,))
+    d_pool = dev(pool)
+    pl = tc.pool(tc.TC_NHD, NB, 1, plane_stride=NB * stride, slot_bytes=pool.size)
+    cases = []
+    for k in range(2):
+        T = np.full(2000, 4 - k, dtype=np.int64)               # one block per request; full or ragged
+        off = np.arange(2001, dtype=np.int64)
+        bt = rng.permutation(NB)[:2000].astype(np.int32)
+        want = np.zeros(oracle.packed_nbytes(shape, T), dtype=np.uint8)
+        oracle.kv_pack(shape, oracle.NHD, stride, planes_of(pool, 2), T, off, bt, oracle.NHD, want, threads=4)
+        cases.append((T, off, bt, torch.from_numpy(want).cuda(), torch.zeros(want.size, dtype=torch.uint8, device="cuda")))
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for it in range(60):
+        T, off, bt, want, out = cases[it % 2]
+        plan = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_PACK, shape, src_pool=pl, packed_layout=tc.TC_NHD, T=T, bt_off=off, bt_src=bt))
+        tc.tc_kv_pack(plan, [d_pool], [out], stream.cuda_stream)
+        stream.synchronize()
+        assert torch.equal(out, want), it
+        out.zero_()
+        torch.cuda.synchronize()
+        plan.destroy()
+
+
 def test_concurrent_threads_create_execute_destroy():
     """Calls on distinct plans are thread safe (plan-storage cache, staging rings, per-thread error
     text): four threads each create, run on their own stream and destroy plans in a loop."""
