@@ -514,8 +514,9 @@ TC_API int tc_trim(void);
  *       waited about a second for its asynchronous bulk copies into shared memory and gave up;
  *       the CTA returned without storing, so the destination of that call is incomplete.  Not
  *       expected to occur; the wait is bounded so that a failure cannot hang the device.
- * flags: host pointer.  The call copies the word back and therefore waits for the device's
- * previously enqueued work (it is a diagnostic, off the data path). */
+ * flags: host pointer.  The call synchronises the device first (every stream's previously
+ * enqueued work, non-blocking streams included) and then copies the word back: it is a
+ * diagnostic, off the data path. */
 #define TC_DEVICE_BULK_WAIT_TIMEOUT 1u
 #define TC_DEVICE_OUT_OF_BOUNDS 2u /* the bounds checker of a TC_PLAN_DEBUG_BOUNDS plan found a descriptor that
                                       reaches outside its table slot; copy kernels of such plans return

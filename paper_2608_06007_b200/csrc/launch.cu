@@ -177,7 +177,10 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
 int read_device_status(unsigned int *out)
 {
     unsigned int zero = 0;
-    cudaError_t e = cudaMemcpyFromSymbol(out, g_device_status, sizeof *out);
+    // a diagnostic: every stream's earlier work first, non-blocking streams included (a copy on
+    // the legacy stream alone would not wait for those)
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpyFromSymbol(out, g_device_status, sizeof *out);
     if (e == cudaSuccess && *out) e = cudaMemcpyToSymbol(g_device_status, &zero, sizeof zero);
     return e == cudaSuccess ? TC_OK : cuda_fail(e, "reading the device status word");
 }
