@@ -427,6 +427,7 @@ def run_ours(args):
         host_tune["max_ctas"] = args.host_ctas
     if args.host_copy_path:
         host_tune["copy_path"] = args.host_copy_path
+    torch.cuda.synchronize()  # the fills above: a first cudaMalloc inside plan creation would wait for them
     t_plan0 = time.perf_counter()
     plans = []
     for src, dst in waves:
