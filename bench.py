@@ -766,7 +766,10 @@ def run_ours(args):
         "roofline": roofline, "rows": per_row, "other_workloads": extras,
         "cpu_baseline": {"value": cpu_v, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": cpu_desc, "parts_GBps": cpu_parts},
     }
-    print(json.dumps(line))
+    print(json.dumps(line), flush=True)
+    if extras and "FAILED" in extras:  # the context may be beyond an orderly teardown
+        sys.stderr.flush()
+        os._exit(0)
     ranks.close()
 
 
@@ -1435,8 +1438,17 @@ def run_extras(args, tc, torch, stream):
     out = {}
     for name, fn in EXTRAS:
         if want is None or name in want:
-            fn(args, tc, torch, stream, out)
-            torch.cuda.empty_cache()
+            try:
+                fn(args, tc, torch, stream, out)
+                torch.cuda.empty_cache()
+            except Exception as e:  # noqa: BLE001
+                # the headline numbers are already taken: report the failure beside them instead of
+                # losing the whole line; a CUDA error is sticky, so the remaining extras are skipped
+                import traceback
+                traceback.print_exc(file=sys.stderr)
+                out["FAILED"] = {"extra": name, "error": repr(e)[:500], "skipped_after_it": [n for n, _ in EXTRAS[[n for n, _ in EXTRAS].index(name) + 1:]
+                                                                                            if want is None or n in want]}
+                break
     return out
 
 
