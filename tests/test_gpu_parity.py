@@ -747,6 +747,17 @@ def test_debug_plans_check_their_descriptors_on_the_device_and_skip_the_copy_whe
         assert tc.tc_device_status() == 0
         tc.tc_plan_check_device(p2, pool.size)                # no slot left at all
         assert tc.tc_device_status() == tc.TC_DEVICE_OUT_OF_BOUNDS
+    # a mixed plan carries extents for both of its groups (offload: pool -> host pool, reload: back)
+    hpool = tc.pool(tc.TC_HND, 24, 1, plane_stride=stride, block_stride=L * 2 * stride, slot_bytes=24 * L * 2 * stride)
+    n_off = int(off[1])
+    mixed = tc.tc_plan_create(tc.kv_spec(tc.TC_KV_MIXED, shape, src_pool=pl, dst_pool=hpool, T=T[:1], bt_off=off[:2], bt_src=bt[:n_off],
+                                         bt_dst=np.arange(n_off, dtype=np.int32),
+                                         reload=dict(T=T[1:2], bt_off=off[1:3] - off[1], bt_src=np.array([23], dtype=np.int32), bt_dst=bt2[:1]),
+                                         flags=tc.TC_PLAN_DEBUG_BOUNDS))
+    tc.tc_plan_check_device(mixed, 0)
+    assert tc.tc_device_status() == 0
+    tc.tc_plan_check_device(mixed, 1)                         # host block 23 ends on the host pool's last byte
+    assert tc.tc_device_status() == tc.TC_DEVICE_OUT_OF_BOUNDS
     ck = small_checkpoint()
     blob = np.zeros(ck.nbytes_total, dtype=np.uint8)
     wl.fill_np(blob, 5, "normal")
