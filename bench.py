@@ -1436,19 +1436,18 @@ def run_extras(args, tc, torch, stream):
     if args.only_misaligned:
         want = {"misaligned"}
     out = {}
-    for name, fn in EXTRAS:
-        if want is None or name in want:
-            try:
-                fn(args, tc, torch, stream, out)
-                torch.cuda.empty_cache()
-            except Exception as e:  # noqa: BLE001
-                # the headline numbers are already taken: report the failure beside them instead of
-                # losing the whole line; a CUDA error is sticky, so the remaining extras are skipped
-                import traceback
-                traceback.print_exc(file=sys.stderr)
-                out["FAILED"] = {"extra": name, "error": repr(e)[:500], "skipped_after_it": [n for n, _ in EXTRAS[[n for n, _ in EXTRAS].index(name) + 1:]
-                                                                                            if want is None or n in want]}
-                break
+    todo = [(name, fn) for name, fn in EXTRAS if want is None or name in want]
+    for k, (name, fn) in enumerate(todo):
+        try:
+            fn(args, tc, torch, stream, out)
+            torch.cuda.empty_cache()
+        except Exception as e:  # noqa: BLE001
+            # the headline numbers are already taken: report the failure beside them instead of
+            # losing the whole line; a CUDA error is sticky, so the remaining extras are skipped
+            import traceback
+            traceback.print_exc(file=sys.stderr)
+            out["FAILED"] = {"extra": name, "error": repr(e)[:500], "skipped_after_it": [n for n, _ in todo[k + 1:]]}
+            break
     return out
 
 
