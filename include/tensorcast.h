@@ -423,8 +423,8 @@ TC_API int tc_plan_destroy(tc_plan_t *plan);
  * launches nothing.  Every GPU that loads the library holds that 1 MiB until the process exits.
  *
  * The first call on a device resolves the scratch area's device address for that device (the
- * device must be current, as for every call of this library); make that first call before any
- * stream capture begins.  All calls on a device share the one scratch area, and it keeps the
+ * device must be current, as for every call of this library).  All calls on a device share
+ * the one scratch area, and it keeps the
  * previous call's contents: each call overwrites the part it uses and nothing in it needs to
  * start at zero.  Because the area is shared, two calls whose GPU work can overlap - calls on
  * different streams, or from several threads - race on it; issue them on one stream (where the
