@@ -357,7 +357,7 @@ TC_API int tc_weights_materialize(const tc_plan_t *plan, const void *blob, void 
 
 /*
  * tc_weights_materialize plus integrity checksums, in one pass over the data (the
- * materialisation pipeline "verifies integrity" before it hands tensors out, Sec. 5).
+ * materialisation pipeline checks integrity before it hands tensors out, Sec. 5).
  * `plan` must have been created with TC_PLAN_CHECKSUM.  checksums: DEVICE pointer to
  * n_tensors uint64 accumulators; the call zeroes them on `stream` and the kernel adds to them.
  * Definition.  Tensor i is read as little-endian 4-byte words x_u at tensor-relative offsets

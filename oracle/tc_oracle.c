@@ -249,8 +249,8 @@ void oracle_weights(int64_t N, const int64_t *blob_off, const int64_t *E,
 }
 
 /*
- * Integrity checksum folded into weight materialisation (the materialisation pipeline
- * "verifies integrity", Sec. 5 "Tensor Materialization and Transfer"; the paper does not
+ * Integrity checksum folded into weight materialisation (the materialisation pipeline checks
+ * integrity, Sec. 5 on tensor materialisation and transfer; the paper does not
  * define the function, this is the library's, stated in its header).
  * Tensor i is read as little-endian 4-byte words x_u at tensor-relative byte offsets 4u:
  *   key(u) = ((u * 0x9E3779B1) << 1 | 1) mod 2^32
