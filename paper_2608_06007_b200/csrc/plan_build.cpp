@@ -938,8 +938,16 @@ int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
         // independent, so their order is free; staged groups keep request order, which their
         // segments are cut from)
         const bool kv_kind = spec->kind != TC_WEIGHTS;
-        if (kv_kind && !(spec->flags & TC_PLAN_STAGED) && spec->tuning.tile_order != 1)
-            std::stable_sort(g.descs.begin(), g.descs.end(), [](const Desc &a, const Desc &b) { return a.dst_off < b.dst_off; });
+        if (kv_kind && !(spec->flags & TC_PLAN_STAGED) && spec->tuning.tile_order != 1 &&
+            !std::is_sorted(g.descs.begin(), g.descs.end(), [](const Desc &a, const Desc &b) { return a.dst_off < b.dst_off; })) {
+            // sort 12-byte keys, then move every 128-byte descriptor once
+            std::vector<std::pair<int64_t, uint32_t>> key(g.descs.size());
+            for (size_t i = 0; i < key.size(); i++) key[i] = {g.descs[i].dst_off, static_cast<uint32_t>(i)};
+            std::sort(key.begin(), key.end());  // ties keep their order: the index is the second key
+            std::vector<Desc> sorted(g.descs.size());
+            for (size_t i = 0; i < key.size(); i++) sorted[i] = g.descs[key[i].second];
+            g.descs.swap(sorted);
+        }
         if ((rc = finish_group(g, tile_bytes))) return rc;
     }
     if ((spec->flags & TC_PLAN_SAME_POOL) && spec->kind != TC_KV_MIGRATE)
