@@ -53,3 +53,29 @@ def test_plain_invocation_with_gpus_2_starts_its_own_two_ranks():
     assert len(lines) == 1, out.stdout
     j = json.loads(lines[0])
     assert j["n_gpus"] == 2 and abs(j["ms_per_step"] - 150.0) < 1e-9
+
+
+def test_a_failing_extra_is_reported_and_the_rest_skipped(monkeypatch):
+    """bench.py's secondary workloads run after the headline numbers are taken: one that raises
+    must leave a record beside the others' results instead of losing the line."""
+    import argparse
+    import importlib
+    import types
+    sys.path.insert(0, ROOT)
+    bench = importlib.import_module("bench")
+
+    def ok(args, tc, torch, stream, out):
+        out["first"] = 1
+
+    def boom(args, tc, torch, stream, out):
+        raise RuntimeError("an illegal memory access was encountered")
+
+    def never(args, tc, torch, stream, out):
+        out["third"] = 3
+
+    monkeypatch.setattr(bench, "EXTRAS", [("a", ok), ("b", boom), ("c", never)])
+    fake_torch = types.SimpleNamespace(cuda=types.SimpleNamespace(empty_cache=lambda: None))
+    args = argparse.Namespace(extras="all", only_kv_shapes=False, only_misaligned=False)
+    out = bench.run_extras(args, None, fake_torch, None)
+    assert out["first"] == 1 and "third" not in out
+    assert out["FAILED"]["extra"] == "b" and out["FAILED"]["skipped_after_it"] == ["c"] and "illegal memory access" in out["FAILED"]["error"]
