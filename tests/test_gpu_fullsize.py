@@ -228,6 +228,44 @@ def test_config3_full_size_weights_full_and_all_shards():
     _free()
 
 
+def test_config3_full_size_shard_does_not_depend_on_pointer_alignment():
+    """The 1-of-8 shard of the full checkpoint through misaligned base pointers - the blob 1 byte
+    and every output 9 bytes off a 16-byte boundary, then only the outputs off - must equal the
+    aligned run byte for byte (which the test above holds against the oracle): long slabs, the
+    strided 1 KiB and 3.5 KiB rows of o_proj / down_proj staged back to back, and the replicated
+    norms, with the bytes around every output untouched."""
+    ck = wl.config3()
+    _need(2.6 * ck.nbytes_total)
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    raw = torch.empty(ck.nbytes_total + 16, **u8)
+    wl.fill_torch(raw, wl.SEED_BASE + 3, "normal")
+    nbytes = [ck.nbytes(i) for i in range(ck.N)]
+    W, rank = 8, 3
+    ssize = [n // (W if ck.split_dim[i] >= 0 else 1) for i, n in enumerate(nbytes)]
+    pitch = [(n + 63) // 32 * 32 for n in ssize]             # room for a shift and a gap after every output
+    soffs = np.concatenate([[0], np.cumsum(pitch)])
+    plan = tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, split_dim=ck.split_dim, rank=rank, world=W, blob_bytes=ck.nbytes_total))
+    outs = {}
+    for a, b in ((0, 0), (0, 1), (1, 9)):
+        blob = raw[a:a + ck.nbytes_total]
+        if a:
+            blob.copy_(raw[:ck.nbytes_total].clone())            # the same bytes, one byte further on
+        out = torch.full((int(soffs[-1]) + 16,), 0xEE, **u8)
+        torch.cuda.synchronize()
+        tc.tc_weights_materialize(plan, blob, [out.data_ptr() + int(o) + b for o in soffs[:-1]])
+        torch.cuda.synchronize()
+        outs[(a, b)] = out
+    ref = outs[(0, 0)]
+    for (a, b), out in outs.items():
+        for i in range(ck.N):
+            lo = int(soffs[i])
+            assert torch.equal(out[lo + b:lo + b + ssize[i]], ref[lo:lo + ssize[i]]), (ck.names[i], a, b)
+            assert bool((out[lo + b + ssize[i]:int(soffs[i + 1]) + b] == 0xEE).all()), (ck.names[i], a, b)
+    assert tc.tc_device_status() == 0
+    del raw, outs
+    _free()
+
+
 def test_config4_full_size_migration_70b_shape():
     shape = wl.LLAMA3_70B_KV
     s, chunk, planes = shape.tuple, shape.chunk_bytes, shape.L * 2
