@@ -48,7 +48,7 @@ def test_config2_full_size_pack_unpack_migrate():
     shape = wl.LLAMA3_8B_KV
     s, chunk, planes = shape.tuple, shape.chunk_bytes, shape.L * 2
     NB, WB = 20000, 8192
-    _need((NB + 2 * WB) * shape.block_bytes)
+    _need((NB + 5 * WB) * shape.block_bytes)
     _, _, _, waves = wl.config2(NB=NB, R=256, wave_blocks=WB, NB_dst=WB)
     src, dst = waves[0]
     u8 = dict(dtype=torch.uint8, device="cuda")
@@ -137,6 +137,18 @@ def test_config2_full_size_pack_unpack_migrate():
     tc.tc_kv_pack(pack, [poolA], [Q])
     tc.tc_kv_unpack(unpack, [Q], [poolB])
     torch.cuda.synchronize()
+    # the packed buffer as a view one byte off a 16-byte boundary (the realigning build at full
+    # size): the same bytes, nothing around them touched, and the same pool after the reload
+    Q2 = torch.full((Q.numel() + 16,), 0x5A, **u8)
+    Qv = Q2[1:1 + Q.numel()]
+    poolC.fill_(0xA5)
+    tc.tc_kv_pack(pack, [poolA], [Qv])
+    tc.tc_kv_unpack(unpack, [Qv], [poolC])
+    torch.cuda.synchronize()
+    assert torch.equal(Qv[:payload], Q[:payload]) and int(Q2[0]) == 0x5A and bool((Qv[payload:] == 0x5A).all())
+    assert torch.equal(poolC, poolB)
+    assert tc.tc_device_status() == 0
+    del Q2, Qv
     # staged host path at full size: offload to pinned host and reload must reproduce the
     # (oracle-checked) direct results byte for byte
     Qh = torch.empty(payload, dtype=torch.uint8).pin_memory()
