@@ -427,6 +427,8 @@ def run_ours(args):
         host_tune["max_ctas"] = args.host_ctas
     if args.host_copy_path:
         host_tune["copy_path"] = args.host_copy_path
+    if args.host_tile_order:
+        host_tune["tile_order"] = args.host_tile_order
     torch.cuda.synchronize()  # the fills above: a first cudaMalloc inside plan creation would wait for them
     t_plan0 = time.perf_counter()
     plans = []
@@ -1345,6 +1347,11 @@ def extra_config4(args, tc, torch, stream, out):
             return 1e3 * (t_d + (h2d_bytes - dup_h2d * GB * t_d) / (ceil_h2d * GB))
         return 1e3 * (t_h + (d2h_bytes - dup_d2h * GB * t_h) / (ceil_d2h * GB))
 
+    burst_tune = {}
+    if args.host_ctas:
+        burst_tune["max_ctas"] = args.host_ctas
+    if args.burst_tile_order:
+        burst_tune["tile_order"] = args.burst_tile_order
     paths = ["zerocopy", "staged", "mixed"] if args.burst_paths == "all" else [args.burst_paths]
     results = {}
     for path in paths:
@@ -1365,7 +1372,7 @@ def extra_config4(args, tc, torch, stream, out):
                 tc.TC_KV_MIXED, shape.tuple, src_pool=dev_pool, dst_pool=host_pool,
                 T=st.offload_T, bt_off=st.offload_off, bt_src=st.offload_dev, bt_dst=st.offload_host,
                 reload=dict(T=st.reload_T, bt_off=st.reload_off, bt_src=st.reload_host, bt_dst=st.reload_dev), flags=flags,
-                tuning=dict(max_ctas=args.host_ctas) if args.host_ctas else None))
+                tuning=burst_tune or None))
             if i >= 1:
                 create.append(1e3 * (time.perf_counter() - t0))
                 h2d += int(st.reload_T.sum()) * shape.token_bytes
@@ -1497,12 +1504,14 @@ def main():
     ap.add_argument("--extras", default="all", help="secondary workloads to run: all, or a comma list of " + ",".join(n for n, _ in EXTRAS))
     ap.add_argument("--host-pool-blocks", type=int, default=0, help="configs[4]: pinned host pool size in 2 MiB blocks (0: min(262144, half of MemAvailable))")
     ap.add_argument("--burst-steps", type=int, default=200, help="configs[4]: scheduler steps timed (the workload has 200)")
+    ap.add_argument("--burst-tile-order", type=int, default=0, help="configs[4]: tuning.tile_order of the step's plans (1: block after block instead of plane after plane)")
     ap.add_argument("--burst-paths", default="all", choices=["staged", "mixed", "zerocopy", "all"],
                     help="configs[4]: host path (all: zerocopy over all the steps, staged and mixed on a tenth of them)")
     ap.add_argument("--cold-layers", type=int, default=8, help="cold-path extra: layers of the checkpoint written to a file (8: 4.0 GB)")
     ap.add_argument("--moe-layers", type=int, default=8, help="expert-stacking extra: layers of the MoE checkpoint (8: 11 GB)")
     ap.add_argument("--host-ctas", type=int, default=0)
     ap.add_argument("--host-copy-path", type=int, default=0, help="tuning.copy_path of the e2e plans (1: through shared memory, bulk copies)")
+    ap.add_argument("--host-tile-order", type=int, default=0, help="tuning.tile_order of the e2e plans")
     ap.add_argument("--host-path", default="staged", choices=["staged", "zerocopy"])
     ap.add_argument("--e2e-schedule", default="duplex", choices=["duplex", "serial"],
                     help="duplex: offload wave k+1 while wave k reloads (two streams, two host buffers)")

@@ -90,7 +90,11 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     // pass writes ascending addresses (and pack / unpack stream through the packed buffer),
     // which measured 3-5 % faster than walking the planes of one block after another.
     Segment whole{0, static_cast<uint32_t>(g.descs.size()), 0, g.descs.empty() ? 0 : g.descs[0].n_outer, 0, 0, 0};
-    if (!win && g.tiles_per_desc && !g.descs.empty() && g.descs[0].n_outer > 1 && plan->tuning.tile_order != 1) win = &whole;
+    // Over the host link (a table entry is pinned host memory) HBM locality is beside the point and
+    // the planes of one block run consecutively instead, so that a paged host pool's 2 MiB page is
+    // read or written in one go (prefix-reload burst: 262 against 271 ms per step).
+    const bool plane_major = plan->tuning.tile_order == 2 || (plan->tuning.tile_order == 0 && !over_host_link);
+    if (!win && g.tiles_per_desc && !g.descs.empty() && g.descs[0].n_outer > 1 && plane_major) win = &whole;
     const int mode = mode_for(plan, g, ptr_align, sums != nullptr);
     if (sums && mode == kModeAny) return fail(TC_ERR_INVALID_ARG, "checksums need 16-byte aligned base pointers");
     const uint32_t grid = grid_for(plan, g, mode, win, over_host_link);

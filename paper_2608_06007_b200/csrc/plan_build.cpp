@@ -913,6 +913,8 @@ int build_plan(const tc_plan_spec_t *spec, tc_plan *plan)
     uint32_t tile_bytes = spec->tuning.tile_bytes > 0 ? static_cast<uint32_t>(spec->tuning.tile_bytes) : default_tile;
     if (tile_bytes < 512 || tile_bytes > kMaxTileBytes || (tile_bytes & (tile_bytes - 1)))
         return fail(TC_ERR_INVALID_ARG, "tuning.tile_bytes %u must be a power of two in [512, %u]", tile_bytes, kMaxTileBytes);
+    if (spec->tuning.tile_order < 0 || spec->tuning.tile_order > 2)
+        return fail(TC_ERR_INVALID_ARG, "tuning.tile_order %d must be 0 (auto), 1 (descriptor order) or 2 (plane-major)", spec->tuning.tile_order);
     if (spec->tuning.copy_path != 0 && spec->tuning.copy_path != 1)
         return fail(TC_ERR_INVALID_ARG, "tuning.copy_path %d must be 0 (auto) or 1 (through shared memory)", spec->tuning.copy_path);
     int rc;
