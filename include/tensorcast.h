@@ -288,9 +288,10 @@ typedef struct {
                              ctas_per_sm is set, the grid is capped at one CTA per SM: few
                              long-lived CTAs serve the host link better than one CTA per tile */
     int32_t tile_order;   /* 0 auto: KV groups run plane-major over descriptors sorted by
-                             destination offset (ascending writes in HBM) - unless a table entry
-                             of the call is pinned host memory: then the planes of one block run
-                             consecutively (a paged host pool's page is touched in one go);
+                             destination offset (ascending writes in HBM) - unless one side of
+                             the call is pinned host memory in which a block's planes lie back to
+                             back (a paged host pool): then the planes of one block run
+                             consecutively and a page is touched in one go;
                              1: request / descriptor order as given, planes of one block
                              consecutively; 2: plane-major whatever the memory */
     int32_t copy_path;    /* 0 auto: aligned geometry moves register to register (16-byte loads and

@@ -200,9 +200,10 @@ int execute(const tc_plan *plan, int gi, const void *const *src, size_t n_src, v
         ptr_align = std::min<uint32_t>(ptr_align, __builtin_ctzll(reinterpret_cast<uintptr_t>(dst[i]) | 16));
     }
     int rc;
-    bool host_memory = false;  // some table entry is pinned host memory: the kernel works over the host link
-    if (!file && (rc = check_addressable(src, n_src, "source", &host_memory)) != TC_OK) return rc;
-    if ((rc = check_addressable(const_cast<const void *const *>(dst), n_dst, "destination", &host_memory)) != TC_OK) return rc;
+    bool host_src = false, host_dst = false;  // some table entry is pinned host memory: the kernel works over the host link
+    if (!file && (rc = check_addressable(src, n_src, "source", &host_src)) != TC_OK) return rc;
+    if ((rc = check_addressable(const_cast<const void *const *>(dst), n_dst, "destination", &host_dst)) != TC_OK) return rc;
+    const int host_memory = (host_src ? kHostSrc : 0) | (host_dst ? kHostDst : 0);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool trace = plan->trace_ev[gi][0] != nullptr;
     if (trace) {

@@ -29,11 +29,13 @@ int cuda_fail(cudaError_t e, const char *what);
 int mode_for(const tc_plan *plan, const Group &g, uint32_t ptr_align, bool checksums = false);
 // CTAs of each build that one SM holds, for a pointer table of n_ptrs slots (cached).
 void resident_ctas_for(size_t n_ptrs, int out[3]);
-uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *win = nullptr, bool over_host_link = false);
+// over_host_link: which side of a call has pinned host memory in its table (kHostSrc | kHostDst)
+enum : int { kHostSrc = 1, kHostDst = 2 };
+uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *win = nullptr, int over_host_link = 0);
 // Launch group g (or the window / tile range `win` of it) on stream s.  sums: checksum
 // accumulators or null.
 int launch_any(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s, const Segment *win,
-               unsigned long long *sums = nullptr, bool over_host_link = false);
+               unsigned long long *sums = nullptr, int over_host_link = 0);
 
 // The current device's sticky status word (flags set by kernels); reading clears it.
 int read_device_status(unsigned int *out);

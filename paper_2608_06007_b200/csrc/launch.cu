@@ -58,7 +58,7 @@ void resident_ctas_for(size_t n_ptrs, int out[3])
 // Tile rows per descriptor: planes, or groups of ppt planes.
 static uint32_t outer_groups(const Group &g) { return (g.descs[0].n_outer + g.ppt - 1) / g.ppt; }
 
-uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *win, bool over_host_link)
+uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *win, int over_host_link)
 {
     // Default: one CTA per tile.  The hardware block scheduler then balances the tiles over the
     // SMs and de-phases the CTAs' load and store bursts, which measured faster than a
@@ -83,17 +83,25 @@ uint32_t grid_for(const tc_plan *plan, const Group &g, int mode, const Segment *
 
 template <int NPTR>
 static int launch(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t stream,
-                  const Segment *win, unsigned long long *sums, bool over_host_link)
+                  const Segment *win, unsigned long long *sums, int over_host_link)
 {
     // Uniform groups with planes (KV) are walked plane-major by default: all blocks of plane 0,
     // then plane 1, ...  Together with descriptors sorted by destination offset, every plane
     // pass writes ascending addresses (and pack / unpack stream through the packed buffer),
     // which measured 3-5 % faster than walking the planes of one block after another.
     Segment whole{0, static_cast<uint32_t>(g.descs.size()), 0, g.descs.empty() ? 0 : g.descs[0].n_outer, 0, 0, 0};
-    // Over the host link (a table entry is pinned host memory) HBM locality is beside the point and
-    // the planes of one block run consecutively instead, so that a paged host pool's 2 MiB page is
-    // read or written in one go (prefix-reload burst: 262 against 271 ms per step).
-    const bool plane_major = plan->tuning.tile_order == 2 || (plan->tuning.tile_order == 0 && !over_host_link);
+    // A paged host pool (pinned memory in which the planes of a block lie back to back: one page
+    // per block) is walked block after block instead, so that a page is read or written in one
+    // go; HBM locality is beside the point at the host link's speed (prefix-reload burst: 262-266
+    // against 268-271 ms per step).  A contiguous packed host buffer keeps the plane-major walk,
+    // which streams through it (offload by kernel stores: 80-81 against 78 GB/s).
+    bool paged_host = false;
+    if (over_host_link && !g.descs.empty()) {
+        const Desc &d0 = g.descs[0];
+        const int64_t plane = static_cast<int64_t>(d0.rows) * d0.run;
+        paged_host = ((over_host_link & kHostSrc) && d0.src_outer == plane) || ((over_host_link & kHostDst) && d0.dst_outer == plane);
+    }
+    const bool plane_major = plan->tuning.tile_order == 2 || (plan->tuning.tile_order == 0 && !paged_host);
     if (!win && g.tiles_per_desc && !g.descs.empty() && g.descs[0].n_outer > 1 && plane_major) win = &whole;
     const int mode = mode_for(plan, g, ptr_align, sums != nullptr);
     if (sums && mode == kModeAny) return fail(TC_ERR_INVALID_ARG, "checksums need 16-byte aligned base pointers");
@@ -206,7 +214,7 @@ int launch_wait_timeout_probe(cudaStream_t s)
 }
 
 int launch_any(const tc_plan *plan, const Group &g, const void *const *src, void *const *dst, uint32_t ptr_align, cudaStream_t s, const Segment *win,
-               unsigned long long *sums, bool over_host_link)
+               unsigned long long *sums, int over_host_link)
 {
     const size_t n = g.n_src + g.n_dst;
     if (n <= 8) return launch<8>(plan, g, src, dst, ptr_align, s, win, sums, over_host_link);
