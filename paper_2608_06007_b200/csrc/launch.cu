@@ -97,9 +97,17 @@ static int launch(const tc_plan *plan, const Group &g, const void *const *src, v
     // which streams through it (offload by kernel stores: 80-81 against 78 GB/s).
     bool paged_host = false;
     if (over_host_link && !g.descs.empty()) {
-        const Desc &d0 = g.descs[0];
-        const int64_t plane = static_cast<int64_t>(d0.rows) * d0.run;
-        paged_host = ((over_host_link & kHostSrc) && d0.src_outer == plane) || ((over_host_link & kHostDst) && d0.dst_outer == plane);
+        // the first, the middle and the last descriptor have one and the same plane stride and it is
+        // the size of their largest plane (a block with a ragged tail has fewer rows than its page
+        // has room for; the requests of a packed buffer differ in their plane strides)
+        bool src_paged = (over_host_link & kHostSrc) != 0, dst_paged = (over_host_link & kHostDst) != 0;
+        int64_t plane = 0;
+        for (size_t i : {size_t(0), g.descs.size() / 2, g.descs.size() - 1}) plane = std::max<int64_t>(plane, static_cast<int64_t>(g.descs[i].rows) * g.descs[i].run);
+        for (size_t i : {size_t(0), g.descs.size() / 2, g.descs.size() - 1}) {
+            src_paged = src_paged && g.descs[i].src_outer == plane;
+            dst_paged = dst_paged && g.descs[i].dst_outer == plane;
+        }
+        paged_host = src_paged || dst_paged;
     }
     const bool plane_major = plan->tuning.tile_order == 2 || (plan->tuning.tile_order == 0 && !paged_host);
     if (!win && g.tiles_per_desc && !g.descs.empty() && g.descs[0].n_outer > 1 && plane_major) win = &whole;
