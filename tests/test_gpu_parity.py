@@ -200,7 +200,7 @@ def test_staged_windows_cut_inside_a_tile_row_of_planes():
     assert np.array_equal(fresh.result(), want_pool)
 
 
-@pytest.mark.parametrize("tune", [dict(tile_order=1), dict(ctas_per_sm=2), dict(max_ctas=7), dict(tile_bytes=65536), dict(tile_bytes=1024, ctas_per_sm=1, tile_order=1)])
+@pytest.mark.parametrize("tune", [dict(tile_order=1), dict(tile_order=2), dict(ctas_per_sm=2), dict(max_ctas=7), dict(tile_bytes=65536), dict(tile_bytes=1024, ctas_per_sm=1, tile_order=1)])
 def test_tuning_knobs_change_the_schedule_not_the_bytes(tune):
     rng = np.random.default_rng(29)
     shape, NB, stride, pool, T, off, bt = kv_case(rng, L=3, NB=90, B=32, H=8, D=128, E=2, T=(700, 33, 0, 64, 1200))

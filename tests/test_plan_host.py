@@ -811,6 +811,8 @@ def test_documented_limits_are_enforced():
     # tile size knob must be a power of two in range
     assert _status(_pack_spec(tuning=dict(tile_bytes=3000))) == tc.TC_ERR_INVALID_ARG
     assert _status(_pack_spec(tuning=dict(tile_bytes=1 << 21))) == tc.TC_ERR_INVALID_ARG
+    assert _status(_pack_spec(tuning=dict(tile_order=3))) == tc.TC_ERR_INVALID_ARG
+    tc.tc_plan_create(_pack_spec(tuning=dict(tile_order=2))).destroy()
     # the longest request the configs allow (32 768 tokens) and a single-token one, in one plan
     T = np.array([32768, 1], dtype=np.int64)
     off = np.array([0, 2048, 2049], dtype=np.int64)
