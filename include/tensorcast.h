@@ -532,7 +532,7 @@ TC_API int tc_device_status(uint32_t *flags);
  * table slots less `shrink` bytes.  shrink = 0 is the real check (a plan that tc_plan_create
  * accepted passes it); a positive shrink pretends every slot is that much smaller and shows the
  * checker firing (tests use it: a plan that uses its slots to the last byte must then raise
- * TC_DEVICE_OUT_OF_BOUNDS).  Nothing is copied.  The verdict arrives through tc_device_status. */
+ * TC_DEVICE_OUT_OF_BOUNDS).  Nothing is copied.  The outcome is read with tc_device_status. */
 TC_API int tc_plan_check_device(const tc_plan_t *plan, int64_t shrink, void *stream);
 
 /* Self-test of that bounded wait: launches one small kernel on `stream` that waits on a barrier

@@ -383,7 +383,7 @@ def tc_device_status() -> int:
 
 def tc_plan_check_device(plan: Plan, shrink: int = 0, stream=None) -> None:
     """Run the device-side bounds checker of a TC_PLAN_DEBUG_BOUNDS plan (slot extents less
-    `shrink` bytes); the verdict arrives through tc_device_status()."""
+    `shrink` bytes); the outcome is read with tc_device_status()."""
     _check(load_library().tc_plan_check_device(plan.handle, int(shrink), _stream(stream)))
 
 
