@@ -1027,7 +1027,7 @@ def misaligned(args, tc, torch, stream):
               tc.tc_plan_create(tc.weights_spec(ck.byte_off, nbytes, ck.E, ck.ndim, ck.shapes, split_dim=ck.split_dim, rank=args.shard_rank, world=W,
                                                 blob_bytes=ck.nbytes_total, tuning=smem)))
     cases = [("aligned", 0, 0, auto), ("aligned, through shared memory (tuning.copy_path = 1)", 0, 0, staged)]
-    cases += [(f"src+{a}", a, 0, auto) for a in (8, 4, 2, 1)] + [("dst+1", 0, 1, auto), ("both+1", 1, 1, auto), ("src+3 dst+9", 3, 9, auto)]
+    cases += [(f"src+{a}", a, 0, auto) for a in (8, 4, 2, 1)] + [("dst+1", 0, 1, auto), ("both+1", 1, 1, auto), ("src+3 dst+9", 3, 9, auto), ("src+9 dst+3", 9, 3, auto)]
     for label, a_src, a_dst, (pk, up, mig, wf, ws) in cases:
         A, B = rawA.data_ptr(), rawB.data_ptr()
         Q, bl, dw = rawQ.data_ptr(), blob.data_ptr(), dstw.data_ptr()

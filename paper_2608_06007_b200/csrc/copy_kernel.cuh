@@ -711,6 +711,127 @@ __device__ __forceinline__ int realign_tile_joined(const Desc &d, const char *sr
     return 1;
 }
 
+// SHORT rows that follow one another in the destination a step of n0 apart (dst_s1 == run: the
+// tokens of a head in a head-major buffer, the heads of a token in a token-major block), through
+// a MISALIGNED destination.  Stored row by row, every row boundary is two half-written 32-byte
+// sectors - the chunk two rows share goes out apart from the chunk next to it - and partial
+// sectors are what the memory system charges for.  Here the rows keep their own slots, each
+// slot is completed after the wait with the first chunk of the row that follows it in the
+// destination (copied from that row's slot, merged with the row's own last bytes when the source
+// is misaligned too), and the store loop walks the DESTINATION: thread t takes the aligned chunks t, t + kThreads, ...
+// of a destination run and finds each in its row's slot, so that a warp's store is 512 contiguous,
+// sector-aligned bytes whatever rows they come from.  Only the two ends of a run are partial.
+// Needs: whole i1-columns in the tile, chunks per row a power of two, and, where all rows of
+// the tile form one run, a power-of-two column count.  Returns 1 done, 0 not this geometry
+// (nothing touched), -1 the bulk copies did not arrive.
+template <int WS, int kThreads>
+__device__ __forceinline__ void realign_store_dest_order(char *out0, uint32_t vstride, uint32_t groups, uint32_t total, uint32_t lcpr, uint32_t pmask, uint32_t pshift,
+                                                         uint32_t n0, uint32_t units, uint32_t s_lo, uint32_t d_lo, uint32_t data_addr)
+{
+    const int delta = static_cast<int>(s_lo) - static_cast<int>(d_lo);
+    const uint32_t bits = (static_cast<uint32_t>(delta) & 3) * 8;
+    const uint32_t shifted = data_addr + 16 * (delta >> 4);
+    const uint32_t cmask = (1u << lcpr) - 1;
+    if (total <= kThreads) {
+        // short runs (a head's 16 tokens): a thread keeps its chunk and steps through the runs
+        const uint32_t m = threadIdx.x;
+        if (m >= 1 && m < total) {  // the run's first chunk is partial
+            const uint32_t p = (m - 1) >> lcpr, c = ((m - 1) & cmask) + 1;
+            uint32_t at = shifted + 16 * (((p & pmask) * n0 + (p >> pshift)) * units + c);
+            char *out = out0 + 16 * static_cast<size_t>(m);
+#pragma unroll 4
+            for (uint32_t g = 0; g < groups; g++, at += 16 * units, out += vstride)
+                st_stream<uint4>(out, shift_words<WS>(lds128(at), lds128(at + 16), bits));
+        }
+    } else {
+        for (uint32_t g = 0; g < groups; g++) {
+            char *out = out0 + static_cast<size_t>(g) * vstride;
+#pragma unroll 2
+            for (uint32_t m = threadIdx.x; m < total; m += kThreads) {
+                if (m == 0) continue;  // the run's first chunk is partial
+                const uint32_t p = (m - 1) >> lcpr, c = ((m - 1) & cmask) + 1;
+                const uint32_t rr = (p & pmask) * n0 + (p >> pshift) + g;
+                const uint32_t at = shifted + 16 * (rr * units + c);
+                st_stream<uint4>(out + 16 * static_cast<size_t>(m), shift_words<WS>(lds128(at), lds128(at + 16), bits));
+            }
+        }
+    }
+    // the first 16 - d_lo and the last d_lo bytes of every run, a thread per byte
+    const uint32_t last_p = (total >> lcpr) - 1;
+    for (uint32_t item = threadIdx.x; item < groups * 16; item += kThreads) {
+        const uint32_t g = item >> 4, k = item & 15;
+        const bool tail = k < d_lo;  // k < d_lo: byte k of the run's last chunk; else byte k of its first
+        const uint32_t p = tail ? last_p : 0;
+        const uint32_t rr = (p & pmask) * n0 + (p >> pshift) + g;
+        const uint32_t row_byte = tail ? (16u << lcpr) - d_lo + k : k - d_lo;
+        uint32_t v;
+        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(data_addr + 16 * rr * units + s_lo + row_byte));
+        out0[static_cast<size_t>(g) * vstride + (tail ? 16 * static_cast<size_t>(total) + k : k)] = static_cast<char>(v);
+    }
+}
+
+template <int kThreads>
+__device__ __forceinline__ int realign_tile_dest_order(const Desc &d, const char *src, char *dst, uint32_t row0, uint32_t nrows, uint32_t data_addr, uint32_t stage_bytes,
+                                                       uint32_t bar, uint32_t &phase, uint32_t *wait_ok)
+{
+    const uint32_t run = d.run, n0 = d.n0, cpr = run >> 4;
+    if ((run & 15) || (cpr & (cpr - 1)) || run >= kJoinMinRun || d.dst_s1 != run || (n0 > 1 && d.dst_s0 == run)) return 0;
+    const uint32_t j1 = fastdiv(row0, d.div_n0), cols = fastdiv(nrows, d.div_n0);
+    if (row0 != j1 * n0 || cols * n0 != nrows || cols < 2) return 0;
+    const char *s0 = src + j1 * d.src_s1;
+    char *d0 = dst + j1 * d.dst_s1;
+    const uint32_t s_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(s0)) & 15;
+    const uint32_t d_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(d0)) & 15;
+    if (d_lo == 0) return 0;  // an aligned destination measured no faster this way (unpack 1.5 % slower)
+    // chunks per slot: the row's own, and what the chunk it shares with the next row needs of that
+    // row - its first aligned chunk, and its second one too when s_lo > d_lo
+    const uint32_t units = cpr + (s_lo > d_lo ? 2 : 1);
+    if (nrows * (units << 4) + 32 > stage_bytes) return 0;
+    // one run per i0, dst_s0 apart - or, where those runs are adjacent too, one run in all
+    const bool one_run = n0 == 1 || d.dst_s0 == cols * run;
+    if (one_run && n0 > 1 && (cols & (cols - 1))) return 0;
+    const uint32_t lcpr = 31 - __clz(cpr);
+    const uint32_t groups = one_run ? 1 : n0, glen = one_run ? nrows : cols;
+    const uint32_t pmask = one_run && n0 > 1 ? cols - 1 : 0xffffffffu, pshift = one_run && n0 > 1 ? 31 - __clz(cols) : 31;
+    const char *base = s0 - s_lo;
+    if (threadIdx.x == 0) mbar_expect_tx(bar, nrows * (s_lo ? run + 16 : run));
+    for (uint32_t rr = threadIdx.x; rr < nrows; rr += kThreads) {
+        const uint32_t k1 = fastdiv(rr, d.div_n0), i0 = rr - k1 * n0;  // the tile starts on an i1 boundary
+        bulk_load(data_addr + 16 * rr * units, base + (k1 * d.src_s1 + i0 * d.src_s0), s_lo ? run + 16 : run, bar);
+    }
+    if (!realign_wait(bar, phase, wait_ok)) return -1;
+    // complete every slot with the first chunk of the row after it in the destination (the next
+    // column of the same i0, or, in a single run, the first column of the next i0): from that
+    // row's own slot - a second copy from global memory per row, bulk or not, cost more than it saved
+    for (uint32_t rr = threadIdx.x; rr < nrows; rr += kThreads) {
+        const uint32_t k1 = fastdiv(rr, d.div_n0), i0 = rr - k1 * n0;
+        uint32_t next;
+        if (k1 + 1 < cols) next = rr + n0;
+        else if (one_run && i0 + 1 < n0) next = i0 + 1;
+        else continue;
+        const uint32_t at = data_addr + 16 * (rr * units + cpr);
+        uint4 v = lds128(data_addr + 16 * next * units);
+        if (s_lo) v = merge_bytes(lds128(at), v, s_lo);
+        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(at), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+        if (s_lo > d_lo) {
+            v = lds128(data_addr + 16 * (next * units + 1));
+            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(at + 16), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+        }
+    }
+    __syncthreads();
+    char *out0 = d0 - d_lo;
+    const uint32_t total = glen * cpr;
+    switch (((s_lo - d_lo) & 15) >> 2) {
+    case 0: realign_store_dest_order<0, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, data_addr); break;
+    case 1: realign_store_dest_order<1, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, data_addr); break;
+    case 2: realign_store_dest_order<2, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, data_addr); break;
+    default: realign_store_dest_order<3, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, data_addr); break;
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // ordinary stores into the slots, bulk copies next
+    __syncthreads();
+    return 1;
+}
+
 // Rows [row0, row0 + nrows) of one outer index of descriptor d, any alignment; src / dst point
 // at row 0.  `stage` is the shared-memory staging area (16-byte aligned, stage_bytes long, of
 // which the first and last 16 are padding that neighbouring-chunk loads may touch): a pass
@@ -732,6 +853,8 @@ __device__ __forceinline__ bool copy_rows_realign(const Desc &d, const char *src
     if (same_alignment) {
         const int joined = realign_tile_joined<kThreads>(d, src, dst, row0, nrows, data_addr, stage_bytes, bar, phase, wait_ok);
         if (joined) return joined > 0;
+        const int walked = realign_tile_dest_order<kThreads>(d, src, dst, row0, nrows, data_addr, stage_bytes, bar, phase, wait_ok);
+        if (walked) return walked > 0;
     }
     for (uint32_t col0 = 0; col0 < run; col0 += column) {
         const uint32_t len = min(column, run - col0);

@@ -261,6 +261,9 @@ static int finish_group(Group &g, uint32_t tile_bytes)
             const uint64_t units = (std::min<uint32_t>(d.run, kRealignColumn) + 30) >> 4;
             const uint64_t rows = std::min<uint64_t>(d.rows_per_tile, d.rows);
             most = std::max<uint64_t>(most, rows * units * 16 * ppt + 32);
+            // short rows a step of n0 apart in the destination: room for one more chunk per slot
+            if (ppt == 1 && (d.run & 15) == 0 && d.run < kJoinMinRun && d.dst_s1 == d.run)
+                most = std::max<uint64_t>(most, rows * (units + 1) * 16 + 32);
             // rows adjacent in the destination are staged back to back, one group per destination
             // run (16 bytes of slack each), plus one 16-byte side chunk per row
             if (ppt == 1 && (d.run & 15) == 0 && d.run >= kJoinMinRun && d.run <= kRealignColumn && (d.dst_s1 == d.run || d.dst_s0 == d.run))

@@ -239,6 +239,92 @@ def run_realign_tile_joined(d, o, part, src, dst, cnt, smem_bytes=52 << 10, thre
     return True
 
 
+def run_realign_tile_dest_order(d, o, part, src, dst, cnt, smem_bytes=52 << 10, threads=256):
+    """The realigning path for SHORT rows that follow one another in the destination a step of n0
+    apart, through a misaligned destination, replayed like run_realign_tile.  Returns False,
+    touching nothing, for a tile the kernel would not take this way.  Every row is loaded into a
+    slot of its own; after the wait each slot is completed with the first chunk (two when
+    s_lo > d_lo) of the row that follows it in the destination, taken from that row's slot; the
+    stores then walk the aligned chunks of every destination run, finding each in its row's slot;
+    the first 16 - d_lo and last d_lo bytes of a run go out byte by byte."""
+    run, n0 = d.run_bytes, d.n0
+    row0 = part * d.rows_per_tile
+    nrows = min(d.rows_per_tile, d.rows - row0)
+    cpr = run >> 4
+    if run % 16 or cpr & (cpr - 1) or run >= JOIN_MIN_RUN or d.dst_s1 != run or (n0 > 1 and d.dst_s0 == run):
+        return False
+    j1, cols = row0 // n0, nrows // n0
+    if row0 != j1 * n0 or cols * n0 != nrows or cols < 2:
+        return False
+    src0 = src.va + d.src_off + o * d.src_outer + j1 * d.src_s1
+    dst0 = dst.va + d.dst_off + o * d.dst_outer + j1 * d.dst_s1
+    s_lo, d_lo = src0 % 16, dst0 % 16
+    if d_lo == 0:
+        return False
+    units = cpr + (2 if s_lo > d_lo else 1)
+    if nrows * (units << 4) + 32 > smem_bytes:
+        return False
+    one_run = n0 == 1 or d.dst_s0 == cols * run
+    if one_run and n0 > 1 and cols & (cols - 1):
+        return False
+    groups, glen = (1, nrows) if one_run else (n0, cols)
+    data = 16
+    stage = np.full(smem_bytes, 0xDD, dtype=np.uint8)
+    loaded = np.zeros(smem_bytes, dtype=bool)
+    nbytes = run + 16 if s_lo else run
+    for rr in range(nrows):                                   # one bulk copy per row
+        k1, i0 = divmod(rr, n0)
+        g = src0 - s_lo + k1 * d.src_s1 + i0 * d.src_s0
+        at = data + 16 * rr * units
+        for c in range(nbytes // 16):
+            stage[at + 16 * c:at + 16 * c + 16] = src.read16(g + 16 * c)
+            loaded[at + 16 * c:at + 16 * c + 16] = True
+    snap, snap_loaded = stage.copy(), loaded.copy()           # the fill reads what the copies brought
+    for rr in range(nrows):
+        k1, i0 = divmod(rr, n0)
+        if k1 + 1 < cols:
+            nxt = rr + n0
+        elif one_run and i0 + 1 < n0:
+            nxt = i0 + 1
+        else:
+            continue
+        at, na = data + 16 * (rr * units + cpr), data + 16 * nxt * units
+        assert snap_loaded[na + s_lo:na + 16].all() and (not s_lo or snap_loaded[at:at + s_lo].all())
+        stage[at + s_lo:at + 16] = snap[na + s_lo:na + 16]
+        loaded[at + s_lo:at + 16] = True
+        if s_lo > d_lo:
+            assert snap_loaded[na + 16:na + 32].all()
+            stage[at + 16:at + 32] = snap[na + 16:na + 32]
+            loaded[at + 16:at + 32] = True
+    delta = s_lo - d_lo
+    sh, shifted = delta % 16, data + 16 * (delta >> 4)
+    total = glen * cpr
+    out0 = dst0 - d_lo
+
+    def row_of(p, g):
+        if one_run and n0 > 1:
+            return (p & (cols - 1)) * n0 + (p // cols) + g
+        return p * n0 + g
+
+    for g in range(groups):
+        out = out0 + g * d.dst_s0
+        for m in range(1, total):
+            p, c = divmod(m - 1, cpr)
+            c += 1
+            at = shifted + 16 * (row_of(p, g) * units + c)
+            assert 0 <= at and at + 32 <= smem_bytes, "staging read outside the area"
+            assert loaded[at + sh:at + sh + 16].all(), "a staged byte that was never loaded is consumed"
+            dst.write(out + 16 * m, stage[at + sh:at + sh + 16].copy(), cnt)
+        for k in range(16):
+            tail = k < d_lo
+            p = glen - 1 if tail else 0
+            row_byte = run - d_lo + k if tail else k - d_lo
+            at = data + 16 * row_of(p, g) * units + s_lo + row_byte
+            assert loaded[at], "a staged byte that was never loaded is consumed"
+            dst.write(out + (16 * total + k if tail else k), stage[at:at + 1], cnt)
+    return True
+
+
 def run_realign_tile(d, o, part, src, dst, cnt, smem_bytes=52 << 10, threads=256):
     """The realigning path of the kernel (rows whose source and destination are not both
     16-byte aligned, all strides multiples of 16), replayed for tile (outer o, part) of
@@ -250,6 +336,8 @@ def run_realign_tile(d, o, part, src, dst, cnt, smem_bytes=52 << 10, threads=256
     assert all(x % 16 == 0 for x in (d.src_s0, d.src_s1, d.dst_s0, d.dst_s1))
     if run_realign_tile_joined(d, o, part, src, dst, cnt, smem_bytes, threads):
         return "joined"
+    if run_realign_tile_dest_order(d, o, part, src, dst, cnt, smem_bytes, threads):
+        return "destination order"
     column_max = smem_bytes - 64
     row0 = part * d.rows_per_tile
     nrows = min(d.rows_per_tile, d.rows - row0)
