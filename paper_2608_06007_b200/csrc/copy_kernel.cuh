@@ -743,6 +743,19 @@ __device__ __forceinline__ void realign_store_dest_order(char *out0, uint32_t vs
             for (uint32_t g = 0; g < groups; g++, at += 16 * units, out += vstride)
                 st_stream<uint4>(out, shift_words<WS>(lds128(at), lds128(at + 16), bits));
         }
+    } else if (const uint32_t rpi = kThreads >> lcpr, rr_inc = pshift == 31 ? rpi * n0 : ((rpi & pmask) == 0 ? rpi >> pshift : 0); rr_inc) {
+        // longer runs whose rows advance by a constant from one round of the CTA to the next
+        // (rpi rows per round): the chunk is decoded once, the loop only adds
+        const uint32_t m0 = threadIdx.x ? threadIdx.x : kThreads;  // chunk 0 is partial: thread 0 starts a round later
+        const uint32_t p = (m0 - 1) >> lcpr, c = ((m0 - 1) & cmask) + 1;
+        const uint32_t at0 = shifted + 16 * (((p & pmask) * n0 + (p >> pshift)) * units + c), step = 16 * units * rr_inc;
+        for (uint32_t g = 0; g < groups; g++) {
+            uint32_t at = at0 + 16 * g * units;
+            char *out = out0 + static_cast<size_t>(g) * vstride + 16 * static_cast<size_t>(m0);
+#pragma unroll 2
+            for (uint32_t m = m0; m < total; m += kThreads, at += step, out += 16 * kThreads)
+                st_stream<uint4>(out, shift_words<WS>(lds128(at), lds128(at + 16), bits));
+        }
     } else {
         for (uint32_t g = 0; g < groups; g++) {
             char *out = out0 + static_cast<size_t>(g) * vstride;
