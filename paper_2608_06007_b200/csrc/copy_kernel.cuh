@@ -1043,6 +1043,46 @@ __device__ __forceinline__ bool copy_multi_realign(const Desc &d, const Params<N
         alive = false;
         return true;
     }
+    // planes of short rows that follow one another in the destination, through a misaligned
+    // destination: complete the slots and walk each plane's destination (realign_tile_dest_order)
+    const uint32_t cpr = d.run >> 4, cols = fastdiv(d.rows, d.div_n0);
+    const RealignPass first = plane(0);
+    if (*same && first.d_lo && first.s_lo <= first.d_lo && (d.run & 15) == 0 && (cpr & (cpr - 1)) == 0 && d.run < kJoinMinRun && d.dst_s1 == d.run &&
+        !(d.n0 > 1 && d.dst_s0 == d.run) && cols >= 2 && cols * d.n0 == d.rows) {
+        const bool one_run = d.n0 == 1 || d.dst_s0 == cols * d.run;
+        if (!(one_run && d.n0 > 1 && (cols & (cols - 1)))) {
+            const uint32_t s_lo = first.s_lo, d_lo = first.d_lo, n0 = d.n0, rows = d.rows;
+            const uint32_t magic = 0xffffffffu / rows + 1;  // rows >= 2
+            for (uint32_t rr = threadIdx.x; rr < n_units * rows; rr += kThreads) {
+                const uint32_t j = __umulhi(rr, magic), r = rr - j * rows;
+                const uint32_t k1 = fastdiv(r, d.div_n0), i0 = r - k1 * n0;
+                uint32_t next;
+                if (k1 + 1 < cols) next = rr + n0;
+                else if (one_run && i0 + 1 < n0) next = j * rows + i0 + 1;
+                else continue;
+                const uint32_t at = data_addr + 16 * (rr * units + cpr);
+                uint4 v = lds128(data_addr + 16 * next * units);
+                if (s_lo) v = merge_bytes(lds128(at), v, s_lo);
+                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(at), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+            }
+            __syncthreads();
+            const uint32_t lcpr = 31 - __clz(cpr), groups = one_run ? 1 : n0, total = (one_run ? rows : cols) * cpr;
+            const uint32_t pmask = one_run && n0 > 1 ? cols - 1 : 0xffffffffu, pshift = one_run && n0 > 1 ? 31 - __clz(cols) : 31;
+            for (uint32_t j = 0; j < n_units; j++) {
+                char *out0 = reinterpret_cast<char *>(plane_dst[j]);
+                const uint32_t at_j = data_addr + j * plane_stage;
+                switch (((s_lo - d_lo) & 15) >> 2) {
+                case 0: realign_store_dest_order<0, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, at_j); break;
+                case 1: realign_store_dest_order<1, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, at_j); break;
+                case 2: realign_store_dest_order<2, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, at_j); break;
+                default: realign_store_dest_order<3, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, at_j); break;
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // ordinary stores into the slots, bulk copies next
+            __syncthreads();
+            return true;
+        }
+    }
     if (*same) {  // one pass of the store loops over the rows of all planes
         RealignPass all = plane(0);
         all.n_rows = n_units * d.rows;
