@@ -726,31 +726,33 @@ __device__ __forceinline__ int realign_tile_joined(const Desc &d, const char *sr
 // (nothing touched), -1 the bulk copies did not arrive.
 template <int WS, int kThreads>
 __device__ __forceinline__ void realign_store_dest_order(char *out0, uint32_t vstride, uint32_t groups, uint32_t total, uint32_t lcpr, uint32_t pmask, uint32_t pshift,
-                                                         uint32_t n0, uint32_t units, uint32_t s_lo, uint32_t d_lo, uint32_t data_addr)
+                                                         uint32_t n0, uint32_t pitch, uint32_t extra, uint32_t s_lo, uint32_t d_lo, uint32_t data_addr)
 {
+    // row rr (column k1 = p & pmask of the tile) keeps its chunks from 16 * (rr * pitch + k1 * extra) on
     const int delta = static_cast<int>(s_lo) - static_cast<int>(d_lo);
     const uint32_t bits = (static_cast<uint32_t>(delta) & 3) * 8;
     const uint32_t shifted = data_addr + 16 * (delta >> 4);
     const uint32_t cmask = (1u << lcpr) - 1;
+    const uint32_t off = d_lo ? 1 : 0;  // through a misaligned destination a run's first chunk is partial
+    auto chunk_of = [&](uint32_t p, uint32_t c) { return ((p & pmask) * n0 + (p >> pshift)) * pitch + (p & pmask) * extra + c; };
     if (total <= kThreads) {
         // short runs (a head's 16 tokens): a thread keeps its chunk and steps through the runs
         const uint32_t m = threadIdx.x;
-        if (m >= 1 && m < total) {  // the run's first chunk is partial
-            const uint32_t p = (m - 1) >> lcpr, c = ((m - 1) & cmask) + 1;
-            uint32_t at = shifted + 16 * (((p & pmask) * n0 + (p >> pshift)) * units + c);
+        if (m >= off && m < total) {
+            uint32_t at = shifted + 16 * chunk_of((m - off) >> lcpr, ((m - off) & cmask) + off);
             char *out = out0 + 16 * static_cast<size_t>(m);
 #pragma unroll 4
-            for (uint32_t g = 0; g < groups; g++, at += 16 * units, out += vstride)
+            for (uint32_t g = 0; g < groups; g++, at += 16 * pitch, out += vstride)
                 st_stream<uint4>(out, shift_words<WS>(lds128(at), lds128(at + 16), bits));
         }
     } else if (const uint32_t rpi = kThreads >> lcpr, rr_inc = pshift == 31 ? rpi * n0 : ((rpi & pmask) == 0 ? rpi >> pshift : 0); rr_inc) {
         // longer runs whose rows advance by a constant from one round of the CTA to the next
         // (rpi rows per round): the chunk is decoded once, the loop only adds
-        const uint32_t m0 = threadIdx.x ? threadIdx.x : kThreads;  // chunk 0 is partial: thread 0 starts a round later
-        const uint32_t p = (m0 - 1) >> lcpr, c = ((m0 - 1) & cmask) + 1;
-        const uint32_t at0 = shifted + 16 * (((p & pmask) * n0 + (p >> pshift)) * units + c), step = 16 * units * rr_inc;
+        const uint32_t m0 = threadIdx.x >= off ? threadIdx.x : kThreads;  // a partial chunk 0: thread 0 starts a round later
+        const uint32_t at0 = shifted + 16 * chunk_of((m0 - off) >> lcpr, ((m0 - off) & cmask) + off);
+        const uint32_t step = 16 * (pitch * rr_inc + (pshift == 31 ? extra * rpi : 0));
         for (uint32_t g = 0; g < groups; g++) {
-            uint32_t at = at0 + 16 * g * units;
+            uint32_t at = at0 + 16 * g * pitch;
             char *out = out0 + static_cast<size_t>(g) * vstride + 16 * static_cast<size_t>(m0);
 #pragma unroll 2
             for (uint32_t m = m0; m < total; m += kThreads, at += step, out += 16 * kThreads)
@@ -761,24 +763,20 @@ __device__ __forceinline__ void realign_store_dest_order(char *out0, uint32_t vs
             char *out = out0 + static_cast<size_t>(g) * vstride;
 #pragma unroll 2
             for (uint32_t m = threadIdx.x; m < total; m += kThreads) {
-                if (m == 0) continue;  // the run's first chunk is partial
-                const uint32_t p = (m - 1) >> lcpr, c = ((m - 1) & cmask) + 1;
-                const uint32_t rr = (p & pmask) * n0 + (p >> pshift) + g;
-                const uint32_t at = shifted + 16 * (rr * units + c);
+                if (m < off) continue;
+                const uint32_t at = shifted + 16 * (chunk_of((m - off) >> lcpr, ((m - off) & cmask) + off) + g * pitch);
                 st_stream<uint4>(out + 16 * static_cast<size_t>(m), shift_words<WS>(lds128(at), lds128(at + 16), bits));
             }
         }
     }
     // the first 16 - d_lo and the last d_lo bytes of every run, a thread per byte
     const uint32_t last_p = (total >> lcpr) - 1;
-    for (uint32_t item = threadIdx.x; item < groups * 16; item += kThreads) {
+    for (uint32_t item = threadIdx.x; item < (d_lo ? groups * 16 : 0); item += kThreads) {
         const uint32_t g = item >> 4, k = item & 15;
         const bool tail = k < d_lo;  // k < d_lo: byte k of the run's last chunk; else byte k of its first
-        const uint32_t p = tail ? last_p : 0;
-        const uint32_t rr = (p & pmask) * n0 + (p >> pshift) + g;
         const uint32_t row_byte = tail ? (16u << lcpr) - d_lo + k : k - d_lo;
         uint32_t v;
-        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(data_addr + 16 * rr * units + s_lo + row_byte));
+        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(data_addr + 16 * (chunk_of(tail ? last_p : 0, 0) + g * pitch) + s_lo + row_byte));
         out0[static_cast<size_t>(g) * vstride + (tail ? 16 * static_cast<size_t>(total) + k : k)] = static_cast<char>(v);
     }
 }
@@ -795,11 +793,16 @@ __device__ __forceinline__ int realign_tile_dest_order(const Desc &d, const char
     char *d0 = dst + j1 * d.dst_s1;
     const uint32_t s_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(s0)) & 15;
     const uint32_t d_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(d0)) & 15;
-    if (d_lo == 0) return 0;  // an aligned destination measured no faster this way (unpack 1.5 % slower)
+    // An aligned destination is taken this way only where the misaligned source is contiguous
+    // along i0 (a packed buffer's tokens): a column of n0 rows then arrives as ONE bulk copy, its
+    // rows at the source's own pitch, instead of n0 overlapping ones (with a slot per row the walk
+    // measured no faster than the per-row loop, and 1.5 % slower for unpack).
+    const bool pieces = d_lo == 0 && s_lo != 0 && d.src_s0 == run;
+    if (d_lo == 0 && !pieces) return 0;
     // chunks per slot: the row's own, and what the chunk it shares with the next row needs of that
     // row - its first aligned chunk, and its second one too when s_lo > d_lo
-    const uint32_t units = cpr + (s_lo > d_lo ? 2 : 1);
-    if (nrows * (units << 4) + 32 > stage_bytes) return 0;
+    const uint32_t units = pieces ? cpr : cpr + (s_lo > d_lo ? 2 : 1);
+    if ((pieces ? cols * (n0 * cpr + 1) * 16 : nrows * (units << 4)) + 32 > stage_bytes) return 0;
     // one run per i0, dst_s0 apart - or, where those runs are adjacent too, one run in all
     const bool one_run = n0 == 1 || d.dst_s0 == cols * run;
     if (one_run && n0 > 1 && (cols & (cols - 1))) return 0;
@@ -807,16 +810,21 @@ __device__ __forceinline__ int realign_tile_dest_order(const Desc &d, const char
     const uint32_t groups = one_run ? 1 : n0, glen = one_run ? nrows : cols;
     const uint32_t pmask = one_run && n0 > 1 ? cols - 1 : 0xffffffffu, pshift = one_run && n0 > 1 ? 31 - __clz(cols) : 31;
     const char *base = s0 - s_lo;
-    if (threadIdx.x == 0) mbar_expect_tx(bar, nrows * (s_lo ? run + 16 : run));
-    for (uint32_t rr = threadIdx.x; rr < nrows; rr += kThreads) {
-        const uint32_t k1 = fastdiv(rr, d.div_n0), i0 = rr - k1 * n0;  // the tile starts on an i1 boundary
-        bulk_load(data_addr + 16 * rr * units, base + (k1 * d.src_s1 + i0 * d.src_s0), s_lo ? run + 16 : run, bar);
+    if (pieces) {
+        if (threadIdx.x == 0) mbar_expect_tx(bar, cols * (n0 * run + 16));
+        for (uint32_t k1 = threadIdx.x; k1 < cols; k1 += kThreads) bulk_load(data_addr + 16 * k1 * (n0 * cpr + 1), base + k1 * d.src_s1, n0 * run + 16, bar);
+    } else {
+        if (threadIdx.x == 0) mbar_expect_tx(bar, nrows * (s_lo ? run + 16 : run));
+        for (uint32_t rr = threadIdx.x; rr < nrows; rr += kThreads) {
+            const uint32_t k1 = fastdiv(rr, d.div_n0), i0 = rr - k1 * n0;  // the tile starts on an i1 boundary
+            bulk_load(data_addr + 16 * rr * units, base + (k1 * d.src_s1 + i0 * d.src_s0), s_lo ? run + 16 : run, bar);
+        }
     }
     if (!realign_wait(bar, phase, wait_ok)) return -1;
     // complete every slot with the first chunk of the row after it in the destination (the next
     // column of the same i0, or, in a single run, the first column of the next i0): from that
     // row's own slot - a second copy from global memory per row, bulk or not, cost more than it saved
-    for (uint32_t rr = threadIdx.x; rr < nrows; rr += kThreads) {
+    for (uint32_t rr = threadIdx.x; rr < (d_lo ? nrows : 0); rr += kThreads) {
         const uint32_t k1 = fastdiv(rr, d.div_n0), i0 = rr - k1 * n0;
         uint32_t next;
         if (k1 + 1 < cols) next = rr + n0;
@@ -831,14 +839,14 @@ __device__ __forceinline__ int realign_tile_dest_order(const Desc &d, const char
             asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(at + 16), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
         }
     }
-    __syncthreads();
+    if (d_lo) __syncthreads();
     char *out0 = d0 - d_lo;
     const uint32_t total = glen * cpr;
     switch (((s_lo - d_lo) & 15) >> 2) {
-    case 0: realign_store_dest_order<0, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, data_addr); break;
-    case 1: realign_store_dest_order<1, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, data_addr); break;
-    case 2: realign_store_dest_order<2, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, data_addr); break;
-    default: realign_store_dest_order<3, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, data_addr); break;
+    case 0: realign_store_dest_order<0, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, pieces ? 1 : 0, s_lo, d_lo, data_addr); break;
+    case 1: realign_store_dest_order<1, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, pieces ? 1 : 0, s_lo, d_lo, data_addr); break;
+    case 2: realign_store_dest_order<2, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, pieces ? 1 : 0, s_lo, d_lo, data_addr); break;
+    default: realign_store_dest_order<3, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, pieces ? 1 : 0, s_lo, d_lo, data_addr); break;
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // ordinary stores into the slots, bulk copies next
     __syncthreads();
@@ -1072,10 +1080,10 @@ __device__ __forceinline__ bool copy_multi_realign(const Desc &d, const Params<N
                 char *out0 = reinterpret_cast<char *>(plane_dst[j]);
                 const uint32_t at_j = data_addr + j * plane_stage;
                 switch (((s_lo - d_lo) & 15) >> 2) {
-                case 0: realign_store_dest_order<0, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, at_j); break;
-                case 1: realign_store_dest_order<1, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, at_j); break;
-                case 2: realign_store_dest_order<2, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, at_j); break;
-                default: realign_store_dest_order<3, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, s_lo, d_lo, at_j); break;
+                case 0: realign_store_dest_order<0, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, 0, s_lo, d_lo, at_j); break;
+                case 1: realign_store_dest_order<1, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, 0, s_lo, d_lo, at_j); break;
+                case 2: realign_store_dest_order<2, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, 0, s_lo, d_lo, at_j); break;
+                default: realign_store_dest_order<3, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, units, 0, s_lo, d_lo, at_j); break;
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // ordinary stores into the slots, bulk copies next

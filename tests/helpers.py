@@ -241,12 +241,14 @@ def run_realign_tile_joined(d, o, part, src, dst, cnt, smem_bytes=52 << 10, thre
 
 def run_realign_tile_dest_order(d, o, part, src, dst, cnt, smem_bytes=52 << 10, threads=256):
     """The realigning path for SHORT rows that follow one another in the destination a step of n0
-    apart, through a misaligned destination, replayed like run_realign_tile.  Returns False,
-    touching nothing, for a tile the kernel would not take this way.  Every row is loaded into a
-    slot of its own; after the wait each slot is completed with the first chunk (two when
-    s_lo > d_lo) of the row that follows it in the destination, taken from that row's slot; the
-    stores then walk the aligned chunks of every destination run, finding each in its row's slot;
-    the first 16 - d_lo and last d_lo bytes of a run go out byte by byte."""
+    apart, replayed like run_realign_tile.  Returns False, touching nothing, for a tile the kernel
+    would not take this way.  Through a misaligned destination every row is loaded into a slot of
+    its own; after the wait each slot is completed with the first chunk (two when s_lo > d_lo) of
+    the row that follows it in the destination, taken from that row's slot; the stores then walk
+    the aligned chunks of every destination run, finding each in its row's slot; the first
+    16 - d_lo and last d_lo bytes of a run go out byte by byte.  With an aligned destination and a
+    misaligned source that is contiguous along i0, a column of n0 rows arrives as one bulk copy,
+    its rows at the source's own pitch, and the same walk stores them."""
     run, n0 = d.run_bytes, d.n0
     row0 = part * d.rows_per_tile
     nrows = min(d.rows_per_tile, d.rows - row0)
@@ -259,10 +261,12 @@ def run_realign_tile_dest_order(d, o, part, src, dst, cnt, smem_bytes=52 << 10, 
     src0 = src.va + d.src_off + o * d.src_outer + j1 * d.src_s1
     dst0 = dst.va + d.dst_off + o * d.dst_outer + j1 * d.dst_s1
     s_lo, d_lo = src0 % 16, dst0 % 16
-    if d_lo == 0:
+    pieces = d_lo == 0 and s_lo != 0 and d.src_s0 == run
+    if d_lo == 0 and not pieces:
         return False
-    units = cpr + (2 if s_lo > d_lo else 1)
-    if nrows * (units << 4) + 32 > smem_bytes:
+    pitch = cpr if pieces else cpr + (2 if s_lo > d_lo else 1)
+    extra = 1 if pieces else 0
+    if (cols * (n0 * cpr + 1) * 16 if pieces else nrows * (pitch << 4)) + 32 > smem_bytes:
         return False
     one_run = n0 == 1 or d.dst_s0 == cols * run
     if one_run and n0 > 1 and cols & (cols - 1):
@@ -271,34 +275,46 @@ def run_realign_tile_dest_order(d, o, part, src, dst, cnt, smem_bytes=52 << 10, 
     data = 16
     stage = np.full(smem_bytes, 0xDD, dtype=np.uint8)
     loaded = np.zeros(smem_bytes, dtype=bool)
-    nbytes = run + 16 if s_lo else run
-    for rr in range(nrows):                                   # one bulk copy per row
-        k1, i0 = divmod(rr, n0)
-        g = src0 - s_lo + k1 * d.src_s1 + i0 * d.src_s0
-        at = data + 16 * rr * units
+
+    def bulk(at, g, nbytes):
+        assert at % 16 == 0 and g % 16 == 0 and nbytes % 16 == 0 and at + nbytes <= smem_bytes
         for c in range(nbytes // 16):
+            assert not loaded[at + 16 * c], "two bulk copies land on one staged chunk"
             stage[at + 16 * c:at + 16 * c + 16] = src.read16(g + 16 * c)
             loaded[at + 16 * c:at + 16 * c + 16] = True
-    snap, snap_loaded = stage.copy(), loaded.copy()           # the fill reads what the copies brought
-    for rr in range(nrows):
-        k1, i0 = divmod(rr, n0)
-        if k1 + 1 < cols:
-            nxt = rr + n0
-        elif one_run and i0 + 1 < n0:
-            nxt = i0 + 1
-        else:
-            continue
-        at, na = data + 16 * (rr * units + cpr), data + 16 * nxt * units
-        assert snap_loaded[na + s_lo:na + 16].all() and (not s_lo or snap_loaded[at:at + s_lo].all())
-        stage[at + s_lo:at + 16] = snap[na + s_lo:na + 16]
-        loaded[at + s_lo:at + 16] = True
-        if s_lo > d_lo:
-            assert snap_loaded[na + 16:na + 32].all()
-            stage[at + 16:at + 32] = snap[na + 16:na + 32]
-            loaded[at + 16:at + 32] = True
+
+    def slot(rr):                                             # chunk index of row rr's first chunk
+        return rr * pitch + (rr // n0) * extra
+
+    if pieces:
+        for k1 in range(cols):                                # one bulk copy per column of n0 rows
+            bulk(data + 16 * k1 * (n0 * cpr + 1), src0 - s_lo + k1 * d.src_s1, n0 * run + 16)
+    else:
+        for rr in range(nrows):                               # one bulk copy per row
+            k1, i0 = divmod(rr, n0)
+            bulk(data + 16 * slot(rr), src0 - s_lo + k1 * d.src_s1 + i0 * d.src_s0, run + 16 if s_lo else run)
+    if d_lo:
+        snap, snap_loaded = stage.copy(), loaded.copy()       # the fill reads what the copies brought
+        for rr in range(nrows):
+            k1, i0 = divmod(rr, n0)
+            if k1 + 1 < cols:
+                nxt = rr + n0
+            elif one_run and i0 + 1 < n0:
+                nxt = i0 + 1
+            else:
+                continue
+            at, na = data + 16 * (slot(rr) + cpr), data + 16 * slot(nxt)
+            assert snap_loaded[na + s_lo:na + 16].all() and (not s_lo or snap_loaded[at:at + s_lo].all())
+            stage[at + s_lo:at + 16] = snap[na + s_lo:na + 16]
+            loaded[at + s_lo:at + 16] = True
+            if s_lo > d_lo:
+                assert snap_loaded[na + 16:na + 32].all()
+                stage[at + 16:at + 32] = snap[na + 16:na + 32]
+                loaded[at + 16:at + 32] = True
     delta = s_lo - d_lo
     sh, shifted = delta % 16, data + 16 * (delta >> 4)
     total = glen * cpr
+    off = 1 if d_lo else 0
     out0 = dst0 - d_lo
 
     def row_of(p, g):
@@ -308,18 +324,18 @@ def run_realign_tile_dest_order(d, o, part, src, dst, cnt, smem_bytes=52 << 10, 
 
     for g in range(groups):
         out = out0 + g * d.dst_s0
-        for m in range(1, total):
-            p, c = divmod(m - 1, cpr)
-            c += 1
-            at = shifted + 16 * (row_of(p, g) * units + c)
+        for m in range(off, total):
+            p, c = divmod(m - off, cpr)
+            c += off
+            at = shifted + 16 * (slot(row_of(p, g)) + c)
             assert 0 <= at and at + 32 <= smem_bytes, "staging read outside the area"
             assert loaded[at + sh:at + sh + 16].all(), "a staged byte that was never loaded is consumed"
             dst.write(out + 16 * m, stage[at + sh:at + sh + 16].copy(), cnt)
-        for k in range(16):
+        for k in range(16 if d_lo else 0):
             tail = k < d_lo
             p = glen - 1 if tail else 0
             row_byte = run - d_lo + k if tail else k - d_lo
-            at = data + 16 * row_of(p, g) * units + s_lo + row_byte
+            at = data + 16 * slot(row_of(p, g)) + s_lo + row_byte
             assert loaded[at], "a staged byte that was never loaded is consumed"
             dst.write(out + (16 * total + k if tail else k), stage[at:at + 1], cnt)
     return True
