@@ -57,7 +57,7 @@
  * any number of bytes.  When every address of a call is a multiple of 16 the kernels move 16-byte
  * vectors register to register.  Otherwise they realign on the fly - aligned 16-byte chunks of
  * the source are staged in shared memory and shifted into aligned 16-byte stores, only the first
- * and last bytes of a row go out in smaller pieces - at 0.85-1.0 of the aligned speed for rows of a
+ * and last bytes of a row go out in smaller pieces - at 0.9-1.0 of the aligned speed for rows of a
  * few hundred bytes and more.  On that path the SOURCE side is read in whole aligned 16-byte
  * chunks: up to 15 bytes before a row's first byte and after its last one are read (always inside
  * a chunk that holds a byte of the row, hence inside the same page) and ignored; destinations are
