@@ -746,9 +746,9 @@ __device__ __forceinline__ void realign_store_dest_order(char *out0, uint32_t vs
                 st_stream<uint4>(out, shift_words<WS>(lds128(at), lds128(at + 16), bits));
         }
     } else if (const uint32_t rpi = kThreads >> lcpr, rr_inc = pshift == 31 ? rpi * n0 : ((rpi & pmask) == 0 ? rpi >> pshift : 0); rr_inc) {
-        // longer runs whose rows advance by a constant from one round of the CTA to the next
-        // (rpi rows per round): the chunk is decoded once, the loop only adds
-        const uint32_t m0 = threadIdx.x >= off ? threadIdx.x : kThreads;  // a partial chunk 0: thread 0 starts a round later
+        // longer runs whose rows advance by a constant from one sweep of the CTA over the run to the next
+        // (rpi rows per sweep): the chunk is decoded once, the loop only adds
+        const uint32_t m0 = threadIdx.x >= off ? threadIdx.x : kThreads;  // a partial chunk 0: thread 0 starts a sweep later
         const uint32_t at0 = shifted + 16 * chunk_of((m0 - off) >> lcpr, ((m0 - off) & cmask) + off);
         const uint32_t step = 16 * (pitch * rr_inc + (pshift == 31 ? extra * rpi : 0));
         for (uint32_t g = 0; g < groups; g++) {
