@@ -1006,6 +1006,45 @@ __device__ __forceinline__ bool copy_multi_realign(const Desc &d, const Params<N
     if (d.run < kRealignMinRun || d.run > kRealignColumn || ((d.src_s0 | d.src_s1 | d.dst_s0 | d.dst_s1) & 15) || n_units * plane_stage + 32 > prm.stage_bytes)
         return false;
     const uint32_t data_addr = static_cast<uint32_t>(__cvta_generic_to_shared(stage + 16));
+    // Planes a byte stride apart whose misaligned source is contiguous along i0 and whose
+    // destination is aligned (a packed buffer at an odd offset unpacked into a pool): every column
+    // of n0 rows of every plane arrives as one bulk copy and each plane's destination is walked
+    // (see realign_tile_dest_order)
+    if (!STEP && ((d.src_outer | d.dst_outer) & 15) == 0) {
+        const uint32_t run = d.run, n0 = d.n0, cpr = run >> 4, rows = d.rows, cols = fastdiv(rows, d.div_n0);
+        const char *src0 = prm.ptr[d.src_slot] + d.src_off + static_cast<long long>(o) * d.src_outer;
+        char *dst0 = prm.ptr[d.dst_slot] + d.dst_off + static_cast<long long>(o) * d.dst_outer;
+        const uint32_t s_lo = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src0)) & 15;
+        const bool one_run = n0 == 1 || d.dst_s0 == cols * run;
+        const uint32_t piece_stage = cols * (n0 * cpr + 1) * 16;
+        if (s_lo && (reinterpret_cast<uintptr_t>(dst0) & 15) == 0 && d.src_s0 == run && (run & 15) == 0 && (cpr & (cpr - 1)) == 0 && run < kJoinMinRun &&
+            d.dst_s1 == run && !(n0 > 1 && d.dst_s0 == run) && cols >= 2 && cols * n0 == rows && !(one_run && n0 > 1 && (cols & (cols - 1))) &&
+            n_units * piece_stage + 32 <= prm.stage_bytes) {
+            if (threadIdx.x == 0) mbar_expect_tx(bar, n_units * cols * (n0 * run + 16));
+            for (uint32_t item = threadIdx.x; item < n_units * cols; item += kThreads) {
+                const uint32_t j = item / cols, k1 = item - j * cols;
+                bulk_load(data_addr + j * piece_stage + 16 * k1 * (n0 * cpr + 1), src0 - s_lo + static_cast<long long>(j) * d.src_outer + k1 * d.src_s1, n0 * run + 16, bar);
+            }
+            if (!realign_wait(bar, phase, wait_ok)) {
+                alive = false;
+                return true;
+            }
+            const uint32_t lcpr = 31 - __clz(cpr), groups = one_run ? 1 : n0, total = (one_run ? rows : cols) * cpr;
+            const uint32_t pmask = one_run && n0 > 1 ? cols - 1 : 0xffffffffu, pshift = one_run && n0 > 1 ? 31 - __clz(cols) : 31;
+            for (uint32_t j = 0; j < n_units; j++) {
+                char *out0 = dst0 + static_cast<long long>(j) * d.dst_outer;
+                const uint32_t at_j = data_addr + j * piece_stage;
+                switch ((s_lo & 15) >> 2) {
+                case 0: realign_store_dest_order<0, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, cpr, 1, s_lo, 0, at_j); break;
+                case 1: realign_store_dest_order<1, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, cpr, 1, s_lo, 0, at_j); break;
+                case 2: realign_store_dest_order<2, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, cpr, 1, s_lo, 0, at_j); break;
+                default: realign_store_dest_order<3, kThreads>(out0, d.dst_s0, groups, total, lcpr, pmask, pshift, n0, cpr, 1, s_lo, 0, at_j); break;
+                }
+            }
+            __syncthreads();
+            return true;
+        }
+    }
     auto plane = [&](uint32_t j) {
         const uint32_t k = o + j;
         RealignPass p;
