@@ -797,7 +797,7 @@ __device__ __forceinline__ int realign_tile_dest_order(const Desc &d, const char
     // along i0 (a packed buffer's tokens): a column of n0 rows then arrives as ONE bulk copy, its
     // rows at the source's own pitch, instead of n0 overlapping ones (with a slot per row the walk
     // measured no faster than the per-row loop, and 1.5 % slower for unpack).
-    const bool pieces = d_lo == 0 && s_lo != 0 && d.src_s0 == run;
+    const bool pieces = d_lo == 0 && d.src_s0 == run;  // (both sides aligned: tuning.copy_path = 1, or an aligned tile of a misaligned call)
     if (d_lo == 0 && !pieces) return 0;
     // chunks per slot: the row's own, and what the chunk it shares with the next row needs of that
     // row - its first aligned chunk, and its second one too when s_lo > d_lo
@@ -811,8 +811,9 @@ __device__ __forceinline__ int realign_tile_dest_order(const Desc &d, const char
     const uint32_t pmask = one_run && n0 > 1 ? cols - 1 : 0xffffffffu, pshift = one_run && n0 > 1 ? 31 - __clz(cols) : 31;
     const char *base = s0 - s_lo;
     if (pieces) {
-        if (threadIdx.x == 0) mbar_expect_tx(bar, cols * (n0 * run + 16));
-        for (uint32_t k1 = threadIdx.x; k1 < cols; k1 += kThreads) bulk_load(data_addr + 16 * k1 * (n0 * cpr + 1), base + k1 * d.src_s1, n0 * run + 16, bar);
+        const uint32_t piece_bytes = n0 * run + (s_lo ? 16 : 0);  // never a chunk without a byte of the column
+        if (threadIdx.x == 0) mbar_expect_tx(bar, cols * piece_bytes);
+        for (uint32_t k1 = threadIdx.x; k1 < cols; k1 += kThreads) bulk_load(data_addr + 16 * k1 * (n0 * cpr + 1), base + k1 * d.src_s1, piece_bytes, bar);
     } else {
         if (threadIdx.x == 0) mbar_expect_tx(bar, nrows * (s_lo ? run + 16 : run));
         for (uint32_t rr = threadIdx.x; rr < nrows; rr += kThreads) {

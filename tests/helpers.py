@@ -261,7 +261,7 @@ def run_realign_tile_dest_order(d, o, part, src, dst, cnt, smem_bytes=52 << 10, 
     src0 = src.va + d.src_off + o * d.src_outer + j1 * d.src_s1
     dst0 = dst.va + d.dst_off + o * d.dst_outer + j1 * d.dst_s1
     s_lo, d_lo = src0 % 16, dst0 % 16
-    pieces = d_lo == 0 and s_lo != 0 and d.src_s0 == run
+    pieces = d_lo == 0 and d.src_s0 == run
     if d_lo == 0 and not pieces:
         return False
     pitch = cpr if pieces else cpr + (2 if s_lo > d_lo else 1)
@@ -288,7 +288,7 @@ def run_realign_tile_dest_order(d, o, part, src, dst, cnt, smem_bytes=52 << 10, 
 
     if pieces:
         for k1 in range(cols):                                # one bulk copy per column of n0 rows
-            bulk(data + 16 * k1 * (n0 * cpr + 1), src0 - s_lo + k1 * d.src_s1, n0 * run + 16)
+            bulk(data + 16 * k1 * (n0 * cpr + 1), src0 - s_lo + k1 * d.src_s1, n0 * run + (16 if s_lo else 0))
     else:
         for rr in range(nrows):                               # one bulk copy per row
             k1, i0 = divmod(rr, n0)
