@@ -736,13 +736,21 @@ __device__ __forceinline__ void realign_store_dest_order(char *out0, uint32_t vs
     const uint32_t off = d_lo ? 1 : 0;  // through a misaligned destination a run's first chunk is partial
     auto chunk_of = [&](uint32_t p, uint32_t c) { return ((p & pmask) * n0 + (p >> pshift)) * pitch + (p & pmask) * extra + c; };
     if (total <= kThreads) {
-        // short runs (a head's 16 tokens): a thread keeps its chunk and steps through the runs
-        const uint32_t m = threadIdx.x;
+        // short runs (a head's 16 tokens): a thread keeps its chunk and steps through the runs;
+        // where a run has fewer chunks than the CTA has threads (128-byte rows), gpar runs go side by side
+        uint32_t m = threadIdx.x, g0 = 0, gpar = 1;
+        if (total < kThreads && (total & (total - 1)) == 0) {
+            const uint32_t lt = 31 - __clz(total);
+            gpar = kThreads >> lt;
+            g0 = m >> lt;
+            m &= total - 1;
+        }
         if (m >= off && m < total) {
-            uint32_t at = shifted + 16 * chunk_of((m - off) >> lcpr, ((m - off) & cmask) + off);
-            char *out = out0 + 16 * static_cast<size_t>(m);
+            uint32_t at = shifted + 16 * (chunk_of((m - off) >> lcpr, ((m - off) & cmask) + off) + g0 * pitch);
+            char *out = out0 + 16 * static_cast<size_t>(m) + static_cast<size_t>(g0) * vstride;
+            const size_t ostep = static_cast<size_t>(gpar) * vstride;
 #pragma unroll 4
-            for (uint32_t g = 0; g < groups; g++, at += 16 * pitch, out += vstride)
+            for (uint32_t g = g0; g < groups; g += gpar, at += 16 * pitch * gpar, out += ostep)
                 st_stream<uint4>(out, shift_words<WS>(lds128(at), lds128(at + 16), bits));
         }
     } else if (const uint32_t rpi = kThreads >> lcpr, rr_inc = pshift == 31 ? rpi * n0 : ((rpi & pmask) == 0 ? rpi >> pshift : 0); rr_inc) {
