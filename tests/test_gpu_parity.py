@@ -904,7 +904,7 @@ def test_dim1_weight_slices_with_long_rows_through_misaligned_pointers(a, b):
     assert tc.tc_device_status() == 0
 
 
-@pytest.mark.parametrize("H,D,E,slots", [(8, 128, 2, "one"), (8, 64, 2, "one"), (8, 32, 2, "planes"), (8, 512, 2, "one"), (2, 512, 2, "one"), (4, 256, 4, "one")])
+@pytest.mark.parametrize("H,D,E,slots", [(8, 128, 2, "one"), (8, 64, 2, "one"), (8, 32, 2, "planes"), (8, 512, 2, "one"), (2, 512, 2, "one"), (4, 256, 4, "one"), (16, 64, 2, "one"), (32, 32, 2, "one")])
 @pytest.mark.parametrize("shift_pool,shift_packed", [(0, 2), (2, 0), (6, 6), (1, 9), (8, 4)])
 def test_kv_pack_unpack_migrate_through_misaligned_pointers(shift_pool, shift_packed, H, D, E, slots):
     """Aligned geometry, misaligned base pointers: the pool and / or the packed buffer start at
@@ -912,7 +912,8 @@ def test_kv_pack_unpack_migrate_through_misaligned_pointers(shift_pool, shift_pa
     planes (same layout) both take the realigning path; with D = 64 and 32 a plane is small enough
     for tiles of two and four planes, in a pool with one pointer or a pointer per plane; rows of
     1 KiB are staged back to back where the destination has them adjacent (a head's tokens, a
-    token's heads)."""
+    token's heads); with 16 and 32 heads of 128- and 64-byte rows a destination run has fewer chunks
+    than the CTA has threads and several runs go side by side."""
     rng = np.random.default_rng(77)
     shape, NB, stride, pool, T, off, bt = kv_case(rng, L=2, NB=40, B=16, H=H, D=D, E=E, T=(100, 16, 7, 333))
     L, B, H, D, E = shape
